@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the RIB window-attention hot path (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one forward and one backward pass of the whole path (window partition + cyclic shift,
+RIB concat, logits, softmax, PV, lse; D pre-pass, the five backward contractions, dPq/dPk
+reduction) over one synthetic batch of the training-patch configuration (B8, 96x96, 6 heads,
+d=32, r=16, window 32, shift 16).  Rank 0 prints ONE JSON line.  With N > 1 every rank runs its
+own batch (pairs are independent: no data-path collective) and the value is the sum over ranks
+divided by the slowest rank's device time.
+
+`--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "rib_window_attn_fwd_bwd_tflops_bf16"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1000 * 1000
+
+
+def load_peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return json.loads(f.read_text()), "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def pick_workload(name):
+    from paper_2603_06738_b200 import synthetic
+    if name is None:
+        base = synthetic.CONFIGS[1]
+        return synthetic.Workload(base.name, base.B, base.H, base.W, base.heads, base.d, base.r, base.window,
+                                  base.shift, base.seed, backward=True)
+    for wl in synthetic.CONFIGS:
+        if wl.name == name or wl.name.startswith(name):
+            return synthetic.Workload(wl.name, wl.B, wl.H, wl.W, wl.heads, wl.d, wl.r, wl.window, wl.shift,
+                                      wl.seed, backward=True)
+    raise SystemExit(f"unknown workload {name!r}; choose from {[w.name for w in synthetic.CONFIGS]}")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.sm, self.reasons, self.max_sm = index, threading.Event(), [], set(), None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            pass
+
+    NAMES = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+             0x80: "hw_power_brake_slowdown"}
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.NAMES.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def summary(self):
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_sm, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.max_sm, "reasons": sorted(self.reasons),
+                "samples": len(self.sm)}
+
+
+def cpu_oracle_sample(wl, budget_pairs=None):
+    """Times the CPU oracle, as it stands, on the first pairs of the workload (forward + backward)."""
+    import numpy as np
+    from oracle import rib_oracle as orc
+    from paper_2603_06738_b200 import synthetic
+    cores = orc.threads()
+    npairs = min(wl.pairs, budget_pairs or 48 * cores)
+    # the sampled pairs live in the first images only: generate just those
+    per_image = wl.pairs // wl.B
+    nb = min(wl.B, -(-npairs // per_image))
+    sub = synthetic.Workload(wl.name, nb, wl.H, wl.W, wl.heads, wl.d, wl.r, wl.window, wl.shift, wl.seed, True)
+    t = {k: v.to(dtype=__import__("torch").float64).numpy() for k, v in synthetic.make_inputs(sub, True).items()}
+    pairs = list(range(npairs))
+    t0 = time.perf_counter()
+    orc.fwd(t["q"], t["k"], t["v"], t["pq"], t["pk"], wl.window, wl.shift, pairs=pairs)
+    t1 = time.perf_counter()
+    orc.bwd(t["q"], t["k"], t["v"], t["pq"], t["pk"], t["dout"], wl.window, wl.shift, pairs=pairs)
+    t2 = time.perf_counter()
+    flops = npairs * 2 * wl.n * wl.n * ((2 * wl.d + wl.r) + (5 * wl.d + 3 * wl.r))
+    return {"value": flops / (t2 - t0) / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {npairs} of {wl.pairs} pairs of {wl.name}, forward {t1 - t0:.2f} s + backward "
+                      f"{t2 - t1:.2f} s, fp64",
+            "seconds": t2 - t0, "tokens_per_s": npairs * wl.n / wl.heads / (t2 - t0)}
+
+
+def run_reference(args, wl, rank):
+    if rank != 0:
+        return
+    samples = []
+    cpu_oracle_sample(wl, budget_pairs=8)   # warm-up: builds and loads the oracle
+    steps = max(1, min(args.steps, 3))
+    for _ in range(steps):
+        samples.append(cpu_oracle_sample(wl))
+    best = max(samples, key=lambda s: s["value"])
+    secs = statistics.mean(s["seconds"] for s in samples)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": best["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": 1, "ms_per_step": secs * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "note": "each step is a bounded sample of the workload: " + best["sample"]},
+        "cpu_baseline": {k: best[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": best["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=None, help="prefix of a configuration name (default: cfg2 shape)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    wl = pick_workload(args.workload)
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_06738_b200 import binding, synthetic
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    binding.library()   # fail loudly if the extension has not been built
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    args.warmup = max(args.warmup, 3)
+
+    # every rank owns a batch of its own (seed offset by rank); pairs are independent
+    my = synthetic.Workload(wl.name, wl.B, wl.H, wl.W, wl.heads, wl.d, wl.r, wl.window, wl.shift,
+                            wl.seed + 1000 * rank, True)
+    host = {k: v.pin_memory() for k, v in synthetic.make_inputs(my, True).items()}
+    step_bytes = sum(host[k].numel() * 2 for k in ("q", "k", "v", "dout")) * 2   # + out, dq, dk, dv
+    nsets = max(2, -(-3 * L2_BYTES // step_bytes))
+    sets = []
+    for i in range(nsets):
+        s = {k: v.to(dev) for k, v in host.items()}
+        if i:   # decorrelate the copies cheaply: rotate the batch dimension
+            for k in ("q", "k", "v", "dout"):
+                s[k] = torch.roll(s[k], i, 0).contiguous()
+        s["out"] = torch.empty_like(s["q"])
+        s["lse"] = torch.empty((wl.B, wl.heads, wl.H, wl.W), dtype=torch.float32, device=dev)
+        sets.append(s)
+    ws_bytes = binding.rib_window_attn_bwd_workspace(wl.B, wl.H, wl.W, wl.heads, wl.d, wl.r, wl.window)
+    workspace = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+
+    def step(s):
+        binding.rib_window_attn_fwd(s["q"], s["k"], s["v"], s["pq"], s["pk"], wl.window, wl.shift,
+                                    out=s["out"], lse=s["lse"])
+        fwd_path = binding.rib_last_path()
+        res = binding.rib_window_attn_bwd(s["q"], s["k"], s["v"], s["pq"], s["pk"], s["out"], s["lse"], s["dout"],
+                                          wl.window, wl.shift, workspace=workspace)
+        return fwd_path, binding.rib_last_path(), res
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        paths = step(sets[i % nsets])[:2]
+    barrier()
+    if binding.rib_query_status() != 0:
+        raise SystemExit("device status word set during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = binding.rib_kernel_launches()
+    sampler.start()
+    barrier()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        s = sets[i % nsets]
+        ev[i][0].record()
+        binding.rib_window_attn_fwd(s["q"], s["k"], s["v"], s["pq"], s["pk"], wl.window, wl.shift,
+                                    out=s["out"], lse=s["lse"])
+        ev[i][1].record()
+        binding.rib_window_attn_bwd(s["q"], s["k"], s["v"], s["pq"], s["pk"], s["out"], s["lse"], s["dout"],
+                                    wl.window, wl.shift, workspace=workspace)
+        ev[i][2].record()
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    sampler.stop_flag.set()
+    sampler.join()
+    launches = binding.rib_kernel_launches() - launches0
+    status = binding.rib_query_status()
+    fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])          # device time of exactly K steps
+
+    # ------------------------------------------------ end to end: pinned host buffers, H2D + D2H inside
+    e2e = None
+    if not args.no_e2e:
+        s = sets[0]
+        hout = {k: torch.empty_like(host["q"]).pin_memory() for k in ("out", "dq", "dk", "dv")}
+        hdp = {k: torch.empty((wl.n, wl.r), dtype=torch.float32).pin_memory() for k in ("dpq", "dpk")}
+        h2d = sum(host[k].numel() * host[k].element_size() for k in ("q", "k", "v", "pq", "pk", "dout"))
+        d2h = sum(t.numel() * t.element_size() for t in list(hout.values()) + list(hdp.values()))
+
+        def e2e_step():
+            for k in ("q", "k", "v", "pq", "pk", "dout"):
+                s[k].copy_(host[k], non_blocking=True)
+            _, _, (dq, dk, dv, dpq, dpk) = step(s)
+            hout["out"].copy_(s["out"], non_blocking=True)
+            for k, t in (("dq", dq), ("dk", dk), ("dv", dv)):
+                hout[k].copy_(t, non_blocking=True)
+            hdp["dpq"].copy_(dpq, non_blocking=True)
+            hdp["dpk"].copy_(dpk, non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2e_steps = max(3, min(args.steps, 10))
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    else:
+        e2e_ms, h2d, d2h = None, 0, 0
+
+    # ------------------------------------------------ reduce over ranks (max time), compose the line
+    times = torch.tensor([total_ms, statistics.median(fwd_ms), statistics.median(bwd_ms), e2e_ms or 0.0],
+                         dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, fwd_med, bwd_med, e2e_ms_max = (float(x) for x in times.tolist())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    ms_per_step = total_ms / args.steps
+    flops_step = (wl.fwd_flops + wl.bwd_flops) * world
+    value = flops_step / (ms_per_step * 1e-3) / 1e12
+    fwd_tf = wl.fwd_flops / (fwd_med * 1e-3) / 1e12
+    bwd_tf = wl.bwd_flops / (bwd_med * 1e-3) / 1e12
+    peak = float(peaks["bf16_tflops"])
+    dominant = "backward (rib_window_attn_bwd kernels)" if bwd_med >= fwd_med else "forward (rib_window_attn_fwd kernel)"
+    dom_tf = bwd_tf if bwd_med >= fwd_med else fwd_tf
+    traffic_file = ROOT / "profiles" / "traffic.json"
+    traffic = None
+    if traffic_file.exists():
+        try:
+            traffic = json.loads(traffic_file.read_text()).get("bwd" if bwd_med >= fwd_med else "fwd")
+        except Exception:
+            traffic = None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name + " (forward + backward)", "B": wl.B, "H": wl.H, "W": wl.W, "heads": wl.heads,
+                   "d": wl.d, "r": wl.r, "window": wl.window, "shift": wl.shift, "pairs": wl.pairs,
+                   "l2": f"rotating {nsets} input/output sets ({nsets * step_bytes >> 20} MiB) > 126 MB L2, no flush",
+                   "paths": {"fwd": paths[0], "bwd": paths[1]}, "multi_gpu": "independent batch per rank, no collective"},
+        "tokens_per_s": wl.tokens * world / (ms_per_step * 1e-3),
+        "fwd": {"ms": fwd_med, "tflops": fwd_tf, "frac_of_peak": fwd_tf / peak},
+        "bwd": {"ms": bwd_med, "tflops": bwd_tf, "frac_of_peak": bwd_tf / peak},
+        "frac_of_peak": value / world / peak,
+        "roofline": {"bound": "tensor", "kernel": dominant, "achieved": dom_tf, "peak": peak, "unit": "TFLOP/s",
+                     "frac": dom_tf / peak, "traffic": traffic, "peak_source": f"bf16_tflops burst, {peak_kind}"},
+        "e2e": None if e2e_ms is None else {
+            "value": flops_step / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_max,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "clocks": sampler.summary(),
+        "wall_s": t_wall,
+        "device_status": status,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = {k: v for k, v in cpu_oracle_sample(wl).items() if k != "seconds"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

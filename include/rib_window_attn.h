@@ -1,0 +1,118 @@
+/*
+ * rib_window_attn.h -- C ABI of the B200 (sm_100a) RIB window-attention library.
+ *
+ * The operation (paper: Sec. 2.2 window attention; Sec. 3.1 "Rank-factorized Implicit Neural
+ * Bias", Eq. 5 and Eq. 6).  A feature map of H x W tokens is cut into M x M windows
+ * (M = `window`, n = M*M tokens per window).  Inside every window, for every head,
+ *
+ *     S_ij = (q_i . k_j) / sqrt(d) + (Pq_i . Pk_j) / sqrt(r)        (Eq. 6)
+ *
+ * which is the single dot product of the concatenated rows [q_i/sqrt(d), Pq_i/sqrt(r)] and
+ * [k_j, Pk_j] (Eq. 5); then P = SoftMax(S) row-wise and O = P V as in standard attention.  The
+ * rank-r positional features Pq, Pk depend only on the position inside the window and are the
+ * same for every window, batch item and head.  The n x n bias matrix is never formed.
+ *
+ * Window geometry.  Token i = y*M + x of window (wy, wx) is image pixel
+ *     ( (wy*M + y + shift) mod H , (wx*M + x + shift) mod W ).
+ * shift = 0 is plain window partition; shift > 0 is a cyclic (torus) shift of the window grid,
+ * with no mask between wrapped regions.  Row i of Pq/Pk belongs to token i.
+ *
+ * Layouts (all DEVICE pointers, owned by the caller, 16-byte aligned, inputs never alias
+ * outputs):
+ *   q, k, v, out, dout, dq, dk, dv : bf16  [B][H][W][heads][d]   (channels last)
+ *   pq, pk                         : bf16  [n][r]
+ *   lse                            : fp32  [B][heads][H][W]      natural log of sum_j exp(S_ij)
+ *   dpq, dpk                       : fp32  [n][r]                summed over batch, windows, heads
+ * Raw q and Pq are passed; the library applies 1/sqrt(d) and 1/sqrt(r) itself.
+ *
+ * Calls only ENQUEUE work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ * and return without synchronising.  They return RIB_OK (0) or a negative RIB_ERR_* code; on an
+ * error nothing has been launched.  No exception crosses this boundary.  There is no CPU
+ * fallback: every step runs in CUDA kernels of this library.
+ *
+ * Supported shapes: H and W multiples of `window`, 0 <= shift < window, 1 <= d <= 64,
+ * 0 <= r <= 64, d and r multiples of 8 (16-byte rows).  Shapes with d = 32, r = 16, window a
+ * multiple of 16 and shift a multiple of 8 take the tcgen05 / TMEM / TMA kernels; every other
+ * supported shape takes a slower any-shape CUDA kernel.
+ */
+#ifndef RIB_WINDOW_ATTN_H
+#define RIB_WINDOW_ATTN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    RIB_OK = 0,
+    RIB_ERR_NULL = -1,         /* a required pointer is NULL */
+    RIB_ERR_SHAPE = -2,        /* non-positive size, H or W not a multiple of window, bad shift */
+    RIB_ERR_UNSUPPORTED = -3,  /* d or r outside the supported range */
+    RIB_ERR_ALIGN = -4,        /* a pointer is not 16-byte aligned */
+    RIB_ERR_WORKSPACE = -5,    /* workspace missing or smaller than rib_window_attn_bwd_workspace() */
+    RIB_ERR_CUDA = -6,         /* a CUDA call (launch, tensor-map encode, memset) failed */
+    RIB_ERR_DEVICE_WAIT = -7   /* reported by rib_query_status: a bounded device-side wait ran out */
+};
+
+/* Which kernel family a call used (see rib_last_path). */
+enum { RIB_PATH_NONE = 0, RIB_PATH_GENERIC = 1, RIB_PATH_SM100 = 2 };
+
+/*
+ * Forward (Eq. 5, Eq. 6, O = SoftMax(S) V).
+ *   q, k, v, pq, pk : inputs, layouts above.
+ *   out             : bf16 [B][H][W][heads][d], overwritten.
+ *   lse             : fp32 [B][heads][H][W], overwritten; may be NULL when not wanted.
+ */
+int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                        int B, int H, int W, int heads, int d, int r, int window, int shift,
+                        void* out, float* lse, void* stream);
+
+/*
+ * Backward of the same definition (chain rule of Eq. 6 and the softmax), given dout = dL/dout:
+ *   dV = P^T dO;  dP = dO V^T;  dS = P o (dP - rowsum(dO o O));
+ *   dq = dS k / sqrt(d);  dk = dS^T q / sqrt(d);
+ *   dPq = sum over pairs dS Pk / sqrt(r);  dPk = sum over pairs dS^T Pq / sqrt(r).
+ *   out, lse  : the forward results for the same inputs (lse is required here).
+ *   dq, dk, dv: bf16, overwritten.   dpq, dpk: fp32 [n][r], zero-filled by this call on `stream`
+ *               and then accumulated with atomic adds (summation order, hence the last bits, may
+ *               differ from run to run).
+ *   workspace : device scratch of at least rib_window_attn_bwd_workspace(...) bytes, 256-byte
+ *               aligned, owned by the caller; contents are undefined afterwards.  Calls that
+ *               share a workspace must not overlap on the GPU.
+ */
+int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                        const void* out, const float* lse, const void* dout,
+                        int B, int H, int W, int heads, int d, int r, int window, int shift,
+                        void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch rib_window_attn_bwd needs for this shape (0 on an invalid shape). */
+size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window);
+
+/*
+ * Synchronises `stream`, then reads and clears the device status word.  Kernels of this library
+ * never spin without a limit: a wait that runs out records RIB_ERR_DEVICE_WAIT there and the
+ * kernel returns (results of that launch are then invalid).  Returns RIB_OK, RIB_ERR_DEVICE_WAIT
+ * or RIB_ERR_CUDA.
+ */
+int rib_query_status(void* stream);
+
+/* Human-readable name of a status code; never NULL; static storage. */
+const char* rib_status_string(int status);
+
+/*
+ * Debugging knobs, per process.  rib_set_path(RIB_PATH_GENERIC) forces the any-shape kernels,
+ * rib_set_path(RIB_PATH_NONE) restores automatic selection; returns the previous setting.
+ * rib_last_path() tells which family the last successful fwd/bwd call of this thread launched.
+ */
+int rib_set_path(int path);
+int rib_last_path(void);
+
+/* Number of CUDA kernels this library has launched in this process so far (memsets excluded). */
+long long rib_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RIB_WINDOW_ATTN_H */

@@ -1,0 +1,156 @@
+"""Thin Python binding of the C ABI in ``include/rib_window_attn.h``.
+
+Argument marshalling only: torch supplies device memory and the current stream, every step of
+the computation runs in the CUDA kernels of ``librib_window_attn.so``.  There is no CPU or
+PyTorch fallback: if the shared library has not been built, importing this module's functions
+raises ``RibLibraryMissing``.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "librib_window_attn.so"
+_lib = None
+
+RIB_OK = 0
+RIB_PATH_NONE, RIB_PATH_GENERIC, RIB_PATH_SM100 = 0, 1, 2
+
+EXPORTS = (
+    "rib_window_attn_fwd", "rib_window_attn_bwd", "rib_window_attn_bwd_workspace",
+    "rib_query_status", "rib_status_string", "rib_set_path", "rib_last_path", "rib_kernel_launches",
+)
+
+
+class RibLibraryMissing(RuntimeError):
+    pass
+
+
+class RibError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"rib call failed with {code}: {rib_status_string(code)}")
+
+
+def library() -> ctypes.CDLL:
+    """Load (once) the in-tree shared library and declare the C signatures."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RibLibraryMissing(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2603_06738_b200.build`")
+        lib = ctypes.CDLL(str(_LIB_PATH))
+        vp, ci, fp = ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p
+        lib.rib_window_attn_fwd.restype = ci
+        lib.rib_window_attn_fwd.argtypes = [vp] * 5 + [ci] * 8 + [vp, fp, vp]
+        lib.rib_window_attn_bwd.restype = ci
+        lib.rib_window_attn_bwd.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_attn_bwd_workspace.restype = ctypes.c_size_t
+        lib.rib_window_attn_bwd_workspace.argtypes = [ci] * 7
+        lib.rib_query_status.restype = ci
+        lib.rib_query_status.argtypes = [vp]
+        lib.rib_status_string.restype = ctypes.c_char_p
+        lib.rib_status_string.argtypes = [ci]
+        lib.rib_set_path.restype = ci
+        lib.rib_set_path.argtypes = [ci]
+        lib.rib_last_path.restype = ci
+        lib.rib_last_path.argtypes = []
+        lib.rib_kernel_launches.restype = ctypes.c_longlong
+        lib.rib_kernel_launches.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else int(t.data_ptr())
+
+
+def _check_image(name, t, shape=None):
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 5:
+        raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor [B,H,W,heads,d]")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+
+
+def _check_pos(name, t, n):
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 2 or t.shape[0] != n:
+        raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor [n={n}, r]")
+
+
+def rib_status_string(code: int) -> str:
+    return library().rib_status_string(int(code)).decode()
+
+
+def rib_set_path(path: int) -> int:
+    return int(library().rib_set_path(int(path)))
+
+
+def rib_last_path() -> int:
+    return int(library().rib_last_path())
+
+
+def rib_kernel_launches() -> int:
+    return int(library().rib_kernel_launches())
+
+
+def rib_query_status(stream=None) -> int:
+    return int(library().rib_query_status(_stream_ptr(stream)))
+
+
+def rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window) -> int:
+    return int(library().rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window))
+
+
+def rib_window_attn_fwd(q, k, v, pq, pk, window, shift=0, out=None, lse=None, stream=None, want_lse=True):
+    """Enqueue the forward pass; returns (out bf16 [B,H,W,heads,d], lse fp32 [B,heads,H,W] or None)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    _check_image("k", k, q.shape)
+    _check_image("v", v, q.shape)
+    n = window * window
+    _check_pos("pq", pq, n)
+    _check_pos("pk", pk, n)
+    r = pq.shape[1]
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None and want_lse:
+        lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device)
+    rc = library().rib_window_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), B, H, W, heads, d, r,
+                                       window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return out, lse
+
+
+def rib_window_attn_bwd(q, k, v, pq, pk, out, lse, dout, window, shift=0, workspace=None, stream=None):
+    """Enqueue the backward pass; returns (dq, dk, dv bf16, dpq, dpk fp32 [n,r])."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    for name, t in (("k", k), ("v", v), ("out", out), ("dout", dout)):
+        _check_image(name, t, q.shape)
+    n = window * window
+    _check_pos("pq", pq, n)
+    _check_pos("pk", pk, n)
+    r = pq.shape[1]
+    if lse.dtype != torch.float32 or tuple(lse.shape) != (B, heads, H, W) or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous fp32 tensor [B,heads,H,W]")
+    need = rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dpq = torch.empty((n, r), dtype=torch.float32, device=q.device)
+    dpk = torch.empty((n, r), dtype=torch.float32, device=q.device)
+    rc = library().rib_window_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), _ptr(out), _ptr(lse),
+                                       _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq), _ptr(dk),
+                                       _ptr(dv), _ptr(dpq), _ptr(dpk), _ptr(workspace), workspace.numel(),
+                                       _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return dq, dk, dv, dpq, dpk

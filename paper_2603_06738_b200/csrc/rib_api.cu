@@ -1,0 +1,169 @@
+// C ABI of the RIB window-attention library: argument validation, kernel selection, status word.
+// The contract of every entry point is stated in include/rib_window_attn.h.
+#include "../../include/rib_window_attn.h"
+#include "rib_common.cuh"
+
+#include <atomic>
+
+namespace {
+
+__device__ int g_status_word = 0;   // written by bounded device-side waits that ran out
+
+std::atomic<int> g_forced_path{RIB_PATH_NONE};
+thread_local int t_last_path = RIB_PATH_NONE;
+std::atomic<long long> g_kernel_launches{0};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int B, int H, int W, int heads, int d, int r, int window, int shift)
+{
+    if (B <= 0 || H <= 0 || W <= 0 || heads <= 0 || d <= 0 || r < 0 || window <= 0) return RIB_ERR_SHAPE;
+    if (H % window || W % window) return RIB_ERR_SHAPE;
+    if (shift < 0 || shift >= window) return RIB_ERR_SHAPE;
+    if (d > 64 || r > 64 || (d % 8) || (r % 8)) return RIB_ERR_UNSUPPORTED;
+    const long long pairs = (long long)B * (H / window) * (W / window) * heads;
+    if (pairs > 0x7fffffffLL || (long long)window * window > (1 << 20)) return RIB_ERR_SHAPE;
+    return RIB_OK;
+}
+
+int device_status_ptr(int** out)
+{
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_status_word) != cudaSuccess) return RIB_ERR_CUDA;
+    *out = static_cast<int*>(ptr);
+    return RIB_OK;
+}
+
+void fill_shape(rib::Problem& p, int B, int H, int W, int heads, int d, int r, int window, int shift)
+{
+    p.B = B; p.H = H; p.W = W; p.heads = heads; p.d = d; p.r = r; p.M = window; p.s = shift;
+    p.n = window * window; p.nWy = H / window; p.nWx = W / window;
+    p.pairs = B * p.nWy * p.nWx * heads;
+}
+
+size_t rowdot_bytes(int B, int H, int W, int heads)
+{
+    const size_t bytes = sizeof(float) * (size_t)B * H * W * heads;
+    return (bytes + 255) & ~(size_t)255;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                        int B, int H, int W, int heads, int d, int r, int window, int shift,
+                        void* out, float* lse, void* stream)
+{
+    if (!q || !k || !v || !out || (r > 0 && (!pq || !pk))) return RIB_ERR_NULL;
+    if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(pq) ||
+        !aligned16(pk) || !aligned16(lse))
+        return RIB_ERR_ALIGN;
+    rib::Problem p{};
+    fill_shape(p, B, H, W, heads, d, r, window, shift);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.pq = static_cast<const __nv_bfloat16*>(pq);
+    p.pk = static_cast<const __nv_bfloat16*>(pk);
+    p.out_w = static_cast<__nv_bfloat16*>(out);
+    p.lse_w = lse;
+    if (int rc = device_status_ptr(&p.status)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
+    const cudaError_t e = fast ? rib::sm100_fwd(p, st) : rib::generic_fwd(p, st);
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
+size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window)
+{
+    if (check_shape(B, H, W, heads, d, r, window, 0) != RIB_OK) return 0;
+    return rowdot_bytes(B, H, W, heads);
+}
+
+int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                        const void* out, const float* lse, const void* dout,
+                        int B, int H, int W, int heads, int d, int r, int window, int shift,
+                        void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                        void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return RIB_ERR_NULL;
+    if (r > 0 && (!pq || !pk || !dpq || !dpk)) return RIB_ERR_NULL;
+    if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    const void* ptrs[] = {q, k, v, pq, pk, out, lse, dout, dq, dk, dv, dpq, dpk};
+    for (const void* ptr : ptrs)
+        if (!aligned16(ptr)) return RIB_ERR_ALIGN;
+    const size_t need = rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window);
+    if (!workspace || workspace_bytes < need) return RIB_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return RIB_ERR_ALIGN;
+    rib::Problem p{};
+    fill_shape(p, B, H, W, heads, d, r, window, shift);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.pq = static_cast<const __nv_bfloat16*>(pq);
+    p.pk = static_cast<const __nv_bfloat16*>(pk);
+    p.out = static_cast<const __nv_bfloat16*>(out);
+    p.dout = static_cast<const __nv_bfloat16*>(dout);
+    p.lse_in = lse;
+    p.dq = static_cast<__nv_bfloat16*>(dq);
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.dpq = dpq;
+    p.dpk = dpk;
+    p.rowdot = static_cast<float*>(workspace);
+    if (int rc = device_status_ptr(&p.status)) return rc;
+    const cudaError_t e = rib::generic_bwd(p, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    t_last_path = RIB_PATH_GENERIC;
+    g_kernel_launches += 3;   // rowdot, dq, dk/dv
+    return RIB_OK;
+}
+
+int rib_query_status(void* stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    if (cudaMemcpyFromSymbolAsync(&word, g_status_word, sizeof(int), 0, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return RIB_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return RIB_ERR_CUDA;
+    if (word != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbolAsync(g_status_word, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return RIB_ERR_CUDA;
+        return RIB_ERR_DEVICE_WAIT;
+    }
+    return RIB_OK;
+}
+
+const char* rib_status_string(int status)
+{
+    switch (status) {
+        case RIB_OK: return "RIB_OK";
+        case RIB_ERR_NULL: return "RIB_ERR_NULL: a required pointer is NULL";
+        case RIB_ERR_SHAPE: return "RIB_ERR_SHAPE: bad sizes, H/W not a multiple of window, or shift out of range";
+        case RIB_ERR_UNSUPPORTED: return "RIB_ERR_UNSUPPORTED: d or r outside the supported range";
+        case RIB_ERR_ALIGN: return "RIB_ERR_ALIGN: a pointer is not sufficiently aligned";
+        case RIB_ERR_WORKSPACE: return "RIB_ERR_WORKSPACE: workspace missing or too small";
+        case RIB_ERR_CUDA: return "RIB_ERR_CUDA: a CUDA call failed";
+        case RIB_ERR_DEVICE_WAIT: return "RIB_ERR_DEVICE_WAIT: a bounded device-side wait ran out";
+        default: return "unknown RIB status";
+    }
+}
+
+int rib_set_path(int path)
+{
+    if (path != RIB_PATH_NONE && path != RIB_PATH_GENERIC) return g_forced_path.load();
+    return g_forced_path.exchange(path);
+}
+
+int rib_last_path(void) { return t_last_path; }
+
+long long rib_kernel_launches(void) { return g_kernel_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,52 @@
+// Shared declarations of the RIB window-attention CUDA library (internal; the public surface is
+// include/rib_window_attn.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace rib {
+
+// One problem instance.  Image tensors are bf16 [B][H][W][heads][d]; pq/pk bf16 [n][r];
+// lse / rowdot fp32 [B][heads][H][W]; dpq/dpk fp32 [n][r].
+struct Problem {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    const __nv_bfloat16* pq;
+    const __nv_bfloat16* pk;
+    const __nv_bfloat16* out;   // forward result (input of the backward pass)
+    const __nv_bfloat16* dout;
+    const float* lse_in;        // backward
+    __nv_bfloat16* out_w;       // forward output
+    float* lse_w;               // forward output, may be null
+    __nv_bfloat16* dq;
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    float* dpq;
+    float* dpk;
+    float* rowdot;              // workspace: D_i = sum_c dout_ic * out_ic, image layout of lse
+    int B, H, W, heads, d, r, M, s;   // M = window side, s = cyclic shift
+    int n, nWy, nWx, pairs;           // n = M*M, windows per image, B*nWy*nWx*heads
+    int* status;                      // device status word (bounded waits report here)
+};
+
+// Launchers; each returns the cudaError_t of its launches.
+cudaError_t generic_fwd(const Problem& p, cudaStream_t stream);
+cudaError_t generic_bwd(const Problem& p, cudaStream_t stream);
+cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream);
+
+bool sm100_fwd_supported(const Problem& p);
+cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
+
+// Window partition with cyclic shift: token i = y*M + x of window (wy, wx) -> image pixel.
+__host__ __device__ inline void token_pixel(int H, int W, int M, int s, int wy, int wx, int i,
+                                            int& Y, int& X)
+{
+    const int y = i / M, x = i - y * M;
+    Y = wy * M + y + s; if (Y >= H) Y -= H;
+    X = wx * M + x + s; if (X >= W) X -= W;
+}
+
+}  // namespace rib

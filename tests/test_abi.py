@@ -1,0 +1,87 @@
+"""The C-ABI library loads and exports every symbol the header declares; host-side validation
+rejects bad arguments before anything is launched (no GPU needed)."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2603_06738_b200 import binding, build
+
+ROOT = Path(__file__).resolve().parent.parent
+HEADER = (ROOT / "include" / "rib_window_attn.h").read_text()
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.library()
+
+
+def declared_functions():
+    text = re.sub(r"/\*.*?\*/", "", HEADER, flags=re.S)
+    return sorted(set(re.findall(r"\b(rib_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    names = declared_functions()
+    assert set(binding.EXPORTS) <= set(names)
+    assert len(names) >= 7
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in the header but not exported"
+
+
+def test_status_strings(lib):
+    for code in range(-7, 1):
+        s = binding.rib_status_string(code)
+        assert s and "unknown" not in s
+    assert "unknown" in binding.rib_status_string(-99)
+
+
+def fwd_args(**over):
+    a = dict(q=256, k=512, v=768, pq=1024, pk=1280, B=1, H=32, W=32, heads=2, d=32, r=16, window=16,
+             shift=0, out=2048, lse=4096, stream=None)
+    a.update(over)
+    return [a[k] for k in ("q", "k", "v", "pq", "pk", "B", "H", "W", "heads", "d", "r", "window", "shift",
+                           "out", "lse", "stream")]
+
+
+@pytest.mark.parametrize("over,code", [
+    (dict(q=None), -1), (dict(out=None), -1), (dict(pq=None), -1),
+    (dict(H=40), -2), (dict(shift=16), -2), (dict(shift=-1), -2), (dict(B=0), -2), (dict(window=0), -2),
+    (dict(d=128), -3), (dict(r=20), -3), (dict(d=12), -3),
+    (dict(k=516), -4), (dict(lse=4100), -4),
+])
+def test_fwd_rejects_bad_arguments_without_launching(lib, over, code):
+    """Validation order: NULL, shape, support, alignment; fake pointers are never dereferenced."""
+    assert lib.rib_window_attn_fwd(*fwd_args(**over)) == code
+
+
+def test_bwd_rejects_bad_arguments(lib):
+    base = dict(q=256, k=512, v=768, pq=1024, pk=1280, out=1536, lse=1792, dout=2048, B=1, H=32, W=32, heads=2,
+                d=32, r=16, window=16, shift=0, dq=4096, dk=8192, dv=12288, dpq=16384, dpk=20480,
+                ws=65536, ws_bytes=1 << 20, stream=None)
+    order = ("q", "k", "v", "pq", "pk", "out", "lse", "dout", "B", "H", "W", "heads", "d", "r", "window", "shift",
+             "dq", "dk", "dv", "dpq", "dpk", "ws", "ws_bytes", "stream")
+
+    def call(**over):
+        a = dict(base); a.update(over)
+        return lib.rib_window_attn_bwd(*[a[k] for k in order])
+
+    assert call(lse=None) == -1
+    assert call(dpq=None) == -1
+    assert call(W=33) == -2
+    assert call(r=72) == -3
+    assert call(dv=12290) == -4
+    assert call(ws=None) == -5
+    assert call(ws_bytes=16) == -5
+    assert call(ws=65536 + 16) == -4
+    need = lib.rib_window_attn_bwd_workspace(1, 32, 32, 2, 32, 16, 16)
+    assert need >= 4 * 32 * 32 * 2 and need % 256 == 0
+    assert lib.rib_window_attn_bwd_workspace(1, 33, 32, 2, 32, 16, 16) == 0
+
+
+def test_path_knob(lib):
+    assert binding.rib_set_path(binding.RIB_PATH_GENERIC) in (0, 1)
+    assert binding.rib_set_path(binding.RIB_PATH_NONE) == binding.RIB_PATH_GENERIC
+    assert binding.rib_set_path(77) == binding.RIB_PATH_NONE   # invalid value: unchanged

@@ -1,0 +1,136 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Small cases compare every element; the full-size benchmark configurations compare
+sampled pairs (and, for the backward pass, the complete dPq/dPk reduction)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_06738_b200 import binding, synthetic
+from paper_2603_06738_b200.synthetic import CONFIGS, Workload
+
+from parity_util import (compare, make, oracle_bwd, oracle_fwd, run_bwd, run_fwd, sample_pairs, to_f64)
+
+pytestmark = pytest.mark.gpu
+
+# name, B, H, W, heads, d, r, window, shift
+SMALL = [
+    Workload("tiny_2x2", 2, 4, 4, 1, 8, 8, 2, 1, seed=11),
+    Workload("w4_s2", 2, 8, 8, 2, 16, 8, 4, 2, seed=12),
+    Workload("w8_s3_d32", 1, 16, 24, 3, 32, 16, 8, 3, seed=13),
+    Workload("w6_ragged_rows", 1, 12, 18, 2, 24, 24, 6, 5, seed=14),       # n = 36: ragged row tile
+    Workload("w20_ragged_tiles", 1, 40, 40, 2, 32, 16, 20, 7, seed=15),    # n = 400: several tiles + tail
+    Workload("d64_r64", 1, 16, 16, 2, 64, 64, 8, 0, seed=16),
+    Workload("rank0", 1, 16, 16, 2, 32, 0, 8, 4, seed=17),
+    Workload("w16_s8_fast_shape", 2, 32, 48, 2, 32, 16, 16, 8, seed=18),   # fast-path shape, small
+    Workload("w32_s16_fast_shape", 1, 64, 32, 3, 32, 16, 32, 16, seed=19),
+    Workload("w48_s24_fast_shape", 1, 48, 96, 1, 32, 16, 48, 24, seed=20),
+    Workload("w16_odd_shift", 1, 32, 32, 2, 32, 16, 16, 5, seed=21),       # fast shape but odd shift
+]
+
+
+def _inputs_for(wl):
+    if wl.r == 0:
+        cpu = synthetic.make_inputs(Workload(wl.name, wl.B, wl.H, wl.W, wl.heads, wl.d, 8, wl.window, wl.shift, wl.seed), True)
+        cpu["pq"] = cpu["pq"][:, :0].contiguous()
+        cpu["pk"] = cpu["pk"][:, :0].contiguous()
+        return cpu, {k: v.cuda() for k, v in cpu.items()}
+    return make(wl, with_dout=True)
+
+
+@pytest.mark.parametrize("wl", SMALL, ids=lambda w: w.name)
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_small_forward_and_backward_every_element(wl, path):
+    cpu, gpu = _inputs_for(wl)
+    binding.rib_set_path(binding.RIB_PATH_GENERIC if path == "generic" else binding.RIB_PATH_NONE)
+    try:
+        out, lse = run_fwd(gpu, wl)
+        fwd_path = binding.rib_last_path()
+        dq, dk, dv, dpq, dpk = run_bwd(gpu, wl, out, lse)
+    finally:
+        binding.rib_set_path(binding.RIB_PATH_NONE)
+    if path == "generic":
+        assert fwd_path == binding.RIB_PATH_GENERIC
+    ref_out, ref_lse = oracle_fwd(cpu, wl)
+    compare("out", to_f64(out), ref_out)
+    compare("lse", to_f64(lse), ref_lse)
+    rdq, rdk, rdv, rdpq, rdpk = oracle_bwd(cpu, wl)
+    compare("dq", to_f64(dq), rdq)
+    compare("dk", to_f64(dk), rdk)
+    compare("dv", to_f64(dv), rdv)
+    if wl.r:
+        compare("dpq", to_f64(dpq), rdpq)
+        compare("dpk", to_f64(dpk), rdpk)
+
+
+def test_lse_is_optional_and_outputs_are_fully_written():
+    wl = SMALL[2]
+    cpu, gpu = make(wl)
+    out = torch.full_like(gpu["q"], float("nan"))
+    binding.rib_window_attn_fwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift,
+                                out=out, want_lse=False)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    ref_out, _ = oracle_fwd(cpu, wl)
+    compare("out", to_f64(out), ref_out)
+
+
+def test_config1_full_forward():
+    wl = CONFIGS[0]
+    cpu, gpu = make(wl, with_dout=False)
+    out, lse = run_fwd(gpu, wl)
+    ref_out, ref_lse = oracle_fwd(cpu, wl)
+    compare("out", to_f64(out), ref_out)
+    compare("lse", to_f64(lse), ref_lse)
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+def test_full_size_forward_sampled_pairs(idx):
+    """Benchmark configurations 2-4 at full size: sampled pairs against the oracle, all tokens finite."""
+    wl = CONFIGS[idx]
+    cpu, gpu = make(wl, with_dout=False)
+    out, lse = run_fwd(gpu, wl)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+    pairs = sample_pairs(wl, 6, seed=idx)
+    ref_out, ref_lse = oracle_fwd(cpu, wl, pairs=pairs)
+    mask = ~np.isnan(ref_out)
+    assert mask.sum() == len(pairs) * wl.n * wl.d
+    compare("out", to_f64(out), ref_out, mask)
+    compare("lse", to_f64(lse), ref_lse, ~np.isnan(ref_lse))
+
+
+def test_config5_full_forward_backward():
+    """Training configuration at full size: dq/dk/dv on sampled pairs, dPq/dPk over all pairs."""
+    wl = CONFIGS[4]
+    cpu, gpu = make(wl, with_dout=True)
+    out, lse = run_fwd(gpu, wl)
+    dq, dk, dv, dpq, dpk = run_bwd(gpu, wl, out, lse)
+    for t in (out, dq, dk, dv):
+        assert torch.isfinite(t.float()).all()
+    pairs = sample_pairs(wl, 6, seed=5)
+    ref_out, ref_lse = oracle_fwd(cpu, wl, pairs=pairs)
+    mask = ~np.isnan(ref_out)
+    compare("out", to_f64(out), ref_out, mask)
+    compare("lse", to_f64(lse), ref_lse, ~np.isnan(ref_lse))
+    rdq, rdk, rdv, _, _ = oracle_bwd(cpu, wl, pairs=pairs)
+    compare("dq", to_f64(dq), rdq, mask)
+    compare("dk", to_f64(dk), rdk, mask)
+    compare("dv", to_f64(dv), rdv, mask)
+    _, _, _, rdpq, rdpk = oracle_bwd(cpu, wl)
+    # dPq/dPk are sums of pairs*n terms; the absolute bound scales with their magnitude.
+    scale = max(1.0, float(np.abs(rdpq).max()), float(np.abs(rdpk).max()))
+    compare("dpq", to_f64(dpq), rdpq, max_abs=1e-2 * scale)
+    compare("dpk", to_f64(dpk), rdpk, max_abs=1e-2 * scale)
+
+
+def test_outputs_do_not_depend_on_stale_memory():
+    """Two calls in a row on the same buffers give the same bits for out/lse/dq/dk/dv."""
+    wl = SMALL[7]
+    cpu, gpu = make(wl)
+    out1, lse1 = run_fwd(gpu, wl)
+    out2, lse2 = run_fwd(gpu, wl)
+    assert torch.equal(out1, out2) and torch.equal(lse1, lse2)
+    a = run_bwd(gpu, wl, out1, lse1)
+    b = run_bwd(gpu, wl, out1, lse1)
+    for x, y in zip(a[:3], b[:3]):
+        assert torch.equal(x, y)
+    torch.testing.assert_close(a[3], b[3], rtol=1e-4, atol=1e-5)
