@@ -1,6 +1,442 @@
-// Placeholder until the tcgen05 forward kernel lands: no shape is claimed by the fast path.
+// Forward RIB window attention for B200 (sm_100a): tcgen05 MMAs with TMEM accumulators, TMA loads
+// whose box coordinates do the window partition and the cyclic shift, online softmax in registers.
+//
+// Shapes: d = 32, r = 16, window side M a multiple of 16, shift a multiple of 8.
+//
+// Work item = one (batch, window, head) pair x two query tiles of 128 tokens.  A persistent CTA
+// walks items; inside an item it streams the window's keys in blocks of 128:
+//     S_q = Q~_q K~^T   (M128 N128 K48: two K16 steps on the 64-byte content rows, one on the
+//                        32-byte RIB rows -- the concatenation of Eq. 5 exists only as three
+//                        accumulating MMAs on separately staged shared-memory slabs)
+//     P_q = exp2((S_q - m) * log2e / sqrt(d))      softmax warps, fp32 -> bf16 written back to TMEM
+//     O_q += P_q V      (M128 N32 K128, A operand from TMEM, V as an MN-major shared-memory tile)
+// for the two query tiles q = 0, 1, so that one tile's softmax overlaps the other's MMAs.
+//
+// A tile is not 128 consecutive tokens of the window but two 8x8-token patches: attention is
+// equivariant to the order of tokens inside a window, so any enumeration works as long as the
+// Pq/Pk rows and the output rows follow it.  An 8x8 patch never straddles the image border when
+// the shift is a multiple of 8, so one TMA box per patch does partition and shift.
+//
+// Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocator, warps 4-7
+// softmax/epilogue of query tile 0, warps 8-11 of query tile 1.  Every wait is bounded.
 #include "rib_common.cuh"
+#include "sm100_primitives.cuh"
+
+#include <mutex>
+
 namespace rib {
-bool sm100_fwd_supported(const Problem&) { return false; }
-cudaError_t sm100_fwd(const Problem&, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+using namespace sm100;
+
+constexpr int kD = 32, kR = 16;
+constexpr int kTile = 128;            // rows of a query tile / keys of a key block
+constexpr int kStages = 4;            // K/V ring depth
+constexpr int kThreads = 384;
+
+constexpr uint32_t kContentBytes = kTile * kD * 2;   // 8192: 128 rows x 64 B, SWIZZLE_64B
+constexpr uint32_t kPosBytes = kTile * kR * 2;       // 4096: 128 rows x 32 B, SWIZZLE_32B
+constexpr uint32_t kPatchContent = kContentBytes / 2, kPatchPos = kPosBytes / 2;
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t kOffQc = 0;                                        // [2] query content
+constexpr uint32_t kOffQp = kOffQc + 2 * kContentBytes;               // [2] query RIB rows (scaled)
+constexpr uint32_t kOffKc = kOffQp + 2 * kPosBytes;                   // [kStages] key content
+constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStages] key RIB rows
+constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
+constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
+enum Bar { kQFull = 0, kQEmpty, kQPos0, kQPos1, kSFull0, kSFull1, kPReady0, kPReady1, kOFull0, kOFull1, kDrain,
+           kKFull, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
+           kNumBars = kVEmpty + kStages };
+constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
+constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;                 // + slack for manual alignment
+
+// tensor-memory columns (fp32 accumulators; P is bf16x2, two keys per column)
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 320, kTmemCols = 512;
+
+constexpr uint32_t kIdescS = idesc_bf16_f32(kTile, kTile, false);
+constexpr uint32_t kIdescPV = idesc_bf16_f32(kTile, kD, true);
+
+struct FwdParams {
+    const __nv_bfloat16* pq;
+    __nv_bfloat16* out;
+    float* lse;
+    int* status;
+    int H, W, heads, M, s, n, nWy, nWx;
+    int tiles_per_item_pair;   // n / 256: items per pair
+    int items;
+    float scale_log2;          // log2(e) / sqrt(d)
+    float inv_sqrt_d;
+    float pos_scale;           // sqrt(d / r): folds 1/sqrt(r) into the content scale
+};
+
+struct ItemCoord { int b, wy, wx, h, tp; };
+
+__device__ __forceinline__ ItemCoord decode_item(const FwdParams& p, int item)
+{
+    ItemCoord c;
+    c.tp = item % p.tiles_per_item_pair; item /= p.tiles_per_item_pair;
+    c.h = item % p.heads; item /= p.heads;
+    c.wx = item % p.nWx; item /= p.nWx;
+    c.wy = item % p.nWy; item /= p.nWy;
+    c.b = item;
+    return c;
+}
+
+// Patch `sp` of a window (patches of 8x8 tokens, row-major over the window): top-left token in
+// window coordinates and in (shifted, wrapped) image coordinates.
+__device__ __forceinline__ void patch_origin(const FwdParams& p, const ItemCoord& c, int sp, int& py, int& px,
+                                             int& Y0, int& X0)
+{
+    const int per_row = p.M >> 3;
+    py = (sp / per_row) << 3;
+    px = (sp % per_row) << 3;
+    Y0 = c.wy * p.M + py + p.s; if (Y0 >= p.H) Y0 -= p.H;
+    X0 = c.wx * p.M + px + p.s; if (X0 >= p.W) X0 -= p.W;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_pk,
+                     const FwdParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    auto bar = [&](int i) { return base + kOffBar + 8u * i; };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kOffMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + kOffMisc + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nblk = p.n / kTile;
+
+    if (threadIdx.x == 0) {
+        abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
+        mbar_init(bar(kQFull), 1); mbar_init(bar(kQEmpty), 1);
+        mbar_init(bar(kQPos0), 4); mbar_init(bar(kQPos1), 4);
+        mbar_init(bar(kSFull0), 1); mbar_init(bar(kSFull1), 1);
+        mbar_init(bar(kPReady0), 4); mbar_init(bar(kPReady1), 4);
+        mbar_init(bar(kOFull0), 1); mbar_init(bar(kOFull1), 1);
+        mbar_init(bar(kDrain), 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 1);
+            mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 1);
+        }
+        fence_barrier_init();
+        prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_pk);
+    }
+    if (warp == 2) {
+        tmem_alloc(base + kOffMisc, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ============================================================ TMA producer (one thread)
+        if (lane == 0) {
+            uint32_t blk = 0, nitem = 0, q_armed = 0, k_armed = 0, v_armed = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+                const ItemCoord c = decode_item(p, item);
+                if (nitem > 0 && !mbar_wait(bar(kQEmpty), (nitem - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_arrive_expect_tx(bar(kQFull), 2 * kContentBytes);
+                ++q_armed;
+                for (int qt = 0; qt < 2; ++qt)
+                    for (int sub = 0; sub < 2; ++sub) {
+                        int py, px, Y0, X0;
+                        patch_origin(p, c, 2 * (2 * c.tp + qt) + sub, py, px, Y0, X0);
+                        tma_load_5d(base + kOffQc + qt * kContentBytes + sub * kPatchContent, &tm_q, bar(kQFull),
+                                    0, c.h, X0, Y0, c.b);
+                    }
+                for (int j = 0; j < nblk; ++j, ++blk) {
+                    const uint32_t st = blk % kStages, use = blk / kStages;
+                    if (use > 0 && !mbar_wait(bar(kKEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(kKFull + st), kContentBytes + kPosBytes);
+                    ++k_armed;
+                    int py[2], px[2], Y0[2], X0[2];
+                    for (int sub = 0; sub < 2; ++sub) {
+                        patch_origin(p, c, 2 * j + sub, py[sub], px[sub], Y0[sub], X0[sub]);
+                        tma_load_5d(base + kOffKc + st * kContentBytes + sub * kPatchContent, &tm_k, bar(kKFull + st),
+                                    0, c.h, X0[sub], Y0[sub], c.b);
+                        tma_load_3d(base + kOffKp + st * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKFull + st),
+                                    0, px[sub], py[sub]);
+                    }
+                    if (use > 0 && !mbar_wait(bar(kVEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(kVFull + st), kContentBytes);
+                    ++v_armed;
+                    for (int sub = 0; sub < 2; ++sub)
+                        tma_load_5d(base + kOffV + st * kContentBytes + sub * kPatchContent, &tm_v, bar(kVFull + st),
+                                    0, c.h, X0[sub], Y0[sub], c.b);
+                }
+            }
+            if (!ok) {
+                // Gave up: let the copies already in flight land before the CTA may exit.
+                if (q_armed) mbar_wait(bar(kQFull), (q_armed - 1) & 1, abort_flag + 1, p.status);
+                for (uint32_t b2 = k_armed > (uint32_t)kStages ? k_armed - kStages : 0; b2 < k_armed; ++b2)
+                    mbar_wait(bar(kKFull + b2 % kStages), (b2 / kStages) & 1, abort_flag + 1, p.status);
+                for (uint32_t b2 = v_armed > (uint32_t)kStages ? v_armed - kStages : 0; b2 < v_armed; ++b2)
+                    mbar_wait(bar(kVFull + b2 % kStages), (b2 / kStages) & 1, abort_flag + 1, p.status);
+            }
+        }
+    } else if (warp == 1) {
+        // ============================================================== MMA issuer (one thread)
+        if (lane == 0) {
+            uint32_t blk = 0, nitem = 0;
+            bool ok = true;
+            auto issue_s = [&](int qt, uint32_t st) {
+                const uint32_t qc = base + kOffQc + qt * kContentBytes, qp = base + kOffQp + qt * kPosBytes;
+                const uint32_t kc = base + kOffKc + st * kContentBytes, kp = base + kOffKp + st * kPosBytes;
+                const uint32_t d_s = tmem + kColS + qt * kTile;
+                mma_ss(d_s, smem_desc(qc, 16, 512, kSwizzle64B), smem_desc(kc, 16, 512, kSwizzle64B), kIdescS, 0);
+                mma_ss(d_s, smem_desc(qc + 32, 16, 512, kSwizzle64B), smem_desc(kc + 32, 16, 512, kSwizzle64B), kIdescS, 1);
+                mma_ss(d_s, smem_desc(qp, 16, 256, kSwizzle32B), smem_desc(kp, 16, 256, kSwizzle32B), kIdescS, 1);
+            };
+            auto issue_pv = [&](int qt, uint32_t st, uint32_t accumulate) {
+                const uint32_t v = base + kOffV + st * kContentBytes;
+                const uint32_t d_o = tmem + kColO + qt * kD, a_p = tmem + kColP + qt * (kTile / 2);
+                for (int kk = 0; kk < kTile / 16; ++kk)
+                    mma_ts(d_o, a_p + 8 * kk, smem_desc(v + 1024 * kk, 16, 512, kSwizzle64B), kIdescPV,
+                           (accumulate || kk) ? 1u : 0u);
+            };
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+                if (!mbar_wait(bar(kQFull), nitem & 1, abort_flag, p.status) ||
+                    !mbar_wait(bar(kQPos0), nitem & 1, abort_flag, p.status) ||
+                    !mbar_wait(bar(kQPos1), nitem & 1, abort_flag, p.status)) { ok = false; break; }
+                {
+                    const uint32_t st = blk % kStages;
+                    if (!mbar_wait(bar(kKFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_s(0, st); mma_commit(bar(kSFull0));
+                    issue_s(1, st); mma_commit(bar(kSFull1));
+                    mma_commit(bar(kKEmpty + st));
+                }
+                for (int j = 0; j < nblk && ok; ++j, ++blk) {
+                    const uint32_t st = blk % kStages, stn = (blk + 1) % kStages;
+                    if (!mbar_wait(bar(kVFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
+                    for (int qt = 0; qt < 2; ++qt) {
+                        if (!mbar_wait(bar(kPReady0 + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        issue_pv(qt, st, j > 0);
+                        if (j + 1 < nblk) {
+                            if (qt == 0 && !mbar_wait(bar(kKFull + stn), ((blk + 1) / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
+                            tc_fence_after();
+                            issue_s(qt, stn); mma_commit(bar(kSFull0 + qt));
+                            if (qt == 1) mma_commit(bar(kKEmpty + stn));
+                        } else {
+                            mma_commit(bar(kOFull0 + qt));
+                        }
+                    }
+                    if (ok) mma_commit(bar(kVEmpty + st));
+                }
+                if (ok) mma_commit(bar(kQEmpty));
+            }
+            // everything issued by this thread must have finished before TMEM is released
+            mma_commit(bar(kDrain));
+            mbar_wait(bar(kDrain), 0, abort_flag + 1, p.status);
+        }
+    } else if (warp >= 4) {
+        // ========================================== softmax + epilogue, one thread per query row
+        const int qt = (warp - 4) >> 2;
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;                 // row of the tile == TMEM lane
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + kColS + qt * kTile;
+        const uint32_t t_o = tmem + lane_base + kColO + qt * kD;
+        const uint32_t t_p = tmem + lane_base + kColP + qt * (kTile / 2);
+        const float rescale_threshold = 8.0f / p.scale_log2;    // raw-logit units: p stays <= 2^8
+        uint32_t blk = 0, nitem = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+            const ItemCoord c = decode_item(p, item);
+            int py, px, Y0, X0;
+            patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+            const int ty = (row >> 3) & 7, tx = row & 7;
+            const int token = (py + ty) * p.M + (px + tx);       // row of Pq that belongs to this query
+            // -- stage this row of the query RIB slab: bf16(Pq * sqrt(d/r)), SWIZZLE_32B K-major
+            {
+                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)token * kR);
+                uint4 v[2] = {__ldg(src), __ldg(src + 1)};
+                uint32_t* w = reinterpret_cast<uint32_t*>(v);
+                for (int i = 0; i < 8; ++i) {
+                    const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
+                    const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
+                    w[i] = pack_bf16x2(lo, hi);
+                }
+                uint8_t* dst = base_ptr + kOffQp + qt * kPosBytes + row * 32;
+                const int sw = (row >> 2) & 1;
+                *reinterpret_cast<uint4*>(dst + ((0 ^ sw) << 4)) = v[0];
+                *reinterpret_cast<uint4*>(dst + ((1 ^ sw) << 4)) = v[1];
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kQPos0 + qt));
+            }
+            float m_used = -INFINITY, l = 0.f;
+            for (int j = 0; j < nblk; ++j, ++blk) {
+                // warp-uniform outcome: the TMEM loads below are warp-collective
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull0 + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
+                tc_fence_after();
+                uint32_t s[4][32];
+                tmem_ld32(t_s, s[0]); tmem_ld32(t_s + 32, s[1]); tmem_ld32(t_s + 64, s[2]); tmem_ld32(t_s + 96, s[3]);
+                tmem_wait_ld();
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[0][i])); mx1 = fmaxf(mx1, __uint_as_float(s[1][i]));
+                    mx2 = fmaxf(mx2, __uint_as_float(s[2][i])); mx3 = fmaxf(mx3, __uint_as_float(s[3][i]));
+                }
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                if (j == 0) {
+                    m_used = mx;
+                } else {
+                    // Rescale O only when the maximum grew by more than the threshold; the result is
+                    // exact after the final normalisation because l carries the same reference.
+                    const bool need = mx > m_used + rescale_threshold;
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
+                        if (need) { l *= factor; m_used = mx; }
+                        uint32_t o[32];
+                        tmem_ld32(t_o, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                        tmem_st32(t_o, o);
+                        tmem_wait_st();
+                    }
+                }
+                const float neg_ms = -m_used * p.scale_log2;
+                float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[ch][2 * i]), p.scale_log2, neg_ms));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[ch][2 * i + 1]), p.scale_log2, neg_ms));
+                        if (i & 1) { sum2 += p0; sum3 += p1; } else { sum0 += p0; sum1 += p1; }
+                        packed[i] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(t_p + 16 * ch, packed);
+                }
+                l += (sum0 + sum1) + (sum2 + sum3);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kPReady0 + qt));
+            }
+            if (!ok) break;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kOFull0 + qt), nitem & 1, abort_flag, p.status))) { ok = false; break; }
+            tc_fence_after();
+            uint32_t o[32];
+            tmem_ld32(t_o, o);
+            tmem_wait_ld();
+            tc_fence_before();
+            const float inv_l = 1.f / l;
+            int Y = Y0 + ty, X = X0 + tx;        // the patch does not straddle the border
+            const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
+            uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 v;
+                v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
+                v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
+                v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
+                v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
+                dst[i] = v;
+            }
+            if (p.lse)
+                p.lse[(((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X] = m_used * p.inv_sqrt_d + logf(l);
+        }
+    }
+    // ================================================================================ common tail
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------- host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+// bf16 [B][H][W][heads][32] image tensor, box = one 8x8-token patch of one head.
+bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p)
+{
+    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)p.heads, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+    const cuuint64_t row = (cuuint64_t)kD * 2;
+    const cuuint64_t strides[4] = {row, row * p.heads, row * p.heads * p.W, row * p.heads * p.W * p.H};
+    const cuuint32_t box[5] = {(cuuint32_t)kD, 1, 8, 8, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// bf16 [M][M][16] positional features, box = one 8x8-token patch.
+bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M};
+    const cuuint64_t strides[2] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M};
+    const cuuint32_t box[3] = {(cuuint32_t)kR, 8, 8};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool sm100_fwd_supported(const Problem& p)
+{
+    return p.d == kD && p.r == kR && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
+}
+
+cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
+{
+    if (!encode_fn()) return cudaErrorNotSupported;
+    CUtensorMap tm_q, tm_k, tm_v, tm_pk;
+    if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
+        !encode_pos_map(&tm_pk, p.pk, p))
+        return cudaErrorInvalidValue;
+    static int sm_count = 0;
+    if (!sm_count) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(rib_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) { sm_count = 0; return e; }
+    }
+    FwdParams fp{};
+    fp.pq = p.pq; fp.out = p.out_w; fp.lse = p.lse_w; fp.status = p.status;
+    fp.H = p.H; fp.W = p.W; fp.heads = p.heads; fp.M = p.M; fp.s = p.s; fp.n = p.n; fp.nWy = p.nWy; fp.nWx = p.nWx;
+    fp.tiles_per_item_pair = p.n / (2 * kTile);
+    fp.items = p.pairs * fp.tiles_per_item_pair;
+    fp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
+    fp.inv_sqrt_d = 1.f / sqrtf((float)p.d);
+    fp.pos_scale = sqrtf((float)p.d / (float)p.r);
+    const int grid = fp.items < sm_count ? fp.items : sm_count;
+    rib_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp);
+    return cudaGetLastError();
+}
+
 }  // namespace rib

@@ -122,6 +122,34 @@ def test_config5_full_forward_backward():
     compare("dpk", to_f64(dpk), rdpk, max_abs=1e-2 * scale)
 
 
+@pytest.mark.parametrize("direction", ["growing", "shrinking"])
+def test_running_maximum_rescale(direction):
+    """Logits that grow (or shrink) steeply along the key order force the online-softmax rescale
+    of the accumulated output in later key blocks."""
+    wl = Workload("w32_rescale", 1, 32, 64, 2, 32, 16, 32, 0, seed=31)
+    cpu, gpu = make(wl, with_dout=False)
+    ramp = torch.linspace(0.2, 6.0, wl.H).view(1, wl.H, 1, 1, 1)
+    if direction == "shrinking":
+        ramp = ramp.flip(1)
+    cpu["k"] = (cpu["k"].float() * ramp).to(torch.bfloat16)      # |k| grows with the row of the window
+    cpu["q"] = (cpu["q"].float() * 2.0).to(torch.bfloat16)
+    gpu = {k: v.cuda() for k, v in cpu.items()}
+    out, lse = run_fwd(gpu, wl)
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    ref_out, ref_lse = oracle_fwd(cpu, wl)
+    assert np.abs(ref_lse).max() > 20          # the case really has large logits
+    compare("out", to_f64(out), ref_out, max_abs=2e-2)
+    compare("lse", to_f64(lse), ref_lse, max_abs=2e-2, rel_l2=5e-3)
+
+
+def test_fast_path_is_taken_for_benchmark_shapes():
+    for wl in CONFIGS:
+        small = Workload(wl.name, 1, wl.window, wl.window, 1, wl.d, wl.r, wl.window, wl.shift, seed=1)
+        cpu, gpu = make(small, with_dout=False)
+        run_fwd(gpu, small)
+        assert binding.rib_last_path() == binding.RIB_PATH_SM100, wl.name
+
+
 def test_outputs_do_not_depend_on_stale_memory():
     """Two calls in a row on the same buffers give the same bits for out/lse/dq/dk/dv."""
     wl = SMALL[7]
