@@ -82,7 +82,14 @@ int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void*
 size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window)
 {
     if (check_shape(B, H, W, heads, d, r, window, 0) != RIB_OK) return 0;
-    return rowdot_bytes(B, H, W, heads);
+    size_t need = rowdot_bytes(B, H, W, heads);
+    rib::Problem p{};
+    fill_shape(p, B, H, W, heads, d, r, window, 0);
+    if (rib::sm100_bwd_supported(p)) {   // whatever the shift: one size per shape
+        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n);
+        if (fast > need) need = fast;
+    }
+    return need;
 }
 
 int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void* pq, const void* pk,
@@ -116,11 +123,15 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
     p.dpq = dpq;
     p.dpk = dpk;
     p.rowdot = static_cast<float*>(workspace);
+    p.workspace = workspace;
+    p.workspace_bytes = workspace_bytes;
     if (int rc = device_status_ptr(&p.status)) return rc;
-    const cudaError_t e = rib::generic_bwd(p, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_bwd_supported(p);
+    const cudaError_t e = fast ? rib::sm100_bwd(p, st) : rib::generic_bwd(p, st);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
-    t_last_path = RIB_PATH_GENERIC;
-    g_kernel_launches += 3;   // rowdot, dq, dk/dv
+    t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
+    g_kernel_launches += fast ? 4 : 3;   // prepare, main, two finishing kernels : rowdot, dq, dk/dv
     return RIB_OK;
 }
 

@@ -1,0 +1,569 @@
+// Backward RIB window attention for B200 (sm_100a): the chain rule of Eq. 6 and the softmax as five
+// tcgen05 contractions per (query tile, key block) with TMEM accumulators and TMA loads.
+//
+// Shapes: d = 32, r = 16, window side M a multiple of 16, shift a multiple of 8 (as the forward).
+//
+// Work item = one (batch, window, head) pair x one key block J of 128 tokens.  A persistent CTA keeps
+// K~_J = [k, Pk] and V_J in shared memory and dV_J, dK~_J in tensor memory, and walks the query tiles
+// I of the window.  Everything is computed transposed (keys on the TMEM lanes) so that P^T and dS^T
+// feed the dV and dK~ contractions straight from tensor memory:
+//     S^T  = K~_J Q~_I^T                    (M128 N128 K48: content rows 2 x K16, RIB rows 1 x K16)
+//     dP^T = V_J dO_I^T                     (M128 N128 K32)
+//     P^T  = exp2(S^T * log2e/sqrt(d) - lse_i * log2e),   dS^T = P^T o (dP^T - D_i)     (ALU warps)
+//     dV_J  += P^T  dO_I                    (A from TMEM, B = dO tile, MN-major)
+//     dK~_J += dS^T Q~_I                    (A from TMEM, B = Q content / RIB slabs, MN-major)
+//     dQ~_I  = dS K~_J                      (A = dS through shared memory, MN-major, B = K~ slabs)
+// dQ~_I is one key block's share of the query gradient: it is added (fp32 red) into a workspace laid
+// out [pair][column][token in window order] and finished by a small kernel that converts dq to
+// bf16 and sums the RIB columns over pairs into dPq.  The RIB columns of dK~ are written per pair
+// and summed over pairs by the same finishing kernel into dPk.
+//
+// Roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocator, warps 4-11
+// P/dS arithmetic (two warpgroups, each half of the tile's columns), warps 12-15 drain dQ~ after every
+// tile and dK~/dV after every item.  Every wait is bounded.
+#include "rib_sm100_common.cuh"
+
+namespace rib {
+namespace {
+
+using namespace sm100;
+
+constexpr int kQStages = 3;           // ring of query-side tiles (Q content, Q RIB rows, dO, lse/D)
+constexpr int kThreads = 512;
+constexpr int kDk = kD + kR;          // 48 columns of dQ~ / dK~
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t kOffKc = 0;                                   // [2] key content (one slot per item in flight)
+constexpr uint32_t kOffKp = kOffKc + 2 * kContentBytes;          // [2] key RIB rows
+constexpr uint32_t kOffV = kOffKp + 2 * kPosBytes;               // [2] values
+constexpr uint32_t kOffRing = kOffV + 2 * kContentBytes;
+constexpr uint32_t kLdBytes = kTile * 8;                         // 128 x (-lse*log2e, D)
+constexpr uint32_t kRingQc = 0, kRingQp = kContentBytes, kRingDO = kRingQp + kPosBytes, kRingLD = kRingDO + kContentBytes;
+constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 21504
+constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
+constexpr uint32_t kDSHalf = kTile * 128;
+constexpr uint32_t kOffBar = kOffDS + 2 * kDSHalf;
+enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kPReady,
+           kPFree, kDQFull, kDQFree, kAccFull, kAccFree, kDrain, kNumBars };
+constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;
+constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
+static_assert(kOffRing % 1024 == 0 && kRingBytes % 1024 == 0 && kOffDS % 1024 == 0, "swizzle atoms need aligned tiles");
+
+// tensor-memory columns
+constexpr uint32_t kColS = 0, kColDP = 128, kColP = 256, kColDS = 320, kColDV = 384, kColDK = 416, kColDQ = 464;
+constexpr uint32_t kTmemCols = 512;
+
+constexpr uint32_t kIdescSS = idesc_bf16_f32(kTile, kTile, false);            // S^T, dP^T: both operands K-major
+constexpr uint32_t kIdescT32 = idesc_bf16_f32(kTile, kD, true);               // A in TMEM, B MN-major, N = 32
+constexpr uint32_t kIdescT16 = idesc_bf16_f32(kTile, kR, true);               // A in TMEM, B MN-major, N = 16
+constexpr uint32_t kIdescQ32 = idesc_bf16_f32_ab(kTile, kD, true, true);      // dQ~: A and B MN-major
+constexpr uint32_t kIdescQ16 = idesc_bf16_f32_ab(kTile, kR, true, true);
+
+struct BwdParams {
+    const float2* ld;          // [pairs][n] window order: (-lse * log2e, D)
+    float* dq_acc;             // [pairs][48][n] fp32, zeroed by the preparation kernel
+    float* dkp;                // [pairs][16][n] fp32, RIB columns of dK~ (already times 1/sqrt d)
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    int* status;
+    int H, W, heads, M, s, n, nWy, nWx, nblk, items;
+    float scale_log2;          // log2(e) / sqrt(d)
+    float inv_sqrt_d;
+};
+
+struct ItemCoord { int pair, b, wy, wx, h, J; };
+
+__device__ __forceinline__ ItemCoord decode_item(const BwdParams& p, int item)
+{
+    ItemCoord c;
+    c.J = item % p.nblk; item /= p.nblk;
+    c.pair = item;
+    c.h = item % p.heads; item /= p.heads;
+    c.wx = item % p.nWx; item /= p.nWx;
+    c.wy = item % p.nWy; item /= p.nWy;
+    c.b = item;
+    return c;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                     const __grid_constant__ CUtensorMap tm_pqs, const __grid_constant__ CUtensorMap tm_pk,
+                     const BwdParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    auto bar = [&](int i) { return base + kOffBar + 8u * i; };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kOffMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + kOffMisc + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const WindowGeom geom{p.H, p.W, p.M, p.s};
+
+    if (threadIdx.x == 0) {
+        abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
+        for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
+        for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
+        mbar_init(bar(kSFull), 1); mbar_init(bar(kPReady), 8); mbar_init(bar(kPFree), 1);
+        mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
+        mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
+        mbar_init(bar(kDrain), 1);
+        fence_barrier_init();
+        prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+        prefetch_tensormap(&tm_do); prefetch_tensormap(&tm_pqs); prefetch_tensormap(&tm_pk);
+    }
+    if (warp == 2) {
+        tmem_alloc(base + kOffMisc, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ============================================================ TMA producer (one thread)
+        if (lane == 0) {
+            uint32_t g = 0, nitem = 0, kv_armed = 0, q_armed = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+                const ItemCoord c = decode_item(p, item);
+                const uint32_t slot = nitem & 1;
+                if (nitem >= 2 && !mbar_wait(bar(kKVEmpty + slot), ((nitem >> 1) - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_arrive_expect_tx(bar(kKVFull + slot), 2 * kContentBytes + kPosBytes);
+                ++kv_armed;
+                for (int sub = 0; sub < 2; ++sub) {
+                    int py, px, Y0, X0;
+                    patch_origin(geom, c.wy, c.wx, 2 * c.J + sub, py, px, Y0, X0);
+                    tma_load_5d(base + kOffKc + slot * kContentBytes + sub * kPatchContent, &tm_k, bar(kKVFull + slot),
+                                0, c.h, X0, Y0, c.b);
+                    tma_load_3d(base + kOffKp + slot * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKVFull + slot), 0, px, py);
+                    tma_load_5d(base + kOffV + slot * kContentBytes + sub * kPatchContent, &tm_v, bar(kKVFull + slot),
+                                0, c.h, X0, Y0, c.b);
+                }
+                for (int I = 0; I < p.nblk; ++I, ++g) {
+                    const uint32_t st = g % kQStages, use = g / kQStages;
+                    if (use > 0 && !mbar_wait(bar(kQEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(kQFull + st), kRingBytes);
+                    ++q_armed;
+                    const uint32_t ring = base + kOffRing + st * kRingBytes;
+                    for (int sub = 0; sub < 2; ++sub) {
+                        int py, px, Y0, X0;
+                        patch_origin(geom, c.wy, c.wx, 2 * I + sub, py, px, Y0, X0);
+                        tma_load_5d(ring + kRingQc + sub * kPatchContent, &tm_q, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
+                        tma_load_3d(ring + kRingQp + sub * kPatchPos, &tm_pqs, bar(kQFull + st), 0, px, py);
+                        tma_load_5d(ring + kRingDO + sub * kPatchContent, &tm_do, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
+                    }
+                    bulk_load_1d(ring + kRingLD, p.ld + (size_t)c.pair * p.n + (size_t)I * kTile, kLdBytes, bar(kQFull + st));
+                }
+            }
+            if (!ok) {
+                // Gave up: let the copies already in flight land before the CTA may exit.
+                for (uint32_t b2 = kv_armed > 2u ? kv_armed - 2 : 0; b2 < kv_armed; ++b2)
+                    mbar_wait(bar(kKVFull + (b2 & 1)), (b2 >> 1) & 1, abort_flag + 1, p.status);
+                for (uint32_t b2 = q_armed > (uint32_t)kQStages ? q_armed - kQStages : 0; b2 < q_armed; ++b2)
+                    mbar_wait(bar(kQFull + b2 % kQStages), (b2 / kQStages) & 1, abort_flag + 1, p.status);
+            }
+        }
+    } else if (warp == 1) {
+        // ============================================================== MMA issuer (one thread)
+        if (lane == 0) {
+            // S^T and dP^T of one tile: key slot `slot`, ring stage `st`
+            auto issue_scores = [&](uint32_t slot, uint32_t st) {
+                const uint32_t kc = base + kOffKc + slot * kContentBytes, kp = base + kOffKp + slot * kPosBytes;
+                const uint32_t v = base + kOffV + slot * kContentBytes;
+                const uint32_t ring = base + kOffRing + st * kRingBytes;
+                const uint32_t qc = ring + kRingQc, qp = ring + kRingQp, go = ring + kRingDO;
+                mma_ss(tmem + kColS, smem_desc(kc, 16, 512, kSwizzle64B), smem_desc(qc, 16, 512, kSwizzle64B), kIdescSS, 0);
+                mma_ss(tmem + kColS, smem_desc(kc + 32, 16, 512, kSwizzle64B), smem_desc(qc + 32, 16, 512, kSwizzle64B), kIdescSS, 1);
+                mma_ss(tmem + kColS, smem_desc(kp, 16, 256, kSwizzle32B), smem_desc(qp, 16, 256, kSwizzle32B), kIdescSS, 1);
+                mma_ss(tmem + kColDP, smem_desc(v, 16, 512, kSwizzle64B), smem_desc(go, 16, 512, kSwizzle64B), kIdescSS, 0);
+                mma_ss(tmem + kColDP, smem_desc(v + 32, 16, 512, kSwizzle64B), smem_desc(go + 32, 16, 512, kSwizzle64B), kIdescSS, 1);
+            };
+            // dV_J, dK~_J (accumulating over the item) and dQ~_I (fresh every tile)
+            auto issue_grads = [&](uint32_t slot, uint32_t st, bool accumulate) {
+                const uint32_t kc = base + kOffKc + slot * kContentBytes, kp = base + kOffKp + slot * kPosBytes;
+                const uint32_t ring = base + kOffRing + st * kRingBytes;
+                const uint32_t qc = ring + kRingQc, qp = ring + kRingQp, go = ring + kRingDO;
+                const uint32_t ds = base + kOffDS;
+                for (int kk = 0; kk < kTile / 16; ++kk)      // K = 16 queries per step
+                    mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, smem_desc(go + 1024 * kk, 16, 512, kSwizzle64B),
+                           kIdescT32, (accumulate || kk) ? 1u : 0u);
+                for (int kk = 0; kk < kTile / 16; ++kk) {
+                    mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, smem_desc(qc + 1024 * kk, 16, 512, kSwizzle64B),
+                           kIdescT32, (accumulate || kk) ? 1u : 0u);
+                    mma_ts(tmem + kColDK + kD, tmem + kColDS + 8 * kk, smem_desc(qp + 512 * kk, 16, 256, kSwizzle32B),
+                           kIdescT16, (accumulate || kk) ? 1u : 0u);
+                }
+                for (int kk = 0; kk < kTile / 16; ++kk) {    // K = 16 keys per step
+                    const uint64_t a = smem_desc(ds + 2048 * kk, kDSHalf, 1024, kSwizzle128B);
+                    mma_ss(tmem + kColDQ, a, smem_desc(kc + 1024 * kk, 16, 512, kSwizzle64B), kIdescQ32, kk ? 1u : 0u);
+                    mma_ss(tmem + kColDQ + kD, a, smem_desc(kp + 512 * kk, 16, 256, kSwizzle32B), kIdescQ16, kk ? 1u : 0u);
+                }
+            };
+            int item = blockIdx.x, I = 0;
+            uint32_t nitem = 0, g = 0;
+            bool valid = item < p.items, ok = true;
+            if (valid) {
+                ok = mbar_wait(bar(kKVFull), 0, abort_flag, p.status) && mbar_wait(bar(kQFull), 0, abort_flag, p.status);
+                if (ok) {
+                    tc_fence_after();
+                    issue_scores(0, 0);
+                    mma_commit(bar(kSFull));
+                }
+            }
+            while (valid && ok) {
+                int item2 = item, I2 = I + 1;
+                uint32_t nitem2 = nitem;
+                if (I2 == p.nblk) { I2 = 0; item2 += gridDim.x; ++nitem2; }
+                const bool valid2 = item2 < p.items;
+                const uint32_t slot = nitem & 1, st = g % kQStages;
+                if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                if (valid2) {
+                    // next tile's S^T, dP^T first: the arithmetic warps start on them while the
+                    // three gradient contractions of this tile run
+                    const uint32_t st2 = (g + 1) % kQStages;
+                    if (I2 == 0 && !mbar_wait(bar(kKVFull + (nitem2 & 1)), (nitem2 >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    if (!mbar_wait(bar(kQFull + st2), ((g + 1) / kQStages) & 1, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_scores(nitem2 & 1, st2);
+                    mma_commit(bar(kSFull));
+                }
+                if (I == 0 && nitem > 0 && !mbar_wait(bar(kAccFree), (nitem - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                if (g > 0 && !mbar_wait(bar(kDQFree), (g - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                issue_grads(slot, st, I > 0);
+                mma_commit(bar(kPFree));
+                mma_commit(bar(kDQFull));
+                mma_commit(bar(kQEmpty + st));
+                if (I == p.nblk - 1) {
+                    mma_commit(bar(kAccFull));
+                    mma_commit(bar(kKVEmpty + slot));
+                }
+                item = item2; I = I2; nitem = nitem2; valid = valid2; ++g;
+            }
+            // everything issued by this thread must have finished before TMEM is released
+            mma_commit(bar(kDrain));
+            mbar_wait(bar(kDrain), 0, abort_flag + 1, p.status);
+        }
+    } else if (warp >= 4 && warp < 12) {
+        // ===================== P^T and dS^T: one thread per key row, one warpgroup per 64 queries
+        const int half = (warp - 4) >> 2;
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;                 // key row of the block == TMEM lane
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        uint8_t* ds_row = base_ptr + kOffDS + half * kDSHalf + row * 128;
+        const int sw = row & 7;
+        uint32_t g = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
+            for (int I = 0; I < p.nblk; ++I, ++g) {
+                const uint32_t st = g % kQStages;
+                // warp-uniform outcome: the TMEM accesses below are warp-collective
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) &&
+                                                 mbar_wait(bar(kSFull), g & 1, abort_flag, p.status))) { ok = false; break; }
+                tc_fence_after();
+                const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD);
+                bool may_store = g == 0;
+#pragma unroll
+                for (int ch = 0; ch < 2; ++ch) {
+                    const int col0 = half * 64 + ch * 32;
+                    uint32_t s[32], dp[32];
+                    tmem_ld32(tmem + lane_base + kColS + col0, s);
+                    tmem_ld32(tmem + lane_base + kColDP + col0, dp);
+                    tmem_wait_ld();
+                    uint32_t pp[16], dd[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float4 t = ld[(col0 >> 1) + i];   // (-lse2, D) of queries col0 + 2i, col0 + 2i + 1
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, t.x));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, t.z));
+                        const float d0 = p0 * (__uint_as_float(dp[2 * i]) - t.y);
+                        const float d1 = p1 * (__uint_as_float(dp[2 * i + 1]) - t.w);
+                        pp[i] = pack_bf16x2(p0, p1);
+                        dd[i] = pack_bf16x2(d0, d1);
+                    }
+                    if (!may_store) {
+                        // the previous tile's contractions still read P^T, dS^T and the dS tile
+                        if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+                        may_store = true;
+                    }
+                    tmem_st16(tmem + lane_base + kColP + (col0 >> 1), pp);
+                    tmem_st16(tmem + lane_base + kColDS + (col0 >> 1), dd);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const int chunk = ch * 4 + q4;
+                        *reinterpret_cast<uint4*>(ds_row + ((chunk ^ sw) << 4)) =
+                            make_uint4(dd[4 * q4], dd[4 * q4 + 1], dd[4 * q4 + 2], dd[4 * q4 + 3]);
+                    }
+                }
+                if (!ok) break;
+                tmem_wait_st();
+                tc_fence_before();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kPReady));
+            }
+        }
+    } else if (warp >= 12) {
+        // ================================ drains: dQ~ after every tile, dV / dK~ after every item
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        uint32_t g = 0, nitem = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+            const ItemCoord c = decode_item(p, item);
+            for (int I = 0; I < p.nblk; ++I, ++g) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kDQFull), g & 1, abort_flag, p.status))) { ok = false; break; }
+                tc_fence_after();
+                uint32_t a[32], b[16];
+                tmem_ld32(tmem + lane_base + kColDQ, a);
+                tmem_ld16(tmem + lane_base + kColDQ + kD, b);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kDQFree));
+                float* dst = p.dq_acc + (size_t)c.pair * kDk * p.n + (size_t)I * kTile + row;
+#pragma unroll
+                for (int col = 0; col < kD; ++col) red_add_f32(dst + (size_t)col * p.n, __uint_as_float(a[col]));
+#pragma unroll
+                for (int col = 0; col < kR; ++col) red_add_f32(dst + (size_t)(kD + col) * p.n, __uint_as_float(b[col]));
+            }
+            if (!ok) break;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kAccFull), nitem & 1, abort_flag, p.status))) { ok = false; break; }
+            tc_fence_after();
+            uint32_t dv[32], dk[32], dkp[16];
+            tmem_ld32(tmem + lane_base + kColDV, dv);
+            tmem_ld32(tmem + lane_base + kColDK, dk);
+            tmem_ld16(tmem + lane_base + kColDK + kD, dkp);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kAccFree));
+            int i, Y, X;
+            window_order_token(geom, c.wy, c.wx, c.J * kTile + row, i, Y, X);
+            const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
+            uint4* dst_v = reinterpret_cast<uint4*>(p.dv + tok * kD);
+            uint4* dst_k = reinterpret_cast<uint4*>(p.dk + tok * kD);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint4 o;
+                o.x = pack_bf16x2(__uint_as_float(dv[8 * q4 + 0]), __uint_as_float(dv[8 * q4 + 1]));
+                o.y = pack_bf16x2(__uint_as_float(dv[8 * q4 + 2]), __uint_as_float(dv[8 * q4 + 3]));
+                o.z = pack_bf16x2(__uint_as_float(dv[8 * q4 + 4]), __uint_as_float(dv[8 * q4 + 5]));
+                o.w = pack_bf16x2(__uint_as_float(dv[8 * q4 + 6]), __uint_as_float(dv[8 * q4 + 7]));
+                dst_v[q4] = o;
+                o.x = pack_bf16x2(__uint_as_float(dk[8 * q4 + 0]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 1]) * p.inv_sqrt_d);
+                o.y = pack_bf16x2(__uint_as_float(dk[8 * q4 + 2]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 3]) * p.inv_sqrt_d);
+                o.z = pack_bf16x2(__uint_as_float(dk[8 * q4 + 4]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 5]) * p.inv_sqrt_d);
+                o.w = pack_bf16x2(__uint_as_float(dk[8 * q4 + 6]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 7]) * p.inv_sqrt_d);
+                dst_k[q4] = o;
+            }
+            float* dst_p = p.dkp + (size_t)c.pair * kR * p.n + (size_t)c.J * kTile + row;
+#pragma unroll
+            for (int col = 0; col < kR; ++col) dst_p[(size_t)col * p.n] = __uint_as_float(dkp[col]) * p.inv_sqrt_d;
+        }
+    }
+    // ================================================================================ common tail
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------ preparation and finishing
+struct AuxParams {
+    const __nv_bfloat16* out;
+    const __nv_bfloat16* dout;
+    const __nv_bfloat16* pq;
+    const float* lse;
+    float2* ld;
+    float* dq_acc;
+    const float* dkp;
+    __nv_bfloat16* pq_scaled;
+    __nv_bfloat16* dq;
+    float* dpq;
+    float* dpk;
+    int H, W, heads, M, s, n, nWy, nWx, pairs;
+    float pos_scale, inv_sqrt_d, inv_sqrt_r;
+};
+
+__device__ __forceinline__ void decode_pair_token(const AuxParams& p, int pair, int w, int& i, size_t& tok, size_t& scalar)
+{
+    const int h = pair % p.heads; pair /= p.heads;
+    const int wx = pair % p.nWx; pair /= p.nWx;
+    const int wy = pair % p.nWy; pair /= p.nWy;
+    const int b = pair;
+    int Y, X;
+    window_order_token(WindowGeom{p.H, p.W, p.M, p.s}, wy, wx, w, i, Y, X);
+    tok = (((size_t)b * p.H + Y) * p.W + X) * p.heads + h;
+    scalar = (((size_t)b * p.heads + h) * p.H + Y) * p.W + X;
+}
+
+// One thread per (pair, token in window order): D = dO . O and lse in the layout the main kernel
+// streams, zero of this token's dQ~ accumulators; the first threads also stage bf16(Pq sqrt(d/r))
+// and clear dPq, dPk.
+__global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
+{
+    const size_t total = (size_t)p.pairs * p.n;
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+    for (size_t e = t; e < (size_t)p.n * kR; e += nthreads) {
+        p.pq_scaled[e] = __float2bfloat16_rn(__bfloat162float(p.pq[e]) * p.pos_scale);
+        p.dpq[e] = 0.f;
+        p.dpk[e] = 0.f;
+    }
+    if (t >= total) return;
+    const int pair = (int)(t / p.n), w = (int)(t % p.n);
+    int i; size_t tok, scalar;
+    decode_pair_token(p, pair, w, i, tok, scalar);
+    const uint4* a = reinterpret_cast<const uint4*>(p.dout + tok * kD);
+    const uint4* b = reinterpret_cast<const uint4*>(p.out + tok * kD);
+    float acc = 0.f;
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+        const uint4 x = __ldg(a + q4), y = __ldg(b + q4);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc = fmaf(__uint_as_float(xs[k] << 16), __uint_as_float(ys[k] << 16), acc);
+            acc = fmaf(__uint_as_float(xs[k] & 0xffff0000u), __uint_as_float(ys[k] & 0xffff0000u), acc);
+        }
+    }
+    p.ld[t] = make_float2(-p.lse[scalar] * 1.4426950408889634f, acc);
+    float* z = p.dq_acc + (size_t)pair * kDk * p.n + w;
+#pragma unroll 8
+    for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
+}
+
+// One thread per (pair, token): dq = dQ~[:, :d] / sqrt(d) as bf16 at the token's pixel.
+__global__ void __launch_bounds__(256) rib_bwd_finish_dq_kernel(const AuxParams p)
+{
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (size_t)p.pairs * p.n) return;
+    const int pair = (int)(t / p.n), w = (int)(t % p.n);
+    int i; size_t tok, scalar;
+    decode_pair_token(p, pair, w, i, tok, scalar);
+    const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
+    uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+        float f[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
+        dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+    }
+}
+
+// dPq[i][c] = sum over pairs of dQ~[:, d + c] / sqrt(r);  dPk[i][c] = sum over pairs of the RIB
+// columns of dK~.  grid (n / 128 * 32, groups of pairs); a thread sums one (token, column) over
+// its group and adds the partial sum to the (zeroed) result.
+__global__ void __launch_bounds__(128) rib_bwd_finish_pos_kernel(const AuxParams p, int pairs_per_group)
+{
+    const int col = blockIdx.x & 31, w = (blockIdx.x >> 5) * 128 + threadIdx.x;
+    const int pair0 = blockIdx.y * pairs_per_group;
+    const int pair1 = min(p.pairs, pair0 + pairs_per_group);
+    float acc = 0.f;
+    if (col < kR) {
+        const float* src = p.dq_acc + (size_t)(kD + col) * p.n + w;
+        for (int pair = pair0; pair < pair1; ++pair) acc += src[(size_t)pair * kDk * p.n];
+        acc *= p.inv_sqrt_r;
+    } else {
+        const float* src = p.dkp + (size_t)(col - kR) * p.n + w;
+        for (int pair = pair0; pair < pair1; ++pair) acc += src[(size_t)pair * kR * p.n];
+    }
+    int i, Y, X;
+    window_order_token(WindowGeom{p.M, p.M, p.M, 0}, 0, 0, w, i, Y, X);
+    atomicAdd((col < kR ? p.dpq : p.dpk) + (size_t)i * kR + (col & (kR - 1)), acc);
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct WorkspaceLayout { size_t ld, dq_acc, dkp, pq_scaled, total; };
+
+WorkspaceLayout workspace_layout(long long pairs, int n)
+{
+    WorkspaceLayout w;
+    w.ld = 0;
+    w.dq_acc = w.ld + align256((size_t)pairs * n * sizeof(float2));
+    w.dkp = w.dq_acc + align256((size_t)pairs * kDk * n * sizeof(float));
+    w.pq_scaled = w.dkp + align256((size_t)pairs * kR * n * sizeof(float));
+    w.total = w.pq_scaled + align256((size_t)n * kR * sizeof(__nv_bfloat16));
+    return w;
+}
+
+}  // namespace
+
+bool sm100_bwd_supported(const Problem& p)
+{
+    return p.d == sm100::kD && p.r == sm100::kR && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
+}
+
+size_t sm100_bwd_workspace_bytes(long long pairs, int n) { return workspace_layout(pairs, n).total; }
+
+cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
+{
+    if (!encode_fn()) return cudaErrorNotSupported;
+    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n);
+    if (p.workspace_bytes < wl.total) return cudaErrorInvalidValue;
+    uint8_t* ws = static_cast<uint8_t*>(p.workspace);
+    float2* ld = reinterpret_cast<float2*>(ws + wl.ld);
+    float* dq_acc = reinterpret_cast<float*>(ws + wl.dq_acc);
+    float* dkp = reinterpret_cast<float*>(ws + wl.dkp);
+    __nv_bfloat16* pq_scaled = reinterpret_cast<__nv_bfloat16*>(ws + wl.pq_scaled);
+
+    CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk;
+    if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
+        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map(&tm_pqs, pq_scaled, p) || !encode_pos_map(&tm_pk, p.pk, p))
+        return cudaErrorInvalidValue;
+    static int sm_count = 0;
+    if (!sm_count) {
+        cudaError_t e = sm_count_of_current_device(&sm_count);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(rib_bwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) { sm_count = 0; return e; }
+    }
+    AuxParams ap{};
+    ap.out = p.out; ap.dout = p.dout; ap.pq = p.pq; ap.lse = p.lse_in;
+    ap.ld = ld; ap.dq_acc = dq_acc; ap.dkp = dkp; ap.pq_scaled = pq_scaled;
+    ap.dq = p.dq; ap.dpq = p.dpq; ap.dpk = p.dpk;
+    ap.H = p.H; ap.W = p.W; ap.heads = p.heads; ap.M = p.M; ap.s = p.s; ap.n = p.n; ap.nWy = p.nWy; ap.nWx = p.nWx;
+    ap.pairs = p.pairs;
+    ap.pos_scale = sqrtf((float)p.d / (float)p.r);
+    ap.inv_sqrt_d = 1.f / sqrtf((float)p.d);
+    ap.inv_sqrt_r = 1.f / sqrtf((float)p.r);
+    const size_t tokens = (size_t)p.pairs * p.n;
+    const unsigned aux_blocks = (unsigned)((tokens + 255) / 256);
+    rib_bwd_prepare_kernel<<<aux_blocks, 256, 0, stream>>>(ap);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+
+    BwdParams bp{};
+    bp.ld = ld; bp.dq_acc = dq_acc; bp.dkp = dkp; bp.dk = p.dk; bp.dv = p.dv; bp.status = p.status;
+    bp.H = p.H; bp.W = p.W; bp.heads = p.heads; bp.M = p.M; bp.s = p.s; bp.n = p.n; bp.nWy = p.nWy; bp.nWx = p.nWx;
+    bp.nblk = p.n / kTile;
+    bp.items = p.pairs * bp.nblk;
+    bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
+    bp.inv_sqrt_d = ap.inv_sqrt_d;
+    const int grid = bp.items < sm_count ? bp.items : sm_count;
+    rib_bwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+
+    rib_bwd_finish_dq_kernel<<<aux_blocks, 256, 0, stream>>>(ap);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int groups = p.pairs < 16 ? p.pairs : 16;
+    const int per_group = (p.pairs + groups - 1) / groups;
+    dim3 grid_pos((unsigned)(p.n / 128 * 32), (unsigned)((p.pairs + per_group - 1) / per_group));
+    rib_bwd_finish_pos_kernel<<<grid_pos, 128, 0, stream>>>(ap, per_group);
+    return cudaGetLastError();
+}
+
+}  // namespace rib

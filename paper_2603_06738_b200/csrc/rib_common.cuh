@@ -26,7 +26,9 @@ struct Problem {
     __nv_bfloat16* dv;
     float* dpq;
     float* dpk;
-    float* rowdot;              // workspace: D_i = sum_c dout_ic * out_ic, image layout of lse
+    float* rowdot;              // any-shape backward: D_i = sum_c dout_ic * out_ic, image layout of lse
+    void* workspace;            // caller's scratch (backward), 256-byte aligned
+    size_t workspace_bytes;
     int B, H, W, heads, d, r, M, s;   // M = window side, s = cyclic shift
     int n, nWy, nWx, pairs;           // n = M*M, windows per image, B*nWy*nWx*heads
     int* status;                      // device status word (bounded waits report here)
@@ -39,6 +41,9 @@ cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream);
 
 bool sm100_fwd_supported(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
+bool sm100_bwd_supported(const Problem& p);
+size_t sm100_bwd_workspace_bytes(long long pairs, int n);
+cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 4 kernels
 
 // Window partition with cyclic shift: token i = y*M + x of window (wy, wx) -> image pixel.
 __host__ __device__ inline void token_pixel(int H, int W, int M, int s, int wy, int wx, int i,

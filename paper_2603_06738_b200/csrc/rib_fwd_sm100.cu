@@ -19,24 +19,15 @@
 //
 // Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocator, warps 4-7
 // softmax/epilogue of query tile 0, warps 8-11 of query tile 1.  Every wait is bounded.
-#include "rib_common.cuh"
-#include "sm100_primitives.cuh"
-
-#include <mutex>
+#include "rib_sm100_common.cuh"
 
 namespace rib {
 namespace {
 
 using namespace sm100;
 
-constexpr int kD = 32, kR = 16;
-constexpr int kTile = 128;            // rows of a query tile / keys of a key block
 constexpr int kStages = 4;            // K/V ring depth
 constexpr int kThreads = 384;
-
-constexpr uint32_t kContentBytes = kTile * kD * 2;   // 8192: 128 rows x 64 B, SWIZZLE_64B
-constexpr uint32_t kPosBytes = kTile * kR * 2;       // 4096: 128 rows x 32 B, SWIZZLE_32B
-constexpr uint32_t kPatchContent = kContentBytes / 2, kPatchPos = kPosBytes / 2;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffQc = 0;                                        // [2] query content
@@ -83,16 +74,10 @@ __device__ __forceinline__ ItemCoord decode_item(const FwdParams& p, int item)
     return c;
 }
 
-// Patch `sp` of a window (patches of 8x8 tokens, row-major over the window): top-left token in
-// window coordinates and in (shifted, wrapped) image coordinates.
 __device__ __forceinline__ void patch_origin(const FwdParams& p, const ItemCoord& c, int sp, int& py, int& px,
                                              int& Y0, int& X0)
 {
-    const int per_row = p.M >> 3;
-    py = (sp / per_row) << 3;
-    px = (sp % per_row) << 3;
-    Y0 = c.wy * p.M + py + p.s; if (Y0 >= p.H) Y0 -= p.H;
-    X0 = c.wx * p.M + px + p.s; if (X0 >= p.W) X0 -= p.W;
+    sm100::patch_origin(WindowGeom{p.H, p.W, p.M, p.s}, c.wy, c.wx, sp, py, px, Y0, X0);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -359,50 +344,6 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
 }
 
-// ---------------------------------------------------------------------------------- host side
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    });
-    return fn;
-}
-
-// bf16 [B][H][W][heads][32] image tensor, box = one 8x8-token patch of one head.
-bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p)
-{
-    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)p.heads, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-    const cuuint64_t row = (cuuint64_t)kD * 2;
-    const cuuint64_t strides[4] = {row, row * p.heads, row * p.heads * p.W, row * p.heads * p.W * p.H};
-    const cuuint32_t box[5] = {(cuuint32_t)kD, 1, 8, 8, 1};
-    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// bf16 [M][M][16] positional features, box = one 8x8-token patch.
-bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p)
-{
-    const cuuint64_t dims[3] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M};
-    const cuuint64_t strides[2] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M};
-    const cuuint32_t box[3] = {(cuuint32_t)kR, 8, 8};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 bool sm100_fwd_supported(const Problem& p)
@@ -419,9 +360,7 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
         return cudaErrorInvalidValue;
     static int sm_count = 0;
     if (!sm_count) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        cudaError_t e = sm_count_of_current_device(&sm_count);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(rib_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) { sm_count = 0; return e; }

@@ -1,0 +1,103 @@
+// Shared between the tcgen05 forward and backward kernels: the tile geometry (tiles of two 8x8-token
+// patches), the work-item decoding and the host-side TMA tensor-map encoders.
+#pragma once
+#include "rib_common.cuh"
+#include "sm100_primitives.cuh"
+
+#include <mutex>
+
+namespace rib {
+namespace sm100 {
+
+constexpr int kD = 32, kR = 16;
+constexpr int kTile = 128;                             // tokens of a query tile / key block
+constexpr uint32_t kContentBytes = kTile * kD * 2;     // 8192: 128 rows x 64 B, SWIZZLE_64B
+constexpr uint32_t kPosBytes = kTile * kR * 2;         // 4096: 128 rows x 32 B, SWIZZLE_32B
+constexpr uint32_t kPatchContent = kContentBytes / 2, kPatchPos = kPosBytes / 2;
+
+// A tile is not 128 consecutive tokens of the window but two 8x8-token patches: attention is
+// equivariant to the order of tokens inside a window, so any enumeration works as long as the
+// Pq/Pk rows and the output rows follow it.  An 8x8 patch never straddles the image border when
+// the shift is a multiple of 8, so one TMA box per patch does partition and shift.
+// "Window order" below means this enumeration: token w of a window lies in patch w / 64 (patches
+// row-major over the window), at row (w / 8) % 8 and column w % 8 of the patch.
+struct WindowGeom { int H, W, M, s; };
+
+// Patch `sp` of window (wy, wx): top-left token in window coordinates (py, px) and in shifted,
+// wrapped image coordinates (Y0, X0).
+__host__ __device__ __forceinline__ void patch_origin(const WindowGeom& g, int wy, int wx, int sp, int& py, int& px,
+                                                      int& Y0, int& X0)
+{
+    const int per_row = g.M >> 3;
+    py = (sp / per_row) << 3;
+    px = (sp % per_row) << 3;
+    Y0 = wy * g.M + py + g.s; if (Y0 >= g.H) Y0 -= g.H;
+    X0 = wx * g.M + px + g.s; if (X0 >= g.W) X0 -= g.W;
+}
+
+// Window-order index w -> row of Pq/Pk (i = y * M + x) and image pixel of window (wy, wx).
+__host__ __device__ __forceinline__ void window_order_token(const WindowGeom& g, int wy, int wx, int w, int& i,
+                                                            int& Y, int& X)
+{
+    int py, px, Y0, X0;
+    patch_origin(g, wy, wx, w >> 6, py, px, Y0, X0);
+    const int ty = (w >> 3) & 7, tx = w & 7;
+    i = (py + ty) * g.M + px + tx;
+    Y = Y0 + ty;
+    X = X0 + tx;
+}
+
+// ---------------------------------------------------------------------------------- host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+// bf16 [B][H][W][heads][32] image tensor, box = one 8x8-token patch of one head.
+inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p)
+{
+    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)p.heads, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+    const cuuint64_t row = (cuuint64_t)kD * 2;
+    const cuuint64_t strides[4] = {row, row * p.heads, row * p.heads * p.W, row * p.heads * p.W * p.H};
+    const cuuint32_t box[5] = {(cuuint32_t)kD, 1, 8, 8, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// bf16 [M][M][16] positional features, box = one 8x8-token patch.
+inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M};
+    const cuuint64_t strides[2] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M};
+    const cuuint32_t box[3] = {(cuuint32_t)kR, 8, 8};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline cudaError_t sm_count_of_current_device(int* count)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(count, cudaDevAttrMultiProcessorCount, dev);
+    return e;
+}
+
+}  // namespace sm100
+}  // namespace rib

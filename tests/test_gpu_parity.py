@@ -146,19 +146,32 @@ def test_fast_path_is_taken_for_benchmark_shapes():
     for wl in CONFIGS:
         small = Workload(wl.name, 1, wl.window, wl.window, 1, wl.d, wl.r, wl.window, wl.shift, seed=1)
         cpu, gpu = make(small, with_dout=False)
-        run_fwd(gpu, small)
+        out, lse = run_fwd(gpu, small)
+        assert binding.rib_last_path() == binding.RIB_PATH_SM100, wl.name
+        gpu["dout"] = torch.ones_like(out)
+        run_bwd(gpu, small, out, lse)
         assert binding.rib_last_path() == binding.RIB_PATH_SM100, wl.name
 
 
 def test_outputs_do_not_depend_on_stale_memory():
-    """Two calls in a row on the same buffers give the same bits for out/lse/dq/dk/dv."""
+    """Two calls in a row on the same buffers (and the same workspace) give the same bits for
+    out/lse/dk/dv; dq, dPq and dPk are fp32 sums whose order may differ from run to run."""
     wl = SMALL[7]
     cpu, gpu = make(wl)
     out1, lse1 = run_fwd(gpu, wl)
     out2, lse2 = run_fwd(gpu, wl)
     assert torch.equal(out1, out2) and torch.equal(lse1, lse2)
-    a = run_bwd(gpu, wl, out1, lse1)
-    b = run_bwd(gpu, wl, out1, lse1)
-    for x, y in zip(a[:3], b[:3]):
+    need = binding.rib_window_attn_bwd_workspace(wl.B, wl.H, wl.W, wl.heads, wl.d, wl.r, wl.window)
+    workspace = torch.full((need,), 0x7f, dtype=torch.uint8, device="cuda")     # stale, non-zero scratch
+    a = binding.rib_window_attn_bwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out1, lse1, gpu["dout"],
+                                    wl.window, wl.shift, workspace=workspace)
+    b = binding.rib_window_attn_bwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out1, lse1, gpu["dout"],
+                                    wl.window, wl.shift, workspace=workspace)
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    for x, y in zip(a[1:3], b[1:3]):
         assert torch.equal(x, y)
-    torch.testing.assert_close(a[3], b[3], rtol=1e-4, atol=1e-5)
+    torch.testing.assert_close(a[0].float(), b[0].float(), rtol=2e-2, atol=1e-3)
+    for x, y in zip(a[3:], b[3:]):
+        torch.testing.assert_close(x, y, rtol=1e-4, atol=1e-4)
