@@ -52,7 +52,8 @@ enum {
     RIB_ERR_ALIGN = -4,        /* a pointer is not 16-byte aligned */
     RIB_ERR_WORKSPACE = -5,    /* workspace missing or smaller than rib_window_attn_bwd_workspace() */
     RIB_ERR_CUDA = -6,         /* a CUDA call (launch, tensor-map encode, memset) failed */
-    RIB_ERR_DEVICE_WAIT = -7   /* reported by rib_query_status: a bounded device-side wait ran out */
+    RIB_ERR_DEVICE_WAIT = -7,  /* reported by rib_query_status: a bounded device-side wait ran out */
+    RIB_ERR_TOO_LARGE = -8     /* rib_window_attn_bwd_noalloc: the shape needs more than the built-in scratch */
 };
 
 /* Which kernel family a call used (see rib_last_path). */
@@ -89,6 +90,35 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
 
 /* Bytes of scratch rib_window_attn_bwd needs for this shape (0 on an invalid shape). */
 size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window);
+
+/*
+ * Backward pass for callers that cannot hand over scratch memory.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a memory pool or
+ * framework that owns every byte of the device and forbids cudaMalloc, in a real-time loop where
+ * an allocation would stall, in a plug-in whose host gives it only input and output buffers.
+ * Such callers cannot size and provide the `workspace` of rib_window_attn_bwd, so this variant
+ * brings its own: a fixed array of RIB_NOALLOC_SCRATCH_BYTES that is part of the library image.
+ * Every GPU on which the library is loaded holds that array from load until the process exits.
+ *
+ * Same arguments, results, kernels and error codes as rib_window_attn_bwd, minus the workspace.
+ * Differences:
+ *   - shapes whose rib_window_attn_bwd_workspace() exceeds RIB_NOALLOC_SCRATCH_BYTES are rejected
+ *     with RIB_ERR_TOO_LARGE and nothing is launched;
+ *   - the call itself allocates nothing and frees nothing (no cudaMalloc / cudaFree, no allocating
+ *     library routine); inputs and outputs are still the caller's;
+ *   - the first call on each device looks up the array's device address (with that device
+ *     current) and keeps it; make that first call outside any stream capture;
+ *   - all calls on one device share the one array, which still holds the previous call's
+ *     leftovers: the kernels clear what they need to start from zero, but two calls that overlap
+ *     on the GPU (different streams) race on it -- keep them on one stream or order them yourself.
+ */
+#define RIB_NOALLOC_SCRATCH_BYTES (32u << 20)
+int rib_window_attn_bwd_noalloc(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                                const void* out, const float* lse, const void* dout,
+                                int B, int H, int W, int heads, int d, int r, int window, int shift,
+                                void* dq, void* dk, void* dv, float* dpq, float* dpk, void* stream);
 
 /*
  * Synchronises `stream`, then reads and clears the device status word.  Kernels of this library

@@ -21,7 +21,9 @@ RIB_PATH_NONE, RIB_PATH_GENERIC, RIB_PATH_SM100 = 0, 1, 2
 EXPORTS = (
     "rib_window_attn_fwd", "rib_window_attn_bwd", "rib_window_attn_bwd_workspace",
     "rib_query_status", "rib_status_string", "rib_set_path", "rib_last_path", "rib_kernel_launches",
+    "rib_window_attn_bwd_noalloc",
 )
+RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
 class RibLibraryMissing(RuntimeError):
@@ -47,6 +49,8 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_fwd.argtypes = [vp] * 5 + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd.restype = ci
         lib.rib_window_attn_bwd.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_attn_bwd_noalloc.restype = ci
+        lib.rib_window_attn_bwd_noalloc.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp]
         lib.rib_window_attn_bwd_workspace.restype = ctypes.c_size_t
         lib.rib_window_attn_bwd_workspace.argtypes = [ci] * 7
         lib.rib_query_status.restype = ci
@@ -154,3 +158,31 @@ def rib_window_attn_bwd(q, k, v, pq, pk, out, lse, dout, window, shift=0, worksp
     if rc != RIB_OK:
         raise RibError(rc)
     return dq, dk, dv, dpq, dpk
+
+
+def rib_window_attn_bwd_noalloc(q, k, v, pq, pk, out, lse, dout, dq, dk, dv, dpq, dpk, window, shift=0, stream=None):
+    """Backward pass into caller-provided result tensors, using the library's built-in scratch.
+
+    For callers that must not allocate on the device: nothing is allocated here either, so every
+    result tensor is passed in.  Shapes that need more than ``RIB_NOALLOC_SCRATCH_BYTES`` of
+    scratch raise ``RibError`` (RIB_ERR_TOO_LARGE).  Calls on one device share the scratch: keep
+    them on one stream.
+    """
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    for name, t in (("k", k), ("v", v), ("out", out), ("dout", dout), ("dq", dq), ("dk", dk), ("dv", dv)):
+        _check_image(name, t, q.shape)
+    n = window * window
+    _check_pos("pq", pq, n)
+    _check_pos("pk", pk, n)
+    r = pq.shape[1]
+    for name, t in (("dpq", dpq), ("dpk", dpk)):
+        if t.dtype != torch.float32 or tuple(t.shape) != (n, r) or not t.is_contiguous() or not t.is_cuda:
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor [n, r]")
+    if lse.dtype != torch.float32 or tuple(lse.shape) != (B, heads, H, W) or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous fp32 tensor [B,heads,H,W]")
+    rc = library().rib_window_attn_bwd_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), _ptr(out), _ptr(lse),
+                                               _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq), _ptr(dk),
+                                               _ptr(dv), _ptr(dpq), _ptr(dpk), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)

@@ -4,6 +4,7 @@
 #include "rib_common.cuh"
 
 #include <atomic>
+#include <mutex>
 
 namespace {
 
@@ -45,6 +46,30 @@ size_t rowdot_bytes(int B, int H, int W, int heads)
 {
     const size_t bytes = sizeof(float) * (size_t)B * H * W * heads;
     return (bytes + 255) & ~(size_t)255;
+}
+
+// ---- built-in scratch of rib_window_attn_bwd_noalloc -------------------------------------------
+// Lives in the library image: every device that loads the library holds these bytes until exit.
+// In host code the name below is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[RIB_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the current device; looked up once per device.
+int noalloc_scratch_ptr(void** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RIB_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return RIB_ERR_CUDA;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return RIB_OK;
 }
 
 }  // namespace
@@ -135,6 +160,20 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
     return RIB_OK;
 }
 
+int rib_window_attn_bwd_noalloc(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                                const void* out, const float* lse, const void* dout,
+                                int B, int H, int W, int heads, int d, int r, int window, int shift,
+                                void* dq, void* dk, void* dv, float* dpq, float* dpk, void* stream)
+{
+    if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    if (rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window) > (size_t)RIB_NOALLOC_SCRATCH_BYTES)
+        return RIB_ERR_TOO_LARGE;
+    void* scratch = nullptr;
+    if (int rc = noalloc_scratch_ptr(&scratch)) return rc;
+    return rib_window_attn_bwd(q, k, v, pq, pk, out, lse, dout, B, H, W, heads, d, r, window, shift, dq, dk, dv,
+                               dpq, dpk, scratch, (size_t)RIB_NOALLOC_SCRATCH_BYTES, stream);
+}
+
 int rib_query_status(void* stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -163,6 +202,7 @@ const char* rib_status_string(int status)
         case RIB_ERR_WORKSPACE: return "RIB_ERR_WORKSPACE: workspace missing or too small";
         case RIB_ERR_CUDA: return "RIB_ERR_CUDA: a CUDA call failed";
         case RIB_ERR_DEVICE_WAIT: return "RIB_ERR_DEVICE_WAIT: a bounded device-side wait ran out";
+        case RIB_ERR_TOO_LARGE: return "RIB_ERR_TOO_LARGE: the shape needs more scratch than the built-in array holds";
         default: return "unknown RIB status";
     }
 }
