@@ -10,14 +10,15 @@
 //                        accumulating MMAs on separately staged shared-memory slabs)
 //     P_q = exp2((S_q - m) * log2e / sqrt(d))      softmax warps, fp32 -> bf16 written back to TMEM
 //     O_q += P_q V      (M128 N32 K128, A operand from TMEM, V as an MN-major shared-memory tile)
-// for the two query tiles q = 0, 1, so that one tile's softmax overlaps the other's MMAs.
+// for the two query tiles q = 0, 1.  The two tiles run as independent pipelines, each with its own
+// MMA-issuing warp: a softmax warp releases its S accumulator as soon as the scores are in
+// registers, so the next block's S_q is computed while the exponentials of this one are still being
+// evaluated.
 //
-// A tile is not 128 consecutive tokens of the window but two 8x8-token patches: attention is
-// equivariant to the order of tokens inside a window, so any enumeration works as long as the
-// Pq/Pk rows and the output rows follow it.  An 8x8 patch never straddles the image border when
-// the shift is a multiple of 8, so one TMA box per patch does partition and shift.
+// Tiles are two 8x8-token patches (see rib_sm100_common.cuh), fetched by one TMA box each.
 //
-// Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocator, warps 4-7
+// Roles (384 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers of query tile 0 and 1, warp 2
+// stages the scaled query RIB rows of the next item (and owns the TMEM allocation), warps 4-7
 // softmax/epilogue of query tile 0, warps 8-11 of query tile 1.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
@@ -30,14 +31,14 @@ constexpr int kStages = 4;            // K/V ring depth
 constexpr int kThreads = 384;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQc = 0;                                        // [2] query content
-constexpr uint32_t kOffQp = kOffQc + 2 * kContentBytes;               // [2] query RIB rows (scaled)
-constexpr uint32_t kOffKc = kOffQp + 2 * kPosBytes;                   // [kStages] key content
+constexpr uint32_t kOffQc = 0;                                        // [2 items][2 tiles] query content
+constexpr uint32_t kOffQp = kOffQc + 4 * kContentBytes;               // [2 items][2 tiles] query RIB rows (scaled)
+constexpr uint32_t kOffKc = kOffQp + 4 * kPosBytes;                   // [kStages] key content
 constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStages] key RIB rows
 constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
 constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
-enum Bar { kQFull = 0, kQEmpty, kQPos0, kQPos1, kSFull0, kSFull1, kPReady0, kPReady1, kOFull0, kOFull1, kDrain,
-           kKFull, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
+enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 12, kOFree = 14, kDrain = 16,
+           kKFull = 18, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
            kNumBars = kVEmpty + kStages };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
 constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;                 // + slack for manual alignment
@@ -97,15 +98,15 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
     if (threadIdx.x == 0) {
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
-        mbar_init(bar(kQFull), 1); mbar_init(bar(kQEmpty), 1);
-        mbar_init(bar(kQPos0), 4); mbar_init(bar(kQPos1), 4);
-        mbar_init(bar(kSFull0), 1); mbar_init(bar(kSFull1), 1);
-        mbar_init(bar(kPReady0), 4); mbar_init(bar(kPReady1), 4);
-        mbar_init(bar(kOFull0), 1); mbar_init(bar(kOFull1), 1);
-        mbar_init(bar(kDrain), 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 1);
-            mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(kQFull + i), 1); mbar_init(bar(kQEmpty + i), 2); mbar_init(bar(kQPos + i), 1);
+            mbar_init(bar(kDrain + i), 1);
+            mbar_init(bar(kSFull + i), 1); mbar_init(bar(kSFree + i), 4);
+            mbar_init(bar(kPReady + i), 4); mbar_init(bar(kPFree + i), 1); mbar_init(bar(kOFree + i), 4);
+        }
+        for (int s = 0; s < kStages; ++s) {     // the "empty" barriers take one commit from each MMA issuer
+            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 2);
+            mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 2);
         }
         fence_barrier_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_pk);
@@ -122,19 +123,20 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (warp == 0) {
         // ============================================================ TMA producer (one thread)
         if (lane == 0) {
-            uint32_t blk = 0, nitem = 0, q_armed = 0, k_armed = 0, v_armed = 0;
+            uint32_t blk = 0, io = 0, q_armed = 0, k_armed = 0, v_armed = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
                 const ItemCoord c = decode_item(p, item);
-                if (nitem > 0 && !mbar_wait(bar(kQEmpty), (nitem - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                mbar_arrive_expect_tx(bar(kQFull), 2 * kContentBytes);
+                const uint32_t buf = io & 1;
+                if (io >= 2 && !mbar_wait(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                mbar_arrive_expect_tx(bar(kQFull + buf), 2 * kContentBytes);
                 ++q_armed;
                 for (int qt = 0; qt < 2; ++qt)
                     for (int sub = 0; sub < 2; ++sub) {
                         int py, px, Y0, X0;
                         patch_origin(p, c, 2 * (2 * c.tp + qt) + sub, py, px, Y0, X0);
-                        tma_load_5d(base + kOffQc + qt * kContentBytes + sub * kPatchContent, &tm_q, bar(kQFull),
-                                    0, c.h, X0, Y0, c.b);
+                        tma_load_5d(base + kOffQc + (2 * buf + qt) * kContentBytes + sub * kPatchContent, &tm_q,
+                                    bar(kQFull + buf), 0, c.h, X0, Y0, c.b);
                     }
                 for (int j = 0; j < nblk; ++j, ++blk) {
                     const uint32_t st = blk % kStages, use = blk / kStages;
@@ -159,70 +161,108 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
             if (!ok) {
                 // Gave up: let the copies already in flight land before the CTA may exit.
-                if (q_armed) mbar_wait(bar(kQFull), (q_armed - 1) & 1, abort_flag + 1, p.status);
+                for (uint32_t b2 = q_armed > 2u ? q_armed - 2 : 0; b2 < q_armed; ++b2)
+                    mbar_wait(bar(kQFull + (b2 & 1)), (b2 >> 1) & 1, abort_flag + 1, p.status);
                 for (uint32_t b2 = k_armed > (uint32_t)kStages ? k_armed - kStages : 0; b2 < k_armed; ++b2)
                     mbar_wait(bar(kKFull + b2 % kStages), (b2 / kStages) & 1, abort_flag + 1, p.status);
                 for (uint32_t b2 = v_armed > (uint32_t)kStages ? v_armed - kStages : 0; b2 < v_armed; ++b2)
                     mbar_wait(bar(kVFull + b2 % kStages), (b2 / kStages) & 1, abort_flag + 1, p.status);
             }
         }
-    } else if (warp == 1) {
-        // ============================================================== MMA issuer (one thread)
-        if (lane == 0) {
-            uint32_t blk = 0, nitem = 0;
-            bool ok = true;
-            auto issue_s = [&](int qt, uint32_t st) {
-                const uint32_t qc = base + kOffQc + qt * kContentBytes, qp = base + kOffQp + qt * kPosBytes;
-                const uint32_t kc = base + kOffKc + st * kContentBytes, kp = base + kOffKp + st * kPosBytes;
-                const uint32_t d_s = tmem + kColS + qt * kTile;
-                mma_ss(d_s, smem_desc(qc, 16, 512, kSwizzle64B), smem_desc(kc, 16, 512, kSwizzle64B), kIdescS, 0);
-                mma_ss(d_s, smem_desc(qc + 32, 16, 512, kSwizzle64B), smem_desc(kc + 32, 16, 512, kSwizzle64B), kIdescS, 1);
-                mma_ss(d_s, smem_desc(qp, 16, 256, kSwizzle32B), smem_desc(kp, 16, 256, kSwizzle32B), kIdescS, 1);
-            };
-            auto issue_pv = [&](int qt, uint32_t st, uint32_t accumulate) {
-                const uint32_t v = base + kOffV + st * kContentBytes;
-                const uint32_t d_o = tmem + kColO + qt * kD, a_p = tmem + kColP + qt * (kTile / 2);
-                for (int kk = 0; kk < kTile / 16; ++kk)
-                    mma_ts(d_o, a_p + 8 * kk, smem_desc(v + 1024 * kk, 16, 512, kSwizzle64B), kIdescPV,
-                           (accumulate || kk) ? 1u : 0u);
-            };
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
-                if (!mbar_wait(bar(kQFull), nitem & 1, abort_flag, p.status) ||
-                    !mbar_wait(bar(kQPos0), nitem & 1, abort_flag, p.status) ||
-                    !mbar_wait(bar(kQPos1), nitem & 1, abort_flag, p.status)) { ok = false; break; }
-                {
-                    const uint32_t st = blk % kStages;
-                    if (!mbar_wait(bar(kKFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_s(0, st); mma_commit(bar(kSFull0));
-                    issue_s(1, st); mma_commit(bar(kSFull1));
-                    mma_commit(bar(kKEmpty + st));
-                }
-                for (int j = 0; j < nblk && ok; ++j, ++blk) {
-                    const uint32_t st = blk % kStages, stn = (blk + 1) % kStages;
-                    if (!mbar_wait(bar(kVFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
-                    for (int qt = 0; qt < 2; ++qt) {
-                        if (!mbar_wait(bar(kPReady0 + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
-                        tc_fence_after();
-                        issue_pv(qt, st, j > 0);
-                        if (j + 1 < nblk) {
-                            if (qt == 0 && !mbar_wait(bar(kKFull + stn), ((blk + 1) / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
-                            tc_fence_after();
-                            issue_s(qt, stn); mma_commit(bar(kSFull0 + qt));
-                            if (qt == 1) mma_commit(bar(kKEmpty + stn));
-                        } else {
-                            mma_commit(bar(kOFull0 + qt));
-                        }
-                    }
-                    if (ok) mma_commit(bar(kVEmpty + st));
-                }
-                if (ok) mma_commit(bar(kQEmpty));
+    } else if (warp == 1 || warp == 3) {
+        // ===================================== MMA issuers: warp 1 drives query tile 0, warp 3 tile 1
+        // Per block b of this CTA's items: S(b) as soon as the softmax warps have taken S(b-1) out
+        // of tensor memory, then PV(b-1) once P(b-1) is there.  The whole warp walks the loop and
+        // waits; lane 0 issues.
+        const int qt = warp >> 1;
+        constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
+        const uint32_t d_s = tmem + kColS + qt * kTile, d_o = tmem + kColO + qt * kD, a_p = tmem + kColP + qt * (kTile / 2);
+        const bool leader = lane == 0;
+        uint32_t b = 0, io = 0;
+        bool ok = true;
+        // O_q += P_q V for block `pb` (first: the first block of item ordinal `pio`)
+        auto do_pv = [&](uint32_t pb, bool first, uint32_t pio) -> bool {
+            const uint32_t st = pb % kStages;
+            // warp-uniform outcome, so that the warp stays converged
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPReady + qt), pb & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kVFull + st), (pb / kStages) & 1, abort_flag, p.status) &&
+                                             (!first || pio == 0 || mbar_wait(bar(kOFree + qt), (pio - 1) & 1, abort_flag, p.status))))
+                return false;
+            tc_fence_after();
+            if (leader) {
+                const uint64_t v = smem_desc_at(kDesc64, base + kOffV + st * kContentBytes);
+                mma_ts(d_o, a_p, v, kIdescPV, first ? 0u : 1u);
+#pragma unroll
+                for (int kk = 1; kk < kTile / 16; ++kk) mma_ts(d_o, a_p + 8 * kk, v + 64 * kk, kIdescPV, 1u);
+                mma_commit(bar(kPFree + qt));
+                mma_commit(bar(kVEmpty + st));
             }
-            // everything issued by this thread must have finished before TMEM is released
-            mma_commit(bar(kDrain));
-            mbar_wait(bar(kDrain), 0, abort_flag + 1, p.status);
+            __syncwarp();
+            return true;
+        };
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
+            const uint32_t buf = io & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status))) { ok = false; break; }
+            const uint64_t qc = smem_desc_at(kDesc64, base + kOffQc + (2 * buf + qt) * kContentBytes);
+            const uint64_t qp = smem_desc_at(kDesc32, base + kOffQp + (2 * buf + qt) * kPosBytes);
+            for (int j = 0; j < nblk; ++j, ++b) {
+                const uint32_t st = b % kStages;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kKFull + st), (b / kStages) & 1, abort_flag, p.status) &&
+                                                 (b == 0 || mbar_wait(bar(kSFree + qt), (b - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+                tc_fence_after();
+                if (leader) {
+                    const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
+                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + st * kPosBytes);
+                    mma_ss(d_s, qc, kc, kIdescS, 0u);
+                    mma_ss(d_s, qc + 2, kc + 2, kIdescS, 1u);          // + 32 bytes: second K16 step of the content rows
+                    mma_ss(d_s, qp, kp, kIdescS, 1u);
+                    mma_commit(bar(kSFull + qt));
+                    mma_commit(bar(kKEmpty + st));
+                    if (j == nblk - 1) mma_commit(bar(kQEmpty + buf));
+                }
+                __syncwarp();
+                if (b > 0 && !do_pv(b - 1, j == 1, io)) { ok = false; break; }
+            }
         }
-    } else if (warp >= 4) {
+        if (ok && b > 0) do_pv(b - 1, false, io);
+        // everything issued by this warp's leader must have finished before TMEM is released
+        if (leader) {
+            mma_commit(bar(kDrain + qt));
+            mbar_wait(bar(kDrain + qt), 0, abort_flag + 1, p.status);
+        }
+    } else if (warp == 2) {
+        // ====================== query RIB rows of the coming items: bf16(Pq * sqrt(d/r)), SWIZZLE_32B
+        uint32_t io = 0;
+        for (int item = blockIdx.x; item < p.items; item += gridDim.x, ++io) {
+            const ItemCoord c = decode_item(p, item);
+            const uint32_t buf = io & 1;
+            if (io >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status))) break;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int r256 = lane + 32 * k, qt = r256 >> 7, row = r256 & 127;
+                int py, px, Y0, X0;
+                patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+                const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
+                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)token * kR);
+                uint4 v[2] = {__ldg(src), __ldg(src + 1)};
+                uint32_t* w = reinterpret_cast<uint32_t*>(v);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
+                    const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
+                    w[i] = pack_bf16x2(lo, hi);
+                }
+                uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * 32;
+                const int sw = (row >> 2) & 1;
+                *reinterpret_cast<uint4*>(dst + ((0 ^ sw) << 4)) = v[0];
+                *reinterpret_cast<uint4*>(dst + ((1 ^ sw) << 4)) = v[1];
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kQPos + buf));
+        }
+    } else {
         // ========================================== softmax + epilogue, one thread per query row
         const int qt = (warp - 4) >> 2;
         const int quarter = warp & 3;
@@ -232,47 +272,32 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const uint32_t t_o = tmem + lane_base + kColO + qt * kD;
         const uint32_t t_p = tmem + lane_base + kColP + qt * (kTile / 2);
         const float rescale_threshold = 8.0f / p.scale_log2;    // raw-logit units: p stays <= 2^8
-        uint32_t blk = 0, nitem = 0;
+        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+        uint32_t blk = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
             const ItemCoord c = decode_item(p, item);
-            int py, px, Y0, X0;
-            patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
-            const int ty = (row >> 3) & 7, tx = row & 7;
-            const int token = (py + ty) * p.M + (px + tx);       // row of Pq that belongs to this query
-            // -- stage this row of the query RIB slab: bf16(Pq * sqrt(d/r)), SWIZZLE_32B K-major
-            {
-                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)token * kR);
-                uint4 v[2] = {__ldg(src), __ldg(src + 1)};
-                uint32_t* w = reinterpret_cast<uint32_t*>(v);
-                for (int i = 0; i < 8; ++i) {
-                    const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
-                    const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
-                    w[i] = pack_bf16x2(lo, hi);
-                }
-                uint8_t* dst = base_ptr + kOffQp + qt * kPosBytes + row * 32;
-                const int sw = (row >> 2) & 1;
-                *reinterpret_cast<uint4*>(dst + ((0 ^ sw) << 4)) = v[0];
-                *reinterpret_cast<uint4*>(dst + ((1 ^ sw) << 4)) = v[1];
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kQPos0 + qt));
-            }
             float m_used = -INFINITY, l = 0.f;
             for (int j = 0; j < nblk; ++j, ++blk) {
                 // warp-uniform outcome: the TMEM loads below are warp-collective
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull0 + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
                 uint32_t s[4][32];
                 tmem_ld32(t_s, s[0]); tmem_ld32(t_s + 32, s[1]); tmem_ld32(t_s + 64, s[2]); tmem_ld32(t_s + 96, s[3]);
                 tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[0][i])); mx1 = fmaxf(mx1, __uint_as_float(s[1][i]));
-                    mx2 = fmaxf(mx2, __uint_as_float(s[2][i])); mx3 = fmaxf(mx3, __uint_as_float(s[3][i]));
+                for (int i = 0; i < 32; i += 2) {
+                    mx0 = max3(mx0, __uint_as_float(s[0][i]), __uint_as_float(s[0][i + 1]));
+                    mx1 = max3(mx1, __uint_as_float(s[1][i]), __uint_as_float(s[1][i + 1]));
+                    mx2 = max3(mx2, __uint_as_float(s[2][i]), __uint_as_float(s[2][i + 1]));
+                    mx3 = max3(mx3, __uint_as_float(s[3][i]), __uint_as_float(s[3][i + 1]));
                 }
                 const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                bool p_free = blk == 0;       // P_q (and O_q) are free once the previous block's PV has completed
                 if (j == 0) {
                     m_used = mx;
                 } else {
@@ -280,6 +305,9 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     // exact after the final normalisation because l carries the same reference.
                     const bool need = mx > m_used + rescale_threshold;
                     if (__any_sync(0xffffffffu, need)) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + qt), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+                        p_free = true;
                         const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
                         if (need) { l *= factor; m_used = mx; }
                         uint32_t o[32];
@@ -292,34 +320,47 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     }
                 }
                 const float neg_ms = -m_used * p.scale_log2;
-                float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+                const float2 neg2 = make_float2(neg_ms, neg_ms);
+                float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[ch][2 * i]), p.scale_log2, neg_ms));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[ch][2 * i + 1]), p.scale_log2, neg_ms));
-                        if (i & 1) { sum2 += p0; sum3 += p1; } else { sum0 += p0; sum1 += p1; }
-                        packed[i] = pack_bf16x2(p0, p1);
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[ch][2 * i]), __uint_as_float(s[ch][2 * i + 1])),
+                                                    scale2, neg2);
+                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        if (i & 1) sum_b = __fadd2_rn(sum_b, e); else sum_a = __fadd2_rn(sum_a, e);
+                        packed[i] = pack_bf16x2(e.x, e.y);
+                    }
+                    if (!p_free) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + qt), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+                        p_free = true;
                     }
                     tmem_st16(t_p + 16 * ch, packed);
                 }
-                l += (sum0 + sum1) + (sum2 + sum3);
+                if (!ok) break;
+                l += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kPReady0 + qt));
+                if (lane == 0) mbar_arrive(bar(kPReady + qt));
             }
             if (!ok) break;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kOFull0 + qt), nitem & 1, abort_flag, p.status))) { ok = false; break; }
+            // the last PV of the item has completed: O_q is final
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + qt), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
             tc_fence_after();
             uint32_t o[32];
             tmem_ld32(t_o, o);
             tmem_wait_ld();
             tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kOFree + qt));
+            int py, px, Y0, X0;
+            patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+            const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
             const float inv_l = 1.f / l;
-            int Y = Y0 + ty, X = X0 + tx;        // the patch does not straddle the border
             const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
             uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD);
 #pragma unroll

@@ -37,6 +37,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Non-blocking test of a phase (used where one thread polls several barriers).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_timer_ns()
 {
     uint64_t t;
@@ -169,6 +180,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (swizzle << 61);
 }
+// The same descriptor split into its constant part and the address: the address field holds
+// (addr >> 4), and shared-memory addresses are below 2^18, so stepping through a tile is one add.
+constexpr uint64_t smem_desc_const(uint32_t lbo_bytes, uint32_t sbo_bytes, uint64_t swizzle)
+{
+    return ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) | ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) |
+           (swizzle << 61);
+}
+__device__ __forceinline__ uint64_t smem_desc_at(uint64_t desc_const, uint32_t addr) { return desc_const + (addr >> 4); }
 // Instruction descriptor of kind::f16 with bf16 operands and fp32 accumulation.
 // b_mn_major: B is stored with N contiguous (a [K][N] row-major tile).
 constexpr uint32_t idesc_bf16_f32(int m, int n, bool b_mn_major)
@@ -214,6 +233,12 @@ __device__ __forceinline__ float ex2_approx(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
