@@ -11,15 +11,22 @@
 //     P_q = exp2((S_q - m) * log2e / sqrt(d))      softmax warps, fp32 -> bf16 written back to TMEM
 //     O_q += P_q V      (M128 N32 K128, A operand from TMEM, V as an MN-major shared-memory tile)
 // for the two query tiles q = 0, 1.  The two tiles run as independent pipelines, each with its own
-// MMA-issuing warp: a softmax warp releases its S accumulator as soon as the scores are in
-// registers, so the next block's S_q is computed while the exponentials of this one are still being
-// evaluated.
+// MMA-issuing warp; the S accumulator is released as soon as the scores are in registers, so the
+// next block's S_q is computed while the exponentials of this one are still being evaluated.
+//
+// The softmax of a query tile is split over the keys: two threads own a query row, one takes keys
+// 0-63 of every block and the other keys 64-127.  Each keeps its own running maximum and sum and
+// its own O accumulator in tensor memory (PV of a block is two K64 contractions), and the two
+// partial results are merged in the epilogue with the usual log-sum-exp combination.  This puts
+// four softmax warps on every SM sub-partition, which is what keeps the exp (XU) pipe fed: with one
+// thread per row the tensor-memory and barrier latencies of a block were exposed.
 //
 // Tiles are two 8x8-token patches (see rib_sm100_common.cuh), fetched by one TMA box each.
 //
-// Roles (384 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers of query tile 0 and 1, warp 2
-// stages the scaled query RIB rows of the next item (and owns the TMEM allocation), warps 4-7
-// softmax/epilogue of query tile 0, warps 8-11 of query tile 1.  Every wait is bounded.
+// Roles (640 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers of query tile 0 and 1, warp 2
+// stages the scaled query RIB rows of the next item (and owns the TMEM allocation), warps 4-11
+// softmax/epilogue of query tile 0 (4-7 first half of the keys, 8-11 second half), warps 12-19 of
+// query tile 1.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -28,7 +35,7 @@ namespace {
 using namespace sm100;
 
 constexpr int kStages = 4;            // K/V ring depth
-constexpr int kThreads = 384;
+constexpr int kThreads = 640;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffQc = 0;                                        // [2 items][2 tiles] query content
@@ -37,14 +44,17 @@ constexpr uint32_t kOffKc = kOffQp + 4 * kPosBytes;                   // [kStage
 constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStages] key RIB rows
 constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
 constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
-enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 12, kOFree = 14, kDrain = 16,
-           kKFull = 18, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
+// kPReady / kPFree: index 2 * tile + key half
+enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 14, kOFree = 18, kDrain = 20, kMerge = 22,
+           kKFull = 30, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
            kNumBars = kVEmpty + kStages };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
-constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;                 // + slack for manual alignment
+constexpr uint32_t kOffMerge = kOffMisc + 16;                         // [2 tiles][2 halves][128 rows] (max, sum)
+constexpr uint32_t kSmemBytes = kOffMerge + 4 * kTile * 8 + 1024;     // + slack for manual alignment
 
 // tensor-memory columns (fp32 accumulators; P is bf16x2, two keys per column)
-constexpr uint32_t kColS = 0, kColO = 256, kColP = 320, kTmemCols = 512;
+// O: [2 tiles][2 key halves][32]
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
 
 constexpr uint32_t kIdescS = idesc_bf16_f32(kTile, kTile, false);
 constexpr uint32_t kIdescPV = idesc_bf16_f32(kTile, kD, true);
@@ -101,8 +111,9 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(kQFull + i), 1); mbar_init(bar(kQEmpty + i), 2); mbar_init(bar(kQPos + i), 1);
             mbar_init(bar(kDrain + i), 1);
-            mbar_init(bar(kSFull + i), 1); mbar_init(bar(kSFree + i), 4);
-            mbar_init(bar(kPReady + i), 4); mbar_init(bar(kPFree + i), 1); mbar_init(bar(kOFree + i), 4);
+            mbar_init(bar(kSFull + i), 1); mbar_init(bar(kSFree + i), 8); mbar_init(bar(kOFree + i), 8);
+            for (int h = 0; h < 2; ++h) { mbar_init(bar(kPReady + 2 * i + h), 4); mbar_init(bar(kPFree + 2 * i + h), 1); }
+            for (int q4 = 0; q4 < 4; ++q4) mbar_init(bar(kMerge + 4 * i + q4), 2);
         }
         for (int s = 0; s < kStages; ++s) {     // the "empty" barriers take one commit from each MMA issuer
             mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 2);
@@ -176,28 +187,32 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         // waits; lane 0 issues.
         const int qt = warp >> 1;
         constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
-        const uint32_t d_s = tmem + kColS + qt * kTile, d_o = tmem + kColO + qt * kD, a_p = tmem + kColP + qt * (kTile / 2);
+        const uint32_t d_s = tmem + kColS + qt * kTile, d_o = tmem + kColO + qt * 2 * kD, a_p = tmem + kColP + qt * (kTile / 2);
         const bool leader = lane == 0;
         uint32_t b = 0, io = 0;
         bool ok = true;
-        // O_q += P_q V for block `pb` (first: the first block of item ordinal `pio`)
+        // O_q[half] += P_q[:, half] V[half] for block `pb` (first: the first block of item ordinal `pio`)
         auto do_pv = [&](uint32_t pb, bool first, uint32_t pio) -> bool {
             const uint32_t st = pb % kStages;
-            // warp-uniform outcome, so that the warp stays converged
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPReady + qt), pb & 1, abort_flag, p.status) &&
-                                             mbar_wait(bar(kVFull + st), (pb / kStages) & 1, abort_flag, p.status) &&
+            // warp-uniform outcomes, so that the warp stays converged
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kVFull + st), (pb / kStages) & 1, abort_flag, p.status) &&
                                              (!first || pio == 0 || mbar_wait(bar(kOFree + qt), (pio - 1) & 1, abort_flag, p.status))))
                 return false;
-            tc_fence_after();
-            if (leader) {
-                const uint64_t v = smem_desc_at(kDesc64, base + kOffV + st * kContentBytes);
-                mma_ts(d_o, a_p, v, kIdescPV, first ? 0u : 1u);
+            const uint64_t v = smem_desc_at(kDesc64, base + kOffV + st * kContentBytes);
 #pragma unroll
-                for (int kk = 1; kk < kTile / 16; ++kk) mma_ts(d_o, a_p + 8 * kk, v + 64 * kk, kIdescPV, 1u);
-                mma_commit(bar(kPFree + qt));
-                mma_commit(bar(kVEmpty + st));
+            for (int half = 0; half < 2; ++half) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kPReady + 2 * qt + half), pb & 1, abort_flag, p.status))) return false;
+                tc_fence_after();
+                if (leader) {
+                    mma_ts(d_o + half * kD, a_p + 32 * half, v + 256 * half, kIdescPV, first ? 0u : 1u);
+#pragma unroll
+                    for (int kk = 1; kk < 4; ++kk)
+                        mma_ts(d_o + half * kD, a_p + 32 * half + 8 * kk, v + 256 * half + 64 * kk, kIdescPV, 1u);
+                    mma_commit(bar(kPFree + 2 * qt + half));
+                    if (half == 1) mma_commit(bar(kVEmpty + st));
+                }
+                __syncwarp();
             }
-            __syncwarp();
             return true;
         };
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
@@ -263,117 +278,151 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (lane == 0) mbar_arrive(bar(kQPos + buf));
         }
     } else {
-        // ========================================== softmax + epilogue, one thread per query row
-        const int qt = (warp - 4) >> 2;
+        // ================ softmax + epilogue: two threads per query row, one per half of the keys
+        const int qt = (warp - 4) >> 3;
+        const int half = ((warp - 4) >> 2) & 1;
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                 // row of the tile == TMEM lane
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + kColS + qt * kTile;
-        const uint32_t t_o = tmem + lane_base + kColO + qt * kD;
-        const uint32_t t_p = tmem + lane_base + kColP + qt * (kTile / 2);
+        const uint32_t t_s = tmem + lane_base + kColS + qt * kTile + half * 64;
+        const uint32_t t_o = tmem + lane_base + kColO + qt * 2 * kD;        // both halves' accumulators
+        const uint32_t t_p = tmem + lane_base + kColP + qt * (kTile / 2) + half * 32;
+        const uint32_t b_ready = bar(kPReady + 2 * qt + half), b_free = bar(kPFree + 2 * qt + half);
+        float2* merge = reinterpret_cast<float2*>(base_ptr + kOffMerge) + qt * 2 * kTile;   // [half][row]
         const float rescale_threshold = 8.0f / p.scale_log2;    // raw-logit units: p stays <= 2^8
         const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
-        uint32_t blk = 0;
+        uint32_t blk = 0, nitem = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
+        // exp2 of 32 scores against the reference -m * log2e/sqrt(d); returns their sum
+        auto exp_chunk = [&](const uint32_t (&s)[32], float neg_ms, uint32_t (&packed)[16]) -> float {
+            const float2 neg2 = make_float2(neg_ms, neg_ms);
+            float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg2);
+                const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                if (i & 1) sum_b = __fadd2_rn(sum_b, e); else sum_a = __fadd2_rn(sum_a, e);
+                packed[i] = pack_bf16x2(e.x, e.y);
+            }
+            return (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+        };
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
             const ItemCoord c = decode_item(p, item);
             float m_used = -INFINITY, l = 0.f;
             for (int j = 0; j < nblk; ++j, ++blk) {
                 // warp-uniform outcome: the TMEM loads below are warp-collective
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
-                uint32_t s[4][32];
-                tmem_ld32(t_s, s[0]); tmem_ld32(t_s + 32, s[1]); tmem_ld32(t_s + 64, s[2]); tmem_ld32(t_s + 96, s[3]);
-                tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                bool p_free = blk == 0;       // P (and O) of this half are free once the previous block's PV has completed
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    mx0 = max3(mx0, __uint_as_float(s[0][i]), __uint_as_float(s[0][i + 1]));
-                    mx1 = max3(mx1, __uint_as_float(s[1][i]), __uint_as_float(s[1][i + 1]));
-                    mx2 = max3(mx2, __uint_as_float(s[2][i]), __uint_as_float(s[2][i + 1]));
-                    mx3 = max3(mx3, __uint_as_float(s[3][i]), __uint_as_float(s[3][i + 1]));
-                }
-                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                bool p_free = blk == 0;       // P_q (and O_q) are free once the previous block's PV has completed
-                if (j == 0) {
-                    m_used = mx;
-                } else {
-                    // Rescale O only when the maximum grew by more than the threshold; the result is
-                    // exact after the final normalisation because l carries the same reference.
-                    const bool need = mx > m_used + rescale_threshold;
-                    if (__any_sync(0xffffffffu, need)) {
-                        if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + qt), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
-                        tc_fence_after();
-                        p_free = true;
-                        const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
-                        if (need) { l *= factor; m_used = mx; }
-                        uint32_t o[32];
-                        tmem_ld32(t_o, o);
-                        tmem_wait_ld();
+                for (int ch = 0; ch < 2; ++ch) {
+                    uint32_t s[32];
+                    tmem_ld32(t_s + 32 * ch, s);
+                    tmem_wait_ld();
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                        tmem_st32(t_o, o);
-                        tmem_wait_st();
+                    for (int i = 0; i < 32; i += 4) {
+                        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+                        mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
                     }
-                }
-                const float neg_ms = -m_used * p.scale_log2;
-                const float2 neg2 = make_float2(neg_ms, neg_ms);
-                float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+                    const float mx = fmaxf(mx0, mx1);
+                    if (j == 0 && ch == 0) {
+                        m_used = mx;
+                    } else {
+                        // Move the reference (and rescale O, l) only when the maximum grew by more than
+                        // the threshold; the result is exact after the final normalisation because l
+                        // carries the same reference.
+                        const bool need = mx > m_used + rescale_threshold;
+                        if (__any_sync(0xffffffffu, need)) {
+                            if (!p_free) {
+                                if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                                tc_fence_after();
+                                p_free = true;
+                            }
+                            const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
+                            if (need) { l *= factor; m_used = mx; }
+                            if (j > 0) {
+                                uint32_t o[32];
+                                tmem_ld32(t_o + half * kD, o);
+                                tmem_wait_ld();
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
+                                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                                tmem_st32(t_o + half * kD, o);
+                            }
+                            if (ch == 1) {
+                                // the first 32 keys of this block were exponentiated against the old
+                                // reference: redo them (their sum is already in l, rescaled above)
+                                uint32_t s0[32], packed0[16];
+                                tmem_ld32(t_s, s0);
+                                tmem_wait_ld();
+                                exp_chunk(s0, -m_used * p.scale_log2, packed0);
+                                tmem_st16(t_p, packed0);
+                            }
+                            tmem_wait_st();
+                        }
+                    }
+                    if (ch == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
+                    }
                     uint32_t packed[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[ch][2 * i]), __uint_as_float(s[ch][2 * i + 1])),
-                                                    scale2, neg2);
-                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-                        if (i & 1) sum_b = __fadd2_rn(sum_b, e); else sum_a = __fadd2_rn(sum_a, e);
-                        packed[i] = pack_bf16x2(e.x, e.y);
-                    }
+                    l += exp_chunk(s, -m_used * p.scale_log2, packed);
                     if (!p_free) {
-                        if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + qt), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
                         tc_fence_after();
                         p_free = true;
                     }
                     tmem_st16(t_p + 16 * ch, packed);
                 }
                 if (!ok) break;
-                l += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kPReady + qt));
+                if (lane == 0) mbar_arrive(b_ready);
             }
             if (!ok) break;
-            // the last PV of the item has completed: O_q is final
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + qt), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+            // ---- merge the two key halves and write this thread's 16 output columns
+            merge[half * kTile + row] = make_float2(m_used, l);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kMerge + 4 * qt + quarter));
+            // both halves' last PV must have completed, and the partner's (m, l) must be there
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + 2 * qt), (blk - 1) & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kPFree + 2 * qt + 1), (blk - 1) & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kMerge + 4 * qt + quarter), nitem & 1, abort_flag, p.status))) { ok = false; break; }
             tc_fence_after();
-            uint32_t o[32];
-            tmem_ld32(t_o, o);
+            uint32_t oa[16], ob[16];
+            tmem_ld16(t_o + half * 16, oa);
+            tmem_ld16(t_o + kD + half * 16, ob);
             tmem_wait_ld();
+            const float2 other = merge[(half ^ 1) * kTile + row];
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kOFree + qt));
+            const float m_a = half ? other.x : m_used, l_a = half ? other.y : l;
+            const float m_b = half ? m_used : other.x, l_b = half ? l : other.y;
+            const float m = fmaxf(m_a, m_b);
+            const float f_a = ex2_approx((m_a - m) * p.scale_log2), f_b = ex2_approx((m_b - m) * p.scale_log2);
+            const float l_all = l_a * f_a + l_b * f_b;
+            const float w_a = f_a / l_all, w_b = f_b / l_all;
             int py, px, Y0, X0;
             patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
             const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
-            const float inv_l = 1.f / l;
             const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD);
+            uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD + half * 16);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint4 v;
-                v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
-                v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
-                v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
-                v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
-                dst[i] = v;
+            for (int i = 0; i < 2; ++i) {
+                uint32_t w[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int e = 8 * i + 2 * k;
+                    w[k] = pack_bf16x2(__uint_as_float(oa[e]) * w_a + __uint_as_float(ob[e]) * w_b,
+                                       __uint_as_float(oa[e + 1]) * w_a + __uint_as_float(ob[e + 1]) * w_b);
+                }
+                dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            if (p.lse)
-                p.lse[(((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X] = m_used * p.inv_sqrt_d + logf(l);
+            if (p.lse && half == 0)
+                p.lse[(((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X] = m * p.inv_sqrt_d + logf(l_all);
         }
     }
     // ================================================================================ common tail
