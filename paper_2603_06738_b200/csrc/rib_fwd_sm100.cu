@@ -23,15 +23,10 @@
 //
 // Tiles are two 8x8-token patches (see rib_sm100_common.cuh), fetched by one TMA box each.
 //
-// Roles (640 threads): warp 0 TMA producer (and TMEM allocation); warp 1 issues the S contractions
-// of both tiles, warps 2 and 3 the PV contractions of tile 0 and 1 (one thread each: several warps
-// can feed the tensor pipe at once, and a single issuer going wait -> issue -> wait was the
-// bottleneck); warps 4-11 softmax and epilogue of query tile 0 (4-7 first half of the keys, 8-11
-// second half), warps 12-19 of tile 1.  The first-half softmax threads also stage, two items
-// ahead, the scaled query RIB row bf16(Pq sqrt(d/r)) of their query row.
-// K and V ring slots are handed back to the producer by the softmax warps (plain mbarrier
-// arrivals once S has been read, or once the PV that read P has completed), not by extra
-// tcgen05.commit instructions.  Every wait is bounded.
+// Roles (640 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers of query tile 0 and 1, warp 2
+// stages the scaled query RIB rows of the next item (and owns the TMEM allocation), warps 4-11
+// softmax/epilogue of query tile 0 (4-7 first half of the keys, 8-11 second half), warps 12-19 of
+// query tile 1.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -50,8 +45,8 @@ constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStage
 constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
 constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
 // kPReady / kPFree: index 2 * tile + key half
-enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 14, kOFree = 18, kDrain = 20, kMerge = 23,
-           kKFull = 31, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
+enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 14, kOFree = 18, kDrain = 20, kMerge = 22,
+           kKFull = 30, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
            kNumBars = kVEmpty + kStages };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
 constexpr uint32_t kOffMerge = kOffMisc + 16;                         // [2 tiles][2 halves][128 rows] (max, sum)
@@ -114,20 +109,20 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (threadIdx.x == 0) {
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(kQFull + i), 1); mbar_init(bar(kQEmpty + i), 1); mbar_init(bar(kQPos + i), 8);
+            mbar_init(bar(kQFull + i), 1); mbar_init(bar(kQEmpty + i), 2); mbar_init(bar(kQPos + i), 1);
+            mbar_init(bar(kDrain + i), 1);
             mbar_init(bar(kSFull + i), 1); mbar_init(bar(kSFree + i), 8); mbar_init(bar(kOFree + i), 8);
             for (int h = 0; h < 2; ++h) { mbar_init(bar(kPReady + 2 * i + h), 4); mbar_init(bar(kPFree + 2 * i + h), 1); }
             for (int q4 = 0; q4 < 4; ++q4) mbar_init(bar(kMerge + 4 * i + q4), 2);
         }
-        for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
-        for (int s = 0; s < kStages; ++s) {     // the "empty" barriers take one arrival from each of the 16 softmax warps
-            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 16);
-            mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 16);
+        for (int s = 0; s < kStages; ++s) {     // the "empty" barriers take one commit from each MMA issuer
+            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 2);
+            mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 2);
         }
         fence_barrier_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v); prefetch_tensormap(&tm_pk);
     }
-    if (warp == 0) {
+    if (warp == 2) {
         tmem_alloc(base + kOffMisc, kTmemCols);
         tmem_relinquish();
     }
@@ -185,86 +180,102 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     mbar_wait(bar(kVFull + b2 % kStages), (b2 / kStages) & 1, abort_flag + 1, p.status);
             }
         }
-    } else if (warp == 1) {
-        // ================================= S issuer (one thread): S_q(b) = Q~_q K~(b)^T for both tiles
-        // S_q(b) goes out as soon as the softmax warps have taken S_q(b-1) out of tensor memory;
-        // the thread polls both tiles.  Counters are block ordinals over all items of this CTA.
-        if (lane == 0) {
-            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
-            const uint32_t my_items = ((uint32_t)p.items - blockIdx.x + gridDim.x - 1) / gridDim.x;
-            const uint32_t total = my_items * (uint32_t)nblk;
-            uint32_t sb[2] = {0, 0}, s_io[2] = {0, 0}, s_j[2] = {0, 0};
-            uint64_t t_idle = 0;
-            uint32_t idle_spins = 0;
-            bool ok = true;
-            while (ok && (sb[0] < total || sb[1] < total)) {
-                bool progressed = false;
+    } else if (warp == 1 || warp == 3) {
+        // ===================================== MMA issuers: warp 1 drives query tile 0, warp 3 tile 1
+        // Per block b of this CTA's items: S(b) as soon as the softmax warps have taken S(b-1) out
+        // of tensor memory, then PV(b-1) once P(b-1) is there.  The whole warp walks the loop and
+        // waits; lane 0 issues.
+        const int qt = warp >> 1;
+        constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
+        const uint32_t d_s = tmem + kColS + qt * kTile, d_o = tmem + kColO + qt * 2 * kD, a_p = tmem + kColP + qt * (kTile / 2);
+        const bool leader = lane == 0;
+        uint32_t b = 0, io = 0;
+        bool ok = true;
+        // O_q[half] += P_q[:, half] V[half] for block `pb` (first: the first block of item ordinal `pio`)
+        auto do_pv = [&](uint32_t pb, bool first, uint32_t pio) -> bool {
+            const uint32_t st = pb % kStages;
+            // warp-uniform outcomes, so that the warp stays converged
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kVFull + st), (pb / kStages) & 1, abort_flag, p.status) &&
+                                             (!first || pio == 0 || mbar_wait(bar(kOFree + qt), (pio - 1) & 1, abort_flag, p.status))))
+                return false;
+            const uint64_t v = smem_desc_at(kDesc64, base + kOffV + st * kContentBytes);
 #pragma unroll
-                for (int qt = 0; qt < 2; ++qt) {
-                    if (sb[qt] >= total) continue;
-                    const uint32_t b = sb[qt], st = b % kStages, buf = s_io[qt] & 1;
-                    if ((s_j[qt] != 0 || (mbar_test(bar(kQFull + buf), (s_io[qt] >> 1) & 1) &&
-                                          mbar_test(bar(kQPos + buf), (s_io[qt] >> 1) & 1))) &&
-                        mbar_test(bar(kKFull + st), (b / kStages) & 1) &&
-                        (b == 0 || mbar_test(bar(kSFree + qt), (b - 1) & 1))) {
-                        tc_fence_after();
-                        const uint64_t qc = smem_desc_at(kDesc64, base + kOffQc + (2 * buf + qt) * kContentBytes);
-                        const uint64_t qp = smem_desc_at(kDesc32, base + kOffQp + (2 * buf + qt) * kPosBytes);
-                        const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
-                        const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + st * kPosBytes);
-                        const uint32_t d_s = tmem + kColS + qt * kTile;
-                        mma_ss(d_s, qc, kc, kIdescS, 0u);
-                        mma_ss(d_s, qc + 2, kc + 2, kIdescS, 1u);      // + 32 bytes: second K16 step of the content rows
-                        mma_ss(d_s, qp, kp, kIdescS, 1u);
-                        mma_commit(bar(kSFull + qt));
-                        ++sb[qt];
-                        // the query tiles of this item are no longer needed once both tiles' last S is done
-                        if (s_j[qt] == (uint32_t)nblk - 1 && sb[qt ^ 1] > b) mma_commit(bar(kQEmpty + buf));
-                        if (++s_j[qt] == (uint32_t)nblk) { s_j[qt] = 0; ++s_io[qt]; }
-                        progressed = true;
-                    }
+            for (int half = 0; half < 2; ++half) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kPReady + 2 * qt + half), pb & 1, abort_flag, p.status))) return false;
+                tc_fence_after();
+                if (leader) {
+                    mma_ts(d_o + half * kD, a_p + 32 * half, v + 256 * half, kIdescPV, first ? 0u : 1u);
+#pragma unroll
+                    for (int kk = 1; kk < 4; ++kk)
+                        mma_ts(d_o + half * kD, a_p + 32 * half + 8 * kk, v + 256 * half + 64 * kk, kIdescPV, 1u);
+                    mma_commit(bar(kPFree + 2 * qt + half));
+                    if (half == 1) mma_commit(bar(kVEmpty + st));
                 }
-                if (progressed) {
-                    idle_spins = 0;
-                } else if ((++idle_spins & 255u) == 0) {
-                    if (*abort_flag) { ok = false; break; }
-                    const uint64_t now = global_timer_ns();
-                    if (idle_spins == 256u) t_idle = now;
-                    else if (now - t_idle > kWaitLimitNs) { *abort_flag = 1; atomicExch(p.status, 1); ok = false; break; }
-                }
+                __syncwarp();
             }
-            // everything issued by this thread must have finished before TMEM is released
-            mma_commit(bar(kDrain));
-            mbar_wait(bar(kDrain), 0, abort_flag + 1, p.status);
+            return true;
+        };
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
+            const uint32_t buf = io & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status))) { ok = false; break; }
+            const uint64_t qc = smem_desc_at(kDesc64, base + kOffQc + (2 * buf + qt) * kContentBytes);
+            const uint64_t qp = smem_desc_at(kDesc32, base + kOffQp + (2 * buf + qt) * kPosBytes);
+            for (int j = 0; j < nblk; ++j, ++b) {
+                const uint32_t st = b % kStages;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(kKFull + st), (b / kStages) & 1, abort_flag, p.status) &&
+                                                 (b == 0 || mbar_wait(bar(kSFree + qt), (b - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+                tc_fence_after();
+                if (leader) {
+                    const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
+                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + st * kPosBytes);
+                    mma_ss(d_s, qc, kc, kIdescS, 0u);
+                    mma_ss(d_s, qc + 2, kc + 2, kIdescS, 1u);          // + 32 bytes: second K16 step of the content rows
+                    mma_ss(d_s, qp, kp, kIdescS, 1u);
+                    mma_commit(bar(kSFull + qt));
+                    mma_commit(bar(kKEmpty + st));
+                    if (j == nblk - 1) mma_commit(bar(kQEmpty + buf));
+                }
+                __syncwarp();
+                if (b > 0 && !do_pv(b - 1, j == 1, io)) { ok = false; break; }
+            }
         }
-    } else if (warp == 2 || warp == 3) {
-        // ===================== PV issuers (one thread per tile): O_q[half] += P_q[:, half] V(b)[half]
-        if (lane == 0) {
-            const int qt = warp - 2;
-            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B);
-            const uint32_t d_o = tmem + kColO + qt * 2 * kD, a_p = tmem + kColP + qt * (kTile / 2);
-            uint32_t b = 0, io = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
-                for (int j = 0; j < nblk && ok; ++j, ++b) {
-                    const uint32_t st = b % kStages;
-                    if (!mbar_wait(bar(kVFull + st), (b / kStages) & 1, abort_flag, p.status) ||
-                        (j == 0 && io > 0 && !mbar_wait(bar(kOFree + qt), (io - 1) & 1, abort_flag, p.status))) { ok = false; break; }
-                    const uint64_t v = smem_desc_at(kDesc64, base + kOffV + st * kContentBytes);
+        if (ok && b > 0) do_pv(b - 1, false, io);
+        // everything issued by this warp's leader must have finished before TMEM is released
+        if (leader) {
+            mma_commit(bar(kDrain + qt));
+            mbar_wait(bar(kDrain + qt), 0, abort_flag + 1, p.status);
+        }
+    } else if (warp == 2) {
+        // ====================== query RIB rows of the coming items: bf16(Pq * sqrt(d/r)), SWIZZLE_32B
+        uint32_t io = 0;
+        for (int item = blockIdx.x; item < p.items; item += gridDim.x, ++io) {
+            const ItemCoord c = decode_item(p, item);
+            const uint32_t buf = io & 1;
+            if (io >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status))) break;
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        if (!mbar_wait(bar(kPReady + 2 * qt + half), b & 1, abort_flag, p.status)) { ok = false; break; }
-                        tc_fence_after();
-                        mma_ts(d_o + half * kD, a_p + 32 * half, v + 256 * half, kIdescPV, j == 0 ? 0u : 1u);
+            for (int k = 0; k < 8; ++k) {
+                const int r256 = lane + 32 * k, qt = r256 >> 7, row = r256 & 127;
+                int py, px, Y0, X0;
+                patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+                const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
+                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)token * kR);
+                uint4 v[2] = {__ldg(src), __ldg(src + 1)};
+                uint32_t* w = reinterpret_cast<uint32_t*>(v);
 #pragma unroll
-                        for (int kk = 1; kk < 4; ++kk)
-                            mma_ts(d_o + half * kD, a_p + 32 * half + 8 * kk, v + 256 * half + 64 * kk, kIdescPV, 1u);
-                        mma_commit(bar(kPFree + 2 * qt + half));
-                    }
+                for (int i = 0; i < 8; ++i) {
+                    const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
+                    const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
+                    w[i] = pack_bf16x2(lo, hi);
                 }
+                uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * 32;
+                const int sw = (row >> 2) & 1;
+                *reinterpret_cast<uint4*>(dst + ((0 ^ sw) << 4)) = v[0];
+                *reinterpret_cast<uint4*>(dst + ((1 ^ sw) << 4)) = v[1];
             }
-            mma_commit(bar(kDrain + 1 + qt));
-            mbar_wait(bar(kDrain + 1 + qt), 0, abort_flag + 1, p.status);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kQPos + buf));
         }
     } else {
         // ================ softmax + epilogue: two threads per query row, one per half of the keys
@@ -281,19 +292,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const float rescale_threshold = 8.0f / p.scale_log2;    // raw-logit units: p stays <= 2^8
         const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
         uint32_t blk = 0, nitem = 0;
-        uint32_t pv_seen = 0;          // PV completions of this half observed so far (V slots handed back)
         bool ok = true;
-        // Waits until the PV of every block before `upto` has completed (P and O of this half are
-        // then free) and hands each such block's V slot back to the producer, once.
-        auto pv_done_before = [&](uint32_t upto) -> bool {
-            while (pv_seen < upto) {
-                if (!__all_sync(0xffffffffu, mbar_wait(b_free, pv_seen & 1, abort_flag, p.status))) return false;
-                if (lane == 0) mbar_arrive(bar(kVEmpty + pv_seen % kStages));
-                ++pv_seen;
-            }
-            tc_fence_after();
-            return true;
-        };
         // exp2 of 32 scores against the reference -m * log2e/sqrt(d); returns their sum
         auto exp_chunk = [&](const uint32_t (&s)[32], float neg_ms, uint32_t (&packed)[16]) -> float {
             const float2 neg2 = make_float2(neg_ms, neg_ms);
@@ -307,34 +306,6 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
             return (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
         };
-        // Query RIB row of this thread's query for `item2`: bf16(Pq * sqrt(d/r)) into the SWIZZLE_32B
-        // K-major slab the S contraction reads (first-half threads only).
-        auto stage_query_rib = [&](int item2, uint32_t buf) {
-            const ItemCoord c2 = decode_item(p, item2);
-            int py, px, Y0, X0;
-            patch_origin(p, c2, 2 * (2 * c2.tp + qt) + (row >> 6), py, px, Y0, X0);
-            const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
-            const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)token * kR);
-            uint4 v[2] = {__ldg(src), __ldg(src + 1)};
-            uint32_t* w = reinterpret_cast<uint32_t*>(v);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
-                const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
-                w[i] = pack_bf16x2(lo, hi);
-            }
-            uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * 32;
-            const int sw = (row >> 2) & 1;
-            *reinterpret_cast<uint4*>(dst + ((0 ^ sw) << 4)) = v[0];
-            *reinterpret_cast<uint4*>(dst + ((1 ^ sw) << 4)) = v[1];
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kQPos + buf));
-        };
-        if (half == 0) {
-            stage_query_rib(blockIdx.x, 0);
-            if (blockIdx.x + gridDim.x < (unsigned)p.items) stage_query_rib(blockIdx.x + gridDim.x, 1);
-        }
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
             const ItemCoord c = decode_item(p, item);
             float m_used = -INFINITY, l = 0.f;
@@ -342,6 +313,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 // warp-uniform outcome: the TMEM loads below are warp-collective
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
+                bool p_free = blk == 0;       // P (and O) of this half are free once the previous block's PV has completed
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     uint32_t s[32];
@@ -362,7 +334,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         // carries the same reference.
                         const bool need = mx > m_used + rescale_threshold;
                         if (__any_sync(0xffffffffu, need)) {
-                            if (!pv_done_before(blk)) { ok = false; break; }
+                            if (!p_free) {
+                                if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                                tc_fence_after();
+                                p_free = true;
+                            }
                             const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
                             if (need) { l *= factor; m_used = mx; }
                             if (j > 0) {
@@ -388,14 +364,15 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     if (ch == 1) {
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) {
-                            mbar_arrive(bar(kSFree + qt));              // the next block's scores may overwrite the accumulator
-                            mbar_arrive(bar(kKEmpty + blk % kStages));  // and this block's keys are no longer needed
-                        }
+                        if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
                     }
                     uint32_t packed[16];
                     l += exp_chunk(s, -m_used * p.scale_log2, packed);
-                    if (!pv_done_before(blk)) { ok = false; break; }     // P of the previous block has been consumed
+                    if (!p_free) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+                        p_free = true;
+                    }
                     tmem_st16(t_p + 16 * ch, packed);
                 }
                 if (!ok) break;
@@ -405,15 +382,13 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) mbar_arrive(b_ready);
             }
             if (!ok) break;
-            // every S of this tile and item has been read: its query RIB slab may take the item after next
-            if (half == 0 && item + 2 * (int)gridDim.x < p.items) stage_query_rib(item + 2 * gridDim.x, nitem & 1);
             // ---- merge the two key halves and write this thread's 16 output columns
             merge[half * kTile + row] = make_float2(m_used, l);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kMerge + 4 * qt + quarter));
             // both halves' last PV must have completed, and the partner's (m, l) must be there
-            if (!pv_done_before(blk) ||
-                !__all_sync(0xffffffffu, mbar_wait(bar(kPFree + 2 * qt + (half ^ 1)), (blk - 1) & 1, abort_flag, p.status) &&
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + 2 * qt), (blk - 1) & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kPFree + 2 * qt + 1), (blk - 1) & 1, abort_flag, p.status) &&
                                              mbar_wait(bar(kMerge + 4 * qt + quarter), nitem & 1, abort_flag, p.status))) { ok = false; break; }
             tc_fence_after();
             uint32_t oa[16], ob[16];
@@ -453,7 +428,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     // ================================================================================ common tail
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 2) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
