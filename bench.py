@@ -15,6 +15,7 @@ divided by the slowest rank's device time.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -146,8 +147,8 @@ def run_reference(args, wl, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=None, help="prefix of a configuration name (default: cfg2 shape)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -164,7 +165,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2603_06738_b200 import binding, synthetic
+    from paper_2603_06738_b200 import binding, multi, synthetic
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
@@ -177,8 +178,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     # every rank owns a batch of its own (seed offset by rank); pairs are independent
-    my = synthetic.Workload(wl.name, wl.B, wl.H, wl.W, wl.heads, wl.d, wl.r, wl.window, wl.shift,
-                            wl.seed + 1000 * rank, True)
+    my = multi.rank_workload(wl, rank)
     host = {k: v.pin_memory() for k, v in synthetic.make_inputs(my, True).items()}
     step_bytes = sum(host[k].numel() * 2 for k in ("q", "k", "v", "dout")) * 2   # + out, dq, dk, dv
     nsets = max(2, -(-3 * L2_BYTES // step_bytes))
@@ -216,6 +216,8 @@ def main():
     sampler = ClockSampler(local_rank)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     launches0 = binding.rib_kernel_launches()
+    prof_capacity = 5 * args.steps + 8
+    binding.rib_profile_begin(prof_capacity)     # CUDA events around every kernel launch of the library
     sampler.start()
     barrier()
     t_wall0 = time.perf_counter()
@@ -233,6 +235,9 @@ def main():
     sampler.stop_flag.set()
     sampler.join()
     launches = binding.rib_kernel_launches() - launches0
+    per_kernel = {}
+    for kid, ms in binding.rib_profile_end(prof_capacity):
+        per_kernel.setdefault(binding.KERNEL_NAMES.get(kid, str(kid)), []).append(ms)
     status = binding.rib_query_status()
     fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
@@ -272,11 +277,8 @@ def main():
         e2e_ms, h2d, d2h = None, 0, 0
 
     # ------------------------------------------------ reduce over ranks (max time), compose the line
-    times = torch.tensor([total_ms, statistics.median(fwd_ms), statistics.median(bwd_ms), e2e_ms or 0.0],
-                         dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, fwd_med, bwd_med, e2e_ms_max = (float(x) for x in times.tolist())
+    total_ms, fwd_med, bwd_med, e2e_ms_max = multi.max_over_ranks(
+        [total_ms, statistics.median(fwd_ms), statistics.median(bwd_ms), e2e_ms or 0.0], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -285,17 +287,29 @@ def main():
     peaks, peak_kind = load_peaks()
     ms_per_step = total_ms / args.steps
     flops_step = (wl.fwd_flops + wl.bwd_flops) * world
-    value = flops_step / (ms_per_step * 1e-3) / 1e12
+    value = multi.job_throughput(wl.fwd_flops + wl.bwd_flops, ms_per_step, world) / 1e12
     fwd_tf = wl.fwd_flops / (fwd_med * 1e-3) / 1e12
     bwd_tf = wl.bwd_flops / (bwd_med * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
-    dominant = "backward (rib_window_attn_bwd kernels)" if bwd_med >= fwd_med else "forward (rib_window_attn_fwd kernel)"
-    dom_tf = bwd_tf if bwd_med >= fwd_med else fwd_tf
-    traffic_file = ROOT / "profiles" / "traffic.json"
+    # per-kernel device time inside the timed region (rank 0); the dominant kernel is the one with
+    # the largest total; its algorithmic flops per launch are the contraction flops of its pass
+    kernels = {name: {"launches": len(v), "avg_ms": sum(v) / len(v), "total_ms": sum(v)} for name, v in per_kernel.items()}
+    tot = sum(k["total_ms"] for k in kernels.values()) or 1.0
+    for k in kernels.values():
+        k["share"] = k["total_ms"] / tot
+    dominant = max(kernels, key=lambda n: kernels[n]["total_ms"])
+    algo_flops = {"rib_fwd_sm100_kernel": wl.fwd_flops, "generic_fwd_kernel": wl.fwd_flops,
+                  "rib_bwd_sm100_kernel": wl.bwd_flops}.get(dominant)
+    dom_tf = None if algo_flops is None else algo_flops / (kernels[dominant]["avg_ms"] * 1e-3) / 1e12
     traffic = None
+    traffic_file = ROOT / "profiles" / "traffic.json"
     if traffic_file.exists():
         try:
-            traffic = json.loads(traffic_file.read_text()).get("bwd" if bwd_med >= fwd_med else "fwd")
+            rec = json.loads(traffic_file.read_text()).get(dominant)
+            src = ROOT / "paper_2603_06738_b200" / "csrc" / rec["source"]
+            # counters taken on an older version of the kernel say nothing about this one
+            if rec["workload"] == wl.name and hashlib.sha256(src.read_bytes()).hexdigest() == rec["source_sha256"]:
+                traffic = rec["dram_bytes_per_launch"]
         except Exception:
             traffic = None
     line = {
@@ -311,7 +325,10 @@ def main():
         "bwd": {"ms": bwd_med, "tflops": bwd_tf, "frac_of_peak": bwd_tf / peak},
         "frac_of_peak": value / world / peak,
         "roofline": {"bound": "tensor", "kernel": dominant, "achieved": dom_tf, "peak": peak, "unit": "TFLOP/s",
-                     "frac": dom_tf / peak, "traffic": traffic, "peak_source": f"bf16_tflops burst, {peak_kind}"},
+                     "frac": None if dom_tf is None else dom_tf / peak, "traffic": traffic,
+                     "peak_source": f"bf16_tflops burst, {peak_kind}",
+                     "algorithmic_flops_per_launch": algo_flops, "avg_launch_ms": kernels[dominant]["avg_ms"]},
+        "kernels": kernels,
         "e2e": None if e2e_ms is None else {
             "value": flops_step / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_max,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

@@ -142,6 +142,22 @@ int rib_last_path(void);
 /* Number of CUDA kernels this library has launched in this process so far (memsets excluded). */
 long long rib_kernel_launches(void);
 
+/*
+ * Per-kernel device timing, for benchmarks (not part of the method).  Between rib_profile_begin and
+ * rib_profile_end every kernel launch of this library is bracketed by two CUDA events on the launch
+ * stream, up to `max_launches` launches (later ones are not recorded).  rib_profile_end waits for
+ * the recorded events, writes for launch i its kernel id (RIB_KERNEL_*) to kernel_ids[i] and its
+ * device time in milliseconds to ms[i] (at most `capacity` entries), releases the events and
+ * returns the number of entries written, or a negative RIB_ERR_* code.  Both calls create or
+ * destroy CUDA events: keep them outside stream capture and outside timed regions.  One profiling
+ * session per process at a time, driven from one host thread.
+ */
+enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH_DQ = 4,
+       RIB_KERNEL_BWD_FINISH_POS = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
+       RIB_KERNEL_ANY_BWD_DKV = 9 };
+int rib_profile_begin(int max_launches);
+int rib_profile_end(int* kernel_ids, float* ms, int capacity);
+
 #ifdef __cplusplus
 }
 #endif

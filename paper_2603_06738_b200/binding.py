@@ -21,8 +21,11 @@ RIB_PATH_NONE, RIB_PATH_GENERIC, RIB_PATH_SM100 = 0, 1, 2
 EXPORTS = (
     "rib_window_attn_fwd", "rib_window_attn_bwd", "rib_window_attn_bwd_workspace",
     "rib_query_status", "rib_status_string", "rib_set_path", "rib_last_path", "rib_kernel_launches",
-    "rib_window_attn_bwd_noalloc",
+    "rib_window_attn_bwd_noalloc", "rib_profile_begin", "rib_profile_end",
 )
+KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
+                4: "rib_bwd_finish_dq_kernel", 5: "rib_bwd_finish_pos_kernel", 6: "generic_fwd_kernel",
+                7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel"}
 RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
@@ -51,6 +54,10 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_bwd.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
         lib.rib_window_attn_bwd_noalloc.restype = ci
         lib.rib_window_attn_bwd_noalloc.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp]
+        lib.rib_profile_begin.restype = ci
+        lib.rib_profile_begin.argtypes = [ci]
+        lib.rib_profile_end.restype = ci
+        lib.rib_profile_end.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ctypes.c_float), ci]
         lib.rib_window_attn_bwd_workspace.restype = ctypes.c_size_t
         lib.rib_window_attn_bwd_workspace.argtypes = [ci] * 7
         lib.rib_query_status.restype = ci
@@ -102,6 +109,22 @@ def rib_last_path() -> int:
 
 def rib_kernel_launches() -> int:
     return int(library().rib_kernel_launches())
+
+
+def rib_profile_begin(max_launches: int) -> None:
+    rc = int(library().rib_profile_begin(int(max_launches)))
+    if rc != RIB_OK:
+        raise RibError(rc)
+
+
+def rib_profile_end(capacity: int) -> list[tuple[int, float]]:
+    """Ends the per-kernel timing session; returns [(kernel id, device milliseconds), ...] in launch order."""
+    ids = (ctypes.c_int * capacity)()
+    ms = (ctypes.c_float * capacity)()
+    n = int(library().rib_profile_end(ids, ms, capacity))
+    if n < 0:
+        raise RibError(n)
+    return [(int(ids[i]), float(ms[i])) for i in range(n)]
 
 
 def rib_query_status(stream=None) -> int:

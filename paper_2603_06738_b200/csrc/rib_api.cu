@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <mutex>
+#include <vector>
 
 namespace {
 
@@ -48,6 +49,17 @@ size_t rowdot_bytes(int B, int H, int W, int heads)
     return (bytes + 255) & ~(size_t)255;
 }
 
+// ---- per-kernel device timing (rib_profile_begin / rib_profile_end) ------------------------------
+struct ProfileState {
+    std::mutex mutex;
+    bool on = false, pending = false;     // pending: a start event without its stop event yet
+    int capacity = 0, count = 0;          // launches
+    std::vector<cudaEvent_t> events;      // 2 per launch
+    std::vector<int> ids;
+};
+ProfileState g_profile;
+std::atomic<bool> g_profile_on{false};
+
 // ---- built-in scratch of rib_window_attn_bwd_noalloc -------------------------------------------
 // Lives in the library image: every device that loads the library holds these bytes until exit.
 // In host code the name below is only a handle for cudaGetSymbolAddress, never a device pointer.
@@ -74,7 +86,69 @@ int noalloc_scratch_ptr(void** out)
 
 }  // namespace
 
+namespace rib {
+
+void profile_mark(int kernel_id, int phase, cudaStream_t stream)
+{
+    if (!g_profile_on.load(std::memory_order_relaxed)) return;
+    std::lock_guard<std::mutex> lock(g_profile.mutex);
+    if (!g_profile.on) return;
+    if (phase == 0) {
+        if (g_profile.count >= g_profile.capacity) return;
+        g_profile.ids[g_profile.count] = kernel_id;
+        cudaEventRecord(g_profile.events[2 * g_profile.count], stream);
+        g_profile.pending = true;
+    } else if (g_profile.pending) {
+        cudaEventRecord(g_profile.events[2 * g_profile.count + 1], stream);
+        ++g_profile.count;
+        g_profile.pending = false;
+    }
+}
+
+}  // namespace rib
+
 extern "C" {
+
+int rib_profile_begin(int max_launches)
+{
+    if (max_launches <= 0 || max_launches > (1 << 20)) return RIB_ERR_SHAPE;
+    std::lock_guard<std::mutex> lock(g_profile.mutex);
+    if (g_profile.on) return RIB_ERR_UNSUPPORTED;
+    g_profile.events.assign(2 * (size_t)max_launches, nullptr);
+    g_profile.ids.assign((size_t)max_launches, 0);
+    for (auto& e : g_profile.events)
+        if (cudaEventCreate(&e) != cudaSuccess) {
+            for (auto& d : g_profile.events) if (d) cudaEventDestroy(d);
+            g_profile.events.clear();
+            return RIB_ERR_CUDA;
+        }
+    g_profile.capacity = max_launches;
+    g_profile.count = 0;
+    g_profile.pending = false;
+    g_profile.on = true;
+    g_profile_on.store(true);
+    return RIB_OK;
+}
+
+int rib_profile_end(int* kernel_ids, float* ms, int capacity)
+{
+    std::lock_guard<std::mutex> lock(g_profile.mutex);
+    if (!g_profile.on) return RIB_ERR_UNSUPPORTED;
+    g_profile_on.store(false);
+    g_profile.on = false;
+    int written = 0, rc = RIB_OK;
+    for (int i = 0; i < g_profile.count; ++i) {
+        float t = 0.f;
+        if (cudaEventSynchronize(g_profile.events[2 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&t, g_profile.events[2 * i], g_profile.events[2 * i + 1]) != cudaSuccess) { rc = RIB_ERR_CUDA; break; }
+        if (kernel_ids && ms && written < capacity) { kernel_ids[written] = g_profile.ids[i]; ms[written] = t; ++written; }
+    }
+    for (auto& e : g_profile.events) cudaEventDestroy(e);
+    g_profile.events.clear();
+    g_profile.ids.clear();
+    g_profile.capacity = g_profile.count = 0;
+    return rc == RIB_OK ? written : rc;
+}
 
 int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void* pq, const void* pk,
                         int B, int H, int W, int heads, int d, int r, int window, int shift,

@@ -540,7 +540,7 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     ap.inv_sqrt_r = 1.f / sqrtf((float)p.r);
     const size_t tokens = (size_t)p.pairs * p.n;
     const unsigned aux_blocks = (unsigned)((tokens + 255) / 256);
-    rib_bwd_prepare_kernel<<<aux_blocks, 256, 0, stream>>>(ap);
+    { ProfileScope scope(RIB_KERNEL_BWD_PREPARE, stream); rib_bwd_prepare_kernel<<<aux_blocks, 256, 0, stream>>>(ap); }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
@@ -552,17 +552,17 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
-    rib_bwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp);
+    { ProfileScope scope(RIB_KERNEL_BWD_MAIN, stream); rib_bwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
-    rib_bwd_finish_dq_kernel<<<aux_blocks, 256, 0, stream>>>(ap);
+    { ProfileScope scope(RIB_KERNEL_BWD_FINISH_DQ, stream); rib_bwd_finish_dq_kernel<<<aux_blocks, 256, 0, stream>>>(ap); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int groups = p.pairs < 16 ? p.pairs : 16;
     const int per_group = (p.pairs + groups - 1) / groups;
     dim3 grid_pos((unsigned)(p.n / 128 * 32), (unsigned)((p.pairs + per_group - 1) / per_group));
-    rib_bwd_finish_pos_kernel<<<grid_pos, 128, 0, stream>>>(ap, per_group);
+    { ProfileScope scope(RIB_KERNEL_BWD_FINISH_POS, stream); rib_bwd_finish_pos_kernel<<<grid_pos, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();
 }
 

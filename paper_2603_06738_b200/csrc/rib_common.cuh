@@ -1,6 +1,7 @@
 // Shared declarations of the RIB window-attention CUDA library (internal; the public surface is
 // include/rib_window_attn.h).
 #pragma once
+#include "../../include/rib_window_attn.h"
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stddef.h>
@@ -44,6 +45,15 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
 bool sm100_bwd_supported(const Problem& p);
 size_t sm100_bwd_workspace_bytes(long long pairs, int n);
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 4 kernels
+
+// Per-kernel device timing (off unless rib_profile_begin was called): records a CUDA event on
+// `stream` before (phase 0) and after (phase 1) the launch of kernel `kernel_id` (RIB_KERNEL_*).
+void profile_mark(int kernel_id, int phase, cudaStream_t stream);
+struct ProfileScope {
+    int id; cudaStream_t stream;
+    ProfileScope(int kernel_id, cudaStream_t s) : id(kernel_id), stream(s) { profile_mark(id, 0, stream); }
+    ~ProfileScope() { profile_mark(id, 1, stream); }
+};
 
 // Window partition with cyclic shift: token i = y*M + x of window (wy, wx) -> image pixel.
 __host__ __device__ inline void token_pixel(int H, int W, int M, int s, int wy, int wx, int i,

@@ -464,7 +464,7 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
     fp.inv_sqrt_d = 1.f / sqrtf((float)p.d);
     fp.pos_scale = sqrtf((float)p.d / (float)p.r);
     const int grid = fp.items < sm_count ? fp.items : sm_count;
-    rib_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp);
+    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
     return cudaGetLastError();
 }
 

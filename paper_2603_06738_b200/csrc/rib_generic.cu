@@ -350,14 +350,14 @@ cudaError_t generic_fwd(const Problem& p, cudaStream_t stream)
     cudaError_t e = set_smem(generic_fwd_kernel, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(p.pairs, (p.n + kRows - 1) / kRows);
-    generic_fwd_kernel<<<grid, kThreads, smem, stream>>>(p);
+    { ProfileScope scope(RIB_KERNEL_ANY_FWD, stream); generic_fwd_kernel<<<grid, kThreads, smem, stream>>>(p); }
     return cudaGetLastError();
 }
 
 cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream)
 {
     const size_t items = (size_t)p.B * p.H * p.W * p.heads;
-    rowdot_kernel<<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(p, items);
+    { ProfileScope scope(RIB_KERNEL_ANY_ROWDOT, stream); rowdot_kernel<<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(p, items); }
     return cudaGetLastError();
 }
 
@@ -375,14 +375,14 @@ cudaError_t generic_bwd(const Problem& p, cudaStream_t stream)
                                            (size_t)kRows * p.d + (size_t)kRows * kTile);
     e = set_smem(generic_bwd_dq_kernel, smem_q);
     if (e != cudaSuccess) return e;
-    generic_bwd_dq_kernel<<<grid, kThreads, smem_q, stream>>>(p);
+    { ProfileScope scope(RIB_KERNEL_ANY_BWD_DQ, stream); generic_bwd_dq_kernel<<<grid, kThreads, smem_q, stream>>>(p); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t smem_k = sizeof(float) * ((size_t)kTile * (dk | 1) + (size_t)kTile * (p.d | 1) + 2 * (size_t)kTile +
                                            (size_t)kRows * dk + (size_t)kRows * p.d + 2 * (size_t)kRows * kTile);
     e = set_smem(generic_bwd_dkv_kernel, smem_k);
     if (e != cudaSuccess) return e;
-    generic_bwd_dkv_kernel<<<grid, kThreads, smem_k, stream>>>(p);
+    { ProfileScope scope(RIB_KERNEL_ANY_BWD_DKV, stream); generic_bwd_dkv_kernel<<<grid, kThreads, smem_k, stream>>>(p); }
     return cudaGetLastError();
 }
 
