@@ -18,9 +18,11 @@
 // bf16 and sums the RIB columns over pairs into dPq.  The RIB columns of dK~ are written per pair
 // and summed over pairs by the same finishing kernel into dPk.
 //
-// Roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocator, warps 4-11
-// P/dS arithmetic (two warpgroups, each half of the tile's columns), warps 12-15 drain dQ~ after every
-// tile and dK~/dV after every item.  Every wait is bounded.
+// Roles (512 threads): warp 0 TMA producer; three MMA-issuing threads, because one thread issuing
+// all 45 contractions of a tile was the bottleneck and the tensor pipe takes instructions from several
+// warps at once: warp 1 issues S^T and dP^T, warp 2 (also the TMEM allocator) dV and dK~, warp 3 dQ~;
+// warps 4-11 P/dS arithmetic (two warpgroups, each half of the tile's columns), warps 12-15 drain dQ~
+// after every tile and dK~/dV after every item.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -44,7 +46,7 @@ constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 halve
 constexpr uint32_t kDSHalf = kTile * 128;
 constexpr uint32_t kOffBar = kOffDS + 2 * kDSHalf;
 enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kPReady,
-           kPFree, kDQFull, kDQFree, kAccFull, kAccFree, kDrain, kNumBars };
+           kPFree, kDQFull, kDQFree, kAccFull, kAccFree, kDrain, kNumBars = kDrain + 3 };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;
 constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
 static_assert(kOffRing % 1024 == 0 && kRingBytes % 1024 == 0 && kOffDS % 1024 == 0, "swizzle atoms need aligned tiles");
@@ -105,10 +107,10 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
         for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
-        mbar_init(bar(kSFull), 1); mbar_init(bar(kPReady), 8); mbar_init(bar(kPFree), 1);
+        mbar_init(bar(kSFull), 1); mbar_init(bar(kPReady), 8); mbar_init(bar(kPFree), 2);
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
         mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
-        mbar_init(bar(kDrain), 1);
+        for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
         fence_barrier_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
         prefetch_tensormap(&tm_do); prefetch_tensormap(&tm_pqs); prefetch_tensormap(&tm_pk);
@@ -166,87 +168,90 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     mbar_wait(bar(kQFull + b2 % kQStages), (b2 / kQStages) & 1, abort_flag + 1, p.status);
             }
         }
-    } else if (warp == 1) {
-        // ============================================================== MMA issuer (one thread)
+    } else if (warp < 4) {
+        // ==================================================== MMA issuers (one thread per warp 1-3)
         if (lane == 0) {
-            // S^T and dP^T of one tile: key slot `slot`, ring stage `st`
-            auto issue_scores = [&](uint32_t slot, uint32_t st) {
-                const uint32_t kc = base + kOffKc + slot * kContentBytes, kp = base + kOffKp + slot * kPosBytes;
-                const uint32_t v = base + kOffV + slot * kContentBytes;
-                const uint32_t ring = base + kOffRing + st * kRingBytes;
-                const uint32_t qc = ring + kRingQc, qp = ring + kRingQp, go = ring + kRingDO;
-                mma_ss(tmem + kColS, smem_desc(kc, 16, 512, kSwizzle64B), smem_desc(qc, 16, 512, kSwizzle64B), kIdescSS, 0);
-                mma_ss(tmem + kColS, smem_desc(kc + 32, 16, 512, kSwizzle64B), smem_desc(qc + 32, 16, 512, kSwizzle64B), kIdescSS, 1);
-                mma_ss(tmem + kColS, smem_desc(kp, 16, 256, kSwizzle32B), smem_desc(qp, 16, 256, kSwizzle32B), kIdescSS, 1);
-                mma_ss(tmem + kColDP, smem_desc(v, 16, 512, kSwizzle64B), smem_desc(go, 16, 512, kSwizzle64B), kIdescSS, 0);
-                mma_ss(tmem + kColDP, smem_desc(v + 32, 16, 512, kSwizzle64B), smem_desc(go + 32, 16, 512, kSwizzle64B), kIdescSS, 1);
-            };
-            // dV_J, dK~_J (accumulating over the item) and dQ~_I (fresh every tile)
-            auto issue_grads = [&](uint32_t slot, uint32_t st, bool accumulate) {
-                const uint32_t kc = base + kOffKc + slot * kContentBytes, kp = base + kOffKp + slot * kPosBytes;
-                const uint32_t ring = base + kOffRing + st * kRingBytes;
-                const uint32_t qc = ring + kRingQc, qp = ring + kRingQp, go = ring + kRingDO;
-                const uint32_t ds = base + kOffDS;
-                for (int kk = 0; kk < kTile / 16; ++kk)      // K = 16 queries per step
-                    mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, smem_desc(go + 1024 * kk, 16, 512, kSwizzle64B),
-                           kIdescT32, (accumulate || kk) ? 1u : 0u);
-                for (int kk = 0; kk < kTile / 16; ++kk) {
-                    mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, smem_desc(qc + 1024 * kk, 16, 512, kSwizzle64B),
-                           kIdescT32, (accumulate || kk) ? 1u : 0u);
-                    mma_ts(tmem + kColDK + kD, tmem + kColDS + 8 * kk, smem_desc(qp + 512 * kk, 16, 256, kSwizzle32B),
-                           kIdescT16, (accumulate || kk) ? 1u : 0u);
-                }
-                for (int kk = 0; kk < kTile / 16; ++kk) {    // K = 16 keys per step
-                    const uint64_t a = smem_desc(ds + 2048 * kk, kDSHalf, 1024, kSwizzle128B);
-                    mma_ss(tmem + kColDQ, a, smem_desc(kc + 1024 * kk, 16, 512, kSwizzle64B), kIdescQ32, kk ? 1u : 0u);
-                    mma_ss(tmem + kColDQ + kD, a, smem_desc(kp + 512 * kk, 16, 256, kSwizzle32B), kIdescQ16, kk ? 1u : 0u);
-                }
-            };
+            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
+            constexpr uint64_t kDescDS = smem_desc_const(kDSHalf, 1024, kSwizzle128B);
             int item = blockIdx.x, I = 0;
             uint32_t nitem = 0, g = 0;
-            bool valid = item < p.items, ok = true;
-            if (valid) {
-                ok = mbar_wait(bar(kKVFull), 0, abort_flag, p.status) && mbar_wait(bar(kQFull), 0, abort_flag, p.status);
-                if (ok) {
-                    tc_fence_after();
-                    issue_scores(0, 0);
-                    mma_commit(bar(kSFull));
+            bool ok = true;
+            if (warp == 1) {
+                // ---- S^T = K~_J Q~_I^T and dP^T = V_J dO_I^T, as soon as the arithmetic warps have taken
+                // the previous tile's scores out of tensor memory
+                for (; item < p.items && ok; item += gridDim.x, ++nitem) {
+                    const uint32_t slot = nitem & 1;
+                    if (!mbar_wait(bar(kKVFull + slot), (nitem >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + slot * kContentBytes);
+                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + slot * kPosBytes);
+                    const uint64_t v = smem_desc_at(kDesc64, base + kOffV + slot * kContentBytes);
+                    for (I = 0; I < p.nblk; ++I, ++g) {
+                        const uint32_t st = g % kQStages;
+                        if (!mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) ||
+                            (g > 0 && !mbar_wait(bar(kPReady), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t ring = base + kOffRing + st * kRingBytes;
+                        const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc32, ring + kRingQp);
+                        const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
+                        mma_ss(tmem + kColS, kc, qc, kIdescSS, 0u);
+                        mma_ss(tmem + kColS, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
+                        mma_ss(tmem + kColS, kp, qp, kIdescSS, 1u);
+                        mma_ss(tmem + kColDP, v, go, kIdescSS, 0u);
+                        mma_ss(tmem + kColDP, v + 2, go + 2, kIdescSS, 1u);
+                        mma_commit(bar(kSFull));
+                    }
                 }
-            }
-            while (valid && ok) {
-                int item2 = item, I2 = I + 1;
-                uint32_t nitem2 = nitem;
-                if (I2 == p.nblk) { I2 = 0; item2 += gridDim.x; ++nitem2; }
-                const bool valid2 = item2 < p.items;
-                const uint32_t slot = nitem & 1, st = g % kQStages;
-                if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status)) { ok = false; break; }
-                tc_fence_after();
-                if (valid2) {
-                    // next tile's S^T, dP^T first: the arithmetic warps start on them while the
-                    // three gradient contractions of this tile run
-                    const uint32_t st2 = (g + 1) % kQStages;
-                    if (I2 == 0 && !mbar_wait(bar(kKVFull + (nitem2 & 1)), (nitem2 >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                    if (!mbar_wait(bar(kQFull + st2), ((g + 1) / kQStages) & 1, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_scores(nitem2 & 1, st2);
-                    mma_commit(bar(kSFull));
+            } else if (warp == 2) {
+                // ---- dV_J += P^T dO_I and dK~_J += dS^T Q~_I (A from tensor memory, 16 queries per step)
+                for (; item < p.items && ok; item += gridDim.x, ++nitem) {
+                    for (I = 0; I < p.nblk; ++I, ++g) {
+                        const uint32_t st = g % kQStages;
+                        if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status) ||
+                            (I == 0 && nitem > 0 && !mbar_wait(bar(kAccFree), (nitem - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t ring = base + kOffRing + st * kRingBytes;
+                        const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc32, ring + kRingQp);
+                        const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
+                        const uint32_t acc0 = I > 0 ? 1u : 0u;
+#pragma unroll
+                        for (int kk = 0; kk < kTile / 16; ++kk)
+                            mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, go + 64 * kk, kIdescT32, kk ? 1u : acc0);
+#pragma unroll
+                        for (int kk = 0; kk < kTile / 16; ++kk) {
+                            mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, qc + 64 * kk, kIdescT32, kk ? 1u : acc0);
+                            mma_ts(tmem + kColDK + kD, tmem + kColDS + 8 * kk, qp + 32 * kk, kIdescT16, kk ? 1u : acc0);
+                        }
+                        mma_commit(bar(kPFree));
+                        mma_commit(bar(kQEmpty + st));
+                        if (I == p.nblk - 1) mma_commit(bar(kAccFull));
+                    }
                 }
-                if (I == 0 && nitem > 0 && !mbar_wait(bar(kAccFree), (nitem - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                if (g > 0 && !mbar_wait(bar(kDQFree), (g - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                tc_fence_after();
-                issue_grads(slot, st, I > 0);
-                mma_commit(bar(kPFree));
-                mma_commit(bar(kDQFull));
-                mma_commit(bar(kQEmpty + st));
-                if (I == p.nblk - 1) {
-                    mma_commit(bar(kAccFull));
-                    mma_commit(bar(kKVEmpty + slot));
+            } else {
+                // ---- dQ~_I = dS K~_J (A = dS through shared memory, 16 keys per step)
+                const uint64_t ds = smem_desc_at(kDescDS, base + kOffDS);
+                for (; item < p.items && ok; item += gridDim.x, ++nitem) {
+                    const uint32_t slot = nitem & 1;
+                    const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + slot * kContentBytes);
+                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + slot * kPosBytes);
+                    for (I = 0; I < p.nblk; ++I, ++g) {
+                        if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status) ||
+                            (g > 0 && !mbar_wait(bar(kDQFree), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int kk = 0; kk < kTile / 16; ++kk) {
+                            mma_ss(tmem + kColDQ, ds + 128 * kk, kc + 64 * kk, kIdescQ32, kk ? 1u : 0u);
+                            mma_ss(tmem + kColDQ + kD, ds + 128 * kk, kp + 32 * kk, kIdescQ16, kk ? 1u : 0u);
+                        }
+                        mma_commit(bar(kPFree));
+                        mma_commit(bar(kDQFull));
+                        // K~_J and V_J may go once the item's last dQ~ is done (S^T, dP^T finished before it)
+                        if (I == p.nblk - 1) mma_commit(bar(kKVEmpty + slot));
+                    }
                 }
-                item = item2; I = I2; nitem = nitem2; valid = valid2; ++g;
             }
             // everything issued by this thread must have finished before TMEM is released
-            mma_commit(bar(kDrain));
-            mbar_wait(bar(kDrain), 0, abort_flag + 1, p.status);
+            mma_commit(bar(kDrain + warp - 1));
+            mbar_wait(bar(kDrain + warp - 1), 0, abort_flag + 1, p.status);
         }
     } else if (warp >= 4 && warp < 12) {
         // ===================== P^T and dS^T: one thread per key row, one warpgroup per 64 queries
