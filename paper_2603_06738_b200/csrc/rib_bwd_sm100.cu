@@ -10,9 +10,12 @@
 //     S^T  = K~_J Q~_I^T                    (M128 N128 K48: content rows 2 x K16, RIB rows 1 x K16)
 //     dP^T = V_J dO_I^T                     (M128 N128 K32)
 //     P^T  = exp2(S^T * log2e/sqrt(d) - lse_i * log2e),   dS^T = P^T o (dP^T - D_i)     (ALU warps)
-//     dV_J  += P^T  dO_I                    (A from TMEM, B = dO tile, MN-major)
-//     dK~_J += dS^T Q~_I                    (A from TMEM, B = Q content / RIB slabs, MN-major)
-//     dQ~_I  = dS K~_J                      (A = dS through shared memory, MN-major, B = K~ slabs)
+//     dV_J  += P^T  dO_I                    (A from TMEM, B = dO tile, MN-major, N = 32)
+//     dK~_J += dS^T Q~_I                    (A from TMEM, B = [Q content | Q RIB] tiles, MN-major, N = 48)
+//     dQ~_I  = dS K~_J                      (A = dS through shared memory, MN-major, B = [K | Pk] tiles, N = 48)
+// The RIB rows are fetched as zero-padded 64-byte rows, so that a RIB tile has the layout of a content
+// tile and the concatenation of Eq. 5 is, for the MN-major operands, one descriptor whose second
+// 32-column atom is the RIB tile: every contraction step is a single instruction.
 // dQ~_I is one key block's share of the query gradient: it is added (fp32 red) into a workspace laid
 // out [pair][column][token in window order] and finished by a small kernel that converts dq to
 // bf16 and sums the RIB columns over pairs into dPq.  The RIB columns of dK~ are written per pair
@@ -36,16 +39,16 @@ constexpr int kDk = kD + kR;          // 48 columns of dQ~ / dK~
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffKc = 0;                                   // [2] key content (one slot per item in flight)
-constexpr uint32_t kOffKp = kOffKc + 2 * kContentBytes;          // [2] key RIB rows
-constexpr uint32_t kOffV = kOffKp + 2 * kPosBytes;               // [2] values
+constexpr uint32_t kOffKp = kOffKc + 2 * kContentBytes;          // [2] key RIB rows, padded to 64 bytes
+constexpr uint32_t kOffV = kOffKp + 2 * kContentBytes;           // [2] values
 constexpr uint32_t kOffRing = kOffV + 2 * kContentBytes;
 constexpr uint32_t kLdBytes = kTile * 8;                         // 128 x (-lse*log2e, D)
-constexpr uint32_t kRingQc = 0, kRingQp = kContentBytes, kRingDO = kRingQp + kPosBytes, kRingLD = kRingDO + kContentBytes;
-constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 21504
+constexpr uint32_t kRingQc = 0, kRingQp = kContentBytes, kRingDO = kRingQp + kContentBytes, kRingLD = kRingDO + kContentBytes;
+constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 25600
 constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
 constexpr uint32_t kDSHalf = kTile * 128;
 constexpr uint32_t kOffBar = kOffDS + 2 * kDSHalf;
-enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kPReady,
+enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kSIssued, kPReady,
            kPFree, kDQFull, kDQFree, kAccFull, kAccFree, kDrain, kNumBars = kDrain + 3 };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;
 constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
@@ -57,9 +60,8 @@ constexpr uint32_t kTmemCols = 512;
 
 constexpr uint32_t kIdescSS = idesc_bf16_f32(kTile, kTile, false);            // S^T, dP^T: both operands K-major
 constexpr uint32_t kIdescT32 = idesc_bf16_f32(kTile, kD, true);               // A in TMEM, B MN-major, N = 32
-constexpr uint32_t kIdescT16 = idesc_bf16_f32(kTile, kR, true);               // A in TMEM, B MN-major, N = 16
-constexpr uint32_t kIdescQ32 = idesc_bf16_f32_ab(kTile, kD, true, true);      // dQ~: A and B MN-major
-constexpr uint32_t kIdescQ16 = idesc_bf16_f32_ab(kTile, kR, true, true);
+constexpr uint32_t kIdescT48 = idesc_bf16_f32(kTile, kDk, true);              // A in TMEM, B MN-major, N = 48
+constexpr uint32_t kIdescQ48 = idesc_bf16_f32_ab(kTile, kDk, true, true);     // dQ~: A and B MN-major, N = 48
 
 struct BwdParams {
     const float2* ld;          // [pairs][n] window order: (-lse * log2e, D)
@@ -107,7 +109,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
         for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
-        mbar_init(bar(kSFull), 1); mbar_init(bar(kPReady), 8); mbar_init(bar(kPFree), 2);
+        mbar_init(bar(kSFull), 1); mbar_init(bar(kSIssued), 1); mbar_init(bar(kPReady), 8); mbar_init(bar(kPFree), 2);
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
         mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
         for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
@@ -133,14 +135,14 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const ItemCoord c = decode_item(p, item);
                 const uint32_t slot = nitem & 1;
                 if (nitem >= 2 && !mbar_wait(bar(kKVEmpty + slot), ((nitem >> 1) - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                mbar_arrive_expect_tx(bar(kKVFull + slot), 2 * kContentBytes + kPosBytes);
+                mbar_arrive_expect_tx(bar(kKVFull + slot), 3 * kContentBytes);
                 ++kv_armed;
                 for (int sub = 0; sub < 2; ++sub) {
                     int py, px, Y0, X0;
                     patch_origin(geom, c.wy, c.wx, 2 * c.J + sub, py, px, Y0, X0);
                     tma_load_5d(base + kOffKc + slot * kContentBytes + sub * kPatchContent, &tm_k, bar(kKVFull + slot),
                                 0, c.h, X0, Y0, c.b);
-                    tma_load_3d(base + kOffKp + slot * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKVFull + slot), 0, px, py);
+                    tma_load_3d(base + kOffKp + slot * kContentBytes + sub * kPatchContent, &tm_pk, bar(kKVFull + slot), 0, px, py);
                     tma_load_5d(base + kOffV + slot * kContentBytes + sub * kPatchContent, &tm_v, bar(kKVFull + slot),
                                 0, c.h, X0, Y0, c.b);
                 }
@@ -154,7 +156,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         int py, px, Y0, X0;
                         patch_origin(geom, c.wy, c.wx, 2 * I + sub, py, px, Y0, X0);
                         tma_load_5d(ring + kRingQc + sub * kPatchContent, &tm_q, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
-                        tma_load_3d(ring + kRingQp + sub * kPatchPos, &tm_pqs, bar(kQFull + st), 0, px, py);
+                        tma_load_3d(ring + kRingQp + sub * kPatchContent, &tm_pqs, bar(kQFull + st), 0, px, py);
                         tma_load_5d(ring + kRingDO + sub * kPatchContent, &tm_do, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
                     }
                     bulk_load_1d(ring + kRingLD, p.ld + (size_t)c.pair * p.n + (size_t)I * kTile, kLdBytes, bar(kQFull + st));
@@ -171,10 +173,14 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     } else if (warp < 4) {
         // ==================================================== MMA issuers (one thread per warp 1-3)
         if (lane == 0) {
-            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
+            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B);
+            // MN-major operands of 48 columns: the content tile and, one leading-dimension step further, the RIB tile
+            constexpr uint64_t kDescQ48 = smem_desc_const(kRingQp - kRingQc, 512, kSwizzle64B);
+            constexpr uint64_t kDescK48 = smem_desc_const(kOffKp - kOffKc, 512, kSwizzle64B);
             constexpr uint64_t kDescDS = smem_desc_const(kDSHalf, 1024, kSwizzle128B);
             int item = blockIdx.x, I = 0;
             uint32_t nitem = 0, g = 0;
+            const uint32_t total_tiles = (((uint32_t)p.items - blockIdx.x + gridDim.x - 1) / gridDim.x) * (uint32_t)p.nblk;
             bool ok = true;
             if (warp == 1) {
                 // ---- S^T = K~_J Q~_I^T and dP^T = V_J dO_I^T, as soon as the arithmetic warps have taken
@@ -183,7 +189,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint32_t slot = nitem & 1;
                     if (!mbar_wait(bar(kKVFull + slot), (nitem >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
                     const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + slot * kContentBytes);
-                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + slot * kPosBytes);
+                    const uint64_t kp = smem_desc_at(kDesc64, base + kOffKp + slot * kContentBytes);
                     const uint64_t v = smem_desc_at(kDesc64, base + kOffV + slot * kContentBytes);
                     for (I = 0; I < p.nblk; ++I, ++g) {
                         const uint32_t st = g % kQStages;
@@ -191,7 +197,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             (g > 0 && !mbar_wait(bar(kPReady), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t ring = base + kOffRing + st * kRingBytes;
-                        const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc32, ring + kRingQp);
+                        const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc64, ring + kRingQp);
                         const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
                         mma_ss(tmem + kColS, kc, qc, kIdescSS, 0u);
                         mma_ss(tmem + kColS, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
@@ -199,6 +205,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         mma_ss(tmem + kColDP, v, go, kIdescSS, 0u);
                         mma_ss(tmem + kColDP, v + 2, go + 2, kIdescSS, 1u);
                         mma_commit(bar(kSFull));
+                        if (g > 0) mbar_arrive(bar(kSIssued));      // the gradient contractions of tile g - 1 may follow
                     }
                 }
             } else if (warp == 2) {
@@ -210,17 +217,17 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             (I == 0 && nitem > 0 && !mbar_wait(bar(kAccFree), (nitem - 1) & 1, abort_flag, p.status))) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t ring = base + kOffRing + st * kRingBytes;
-                        const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc32, ring + kRingQp);
+                        const uint64_t q48 = smem_desc_at(kDescQ48, ring + kRingQc);
                         const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
                         const uint32_t acc0 = I > 0 ? 1u : 0u;
+                        // let the next tile's S^T, dP^T into the tensor pipe first: the arithmetic warps wait for them
+                        if (g + 1 < total_tiles && !mbar_wait(bar(kSIssued), g & 1, abort_flag, p.status)) { ok = false; break; }
 #pragma unroll
                         for (int kk = 0; kk < kTile / 16; ++kk)
                             mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, go + 64 * kk, kIdescT32, kk ? 1u : acc0);
 #pragma unroll
-                        for (int kk = 0; kk < kTile / 16; ++kk) {
-                            mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, qc + 64 * kk, kIdescT32, kk ? 1u : acc0);
-                            mma_ts(tmem + kColDK + kD, tmem + kColDS + 8 * kk, qp + 32 * kk, kIdescT16, kk ? 1u : acc0);
-                        }
+                        for (int kk = 0; kk < kTile / 16; ++kk)
+                            mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, q48 + 64 * kk, kIdescT48, kk ? 1u : acc0);
                         mma_commit(bar(kPFree));
                         mma_commit(bar(kQEmpty + st));
                         if (I == p.nblk - 1) mma_commit(bar(kAccFull));
@@ -231,17 +238,15 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint64_t ds = smem_desc_at(kDescDS, base + kOffDS);
                 for (; item < p.items && ok; item += gridDim.x, ++nitem) {
                     const uint32_t slot = nitem & 1;
-                    const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + slot * kContentBytes);
-                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + slot * kPosBytes);
+                    const uint64_t k48 = smem_desc_at(kDescK48, base + kOffKc + slot * kContentBytes);
                     for (I = 0; I < p.nblk; ++I, ++g) {
                         if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status) ||
-                            (g > 0 && !mbar_wait(bar(kDQFree), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                            (g > 0 && !mbar_wait(bar(kDQFree), (g - 1) & 1, abort_flag, p.status)) ||
+                            (g + 1 < total_tiles && !mbar_wait(bar(kSIssued), g & 1, abort_flag, p.status))) { ok = false; break; }
                         tc_fence_after();
 #pragma unroll
-                        for (int kk = 0; kk < kTile / 16; ++kk) {
-                            mma_ss(tmem + kColDQ, ds + 128 * kk, kc + 64 * kk, kIdescQ32, kk ? 1u : 0u);
-                            mma_ss(tmem + kColDQ + kD, ds + 128 * kk, kp + 32 * kk, kIdescQ16, kk ? 1u : 0u);
-                        }
+                        for (int kk = 0; kk < kTile / 16; ++kk)
+                            mma_ss(tmem + kColDQ, ds + 128 * kk, k48 + 64 * kk, kIdescQ48, kk ? 1u : 0u);
                         mma_commit(bar(kPFree));
                         mma_commit(bar(kDQFull));
                         // K~_J and V_J may go once the item's last dQ~ is done (S^T, dP^T finished before it)
@@ -525,7 +530,8 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 
     CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
-        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map(&tm_pqs, pq_scaled, p) || !encode_pos_map(&tm_pk, p.pk, p))
+        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p) ||
+        !encode_pos_map_padded(&tm_pk, p.pk, p))
         return cudaErrorInvalidValue;
     static int sm_count = 0;
     if (!sm_count) {

@@ -91,6 +91,20 @@ inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p)
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same features fetched as 64-byte rows: the box is 32 elements wide on a 16-element dimension, so
+// TMA fills the upper half of every row with zeros.  A 64-byte-row RIB tile has the layout of a content
+// tile (SWIZZLE_64B) and can sit behind it as the second 32-column atom of one MN-major operand.
+inline bool encode_pos_map_padded(CUtensorMap* map, const void* ptr, const Problem& p)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M};
+    const cuuint64_t strides[2] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M};
+    const cuuint32_t box[3] = {(cuuint32_t)kD, 8, 8};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline cudaError_t sm_count_of_current_device(int* count)
 {
     int dev = 0;
