@@ -21,11 +21,12 @@
 // bf16 and sums the RIB columns over pairs into dPq.  The RIB columns of dK~ are written per pair
 // and summed over pairs by the same finishing kernel into dPk.
 //
-// Roles (512 threads): warp 0 TMA producer; three MMA-issuing threads, because one thread issuing
-// all 45 contractions of a tile was the bottleneck and the tensor pipe takes instructions from several
+// Roles (768 threads): warp 0 TMA producer; three MMA-issuing threads, because one thread issuing
+// all contractions of a tile was the bottleneck and the tensor pipe takes instructions from several
 // warps at once: warp 1 issues S^T and dP^T, warp 2 (also the TMEM allocator) dV and dK~, warp 3 dQ~;
-// warps 4-11 P/dS arithmetic (two warpgroups, each half of the tile's columns), warps 12-15 drain dQ~
-// after every tile and dK~/dV after every item.  Every wait is bounded.
+// warps 4-19 P/dS arithmetic (four warpgroups, each a quarter of the tile's columns: four warps per SM
+// sub-partition hide each other's tensor-memory and barrier latencies), warps 20-23 drain dQ~ after
+// every tile and dK~/dV after every item.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -34,7 +35,7 @@ namespace {
 using namespace sm100;
 
 constexpr int kQStages = 3;           // ring of query-side tiles (Q content, Q RIB rows, dO, lse/D)
-constexpr int kThreads = 512;
+constexpr int kThreads = 768;
 constexpr int kDk = kD + kR;          // 48 columns of dQ~ / dK~
 
 // shared-memory map (offsets from a 1024-byte aligned base)
@@ -42,7 +43,7 @@ constexpr uint32_t kOffKc = 0;                                   // [2] key cont
 constexpr uint32_t kOffKp = kOffKc + 2 * kContentBytes;          // [2] key RIB rows, padded to 64 bytes
 constexpr uint32_t kOffV = kOffKp + 2 * kContentBytes;           // [2] values
 constexpr uint32_t kOffRing = kOffV + 2 * kContentBytes;
-constexpr uint32_t kLdBytes = kTile * 8;                         // 128 x (-lse*log2e, D)
+constexpr uint32_t kLdBytes = kTile * 8;                         // 64 query pairs x (-lse2, -lse2', -D, -D')
 constexpr uint32_t kRingQc = 0, kRingQp = kContentBytes, kRingDO = kRingQp + kContentBytes, kRingLD = kRingDO + kContentBytes;
 constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 25600
 constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
@@ -64,7 +65,7 @@ constexpr uint32_t kIdescT48 = idesc_bf16_f32(kTile, kDk, true);              //
 constexpr uint32_t kIdescQ48 = idesc_bf16_f32_ab(kTile, kDk, true, true);     // dQ~: A and B MN-major, N = 48
 
 struct BwdParams {
-    const float2* ld;          // [pairs][n] window order: (-lse * log2e, D)
+    const float2* ld;          // [pairs][n / 2] window order, per query pair: (-lse2, -lse2', -D, -D') as two float2
     float* dq_acc;             // [pairs][48][n] fp32, zeroed by the preparation kernel
     float* dkp;                // [pairs][16][n] fp32, RIB columns of dK~ (already times 1/sqrt d)
     __nv_bfloat16* dk;
@@ -109,7 +110,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
         for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
-        mbar_init(bar(kSFull), 1); mbar_init(bar(kSIssued), 1); mbar_init(bar(kPReady), 8); mbar_init(bar(kPFree), 2);
+        mbar_init(bar(kSFull), 1); mbar_init(bar(kSIssued), 1); mbar_init(bar(kPReady), 16); mbar_init(bar(kPFree), 2);
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
         mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
         for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
@@ -258,14 +259,15 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             mma_commit(bar(kDrain + warp - 1));
             mbar_wait(bar(kDrain + warp - 1), 0, abort_flag + 1, p.status);
         }
-    } else if (warp >= 4 && warp < 12) {
-        // ===================== P^T and dS^T: one thread per key row, one warpgroup per 64 queries
-        const int half = (warp - 4) >> 2;
+    } else if (warp >= 4 && warp < 20) {
+        // ===================== P^T and dS^T: one thread per key row, one warpgroup per 32 queries
+        const int cg = (warp - 4) >> 2;                      // column group: queries 32 cg .. 32 cg + 31 of the tile
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                 // key row of the block == TMEM lane
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        uint8_t* ds_row = base_ptr + kOffDS + half * kDSHalf + row * 128;
+        uint8_t* ds_row = base_ptr + kOffDS + (cg >> 1) * kDSHalf + row * 128;
         const int sw = row & 7;
+        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
         uint32_t g = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
@@ -275,25 +277,26 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) &&
                                                  mbar_wait(bar(kSFull), g & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
-                const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD);
+                const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 16 * cg;
                 bool may_store = g == 0;
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
-                    const int col0 = half * 64 + ch * 32;
-                    uint32_t s[32], dp[32];
-                    tmem_ld32(tmem + lane_base + kColS + col0, s);
-                    tmem_ld32(tmem + lane_base + kColDP + col0, dp);
+                    const int col0 = cg * 32 + ch * 16;
+                    uint32_t s[16], dp[16];
+                    tmem_ld16(tmem + lane_base + kColS + col0, s);
+                    tmem_ld16(tmem + lane_base + kColDP + col0, dp);
                     tmem_wait_ld();
-                    uint32_t pp[16], dd[16];
+                    uint32_t pp[8], dd[8];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float4 t = ld[(col0 >> 1) + i];   // (-lse2, D) of queries col0 + 2i, col0 + 2i + 1
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, t.x));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, t.z));
-                        const float d0 = p0 * (__uint_as_float(dp[2 * i]) - t.y);
-                        const float d1 = p1 * (__uint_as_float(dp[2 * i + 1]) - t.w);
-                        pp[i] = pack_bf16x2(p0, p1);
-                        dd[i] = pack_bf16x2(d0, d1);
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 t = ld[8 * ch + i];        // (-lse2, -lse2', -D, -D') of queries col0 + 2i, col0 + 2i + 1
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2,
+                                                    make_float2(t.x, t.y));
+                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])),
+                                                                 make_float2(t.z, t.w)));
+                        pp[i] = pack_bf16x2(e.x, e.y);
+                        dd[i] = pack_bf16x2(d.x, d.y);
                     }
                     if (!may_store) {
                         // the previous tile's contractions still read P^T, dS^T and the dS tile
@@ -301,13 +304,13 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         tc_fence_after();
                         may_store = true;
                     }
-                    tmem_st16(tmem + lane_base + kColP + (col0 >> 1), pp);
-                    tmem_st16(tmem + lane_base + kColDS + (col0 >> 1), dd);
+                    tmem_st8(tmem + lane_base + kColP + (col0 >> 1), pp);
+                    tmem_st8(tmem + lane_base + kColDS + (col0 >> 1), dd);
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const int chunk = ch * 4 + q4;
+                    for (int q2 = 0; q2 < 2; ++q2) {
+                        const int chunk = (cg & 1) * 4 + ch * 2 + q2;
                         *reinterpret_cast<uint4*>(ds_row + ((chunk ^ sw) << 4)) =
-                            make_uint4(dd[4 * q4], dd[4 * q4 + 1], dd[4 * q4 + 2], dd[4 * q4 + 3]);
+                            make_uint4(dd[4 * q2], dd[4 * q2 + 1], dd[4 * q2 + 2], dd[4 * q2 + 3]);
                     }
                 }
                 if (!ok) break;
@@ -318,7 +321,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) mbar_arrive(bar(kPReady));
             }
         }
-    } else if (warp >= 12) {
+    } else if (warp >= 20) {
         // ================================ drains: dQ~ after every tile, dV / dK~ after every item
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
@@ -330,52 +333,52 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             for (int I = 0; I < p.nblk; ++I, ++g) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kDQFull), g & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
-                uint32_t a[32], b[16];
-                tmem_ld32(tmem + lane_base + kColDQ, a);
-                tmem_ld16(tmem + lane_base + kColDQ + kD, b);
-                tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kDQFree));
                 float* dst = p.dq_acc + (size_t)c.pair * kDk * p.n + (size_t)I * kTile + row;
 #pragma unroll
-                for (int col = 0; col < kD; ++col) red_add_f32(dst + (size_t)col * p.n, __uint_as_float(a[col]));
+                for (int part = 0; part < 3; ++part) {       // 16 columns at a time keeps the register count low
+                    uint32_t a[16];
+                    tmem_ld16(tmem + lane_base + kColDQ + 16 * part, a);
+                    tmem_wait_ld();
+                    if (part == 2) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kDQFree));
+                    }
 #pragma unroll
-                for (int col = 0; col < kR; ++col) red_add_f32(dst + (size_t)(kD + col) * p.n, __uint_as_float(b[col]));
+                    for (int col = 0; col < 16; ++col) red_add_f32(dst + (size_t)(16 * part + col) * p.n, __uint_as_float(a[col]));
+                }
             }
             if (!ok) break;
             if (!__all_sync(0xffffffffu, mbar_wait(bar(kAccFull), nitem & 1, abort_flag, p.status))) { ok = false; break; }
             tc_fence_after();
-            uint32_t dv[32], dk[32], dkp[16];
-            tmem_ld32(tmem + lane_base + kColDV, dv);
-            tmem_ld32(tmem + lane_base + kColDK, dk);
-            tmem_ld16(tmem + lane_base + kColDK + kD, dkp);
-            tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kAccFree));
             int i, Y, X;
             window_order_token(geom, c.wy, c.wx, c.J * kTile + row, i, Y, X);
             const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
             uint4* dst_v = reinterpret_cast<uint4*>(p.dv + tok * kD);
             uint4* dst_k = reinterpret_cast<uint4*>(p.dk + tok * kD);
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                uint4 o;
-                o.x = pack_bf16x2(__uint_as_float(dv[8 * q4 + 0]), __uint_as_float(dv[8 * q4 + 1]));
-                o.y = pack_bf16x2(__uint_as_float(dv[8 * q4 + 2]), __uint_as_float(dv[8 * q4 + 3]));
-                o.z = pack_bf16x2(__uint_as_float(dv[8 * q4 + 4]), __uint_as_float(dv[8 * q4 + 5]));
-                o.w = pack_bf16x2(__uint_as_float(dv[8 * q4 + 6]), __uint_as_float(dv[8 * q4 + 7]));
-                dst_v[q4] = o;
-                o.x = pack_bf16x2(__uint_as_float(dk[8 * q4 + 0]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 1]) * p.inv_sqrt_d);
-                o.y = pack_bf16x2(__uint_as_float(dk[8 * q4 + 2]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 3]) * p.inv_sqrt_d);
-                o.z = pack_bf16x2(__uint_as_float(dk[8 * q4 + 4]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 5]) * p.inv_sqrt_d);
-                o.w = pack_bf16x2(__uint_as_float(dk[8 * q4 + 6]) * p.inv_sqrt_d, __uint_as_float(dk[8 * q4 + 7]) * p.inv_sqrt_d);
-                dst_k[q4] = o;
-            }
             float* dst_p = p.dkp + (size_t)c.pair * kR * p.n + (size_t)c.J * kTile + row;
 #pragma unroll
-            for (int col = 0; col < kR; ++col) dst_p[(size_t)col * p.n] = __uint_as_float(dkp[col]) * p.inv_sqrt_d;
+            for (int part = 0; part < 5; ++part) {           // dV (2 x 16 columns), dK~ content (2 x 16), dK~ RIB (16)
+                uint32_t a[16];
+                tmem_ld16(tmem + lane_base + kColDV + 16 * part, a);     // dV, dK~ are adjacent in tensor memory
+                tmem_wait_ld();
+                if (part == 4) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kAccFree));
+#pragma unroll
+                    for (int col = 0; col < kR; ++col) dst_p[(size_t)col * p.n] = __uint_as_float(a[col]) * p.inv_sqrt_d;
+                } else {
+                    const float f = part < 2 ? 1.f : p.inv_sqrt_d;
+                    uint4* dst16 = (part < 2 ? dst_v : dst_k) + 2 * (part & 1);
+#pragma unroll
+                    for (int q2 = 0; q2 < 2; ++q2)
+                        dst16[q2] = make_uint4(pack_bf16x2(__uint_as_float(a[8 * q2 + 0]) * f, __uint_as_float(a[8 * q2 + 1]) * f),
+                                               pack_bf16x2(__uint_as_float(a[8 * q2 + 2]) * f, __uint_as_float(a[8 * q2 + 3]) * f),
+                                               pack_bf16x2(__uint_as_float(a[8 * q2 + 4]) * f, __uint_as_float(a[8 * q2 + 5]) * f),
+                                               pack_bf16x2(__uint_as_float(a[8 * q2 + 6]) * f, __uint_as_float(a[8 * q2 + 7]) * f));
+                }
+            }
         }
     }
     // ================================================================================ common tail
@@ -446,7 +449,10 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
             acc = fmaf(__uint_as_float(xs[k] & 0xffff0000u), __uint_as_float(ys[k] & 0xffff0000u), acc);
         }
     }
-    p.ld[t] = make_float2(-p.lse[scalar] * 1.4426950408889634f, acc);
+    // per query pair (w even, w + 1): (-lse2, -lse2', -D, -D'), the operand order of the packed arithmetic
+    float* ldf = reinterpret_cast<float*>(p.ld) + ((t >> 1) << 2) + (t & 1);
+    ldf[0] = -p.lse[scalar] * 1.4426950408889634f;
+    ldf[2] = -acc;
     float* z = p.dq_acc + (size_t)pair * kDk * p.n + w;
 #pragma unroll 8
     for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
