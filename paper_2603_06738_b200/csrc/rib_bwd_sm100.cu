@@ -23,7 +23,8 @@
 //
 // Roles (768 threads): warp 0 TMA producer; three MMA-issuing threads, because one thread issuing
 // all contractions of a tile was the bottleneck and the tensor pipe takes instructions from several
-// warps at once: warp 1 issues S^T and dP^T, warp 2 (also the TMEM allocator) dV and dK~, warp 3 dQ~;
+// warps at once: warp 1 issues S^T, dP^T (next tile first) and dV, warp 2 (also the TMEM allocator) dK~,
+// warp 3 dQ~;
 // warps 4-19 P/dS arithmetic (four warpgroups, each a quarter of the tile's columns: four warps per SM
 // sub-partition hide each other's tensor-memory and barrier latencies), warps 20-23 drain dQ~ after
 // every tile and dK~/dV after every item.  Every wait is bounded.
@@ -109,10 +110,10 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (threadIdx.x == 0) {
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
-        for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
-        mbar_init(bar(kSFull), 1); mbar_init(bar(kSIssued), 1); mbar_init(bar(kPReady), 16); mbar_init(bar(kPFree), 2);
+        for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 2); }
+        mbar_init(bar(kSFull), 1); mbar_init(bar(kSIssued), 1); mbar_init(bar(kPReady), 16); mbar_init(bar(kPFree), 3);
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
-        mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
+        mbar_init(bar(kAccFull), 2); mbar_init(bar(kAccFree), 4);
         for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
         fence_barrier_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
@@ -185,7 +186,20 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             bool ok = true;
             if (warp == 1) {
                 // ---- S^T = K~_J Q~_I^T and dP^T = V_J dO_I^T, as soon as the arithmetic warps have taken
-                // the previous tile's scores out of tensor memory
+                // the previous tile's scores out of tensor memory; then dV_J += P^T dO_I of that previous tile
+                bool have_prev = false, prev_first = false, prev_last = false;
+                uint32_t prev_st = 0, prev_nitem = 0;
+                auto issue_dv = [&]() -> bool {
+                    if (prev_first && prev_nitem > 0 && !mbar_wait(bar(kAccFree), (prev_nitem - 1) & 1, abort_flag, p.status)) return false;
+                    const uint64_t go = smem_desc_at(kDesc64, base + kOffRing + prev_st * kRingBytes + kRingDO);
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 16; ++kk)
+                        mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, go + 64 * kk, kIdescT32, (kk || !prev_first) ? 1u : 0u);
+                    mma_commit(bar(kPFree));
+                    mma_commit(bar(kQEmpty + prev_st));
+                    if (prev_last) mma_commit(bar(kAccFull));
+                    return true;
+                };
                 for (; item < p.items && ok; item += gridDim.x, ++nitem) {
                     const uint32_t slot = nitem & 1;
                     if (!mbar_wait(bar(kKVFull + slot), (nitem >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
@@ -207,25 +221,26 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         mma_ss(tmem + kColDP, v + 2, go + 2, kIdescSS, 1u);
                         mma_commit(bar(kSFull));
                         if (g > 0) mbar_arrive(bar(kSIssued));      // the gradient contractions of tile g - 1 may follow
+                        if (have_prev && !issue_dv()) { ok = false; break; }
+                        have_prev = true; prev_first = I == 0; prev_last = I == p.nblk - 1; prev_st = st; prev_nitem = nitem;
                     }
                 }
+                if (ok && have_prev && mbar_wait(bar(kPReady), (g - 1) & 1, abort_flag, p.status)) {
+                    tc_fence_after();
+                    issue_dv();
+                }
             } else if (warp == 2) {
-                // ---- dV_J += P^T dO_I and dK~_J += dS^T Q~_I (A from tensor memory, 16 queries per step)
+                // ---- dK~_J += dS^T Q~_I (A from tensor memory, 16 queries per step)
                 for (; item < p.items && ok; item += gridDim.x, ++nitem) {
                     for (I = 0; I < p.nblk; ++I, ++g) {
                         const uint32_t st = g % kQStages;
                         if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status) ||
                             (I == 0 && nitem > 0 && !mbar_wait(bar(kAccFree), (nitem - 1) & 1, abort_flag, p.status))) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t ring = base + kOffRing + st * kRingBytes;
-                        const uint64_t q48 = smem_desc_at(kDescQ48, ring + kRingQc);
-                        const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
+                        const uint64_t q48 = smem_desc_at(kDescQ48, base + kOffRing + st * kRingBytes + kRingQc);
                         const uint32_t acc0 = I > 0 ? 1u : 0u;
                         // let the next tile's S^T, dP^T into the tensor pipe first: the arithmetic warps wait for them
                         if (g + 1 < total_tiles && !mbar_wait(bar(kSIssued), g & 1, abort_flag, p.status)) { ok = false; break; }
-#pragma unroll
-                        for (int kk = 0; kk < kTile / 16; ++kk)
-                            mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, go + 64 * kk, kIdescT32, kk ? 1u : acc0);
 #pragma unroll
                         for (int kk = 0; kk < kTile / 16; ++kk)
                             mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, q48 + 64 * kk, kIdescT48, kk ? 1u : acc0);
