@@ -6,13 +6,18 @@
 // Work item = one (batch, window, head) pair x one key block J of 128 tokens.  A persistent CTA keeps
 // K~_J = [k, Pk] and V_J in shared memory and dV_J, dK~_J in tensor memory, and walks the query tiles
 // I of the window.  Everything is computed transposed (keys on the TMEM lanes) so that P^T and dS^T
-// feed the dV and dK~ contractions straight from tensor memory:
-//     S^T  = K~_J Q~_I^T                    (M128 N128 K48: content rows 2 x K16, RIB rows 1 x K16)
-//     dP^T = V_J dO_I^T                     (M128 N128 K32)
+// feed the dV and dK~ contractions straight from tensor memory.  The unit of the pipeline is a
+// half-tile u = (I, h): the 64 queries of patch h of tile I,
+//     S^T  = K~_J Q~_u^T                    (M128 N64 K48: content rows 2 x K16, RIB rows 1 x K16)
+//     dP^T = V_J dO_u^T                     (M128 N64 K32)
 //     P^T  = exp2(S^T * log2e/sqrt(d) - lse_i * log2e),   dS^T = P^T o (dP^T - D_i)     (ALU warps)
-//     dV_J  += P^T  dO_I                    (A from TMEM, B = dO tile, MN-major, N = 32)
-//     dK~_J += dS^T Q~_I                    (A from TMEM, B = [Q content | Q RIB] tiles, MN-major, N = 48)
-//     dQ~_I  = dS K~_J                      (A = dS through shared memory, MN-major, B = [K | Pk] tiles, N = 48)
+//     dV_J  += P^T  dO_u                    (A from TMEM, B = dO rows, MN-major, N = 32)
+//     dK~_J += dS^T Q~_u                    (A from TMEM, B = [Q content | Q RIB] tiles, MN-major, N = 48)
+// and once per tile, when both halves of dS are in shared memory,
+//     dQ~_I  = dS K~_J                      (A = dS, MN-major, B = [K | Pk] tiles, N = 48).
+// Score accumulators, P^T and dS^T are double-buffered by h, and two groups of arithmetic warps take
+// the even and the odd half-tiles: while one group evaluates exponentials the other one's scores are
+// being contracted, so neither the tensor pipe nor the exp pipe waits for a whole tile of the other.
 // The RIB rows are fetched as zero-padded 64-byte rows, so that a RIB tile has the layout of a content
 // tile and the concatenation of Eq. 5 is, for the MN-major operands, one descriptor whose second
 // 32-column atom is the RIB tile: every contraction step is a single instruction.
@@ -21,13 +26,11 @@
 // bf16 and sums the RIB columns over pairs into dPq.  The RIB columns of dK~ are written per pair
 // and summed over pairs by the same finishing kernel into dPk.
 //
-// Roles (768 threads): warp 0 TMA producer; three MMA-issuing threads, because one thread issuing
-// all contractions of a tile was the bottleneck and the tensor pipe takes instructions from several
-// warps at once: warp 1 issues S^T, dP^T (next tile first) and dV, warp 2 (also the TMEM allocator) dK~,
-// warp 3 dQ~;
-// warps 4-19 P/dS arithmetic (four warpgroups, each a quarter of the tile's columns: four warps per SM
-// sub-partition hide each other's tensor-memory and barrier latencies), warps 20-23 drain dQ~ after
-// every tile and dK~/dV after every item.  Every wait is bounded.
+// Roles (768 threads): warp 0 TMA producer; three MMA-issuing threads (the tensor pipe takes
+// instructions from several warps at once, and one thread issuing everything was the bottleneck):
+// warp 1 issues S^T, dP^T and dV, warp 2 (also the TMEM allocator) dK~, warp 3 dQ~; warps 4-11
+// P/dS arithmetic of the even half-tiles, warps 12-19 of the odd ones (one thread per key row and 32
+// queries); warps 20-23 drain dQ~ after every tile and dK~/dV after every item.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -47,20 +50,23 @@ constexpr uint32_t kOffRing = kOffV + 2 * kContentBytes;
 constexpr uint32_t kLdBytes = kTile * 8;                         // 64 query pairs x (-lse2, -lse2', -D, -D')
 constexpr uint32_t kRingQc = 0, kRingQp = kContentBytes, kRingDO = kRingQp + kContentBytes, kRingLD = kRingDO + kContentBytes;
 constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 25600
-constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
+constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 tiles][2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
 constexpr uint32_t kDSHalf = kTile * 128;
-constexpr uint32_t kOffBar = kOffDS + 2 * kDSHalf;
-enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kSIssued, kPReady,
-           kPFree, kDQFull, kDQFree, kAccFull, kAccFree, kDrain, kNumBars = kDrain + 3 };
+constexpr uint32_t kOffBar = kOffDS + 4 * kDSHalf;
+// kSFull, kPReady, kPFree: one per half h; kDSFree: one per dS tile buffer
+enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kSIssued = kSFull + 2,
+           kPReady, kPFree = kPReady + 2, kDSFree = kPFree + 2, kDQFull = kDSFree + 2, kDQFree, kAccFull, kAccFree, kDrain,
+           kNumBars = kDrain + 3 };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;
 constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
 static_assert(kOffRing % 1024 == 0 && kRingBytes % 1024 == 0 && kOffDS % 1024 == 0, "swizzle atoms need aligned tiles");
 
-// tensor-memory columns
+// tensor-memory columns; S^T, dP^T (64 fp32 columns) and P^T, dS^T (32 columns of bf16 pairs) exist once per half h
 constexpr uint32_t kColS = 0, kColDP = 128, kColP = 256, kColDS = 320, kColDV = 384, kColDK = 416, kColDQ = 464;
+constexpr uint32_t kHalfCols = kTile / 2;
 constexpr uint32_t kTmemCols = 512;
 
-constexpr uint32_t kIdescSS = idesc_bf16_f32(kTile, kTile, false);            // S^T, dP^T: both operands K-major
+constexpr uint32_t kIdescSS = idesc_bf16_f32(kTile, kTile / 2, false);        // S^T, dP^T of a half-tile: both operands K-major
 constexpr uint32_t kIdescT32 = idesc_bf16_f32(kTile, kD, true);               // A in TMEM, B MN-major, N = 32
 constexpr uint32_t kIdescT48 = idesc_bf16_f32(kTile, kDk, true);              // A in TMEM, B MN-major, N = 48
 constexpr uint32_t kIdescQ48 = idesc_bf16_f32_ab(kTile, kDk, true, true);     // dQ~: A and B MN-major, N = 48
@@ -111,7 +117,10 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
         for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 2); }
-        mbar_init(bar(kSFull), 1); mbar_init(bar(kSIssued), 1); mbar_init(bar(kPReady), 16); mbar_init(bar(kPFree), 3);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(bar(kSFull + h), 1); mbar_init(bar(kPReady + h), 8); mbar_init(bar(kPFree + h), 2); mbar_init(bar(kDSFree + h), 1);
+        }
+        mbar_init(bar(kSIssued), 1);
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
         mbar_init(bar(kAccFull), 2); mbar_init(bar(kAccFree), 4);
         for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
@@ -173,114 +182,133 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
         }
     } else if (warp < 4) {
-        // ==================================================== MMA issuers (one thread per warp 1-3)
-        if (lane == 0) {
-            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B);
-            // MN-major operands of 48 columns: the content tile and, one leading-dimension step further, the RIB tile
-            constexpr uint64_t kDescQ48 = smem_desc_const(kRingQp - kRingQc, 512, kSwizzle64B);
-            constexpr uint64_t kDescK48 = smem_desc_const(kOffKp - kOffKc, 512, kSwizzle64B);
-            constexpr uint64_t kDescDS = smem_desc_const(kDSHalf, 1024, kSwizzle128B);
-            int item = blockIdx.x, I = 0;
-            uint32_t nitem = 0, g = 0;
-            const uint32_t total_tiles = (((uint32_t)p.items - blockIdx.x + gridDim.x - 1) / gridDim.x) * (uint32_t)p.nblk;
-            bool ok = true;
-            if (warp == 1) {
-                // ---- S^T = K~_J Q~_I^T and dP^T = V_J dO_I^T, as soon as the arithmetic warps have taken
-                // the previous tile's scores out of tensor memory; then dV_J += P^T dO_I of that previous tile
-                bool have_prev = false, prev_first = false, prev_last = false;
-                uint32_t prev_st = 0, prev_nitem = 0;
-                auto issue_dv = [&]() -> bool {
-                    if (prev_first && prev_nitem > 0 && !mbar_wait(bar(kAccFree), (prev_nitem - 1) & 1, abort_flag, p.status)) return false;
-                    const uint64_t go = smem_desc_at(kDesc64, base + kOffRing + prev_st * kRingBytes + kRingDO);
-#pragma unroll
-                    for (int kk = 0; kk < kTile / 16; ++kk)
-                        mma_ts(tmem + kColDV, tmem + kColP + 8 * kk, go + 64 * kk, kIdescT32, (kk || !prev_first) ? 1u : 0u);
-                    mma_commit(bar(kPFree));
-                    mma_commit(bar(kQEmpty + prev_st));
-                    if (prev_last) mma_commit(bar(kAccFull));
-                    return true;
-                };
-                for (; item < p.items && ok; item += gridDim.x, ++nitem) {
-                    const uint32_t slot = nitem & 1;
-                    if (!mbar_wait(bar(kKVFull + slot), (nitem >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                    const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + slot * kContentBytes);
-                    const uint64_t kp = smem_desc_at(kDesc64, base + kOffKp + slot * kContentBytes);
-                    const uint64_t v = smem_desc_at(kDesc64, base + kOffV + slot * kContentBytes);
-                    for (I = 0; I < p.nblk; ++I, ++g) {
-                        const uint32_t st = g % kQStages;
-                        if (!mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) ||
-                            (g > 0 && !mbar_wait(bar(kPReady), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
-                        tc_fence_after();
-                        const uint32_t ring = base + kOffRing + st * kRingBytes;
+        // ============================================ MMA issuers: warps 1-3, the whole warp walks the
+        // loops and waits (warp-uniform outcomes), one elected lane issues
+        constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B);
+        // MN-major operands of 48 columns: the content tile and, one leading-dimension step further, the RIB tile
+        constexpr uint64_t kDescQ48 = smem_desc_const(kRingQp - kRingQc, 512, kSwizzle64B);
+        constexpr uint64_t kDescK48 = smem_desc_const(kOffKp - kOffKc, 512, kSwizzle64B);
+        constexpr uint64_t kDescDS = smem_desc_const(kDSHalf, 1024, kSwizzle128B);
+        const int nblk = p.nblk;
+        const uint32_t total_tiles = (((uint32_t)p.items - blockIdx.x + gridDim.x - 1) / gridDim.x) * (uint32_t)nblk;
+        const uint32_t total_units = 2 * total_tiles;       // half-tiles of this CTA, in order
+        auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status)) != 0; };
+        bool ok = true;
+        if (warp == 1) {
+            // ---- per unit u: S^T, dP^T of u as soon as the arithmetic group has taken unit u - 2 (same
+            // buffers) out of tensor memory, then dV_J += P^T dO of that unit u - 2
+            uint32_t s_nitem = 0, s_I = 0;                  // item ordinal / tile of the unit whose scores come next
+            uint32_t v_nitem = 0, v_I = 0;                  // the same for the unit whose dV comes next
+            uint32_t slot_base = 0;
+            for (uint32_t u = 0; u < total_units + 2 && ok; ++u) {
+                const uint32_t h = u & 1;
+                if (u >= 2 && !wait_all(bar(kPReady + h), ((u - 2) >> 1) & 1)) { ok = false; break; }
+                if (u < total_units) {
+                    const uint32_t g = u >> 1, st = g % kQStages, slot = s_nitem & 1;
+                    if (h == 0 && s_I == 0) {
+                        if (!wait_all(bar(kKVFull + slot), (s_nitem >> 1) & 1)) { ok = false; break; }
+                        slot_base = base + slot * kContentBytes;
+                    }
+                    if (h == 0 && !wait_all(bar(kQFull + st), (g / kQStages) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t ring = base + kOffRing + st * kRingBytes + h * kPatchContent;   // rows of patch h
+                    if (elect_one()) {
+                        const uint64_t kc = smem_desc_at(kDesc64, slot_base + kOffKc), kp = smem_desc_at(kDesc64, slot_base + kOffKp);
+                        const uint64_t v = smem_desc_at(kDesc64, slot_base + kOffV);
                         const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc64, ring + kRingQp);
                         const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
-                        mma_ss(tmem + kColS, kc, qc, kIdescSS, 0u);
-                        mma_ss(tmem + kColS, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
-                        mma_ss(tmem + kColS, kp, qp, kIdescSS, 1u);
-                        mma_ss(tmem + kColDP, v, go, kIdescSS, 0u);
-                        mma_ss(tmem + kColDP, v + 2, go + 2, kIdescSS, 1u);
-                        mma_commit(bar(kSFull));
-                        if (g > 0) mbar_arrive(bar(kSIssued));      // the gradient contractions of tile g - 1 may follow
-                        if (have_prev && !issue_dv()) { ok = false; break; }
-                        have_prev = true; prev_first = I == 0; prev_last = I == p.nblk - 1; prev_st = st; prev_nitem = nitem;
+                        const uint32_t d_s = tmem + kColS + h * kHalfCols, d_p = tmem + kColDP + h * kHalfCols;
+                        mma_ss(d_s, kc, qc, kIdescSS, 0u);
+                        mma_ss(d_s, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
+                        mma_ss(d_s, kp, qp, kIdescSS, 1u);
+                        mma_ss(d_p, v, go, kIdescSS, 0u);
+                        mma_ss(d_p, v + 2, go + 2, kIdescSS, 1u);
+                        mma_commit(bar(kSFull + h));
+                        if (u >= 2) mbar_arrive(bar(kSIssued));     // the gradient contractions of unit u - 2 may follow
                     }
+                    __syncwarp();
+                    if (h == 1 && ++s_I == (uint32_t)nblk) { s_I = 0; ++s_nitem; }
                 }
-                if (ok && have_prev && mbar_wait(bar(kPReady), (g - 1) & 1, abort_flag, p.status)) {
+                if (u >= 2) {
+                    // dV of unit u - 2 (tile v_I of item ordinal v_nitem, half h)
+                    const uint32_t g2 = (u - 2) >> 1, st2 = g2 % kQStages;
+                    const bool first = v_I == 0 && h == 0, last = v_I == (uint32_t)nblk - 1 && h == 1;
+                    if (first && v_nitem > 0 && !wait_all(bar(kAccFree), (v_nitem - 1) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    issue_dv();
-                }
-            } else if (warp == 2) {
-                // ---- dK~_J += dS^T Q~_I (A from tensor memory, 16 queries per step)
-                for (; item < p.items && ok; item += gridDim.x, ++nitem) {
-                    for (I = 0; I < p.nblk; ++I, ++g) {
-                        const uint32_t st = g % kQStages;
-                        if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status) ||
-                            (I == 0 && nitem > 0 && !mbar_wait(bar(kAccFree), (nitem - 1) & 1, abort_flag, p.status))) { ok = false; break; }
-                        tc_fence_after();
-                        const uint64_t q48 = smem_desc_at(kDescQ48, base + kOffRing + st * kRingBytes + kRingQc);
-                        const uint32_t acc0 = I > 0 ? 1u : 0u;
-                        // let the next tile's S^T, dP^T into the tensor pipe first: the arithmetic warps wait for them
-                        if (g + 1 < total_tiles && !mbar_wait(bar(kSIssued), g & 1, abort_flag, p.status)) { ok = false; break; }
+                    if (elect_one()) {
+                        const uint64_t go = smem_desc_at(kDesc64, base + kOffRing + st2 * kRingBytes + kRingDO + h * kPatchContent);
+                        const uint32_t a_p = tmem + kColP + h * (kHalfCols / 2);
 #pragma unroll
-                        for (int kk = 0; kk < kTile / 16; ++kk)
-                            mma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, q48 + 64 * kk, kIdescT48, kk ? 1u : acc0);
-                        mma_commit(bar(kPFree));
-                        mma_commit(bar(kQEmpty + st));
-                        if (I == p.nblk - 1) mma_commit(bar(kAccFull));
+                        for (int kk = 0; kk < kTile / 32; ++kk)     // 16 queries per step
+                            mma_ts(tmem + kColDV, a_p + 8 * kk, go + 64 * kk, kIdescT32, (kk || !first) ? 1u : 0u);
+                        mma_commit(bar(kPFree + h));
+                        if (h == 1) mma_commit(bar(kQEmpty + st2));
+                        if (last) mma_commit(bar(kAccFull));
                     }
-                }
-            } else {
-                // ---- dQ~_I = dS K~_J (A = dS through shared memory, 16 keys per step)
-                const uint64_t ds = smem_desc_at(kDescDS, base + kOffDS);
-                for (; item < p.items && ok; item += gridDim.x, ++nitem) {
-                    const uint32_t slot = nitem & 1;
-                    const uint64_t k48 = smem_desc_at(kDescK48, base + kOffKc + slot * kContentBytes);
-                    for (I = 0; I < p.nblk; ++I, ++g) {
-                        if (!mbar_wait(bar(kPReady), g & 1, abort_flag, p.status) ||
-                            (g > 0 && !mbar_wait(bar(kDQFree), (g - 1) & 1, abort_flag, p.status)) ||
-                            (g + 1 < total_tiles && !mbar_wait(bar(kSIssued), g & 1, abort_flag, p.status))) { ok = false; break; }
-                        tc_fence_after();
-#pragma unroll
-                        for (int kk = 0; kk < kTile / 16; ++kk)
-                            mma_ss(tmem + kColDQ, ds + 128 * kk, k48 + 64 * kk, kIdescQ48, kk ? 1u : 0u);
-                        mma_commit(bar(kPFree));
-                        mma_commit(bar(kDQFull));
-                        // K~_J and V_J may go once the item's last dQ~ is done (S^T, dP^T finished before it)
-                        if (I == p.nblk - 1) mma_commit(bar(kKVEmpty + slot));
-                    }
+                    __syncwarp();
+                    if (h == 1 && ++v_I == (uint32_t)nblk) { v_I = 0; ++v_nitem; }
                 }
             }
-            // everything issued by this thread must have finished before TMEM is released
-            mma_commit(bar(kDrain + warp - 1));
-            mbar_wait(bar(kDrain + warp - 1), 0, abort_flag + 1, p.status);
+        } else if (warp == 2) {
+            // ---- dK~_J += dS^T Q~_u (A from tensor memory, 16 queries per step)
+            uint32_t nitem = 0, I = 0;
+            for (uint32_t u = 0; u < total_units && ok; ++u) {
+                const uint32_t h = u & 1, g = u >> 1, st = g % kQStages;
+                const bool first = I == 0 && h == 0, last = I == (uint32_t)nblk - 1 && h == 1;
+                if (!wait_all(bar(kPReady + h), g & 1) ||
+                    (first && nitem > 0 && !wait_all(bar(kAccFree), (nitem - 1) & 1)) ||
+                    // let the scores of unit u + 2 into the tensor pipe first: an arithmetic group waits for them
+                    (u + 2 < total_units && !wait_all(bar(kSIssued), u & 1))) { ok = false; break; }
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t q48 = smem_desc_at(kDescQ48, base + kOffRing + st * kRingBytes + kRingQc + h * kPatchContent);
+                    const uint32_t a_ds = tmem + kColDS + h * (kHalfCols / 2);
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 32; ++kk)
+                        mma_ts(tmem + kColDK, a_ds + 8 * kk, q48 + 64 * kk, kIdescT48, (kk || !first) ? 1u : 0u);
+                    mma_commit(bar(kPFree + h));
+                    if (h == 1) mma_commit(bar(kQEmpty + st));
+                    if (last) mma_commit(bar(kAccFull));
+                }
+                __syncwarp();
+                if (h == 1 && ++I == (uint32_t)nblk) { I = 0; ++nitem; }
+            }
+        } else if (warp == 3) {
+            // ---- dQ~_I = dS K~_J once both halves of dS are in shared memory (16 keys per step)
+            uint32_t nitem = 0, I = 0;
+            for (uint32_t g = 0; g < total_tiles && ok; ++g) {
+                if (!wait_all(bar(kPReady), g & 1) || !wait_all(bar(kPReady + 1), g & 1) ||
+                    (g > 0 && !wait_all(bar(kDQFree), (g - 1) & 1)) ||
+                    (2 * g + 3 < total_units && !wait_all(bar(kSIssued), (2 * g + 1) & 1))) { ok = false; break; }
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t k48 = smem_desc_at(kDescK48, base + kOffKc + (nitem & 1) * kContentBytes);
+                    const uint64_t ds = smem_desc_at(kDescDS, base + kOffDS + (g & 1) * 2 * kDSHalf);
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 16; ++kk)
+                        mma_ss(tmem + kColDQ, ds + 128 * kk, k48 + 64 * kk, kIdescQ48, kk ? 1u : 0u);
+                    mma_commit(bar(kDSFree + (g & 1)));
+                    mma_commit(bar(kDQFull));
+                    // K~_J and V_J may go once the item's last dQ~ is done (S^T, dP^T finished before it)
+                    if (I == (uint32_t)nblk - 1) mma_commit(bar(kKVEmpty + (nitem & 1)));
+                }
+                __syncwarp();
+                if (++I == (uint32_t)nblk) { I = 0; ++nitem; }
+            }
         }
+        // everything issued by this warp must have finished before TMEM is released
+        if (elect_one()) mma_commit(bar(kDrain + warp - 1));
+        __syncwarp();
+        mbar_wait(bar(kDrain + warp - 1), 0, abort_flag + 1, p.status);
     } else if (warp >= 4 && warp < 20) {
-        // ===================== P^T and dS^T: one thread per key row, one warpgroup per 32 queries
-        const int cg = (warp - 4) >> 2;                      // column group: queries 32 cg .. 32 cg + 31 of the tile
+        // ===== P^T and dS^T: group h = warps 4 + 8h .. 11 + 8h takes half-tile (I, h); one thread per key row and 32 queries
+        const int h = (warp - 4) >> 3;
+        const int cg = ((warp - 4) >> 2) & 1;                // queries 32 cg .. 32 cg + 31 of the half-tile
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                 // key row of the block == TMEM lane
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        uint8_t* ds_row = base_ptr + kOffDS + (cg >> 1) * kDSHalf + row * 128;
+        const uint32_t t_s = tmem + lane_base + kColS + h * kHalfCols + 32 * cg, t_dp = tmem + lane_base + kColDP + h * kHalfCols + 32 * cg;
+        const uint32_t t_p = tmem + lane_base + kColP + h * (kHalfCols / 2) + 16 * cg, t_ds = tmem + lane_base + kColDS + h * (kHalfCols / 2) + 16 * cg;
         const int sw = row & 7;
         const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
         uint32_t g = 0;
@@ -290,21 +318,21 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint32_t st = g % kQStages;
                 // warp-uniform outcome: the TMEM accesses below are warp-collective
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) &&
-                                                 mbar_wait(bar(kSFull), g & 1, abort_flag, p.status))) { ok = false; break; }
+                                                 mbar_wait(bar(kSFull + h), g & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
-                const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 16 * cg;
-                bool may_store = g == 0;
+                const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 32 * h + 16 * cg;
+                uint8_t* ds_row = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf + row * 128;
+                bool may_store = false;
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
-                    const int col0 = cg * 32 + ch * 16;
                     uint32_t s[16], dp[16];
-                    tmem_ld16(tmem + lane_base + kColS + col0, s);
-                    tmem_ld16(tmem + lane_base + kColDP + col0, dp);
+                    tmem_ld16(t_s + 16 * ch, s);
+                    tmem_ld16(t_dp + 16 * ch, dp);
                     tmem_wait_ld();
                     uint32_t pp[8], dd[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const float4 t = ld[8 * ch + i];        // (-lse2, -lse2', -D, -D') of queries col0 + 2i, col0 + 2i + 1
+                        const float4 t = ld[8 * ch + i];        // (-lse2, -lse2', -D, -D') of two neighbouring queries
                         const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2,
                                                     make_float2(t.x, t.y));
                         const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
@@ -314,16 +342,18 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         dd[i] = pack_bf16x2(d.x, d.y);
                     }
                     if (!may_store) {
-                        // the previous tile's contractions still read P^T, dS^T and the dS tile
-                        if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree), (g - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the
+                        // previous one still reads this dS buffer
+                        if (!__all_sync(0xffffffffu, (g == 0 || mbar_wait(bar(kPFree + h), (g - 1) & 1, abort_flag, p.status)) &&
+                                                         (g < 2 || mbar_wait(bar(kDSFree + (g & 1)), ((g >> 1) - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
                         tc_fence_after();
                         may_store = true;
                     }
-                    tmem_st8(tmem + lane_base + kColP + (col0 >> 1), pp);
-                    tmem_st8(tmem + lane_base + kColDS + (col0 >> 1), dd);
+                    tmem_st8(t_p + 8 * ch, pp);
+                    tmem_st8(t_ds + 8 * ch, dd);
 #pragma unroll
                     for (int q2 = 0; q2 < 2; ++q2) {
-                        const int chunk = (cg & 1) * 4 + ch * 2 + q2;
+                        const int chunk = cg * 4 + ch * 2 + q2;
                         *reinterpret_cast<uint4*>(ds_row + ((chunk ^ sw) << 4)) =
                             make_uint4(dd[4 * q2], dd[4 * q2 + 1], dd[4 * q2 + 2], dd[4 * q2 + 3]);
                     }
@@ -333,7 +363,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tc_fence_before();
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kPReady));
+                if (lane == 0) mbar_arrive(bar(kPReady + h));
             }
         }
     } else if (warp >= 20) {
