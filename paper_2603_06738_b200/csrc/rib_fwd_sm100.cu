@@ -184,11 +184,10 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         // ===================================== MMA issuers: warp 1 drives query tile 0, warp 3 tile 1
         // Per block b of this CTA's items: S(b) as soon as the softmax warps have taken S(b-1) out
         // of tensor memory, then PV(b-1) once P(b-1) is there.  The whole warp walks the loop and
-        // waits; lane 0 issues.
+        // waits; one elected lane issues (this keeps descriptors in uniform registers).
         const int qt = warp >> 1;
         constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
         const uint32_t d_s = tmem + kColS + qt * kTile, d_o = tmem + kColO + qt * 2 * kD, a_p = tmem + kColP + qt * (kTile / 2);
-        const bool leader = lane == 0;
         uint32_t b = 0, io = 0;
         bool ok = true;
         // O_q[half] += P_q[:, half] V[half] for block `pb` (first: the first block of item ordinal `pio`)
@@ -203,7 +202,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             for (int half = 0; half < 2; ++half) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kPReady + 2 * qt + half), pb & 1, abort_flag, p.status))) return false;
                 tc_fence_after();
-                if (leader) {
+                if (elect_one()) {
                     mma_ts(d_o + half * kD, a_p + 32 * half, v + 256 * half, kIdescPV, first ? 0u : 1u);
 #pragma unroll
                     for (int kk = 1; kk < 4; ++kk)
@@ -226,7 +225,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kKFull + st), (b / kStages) & 1, abort_flag, p.status) &&
                                                  (b == 0 || mbar_wait(bar(kSFree + qt), (b - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
                 tc_fence_after();
-                if (leader) {
+                if (elect_one()) {
                     const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
                     const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + st * kPosBytes);
                     mma_ss(d_s, qc, kc, kIdescS, 0u);
@@ -242,10 +241,9 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
         if (ok && b > 0) do_pv(b - 1, false, io);
         // everything issued by this warp's leader must have finished before TMEM is released
-        if (leader) {
-            mma_commit(bar(kDrain + qt));
-            mbar_wait(bar(kDrain + qt), 0, abort_flag + 1, p.status);
-        }
+        if (elect_one()) mma_commit(bar(kDrain + qt));
+        __syncwarp();
+        mbar_wait(bar(kDrain + qt), 0, abort_flag + 1, p.status);
     } else if (warp == 2) {
         // ====================== query RIB rows of the coming items: bf16(Pq * sqrt(d/r)), SWIZZLE_32B
         uint32_t io = 0;
