@@ -152,8 +152,8 @@ long long rib_kernel_launches(void);
  * destroy CUDA events: keep them outside stream capture and outside timed regions.  One profiling
  * session per process at a time, driven from one host thread.
  */
-enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH_DQ = 4,
-       RIB_KERNEL_BWD_FINISH_POS = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
+enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH = 4,
+       RIB_KERNEL_RESERVED = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
        RIB_KERNEL_ANY_BWD_DKV = 9 };
 int rib_profile_begin(int max_launches);
 int rib_profile_end(int* kernel_ids, float* ms, int capacity);

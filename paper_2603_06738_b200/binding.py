@@ -24,7 +24,7 @@ EXPORTS = (
     "rib_window_attn_bwd_noalloc", "rib_profile_begin", "rib_profile_end",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
-                4: "rib_bwd_finish_dq_kernel", 5: "rib_bwd_finish_pos_kernel", 6: "generic_fwd_kernel",
+                4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
                 7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel"}
 RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 

@@ -230,7 +230,7 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
     const cudaError_t e = fast ? rib::sm100_bwd(p, st) : rib::generic_bwd(p, st);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
-    g_kernel_launches += fast ? 4 : 3;   // prepare, main, two finishing kernels : rowdot, dq, dk/dv
+    g_kernel_launches += 3;   // prepare, main, finish : rowdot, dq, dk/dv
     return RIB_OK;
 }
 

@@ -503,45 +503,48 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
 }
 
-// One thread per (pair, token): dq = dQ~[:, :d] / sqrt(d) as bf16 at the token's pixel.
-__global__ void __launch_bounds__(256) rib_bwd_finish_dq_kernel(const AuxParams p)
+// Finishing pass over the fp32 accumulators.  grid (n / 128, groups of pairs), 128 threads: a thread
+// owns one token position w of the window and walks the pairs of its group.  Per pair it turns
+// dQ~[:, :d] / sqrt(d) into the bf16 dq row of that token, and it keeps running sums of the 16 RIB
+// columns of dQ~ (-> dPq, times 1/sqrt(r)) and of dK~ (-> dPk); the group's partial sums go to the
+// zeroed results with one vector atomic per 4 columns.
+__global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_group)
 {
-    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= (size_t)p.pairs * p.n) return;
-    const int pair = (int)(t / p.n), w = (int)(t % p.n);
-    int i; size_t tok, scalar;
-    decode_pair_token(p, pair, w, i, tok, scalar);
-    const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
-    uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
-#pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-        float f[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
-        dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
-    }
-}
-
-// dPq[i][c] = sum over pairs of dQ~[:, d + c] / sqrt(r);  dPk[i][c] = sum over pairs of the RIB
-// columns of dK~.  grid (n / 128 * 32, groups of pairs); a thread sums one (token, column) over
-// its group and adds the partial sum to the (zeroed) result.
-__global__ void __launch_bounds__(128) rib_bwd_finish_pos_kernel(const AuxParams p, int pairs_per_group)
-{
-    const int col = blockIdx.x & 31, w = (blockIdx.x >> 5) * 128 + threadIdx.x;
+    const int w = blockIdx.x * 128 + threadIdx.x;
     const int pair0 = blockIdx.y * pairs_per_group;
     const int pair1 = min(p.pairs, pair0 + pairs_per_group);
-    float acc = 0.f;
-    if (col < kR) {
-        const float* src = p.dq_acc + (size_t)(kD + col) * p.n + w;
-        for (int pair = pair0; pair < pair1; ++pair) acc += src[(size_t)pair * kDk * p.n];
-        acc *= p.inv_sqrt_r;
-    } else {
-        const float* src = p.dkp + (size_t)(col - kR) * p.n + w;
-        for (int pair = pair0; pair < pair1; ++pair) acc += src[(size_t)pair * kR * p.n];
+    float sq[kR], sk[kR];
+#pragma unroll
+    for (int c = 0; c < kR; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
+    int i = 0;
+    for (int pair = pair0; pair < pair1; ++pair) {
+        size_t tok, scalar;
+        decode_pair_token(p, pair, w, i, tok, scalar);
+        const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
+        uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            float f[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
+            dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+        }
+        const float* srk = p.dkp + (size_t)pair * kR * p.n + w;
+#pragma unroll
+        for (int c = 0; c < kR; ++c) {
+            sq[c] += src[(size_t)(kD + c) * p.n];
+            sk[c] += srk[(size_t)c * p.n];
+        }
     }
-    int i, Y, X;
-    window_order_token(WindowGeom{p.M, p.M, p.M, 0}, 0, 0, w, i, Y, X);
-    atomicAdd((col < kR ? p.dpq : p.dpk) + (size_t)i * kR + (col & (kR - 1)), acc);
+    if (pair0 >= pair1) return;
+    float4* out_q = reinterpret_cast<float4*>(p.dpq + (size_t)i * kR);
+    float4* out_k = reinterpret_cast<float4*>(p.dpk + (size_t)i * kR);
+#pragma unroll
+    for (int c4 = 0; c4 < kR / 4; ++c4) {
+        atomicAdd(out_q + c4, make_float4(sq[4 * c4] * p.inv_sqrt_r, sq[4 * c4 + 1] * p.inv_sqrt_r, sq[4 * c4 + 2] * p.inv_sqrt_r,
+                                          sq[4 * c4 + 3] * p.inv_sqrt_r));
+        atomicAdd(out_k + c4, make_float4(sk[4 * c4], sk[4 * c4 + 1], sk[4 * c4 + 2], sk[4 * c4 + 3]));
+    }
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -618,13 +621,9 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
-    { ProfileScope scope(RIB_KERNEL_BWD_FINISH_DQ, stream); rib_bwd_finish_dq_kernel<<<aux_blocks, 256, 0, stream>>>(ap); }
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const int groups = p.pairs < 16 ? p.pairs : 16;
-    const int per_group = (p.pairs + groups - 1) / groups;
-    dim3 grid_pos((unsigned)(p.n / 128 * 32), (unsigned)((p.pairs + per_group - 1) / per_group));
-    { ProfileScope scope(RIB_KERNEL_BWD_FINISH_POS, stream); rib_bwd_finish_pos_kernel<<<grid_pos, 128, 0, stream>>>(ap, per_group); }
+    const int per_group = p.pairs < 8 ? 1 : 4;
+    dim3 grid_fin((unsigned)(p.n / 128), (unsigned)((p.pairs + per_group - 1) / per_group));
+    { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<<<grid_fin, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();
 }
 

@@ -44,7 +44,7 @@ bool sm100_fwd_supported(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
 bool sm100_bwd_supported(const Problem& p);
 size_t sm100_bwd_workspace_bytes(long long pairs, int n);
-cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 4 kernels
+cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 3 kernels
 
 // Per-kernel device timing (off unless rib_profile_begin was called): records a CUDA event on
 // `stream` before (phase 0) and after (phase 1) the launch of kernel `kernel_id` (RIB_KERNEL_*).
