@@ -384,10 +384,12 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             merge[half * kTile + row] = make_float2(m_used, l);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kMerge + 4 * qt + quarter));
-            // both halves' last PV must have completed, and the partner's (m, l) must be there
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kPFree + 2 * qt), (blk - 1) & 1, abort_flag, p.status) &&
-                                             mbar_wait(bar(kPFree + 2 * qt + 1), (blk - 1) & 1, abort_flag, p.status) &&
-                                             mbar_wait(bar(kMerge + 4 * qt + quarter), nitem & 1, abort_flag, p.status))) { ok = false; break; }
+            // The partner's (m, l) must be there and both halves' last PV must have completed.  The
+            // merge barrier comes first: a parity wait on the partner's PV barrier is only meaningful once
+            // the partner has passed its own last block (otherwise an older phase of equal parity answers).
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(kMerge + 4 * qt + quarter), nitem & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kPFree + 2 * qt + half), (blk - 1) & 1, abort_flag, p.status) &&
+                                             mbar_wait(bar(kPFree + 2 * qt + (half ^ 1)), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
             tc_fence_after();
             uint32_t oa[16], ob[16];
             tmem_ld16(t_o + half * 16, oa);
