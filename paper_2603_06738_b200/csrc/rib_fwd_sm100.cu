@@ -298,7 +298,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg2);
-                const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                // the exp (MUFU) pipe is the busiest unit of this kernel: every fourth pair goes to the FMA pipe instead
+                const float2 e = (i & 3) == 3 ? ex2_poly2(x) : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                 if (i & 1) sum_b = __fadd2_rn(sum_b, e); else sum_a = __fadd2_rn(sum_a, e);
                 packed[i] = pack_bf16x2(e.x, e.y);
             }
