@@ -276,6 +276,31 @@ def main():
     else:
         e2e_ms, h2d, d2h = None, 0, 0
 
+    # ------------------------------------------------ RIB feature generator (Eq. 1-3), the step before the path
+    gen = None
+    if rank == 0:
+        gL, gdh = 10, 32                                    # the paper's L and d_h
+        gw = [torch.randn(sz, device=dev) * 0.3 for sz in ((2 + 4 * gL, gdh), (gdh,), (gdh, wl.r), (gdh, wl.r))]
+        gd = [torch.randn((wl.n, wl.r), device=dev) for _ in range(2)]
+        for _ in range(5):
+            binding.rib_generate_features(*gw, wl.window)
+            binding.rib_generate_features_bwd(*gw, *gd, wl.window)
+        torch.cuda.synchronize()
+        g0, g1, g2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        reps = 50
+        g0.record()
+        for _ in range(reps):
+            binding.rib_generate_features(*gw, wl.window)
+        g1.record()
+        for _ in range(reps):
+            binding.rib_generate_features_bwd(*gw, *gd, wl.window)
+        g2.record()
+        torch.cuda.synchronize()
+        gen = {"window": wl.window, "L": gL, "dh": gdh, "r": wl.r, "fwd_us": g0.elapsed_time(g1) * 1e3 / reps,
+               "bwd_us": g1.elapsed_time(g2) * 1e3 / reps, "bound": "launch latency",
+               "algorithmic_bytes_fwd": 4 * ((2 + 4 * gL) * gdh + gdh + 2 * gdh * wl.r) + 2 * 2 * wl.n * wl.r,
+               "algorithmic_flops_fwd": 2 * wl.n * ((2 + 4 * gL) * gdh + 2 * gdh * wl.r)}
+
     # ------------------------------------------------ reduce over ranks (max time), compose the line
     total_ms, fwd_med, bwd_med, e2e_ms_max = multi.max_over_ranks(
         [total_ms, statistics.median(fwd_ms), statistics.median(bwd_ms), e2e_ms or 0.0], device=dev)
@@ -333,6 +358,7 @@ def main():
             "value": flops_step / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_max,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
+        "generator": gen,
         "clocks": sampler.summary(),
         "wall_s": t_wall,
         "device_status": status,

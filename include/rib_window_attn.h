@@ -121,6 +121,31 @@ int rib_window_attn_bwd_noalloc(const void* q, const void* k, const void* v, con
                                 void* dq, void* dk, void* dv, float* dpq, float* dpk, void* stream);
 
 /*
+ * RIB feature generator (paper: Sec. 3.1, Eq. 1, Eq. 2, Eq. 3): the step right before the attention
+ * path.  Every token of a window x window attention window gets a normalised 2-D coordinate, the
+ * Fourier embedding r_in = [x, sin(2^0 x), cos(2^0 x), ..., sin(2^(L-1) x), cos(2^(L-1) x)] of width
+ * 2 + 4 L (Eq. 1), a hidden vector h = ReLU(r_in W_h + b_h) of width dh (Eq. 2), and the positional
+ * features Pq = h W_pq, Pk = h W_pk of width r (Eq. 3), which are the pq / pk arguments above.
+ * The features depend only on the window geometry and the weights, so at inference they are
+ * computed once and cached.
+ *   Coordinates (the paper does not fix them): `window` points from -1 to 1 inclusive per axis (one
+ *   point: 0); token i = y * window + x has the coordinate (row, column).  Frequencies 2^l, no pi.
+ *   w_h  : fp32 [2 + 4 L][dh]   b_h : fp32 [dh]   w_pq, w_pk : fp32 [dh][r]        (device, row-major)
+ *   pq, pk : bf16 [window * window][r], overwritten.
+ * Backward: given dpq, dpk (fp32 [n][r], e.g. from rib_window_attn_bwd) it overwrites
+ *   dw_h [2 + 4 L][dh], db_h [dh], dw_pq, dw_pk [dh][r] (fp32) with the gradients of
+ *   sum(Pq o dpq) + sum(Pk o dpk); the bf16 rounding of pq / pk is treated as the identity.
+ *   The results are zero-filled on `stream` and accumulated with atomic adds over slices of 128 tokens.
+ * Limits: 1 <= window <= 256, 0 <= L <= 16, 1 <= dh <= 64, 1 <= r <= 64; otherwise RIB_ERR_UNSUPPORTED
+ * (RIB_ERR_SHAPE for non-positive sizes).  Pointers 16-byte aligned.  Both calls only enqueue work.
+ */
+int rib_generate_features(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk,
+                          int window, int L, int dh, int r, void* pq, void* pk, void* stream);
+int rib_generate_features_bwd(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk,
+                              const float* dpq, const float* dpk, int window, int L, int dh, int r,
+                              float* dw_h, float* db_h, float* dw_pq, float* dw_pk, void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the device status word.  Kernels of this library
  * never spin without a limit: a wait that runs out records RIB_ERR_DEVICE_WAIT there and the
  * kernel returns (results of that launch are then invalid).  Returns RIB_OK, RIB_ERR_DEVICE_WAIT
@@ -154,7 +179,7 @@ long long rib_kernel_launches(void);
  */
 enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH = 4,
        RIB_KERNEL_RESERVED = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
-       RIB_KERNEL_ANY_BWD_DKV = 9 };
+       RIB_KERNEL_ANY_BWD_DKV = 9, RIB_KERNEL_GENERATOR_FWD = 10, RIB_KERNEL_GENERATOR_BWD = 11 };
 int rib_profile_begin(int max_launches);
 int rib_profile_end(int* kernel_ids, float* ms, int capacity);
 

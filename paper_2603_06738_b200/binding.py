@@ -22,10 +22,12 @@ EXPORTS = (
     "rib_window_attn_fwd", "rib_window_attn_bwd", "rib_window_attn_bwd_workspace",
     "rib_query_status", "rib_status_string", "rib_set_path", "rib_last_path", "rib_kernel_launches",
     "rib_window_attn_bwd_noalloc", "rib_profile_begin", "rib_profile_end",
+    "rib_generate_features", "rib_generate_features_bwd",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
-                7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel"}
+                7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel",
+                10: "rib_generator_fwd_kernel", 11: "rib_generator_bwd_kernel"}
 RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
@@ -54,6 +56,10 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_bwd.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
         lib.rib_window_attn_bwd_noalloc.restype = ci
         lib.rib_window_attn_bwd_noalloc.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp]
+        lib.rib_generate_features.restype = ci
+        lib.rib_generate_features.argtypes = [vp] * 4 + [ci] * 4 + [vp] * 3
+        lib.rib_generate_features_bwd.restype = ci
+        lib.rib_generate_features_bwd.argtypes = [vp] * 6 + [ci] * 4 + [vp] * 5
         lib.rib_profile_begin.restype = ci
         lib.rib_profile_begin.argtypes = [ci]
         lib.rib_profile_end.restype = ci
@@ -209,3 +215,38 @@ def rib_window_attn_bwd_noalloc(q, k, v, pq, pk, out, lse, dout, dq, dk, dv, dpq
                                                _ptr(dv), _ptr(dpq), _ptr(dpk), _stream_ptr(stream))
     if rc != RIB_OK:
         raise RibError(rc)
+
+
+def _check_f32(name, t, shape):
+    if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must be a contiguous CUDA float32 tensor of shape {tuple(shape)}")
+
+
+def rib_generate_features(w_h, b_h, w_pq, w_pk, window, stream=None):
+    """Pq, Pk (bf16 [window^2, r]) from the generator weights (Eq. 1-3); L is read off w_h's height 2 + 4 L."""
+    rows, dh = w_h.shape
+    L, r = (rows - 2) // 4, w_pq.shape[1]
+    _check_f32("w_h", w_h, (2 + 4 * L, dh)); _check_f32("b_h", b_h, (dh,))
+    _check_f32("w_pq", w_pq, (dh, r)); _check_f32("w_pk", w_pk, (dh, r))
+    pq = torch.empty((window * window, r), dtype=torch.bfloat16, device=w_h.device)
+    pk = torch.empty_like(pq)
+    rc = library().rib_generate_features(_ptr(w_h), _ptr(b_h), _ptr(w_pq), _ptr(w_pk), window, L, dh, r, _ptr(pq), _ptr(pk),
+                                         _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return pq, pk
+
+
+def rib_generate_features_bwd(w_h, b_h, w_pq, w_pk, dpq, dpk, window, stream=None):
+    """Gradients (dw_h, db_h, dw_pq, dw_pk) of the generator weights given dpq, dpk fp32 [window^2, r]."""
+    rows, dh = w_h.shape
+    L, r = (rows - 2) // 4, w_pq.shape[1]
+    _check_f32("w_h", w_h, (2 + 4 * L, dh)); _check_f32("b_h", b_h, (dh,))
+    _check_f32("w_pq", w_pq, (dh, r)); _check_f32("w_pk", w_pk, (dh, r))
+    _check_f32("dpq", dpq, (window * window, r)); _check_f32("dpk", dpk, (window * window, r))
+    outs = tuple(torch.empty_like(t) for t in (w_h, b_h, w_pq, w_pk))
+    rc = library().rib_generate_features_bwd(_ptr(w_h), _ptr(b_h), _ptr(w_pq), _ptr(w_pk), _ptr(dpq), _ptr(dpk), window, L, dh, r,
+                                             *[_ptr(t) for t in outs], _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return outs

@@ -248,6 +248,39 @@ int rib_window_attn_bwd_noalloc(const void* q, const void* k, const void* v, con
                                dpq, dpk, scratch, (size_t)RIB_NOALLOC_SCRATCH_BYTES, stream);
 }
 
+int rib_generate_features(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk,
+                          int window, int L, int dh, int r, void* pq, void* pk, void* stream)
+{
+    if (!w_h || !b_h || !w_pq || !w_pk || !pq || !pk) return RIB_ERR_NULL;
+    if (window <= 0 || L < 0 || dh <= 0 || r <= 0) return RIB_ERR_SHAPE;
+    if (!rib::generator_supported(window, L, dh, r)) return RIB_ERR_UNSUPPORTED;
+    const void* ptrs[] = {w_h, b_h, w_pq, w_pk, pq, pk};
+    for (const void* ptr : ptrs)
+        if (!aligned16(ptr)) return RIB_ERR_ALIGN;
+    const cudaError_t e = rib::generator_fwd(w_h, b_h, w_pq, w_pk, window, L, dh, r, static_cast<__nv_bfloat16*>(pq),
+                                             static_cast<__nv_bfloat16*>(pk), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
+int rib_generate_features_bwd(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk,
+                              const float* dpq, const float* dpk, int window, int L, int dh, int r,
+                              float* dw_h, float* db_h, float* dw_pq, float* dw_pk, void* stream)
+{
+    if (!w_h || !b_h || !w_pq || !w_pk || !dpq || !dpk || !dw_h || !db_h || !dw_pq || !dw_pk) return RIB_ERR_NULL;
+    if (window <= 0 || L < 0 || dh <= 0 || r <= 0) return RIB_ERR_SHAPE;
+    if (!rib::generator_supported(window, L, dh, r)) return RIB_ERR_UNSUPPORTED;
+    const void* ptrs[] = {w_h, b_h, w_pq, w_pk, dpq, dpk, dw_h, db_h, dw_pq, dw_pk};
+    for (const void* ptr : ptrs)
+        if (!aligned16(ptr)) return RIB_ERR_ALIGN;
+    const cudaError_t e = rib::generator_bwd(w_h, b_h, w_pq, w_pk, dpq, dpk, window, L, dh, r, dw_h, db_h, dw_pq, dw_pk,
+                                             static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
 int rib_query_status(void* stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);

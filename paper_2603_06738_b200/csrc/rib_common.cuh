@@ -46,6 +46,12 @@ bool sm100_bwd_supported(const Problem& p);
 size_t sm100_bwd_workspace_bytes(long long pairs, int n);
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 3 kernels
 
+bool generator_supported(int window, int L, int dh, int r);
+cudaError_t generator_fwd(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk, int window, int L, int dh, int r,
+                          __nv_bfloat16* pq, __nv_bfloat16* pk, cudaStream_t stream);
+cudaError_t generator_bwd(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk, const float* dpq, const float* dpk,
+                          int window, int L, int dh, int r, float* dw_h, float* db_h, float* dw_pq, float* dw_pk, cudaStream_t stream);
+
 // Per-kernel device timing (off unless rib_profile_begin was called): records a CUDA event on
 // `stream` before (phase 0) and after (phase 1) the launch of kernel `kernel_id` (RIB_KERNEL_*).
 void profile_mark(int kernel_id, int phase, cudaStream_t stream);
