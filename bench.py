@@ -136,7 +136,8 @@ def run_reference(args, wl, rank):
         "impl": "reference", "metric": METRIC, "value": best["value"], "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": 1, "ms_per_step": secs * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "note": "each step is a bounded sample of the workload: " + best["sample"]},
+        "config": {"workload": wl.name + " (forward + backward)",
+                   "note": "each step is a bounded sample of the workload: " + best["sample"]},
         "cpu_baseline": {k: best[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": best["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,

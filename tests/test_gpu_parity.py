@@ -122,6 +122,26 @@ def test_config5_full_forward_backward():
     compare("dpk", to_f64(dpk), rdpk, max_abs=1e-2 * scale)
 
 
+def test_largest_paper_window_96_forward_and_backward():
+    """The paper's largest attention window (96 x 96 = 9216 tokens per window, 72 key blocks): the
+    whole 96 x 96 map is one shifted window per head."""
+    wl = Workload("w96_s48", 1, 96, 96, 2, 32, 16, 96, 48, seed=33)
+    cpu, gpu = make(wl, with_dout=True)
+    out, lse = run_fwd(gpu, wl)
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    dq, dk, dv, dpq, dpk = run_bwd(gpu, wl, out, lse)
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    ref_out, ref_lse = oracle_fwd(cpu, wl)
+    compare("out", to_f64(out), ref_out)
+    compare("lse", to_f64(lse), ref_lse)
+    rdq, rdk, rdv, rdpq, rdpk = oracle_bwd(cpu, wl)
+    compare("dq", to_f64(dq), rdq)
+    compare("dk", to_f64(dk), rdk)
+    compare("dv", to_f64(dv), rdv)
+    compare("dpq", to_f64(dpq), rdpq)
+    compare("dpk", to_f64(dpk), rdpk)
+
+
 @pytest.mark.parametrize("direction", ["growing", "shrinking"])
 def test_running_maximum_rescale(direction):
     """Logits that grow (or shrink) steeply along the key order force the online-softmax rescale
