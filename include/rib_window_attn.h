@@ -92,6 +92,31 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
 size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window);
 
 /*
+ * Head-wise positional features (Sec. 3.1, the remark after Eq. 3: the hidden vector h is shared by
+ * the heads and every head has its own projections, hence its own Pq and Pk).  The three entry
+ * points below are rib_window_attn_fwd / _bwd / _bwd_workspace with one more argument:
+ *   pos_head_stride : elements between the tables of consecutive heads.  pq and pk are then
+ *                     bf16 [heads][n][r] and dpq, dpk fp32 with the same element stride; head h
+ *                     reads pq + h * pos_head_stride and its gradients are summed over the
+ *                     batch and the windows only.  Must be a multiple of 8 and at least n * r.
+ *                     0 means one [n][r] table for all heads, i.e. exactly the calls above.
+ * Anything else (layouts, workspace ownership, error codes, zero-fill of dpq / dpk over the
+ * tables' extent) is as stated above.  A bad stride returns RIB_ERR_SHAPE.
+ */
+int rib_window_attn_fwd_headwise(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                                 long long pos_head_stride,
+                                 int B, int H, int W, int heads, int d, int r, int window, int shift,
+                                 void* out, float* lse, void* stream);
+int rib_window_attn_bwd_headwise(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                                 long long pos_head_stride,
+                                 const void* out, const float* lse, const void* dout,
+                                 int B, int H, int W, int heads, int d, int r, int window, int shift,
+                                 void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+size_t rib_window_attn_bwd_headwise_workspace(long long pos_head_stride, int B, int H, int W, int heads, int d, int r,
+                                              int window);
+
+/*
  * Backward pass for callers that cannot hand over scratch memory.  (The paper has no counterpart:
  * this entry point exists for the library's users, not for the method.)
  *

@@ -23,6 +23,7 @@ EXPORTS = (
     "rib_query_status", "rib_status_string", "rib_set_path", "rib_last_path", "rib_kernel_launches",
     "rib_window_attn_bwd_noalloc", "rib_profile_begin", "rib_profile_end",
     "rib_generate_features", "rib_generate_features_bwd",
+    "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
@@ -54,6 +55,13 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_fwd.argtypes = [vp] * 5 + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd.restype = ci
         lib.rib_window_attn_bwd.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        ll = ctypes.c_longlong
+        lib.rib_window_attn_fwd_headwise.restype = ci
+        lib.rib_window_attn_fwd_headwise.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
+        lib.rib_window_attn_bwd_headwise.restype = ci
+        lib.rib_window_attn_bwd_headwise.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_attn_bwd_headwise_workspace.restype = ctypes.c_size_t
+        lib.rib_window_attn_bwd_headwise_workspace.argtypes = [ll] + [ci] * 7
         lib.rib_window_attn_bwd_noalloc.restype = ci
         lib.rib_window_attn_bwd_noalloc.argtypes = [vp] * 8 + [ci] * 8 + [vp] * 5 + [vp]
         lib.rib_generate_features.restype = ci
@@ -99,6 +107,12 @@ def _check_image(name, t, shape=None):
 def _check_pos(name, t, n):
     if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 2 or t.shape[0] != n:
         raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor [n={n}, r]")
+
+
+def _check_pos_headwise(name, t, heads, n):
+    if (t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 3
+            or t.shape[0] != heads or t.shape[1] != n):
+        raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor [heads={heads}, n={n}, r]")
 
 
 def rib_status_string(code: int) -> str:
@@ -184,6 +198,56 @@ def rib_window_attn_bwd(q, k, v, pq, pk, out, lse, dout, window, shift=0, worksp
                                        _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq), _ptr(dk),
                                        _ptr(dv), _ptr(dpq), _ptr(dpk), _ptr(workspace), workspace.numel(),
                                        _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return dq, dk, dv, dpq, dpk
+
+
+def rib_window_attn_bwd_headwise_workspace(pos_head_stride, B, H, W, heads, d, r, window) -> int:
+    return int(library().rib_window_attn_bwd_headwise_workspace(pos_head_stride, B, H, W, heads, d, r, window))
+
+
+def rib_window_attn_fwd_headwise(q, k, v, pq, pk, window, shift=0, stream=None, want_lse=True):
+    """Forward pass with one Pq/Pk table per head: pq, pk bf16 [heads, n, r]; returns (out, lse)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    _check_image("k", k, q.shape)
+    _check_image("v", v, q.shape)
+    n = window * window
+    _check_pos_headwise("pq", pq, heads, n)
+    _check_pos_headwise("pk", pk, heads, n)
+    r = pq.shape[2]
+    out = torch.empty_like(q)
+    lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device) if want_lse else None
+    rc = library().rib_window_attn_fwd_headwise(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r, B, H, W, heads,
+                                                d, r, window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return out, lse
+
+
+def rib_window_attn_bwd_headwise(q, k, v, pq, pk, out, lse, dout, window, shift=0, workspace=None, stream=None):
+    """Backward pass with one Pq/Pk table per head; returns (dq, dk, dv bf16, dpq, dpk fp32 [heads, n, r])."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    for name, t in (("k", k), ("v", v), ("out", out), ("dout", dout)):
+        _check_image(name, t, q.shape)
+    n = window * window
+    _check_pos_headwise("pq", pq, heads, n)
+    _check_pos_headwise("pk", pk, heads, n)
+    r = pq.shape[2]
+    if lse.dtype != torch.float32 or tuple(lse.shape) != (B, heads, H, W) or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous fp32 tensor [B,heads,H,W]")
+    need = rib_window_attn_bwd_headwise_workspace(n * r, B, H, W, heads, d, r, window)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dpq = torch.empty((heads, n, r), dtype=torch.float32, device=q.device)
+    dpk = torch.empty((heads, n, r), dtype=torch.float32, device=q.device)
+    rc = library().rib_window_attn_bwd_headwise(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r, _ptr(out),
+                                                _ptr(lse), _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq),
+                                                _ptr(dk), _ptr(dv), _ptr(dpq), _ptr(dpk), _ptr(workspace),
+                                                workspace.numel(), _stream_ptr(stream))
     if rc != RIB_OK:
         raise RibError(rc)
     return dq, dk, dv, dpq, dpk

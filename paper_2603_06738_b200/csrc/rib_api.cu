@@ -43,6 +43,13 @@ void fill_shape(rib::Problem& p, int B, int H, int W, int heads, int d, int r, i
     p.pairs = B * p.nWy * p.nWx * heads;
 }
 
+int check_pos_stride(long long stride, int window, int r)
+{
+    if (stride == 0) return RIB_OK;
+    if (stride < (long long)window * window * r || (stride & 7)) return RIB_ERR_SHAPE;
+    return RIB_OK;
+}
+
 size_t rowdot_bytes(int B, int H, int W, int heads)
 {
     const size_t bytes = sizeof(float) * (size_t)B * H * W * heads;
@@ -154,8 +161,17 @@ int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void*
                         int B, int H, int W, int heads, int d, int r, int window, int shift,
                         void* out, float* lse, void* stream)
 {
+    return rib_window_attn_fwd_headwise(q, k, v, pq, pk, 0, B, H, W, heads, d, r, window, shift, out, lse, stream);
+}
+
+int rib_window_attn_fwd_headwise(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                                 long long pos_head_stride,
+                                 int B, int H, int W, int heads, int d, int r, int window, int shift,
+                                 void* out, float* lse, void* stream)
+{
     if (!q || !k || !v || !out || (r > 0 && (!pq || !pk))) return RIB_ERR_NULL;
     if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    if (int rc = check_pos_stride(pos_head_stride, window, r)) return rc;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(pq) ||
         !aligned16(pk) || !aligned16(lse))
         return RIB_ERR_ALIGN;
@@ -168,6 +184,7 @@ int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void*
     p.pk = static_cast<const __nv_bfloat16*>(pk);
     p.out_w = static_cast<__nv_bfloat16*>(out);
     p.lse_w = lse;
+    p.pos_head_stride = pos_head_stride;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
@@ -180,12 +197,19 @@ int rib_window_attn_fwd(const void* q, const void* k, const void* v, const void*
 
 size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window)
 {
+    return rib_window_attn_bwd_headwise_workspace(0, B, H, W, heads, d, r, window);
+}
+
+size_t rib_window_attn_bwd_headwise_workspace(long long pos_head_stride, int B, int H, int W, int heads, int d, int r,
+                                              int window)
+{
     if (check_shape(B, H, W, heads, d, r, window, 0) != RIB_OK) return 0;
+    if (check_pos_stride(pos_head_stride, window, r) != RIB_OK) return 0;
     size_t need = rowdot_bytes(B, H, W, heads);
     rib::Problem p{};
     fill_shape(p, B, H, W, heads, d, r, window, 0);
     if (rib::sm100_bwd_supported(p)) {   // whatever the shift: one size per shape
-        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n);
+        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1);
         if (fast > need) need = fast;
     }
     return need;
@@ -197,13 +221,25 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
                         void* dq, void* dk, void* dv, float* dpq, float* dpk,
                         void* workspace, size_t workspace_bytes, void* stream)
 {
+    return rib_window_attn_bwd_headwise(q, k, v, pq, pk, 0, out, lse, dout, B, H, W, heads, d, r, window, shift, dq, dk, dv,
+                                        dpq, dpk, workspace, workspace_bytes, stream);
+}
+
+int rib_window_attn_bwd_headwise(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                                 long long pos_head_stride,
+                                 const void* out, const float* lse, const void* dout,
+                                 int B, int H, int W, int heads, int d, int r, int window, int shift,
+                                 void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                                 void* workspace, size_t workspace_bytes, void* stream)
+{
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return RIB_ERR_NULL;
     if (r > 0 && (!pq || !pk || !dpq || !dpk)) return RIB_ERR_NULL;
     if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    if (int rc = check_pos_stride(pos_head_stride, window, r)) return rc;
     const void* ptrs[] = {q, k, v, pq, pk, out, lse, dout, dq, dk, dv, dpq, dpk};
     for (const void* ptr : ptrs)
         if (!aligned16(ptr)) return RIB_ERR_ALIGN;
-    const size_t need = rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window);
+    const size_t need = rib_window_attn_bwd_headwise_workspace(pos_head_stride, B, H, W, heads, d, r, window);
     if (!workspace || workspace_bytes < need) return RIB_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return RIB_ERR_ALIGN;
     rib::Problem p{};
@@ -224,6 +260,7 @@ int rib_window_attn_bwd(const void* q, const void* k, const void* v, const void*
     p.rowdot = static_cast<float*>(workspace);
     p.workspace = workspace;
     p.workspace_bytes = workspace_bytes;
+    p.pos_head_stride = pos_head_stride;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_bwd_supported(p);

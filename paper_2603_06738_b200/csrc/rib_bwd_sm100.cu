@@ -79,6 +79,7 @@ struct BwdParams {
     __nv_bfloat16* dv;
     int* status;
     int H, W, heads, M, s, n, nWy, nWx, nblk, items;
+    int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
     float scale_log2;          // log2(e) / sqrt(d)
     float inv_sqrt_d;
 };
@@ -153,7 +154,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     patch_origin(geom, c.wy, c.wx, 2 * c.J + sub, py, px, Y0, X0);
                     tma_load_5d(base + kOffKc + slot * kContentBytes + sub * kPatchContent, &tm_k, bar(kKVFull + slot),
                                 0, c.h, X0, Y0, c.b);
-                    tma_load_3d(base + kOffKp + slot * kContentBytes + sub * kPatchContent, &tm_pk, bar(kKVFull + slot), 0, px, py);
+                    tma_load_4d(base + kOffKp + slot * kContentBytes + sub * kPatchContent, &tm_pk, bar(kKVFull + slot), 0, px, py, c.h * p.pos_per_head);
                     tma_load_5d(base + kOffV + slot * kContentBytes + sub * kPatchContent, &tm_v, bar(kKVFull + slot),
                                 0, c.h, X0, Y0, c.b);
                 }
@@ -167,7 +168,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         int py, px, Y0, X0;
                         patch_origin(geom, c.wy, c.wx, 2 * I + sub, py, px, Y0, X0);
                         tma_load_5d(ring + kRingQc + sub * kPatchContent, &tm_q, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
-                        tma_load_3d(ring + kRingQp + sub * kPatchContent, &tm_pqs, bar(kQFull + st), 0, px, py);
+                        tma_load_4d(ring + kRingQp + sub * kPatchContent, &tm_pqs, bar(kQFull + st), 0, px, py, c.h * p.pos_per_head);
                         tma_load_5d(ring + kRingDO + sub * kPatchContent, &tm_do, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
                     }
                     bulk_load_1d(ring + kRingLD, p.ld + (size_t)c.pair * p.n + (size_t)I * kTile, kLdBytes, bar(kQFull + st));
@@ -449,6 +450,8 @@ struct AuxParams {
     float* dpq;
     float* dpk;
     int H, W, heads, M, s, n, nWy, nWx, pairs;
+    int tables;                  // Pq/Pk tables: 1 (shared by the heads) or heads
+    long long pos_head_stride;   // elements between the tables in pq, dpq, dpk (pq_scaled is packed: n * 16 apart)
     float pos_scale, inv_sqrt_d, inv_sqrt_r;
 };
 
@@ -472,10 +475,12 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     const size_t total = (size_t)p.pairs * p.n;
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-    for (size_t e = t; e < (size_t)p.n * kR; e += nthreads) {
-        p.pq_scaled[e] = __float2bfloat16_rn(__bfloat162float(p.pq[e]) * p.pos_scale);
-        p.dpq[e] = 0.f;
-        p.dpk[e] = 0.f;
+    const size_t per_table = (size_t)p.n * kR;
+    for (size_t e = t; e < per_table * p.tables; e += nthreads) {
+        const size_t user = (e / per_table) * (size_t)p.pos_head_stride + e % per_table;
+        p.pq_scaled[e] = __float2bfloat16_rn(__bfloat162float(p.pq[user]) * p.pos_scale);
+        p.dpq[user] = 0.f;
+        p.dpk[user] = 0.f;
     }
     if (t >= total) return;
     const int pair = (int)(t / p.n), w = (int)(t % p.n);
@@ -504,20 +509,32 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
 }
 
 // Finishing pass over the fp32 accumulators.  grid (n / 128, groups of pairs), 128 threads: a thread
-// owns one token position w of the window and walks the pairs of its group.  Per pair it turns
+// owns one token position w of the window and walks the pairs of its group.  With one table for all
+// heads a group is a run of consecutive pairs; with head-wise tables it is a run of windows of one
+// head (pair = head + heads * window), so that its sums belong to one table.  Per pair it turns
 // dQ~[:, :d] / sqrt(d) into the bf16 dq row of that token, and it keeps running sums of the 16 RIB
 // columns of dQ~ (-> dPq, times 1/sqrt(r)) and of dK~ (-> dPk); the group's partial sums go to the
 // zeroed results with one vector atomic per 4 columns.
 __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_group)
 {
     const int w = blockIdx.x * 128 + threadIdx.x;
-    const int pair0 = blockIdx.y * pairs_per_group;
-    const int pair1 = min(p.pairs, pair0 + pairs_per_group);
+    int pair0, pair1, step = 1;
+    size_t table = 0;
+    if (p.tables == 1) {
+        pair0 = blockIdx.y * pairs_per_group;
+        pair1 = min(p.pairs, pair0 + pairs_per_group);
+    } else {
+        const int head = blockIdx.y % p.heads, first = (blockIdx.y / p.heads) * pairs_per_group;
+        step = p.heads;
+        pair0 = head + first * step;
+        pair1 = min(p.pairs, pair0 + pairs_per_group * step);
+        table = (size_t)head * (size_t)p.pos_head_stride;
+    }
     float sq[kR], sk[kR];
 #pragma unroll
     for (int c = 0; c < kR; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
     int i = 0;
-    for (int pair = pair0; pair < pair1; ++pair) {
+    for (int pair = pair0; pair < pair1; pair += step) {
         size_t tok, scalar;
         decode_pair_token(p, pair, w, i, tok, scalar);
         const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
@@ -537,8 +554,8 @@ __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, 
         }
     }
     if (pair0 >= pair1) return;
-    float4* out_q = reinterpret_cast<float4*>(p.dpq + (size_t)i * kR);
-    float4* out_k = reinterpret_cast<float4*>(p.dpk + (size_t)i * kR);
+    float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * kR);
+    float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * kR);
 #pragma unroll
     for (int c4 = 0; c4 < kR / 4; ++c4) {
         atomicAdd(out_q + c4, make_float4(sq[4 * c4] * p.inv_sqrt_r, sq[4 * c4 + 1] * p.inv_sqrt_r, sq[4 * c4 + 2] * p.inv_sqrt_r,
@@ -551,14 +568,14 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WorkspaceLayout { size_t ld, dq_acc, dkp, pq_scaled, total; };
 
-WorkspaceLayout workspace_layout(long long pairs, int n)
+WorkspaceLayout workspace_layout(long long pairs, int n, int tables)
 {
     WorkspaceLayout w;
     w.ld = 0;
     w.dq_acc = w.ld + align256((size_t)pairs * n * sizeof(float2));
     w.dkp = w.dq_acc + align256((size_t)pairs * kDk * n * sizeof(float));
     w.pq_scaled = w.dkp + align256((size_t)pairs * kR * n * sizeof(float));
-    w.total = w.pq_scaled + align256((size_t)n * kR * sizeof(__nv_bfloat16));
+    w.total = w.pq_scaled + align256((size_t)tables * n * kR * sizeof(__nv_bfloat16));
     return w;
 }
 
@@ -569,12 +586,13 @@ bool sm100_bwd_supported(const Problem& p)
     return p.d == sm100::kD && p.r == sm100::kR && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
 }
 
-size_t sm100_bwd_workspace_bytes(long long pairs, int n) { return workspace_layout(pairs, n).total; }
+size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables) { return workspace_layout(pairs, n, tables).total; }
 
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
-    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n);
+    const int tables = pos_tables(p);
+    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n, tables);
     if (p.workspace_bytes < wl.total) return cudaErrorInvalidValue;
     uint8_t* ws = static_cast<uint8_t*>(p.workspace);
     float2* ld = reinterpret_cast<float2*>(ws + wl.ld);
@@ -584,8 +602,8 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 
     CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
-        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p) ||
-        !encode_pos_map_padded(&tm_pk, p.pk, p))
+        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * kR) ||
+        !encode_pos_map_padded(&tm_pk, p.pk, p, tables, p.pos_head_stride))
         return cudaErrorInvalidValue;
     static int sm_count = 0;
     if (!sm_count) {
@@ -600,6 +618,8 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     ap.dq = p.dq; ap.dpq = p.dpq; ap.dpk = p.dpk;
     ap.H = p.H; ap.W = p.W; ap.heads = p.heads; ap.M = p.M; ap.s = p.s; ap.n = p.n; ap.nWy = p.nWy; ap.nWx = p.nWx;
     ap.pairs = p.pairs;
+    ap.tables = tables;
+    ap.pos_head_stride = p.pos_head_stride;
     ap.pos_scale = sqrtf((float)p.d / (float)p.r);
     ap.inv_sqrt_d = 1.f / sqrtf((float)p.d);
     ap.inv_sqrt_r = 1.f / sqrtf((float)p.r);
@@ -614,6 +634,7 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     bp.H = p.H; bp.W = p.W; bp.heads = p.heads; bp.M = p.M; bp.s = p.s; bp.n = p.n; bp.nWy = p.nWy; bp.nWx = p.nWx;
     bp.nblk = p.n / kTile;
     bp.items = p.pairs * bp.nblk;
+    bp.pos_per_head = tables > 1 ? 1 : 0;
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
@@ -622,7 +643,10 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     if (e != cudaSuccess) return e;
 
     const int per_group = p.pairs < 8 ? 1 : 4;
-    dim3 grid_fin((unsigned)(p.n / 128), (unsigned)((p.pairs + per_group - 1) / per_group));
+    const int windows = p.pairs / p.heads;   // pairs of one head
+    const unsigned groups = tables == 1 ? (unsigned)((p.pairs + per_group - 1) / per_group)
+                                        : (unsigned)(p.heads * ((windows + per_group - 1) / per_group));
+    dim3 grid_fin((unsigned)(p.n / 128), groups);
     { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<<<grid_fin, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();
 }

@@ -30,10 +30,19 @@ struct Problem {
     float* rowdot;              // any-shape backward: D_i = sum_c dout_ic * out_ic, image layout of lse
     void* workspace;            // caller's scratch (backward), 256-byte aligned
     size_t workspace_bytes;
+    long long pos_head_stride;        // elements between the heads' tables in pq/pk/dpq/dpk; 0 = one table for all heads
     int B, H, W, heads, d, r, M, s;   // M = window side, s = cyclic shift
     int n, nWy, nWx, pairs;           // n = M*M, windows per image, B*nWy*nWx*heads
     int* status;                      // device status word (bounded waits report here)
 };
+
+// Pq/Pk tables: one shared by the heads, or one per head (Sec. 3.1, after Eq. 3: head-wise projections of the shared h).
+inline int pos_tables(const Problem& p) { return p.pos_head_stride ? p.heads : 1; }
+// Elements from the first entry of the first table to the end of the last one.
+inline size_t pos_extent(const Problem& p)
+{
+    return (size_t)(pos_tables(p) - 1) * (size_t)p.pos_head_stride + (size_t)p.n * p.r;
+}
 
 // Launchers; each returns the cudaError_t of its launches.
 cudaError_t generic_fwd(const Problem& p, cudaStream_t stream);
@@ -43,7 +52,7 @@ cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream);
 bool sm100_fwd_supported(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
 bool sm100_bwd_supported(const Problem& p);
-size_t sm100_bwd_workspace_bytes(long long pairs, int n);
+size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables);
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 3 kernels
 
 bool generator_supported(int window, int L, int dh, int r);

@@ -70,6 +70,8 @@ struct FwdParams {
     float scale_log2;          // log2(e) / sqrt(d)
     float inv_sqrt_d;
     float pos_scale;           // sqrt(d / r): folds 1/sqrt(r) into the content scale
+    long long pos_head_stride; // elements between the heads' Pq tables (0: one table for all heads)
+    int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
 };
 
 struct ItemCoord { int b, wy, wx, h, tp; };
@@ -159,8 +161,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         patch_origin(p, c, 2 * j + sub, py[sub], px[sub], Y0[sub], X0[sub]);
                         tma_load_5d(base + kOffKc + st * kContentBytes + sub * kPatchContent, &tm_k, bar(kKFull + st),
                                     0, c.h, X0[sub], Y0[sub], c.b);
-                        tma_load_3d(base + kOffKp + st * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKFull + st),
-                                    0, px[sub], py[sub]);
+                        tma_load_4d(base + kOffKp + st * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKFull + st),
+                                    0, px[sub], py[sub], c.h * p.pos_per_head);
                     }
                     if (use > 0 && !mbar_wait(bar(kVEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar(kVFull + st), kContentBytes);
@@ -257,7 +259,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 int py, px, Y0, X0;
                 patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
                 const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
-                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)token * kR);
+                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * kR);
                 uint4 v[2] = {__ldg(src), __ldg(src + 1)};
                 uint32_t* w = reinterpret_cast<uint32_t*>(v);
 #pragma unroll
@@ -447,7 +449,7 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
     if (!encode_fn()) return cudaErrorNotSupported;
     CUtensorMap tm_q, tm_k, tm_v, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
-        !encode_pos_map(&tm_pk, p.pk, p))
+        !encode_pos_map(&tm_pk, p.pk, p, pos_tables(p), p.pos_head_stride))
         return cudaErrorInvalidValue;
     static int sm_count = 0;
     if (!sm_count) {
@@ -464,6 +466,8 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
     fp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     fp.inv_sqrt_d = 1.f / sqrtf((float)p.d);
     fp.pos_scale = sqrtf((float)p.d / (float)p.r);
+    fp.pos_head_stride = p.pos_head_stride;
+    fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     const int grid = fp.items < sm_count ? fp.items : sm_count;
     { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
     return cudaGetLastError();

@@ -69,7 +69,7 @@ __device__ inline void stage_concat(const Problem& p, const PairCoord& c, const 
         float val = 0.f;
         if (i < p.n) {
             val = col < p.d ? __bfloat162float(x[token_offset(p, c, i) + col]) * sx
-                            : __bfloat162float(pos[(size_t)i * p.r + (col - p.d)]) * sp;
+                            : __bfloat162float(pos[(size_t)c.h * p.pos_head_stride + (size_t)i * p.r + (col - p.d)]) * sp;
         }
         dst[rr * ld + col] = val;
     }
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dq_kernel(const Problem 
         for (int t = 0; t < kMaxCols; ++t) {
             const int col = lane + 32 * t;
             if (col < p.d) p.dq[off + col] = __float2bfloat16_rn(acc[rr][t] * isd);
-            else if (col < dk) atomicAdd(p.dpq + (size_t)i * p.r + (col - p.d), acc[rr][t] * isr);
+            else if (col < dk) atomicAdd(p.dpq + (size_t)c.h * p.pos_head_stride + (size_t)i * p.r + (col - p.d), acc[rr][t] * isr);
         }
     }
 }
@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dkv_kernel(const Problem
         for (int t = 0; t < kMaxCols; ++t) {
             const int col = lane + 32 * t;
             if (col < p.d) p.dk[off + col] = __float2bfloat16_rn(accK[rr][t]);          // 1/sqrt d is in Qt
-            else if (col < dk) atomicAdd(p.dpk + (size_t)j * p.r + (col - p.d), accK[rr][t]);  // 1/sqrt r is in Qt
+            else if (col < dk) atomicAdd(p.dpk + (size_t)c.h * p.pos_head_stride + (size_t)j * p.r + (col - p.d), accK[rr][t]);  // 1/sqrt r is in Qt
         }
     }
 }
@@ -364,9 +364,10 @@ cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream)
 cudaError_t generic_bwd(const Problem& p, cudaStream_t stream)
 {
     const int dk = p.d + p.r;
-    cudaError_t e = cudaMemsetAsync(p.dpq, 0, sizeof(float) * (size_t)p.n * p.r, stream);
+    const size_t pos_floats = pos_extent(p);
+    cudaError_t e = cudaMemsetAsync(p.dpq, 0, sizeof(float) * pos_floats, stream);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(p.dpk, 0, sizeof(float) * (size_t)p.n * p.r, stream);
+    e = cudaMemsetAsync(p.dpk, 0, sizeof(float) * pos_floats, stream);
     if (e != cudaSuccess) return e;
     e = rowdot_prepass(p, stream);
     if (e != cudaSuccess) return e;

@@ -79,30 +79,32 @@ inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// bf16 [M][M][16] positional features, box = one 8x8-token patch.
-inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p)
+// bf16 [tables][M][M][16] positional features (one table shared by all heads, or one per head), box = one
+// 8x8-token patch of one table.  `tables` = 1 or heads, `table_stride` elements apart (a multiple of 8,
+// at least M * M * 16); a kernel addresses table h * (tables > 1).
+inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
+                                cuuint32_t box_inner, CUtensorMapSwizzle swz)
 {
-    const cuuint64_t dims[3] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M};
-    const cuuint64_t strides[2] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M};
-    const cuuint32_t box[3] = {(cuuint32_t)kR, 8, 8};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+    const cuuint64_t dims[4] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
+    const cuuint64_t one_table = (cuuint64_t)kR * 2 * p.M * p.M;
+    const cuuint64_t strides[3] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M,
+                                   tables > 1 ? (cuuint64_t)table_stride * 2 : one_table};
+    const cuuint32_t box[4] = {box_inner, 8, 8, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
+inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
+{
+    return encode_pos_map_impl(map, ptr, p, tables, table_stride, kR, CU_TENSOR_MAP_SWIZZLE_32B);
+}
 // The same features fetched as 64-byte rows: the box is 32 elements wide on a 16-element dimension, so
 // TMA fills the upper half of every row with zeros.  A 64-byte-row RIB tile has the layout of a content
 // tile (SWIZZLE_64B) and can sit behind it as the second 32-column atom of one MN-major operand.
-inline bool encode_pos_map_padded(CUtensorMap* map, const void* ptr, const Problem& p)
+inline bool encode_pos_map_padded(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
 {
-    const cuuint64_t dims[3] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M};
-    const cuuint64_t strides[2] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M};
-    const cuuint32_t box[3] = {(cuuint32_t)kD, 8, 8};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return encode_pos_map_impl(map, ptr, p, tables, table_stride, kD, CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
 inline cudaError_t sm_count_of_current_device(int* count)

@@ -69,6 +69,7 @@ class Workload:
     shift: int
     seed: int
     backward: bool = False
+    headwise: bool = False    # one Pq/Pk table per head ([heads, n, r]) instead of one for all heads
 
     @property
     def n(self) -> int:
@@ -104,11 +105,12 @@ CONFIGS = (
 
 
 def make_inputs(wl: Workload, with_dout: bool | None = None) -> dict[str, torch.Tensor]:
-    """CPU bf16 tensors q, k, v [B,H,W,heads,d], pq, pk [n,r] (and dout) for a workload."""
+    """CPU bf16 tensors q, k, v [B,H,W,heads,d], pq, pk [n,r] or [heads,n,r] (and dout) for a workload."""
     shape = (wl.B, wl.H, wl.W, wl.heads, wl.d)
     t = {name: bf16_tensor(wl.seed, name, shape, 1.0) for name in ("q", "k", "v")}
-    t["pq"] = bf16_tensor(wl.seed, "pq", (wl.n, wl.r), 0.5)
-    t["pk"] = bf16_tensor(wl.seed, "pk", (wl.n, wl.r), 0.5)
+    pos_shape = (wl.heads, wl.n, wl.r) if wl.headwise else (wl.n, wl.r)
+    t["pq"] = bf16_tensor(wl.seed, "pq", pos_shape, 0.5)
+    t["pk"] = bf16_tensor(wl.seed, "pk", pos_shape, 0.5)
     if wl.backward if with_dout is None else with_dout:
         t["dout"] = bf16_tensor(wl.seed, "dout", shape, 1.0)
     return t

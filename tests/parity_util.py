@@ -37,15 +37,16 @@ def make(wl: synthetic.Workload, with_dout=True):
 
 
 def run_fwd(gpu, wl):
-    out, lse = binding.rib_window_attn_fwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+    fwd = binding.rib_window_attn_fwd_headwise if wl.headwise else binding.rib_window_attn_fwd
+    out, lse = fwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
     return out, lse
 
 
 def run_bwd(gpu, wl, out, lse):
-    res = binding.rib_window_attn_bwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse, gpu["dout"],
-                                      wl.window, wl.shift)
+    bwd = binding.rib_window_attn_bwd_headwise if wl.headwise else binding.rib_window_attn_bwd
+    res = bwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse, gpu["dout"], wl.window, wl.shift)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
     return res
