@@ -26,11 +26,15 @@
 // bf16 and sums the RIB columns over pairs into dPq.  The RIB columns of dK~ are written per pair
 // and summed over pairs by the same finishing kernel into dPk.
 //
-// Roles (768 threads): warp 0 TMA producer; three MMA-issuing threads (the tensor pipe takes
+// Roles (768 threads): warp 0 TMA producer; three MMA-issuing warps (the tensor pipe takes
 // instructions from several warps at once, and one thread issuing everything was the bottleneck):
-// warp 1 issues S^T, dP^T and dV, warp 2 (also the TMEM allocator) dK~, warp 3 dQ~; warps 4-11
+// warp 1 issues S^T and dP^T, warp 2 (also the TMEM allocator) dV and dK~, warp 3 dQ~; warps 4-11
 // P/dS arithmetic of the even half-tiles, warps 12-19 of the odd ones (one thread per key row and 32
 // queries); warps 20-23 drain dQ~ after every tile and dK~/dV after every item.  Every wait is bounded.
+// What sets the pace is the latency of the loop  scores -> arithmetic -> gradient MMAs -> buffers free
+// divided by the two half-tiles in flight, so every buffer is handed back as early as its last reader
+// allows: the score accumulators when the arithmetic warps hold them in registers (long before their
+// exponentials are done), P^T / dS^T when dV and dK~ have consumed them.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -53,9 +57,9 @@ constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 25600
 constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 tiles][2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
 constexpr uint32_t kDSHalf = kTile * 128;
 constexpr uint32_t kOffBar = kOffDS + 4 * kDSHalf;
-// kSFull, kPReady, kPFree: one per half h; kDSFree: one per dS tile buffer
-enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kSIssued = kSFull + 2,
-           kPReady, kPFree = kPReady + 2, kDSFree = kPFree + 2, kDQFull = kDSFree + 2, kDQFree, kAccFull, kAccFree, kDrain,
+// kSFull, kSFree, kPReady, kPFree: one per half h; kDSFree: one per dS tile buffer
+enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kSFree = kSFull + 2,
+           kPReady = kSFree + 2, kPFree = kPReady + 2, kDSFree = kPFree + 2, kDQFull = kDSFree + 2, kDQFree, kAccFull, kAccFree, kDrain,
            kNumBars = kDrain + 3 };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;
 constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
@@ -117,13 +121,13 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (threadIdx.x == 0) {
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
-        for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 2); }
+        for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
         for (int h = 0; h < 2; ++h) {
-            mbar_init(bar(kSFull + h), 1); mbar_init(bar(kPReady + h), 8); mbar_init(bar(kPFree + h), 2); mbar_init(bar(kDSFree + h), 1);
+            mbar_init(bar(kSFull + h), 1); mbar_init(bar(kSFree + h), 8); mbar_init(bar(kPReady + h), 8); mbar_init(bar(kPFree + h), 1);
+            mbar_init(bar(kDSFree + h), 1);
         }
-        mbar_init(bar(kSIssued), 1);
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
-        mbar_init(bar(kAccFull), 2); mbar_init(bar(kAccFree), 4);
+        mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
         for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
         fence_barrier_init();
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
@@ -196,78 +200,58 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, p.status)) != 0; };
         bool ok = true;
         if (warp == 1) {
-            // ---- per unit u: S^T, dP^T of u as soon as the arithmetic group has taken unit u - 2 (same
-            // buffers) out of tensor memory, then dV_J += P^T dO of that unit u - 2
-            uint32_t s_nitem = 0, s_I = 0;                  // item ordinal / tile of the unit whose scores come next
-            uint32_t v_nitem = 0, v_I = 0;                  // the same for the unit whose dV comes next
+            // ---- S^T, dP^T of unit u as soon as the arithmetic group has read unit u - 2 (same buffers)
+            // out of tensor memory; the group is then still busy with that unit's exponentials
+            uint32_t nitem = 0, I = 0;
             uint32_t slot_base = 0;
-            for (uint32_t u = 0; u < total_units + 2 && ok; ++u) {
-                const uint32_t h = u & 1;
-                if (u >= 2 && !wait_all(bar(kPReady + h), ((u - 2) >> 1) & 1)) { ok = false; break; }
-                if (u < total_units) {
-                    const uint32_t g = u >> 1, st = g % kQStages, slot = s_nitem & 1;
-                    if (h == 0 && s_I == 0) {
-                        if (!wait_all(bar(kKVFull + slot), (s_nitem >> 1) & 1)) { ok = false; break; }
-                        slot_base = base + slot * kContentBytes;
-                    }
-                    if (h == 0 && !wait_all(bar(kQFull + st), (g / kQStages) & 1)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t ring = base + kOffRing + st * kRingBytes + h * kPatchContent;   // rows of patch h
-                    if (elect_one()) {
-                        const uint64_t kc = smem_desc_at(kDesc64, slot_base + kOffKc), kp = smem_desc_at(kDesc64, slot_base + kOffKp);
-                        const uint64_t v = smem_desc_at(kDesc64, slot_base + kOffV);
-                        const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc64, ring + kRingQp);
-                        const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
-                        const uint32_t d_s = tmem + kColS + h * kHalfCols, d_p = tmem + kColDP + h * kHalfCols;
-                        mma_ss(d_s, kc, qc, kIdescSS, 0u);
-                        mma_ss(d_s, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
-                        mma_ss(d_s, kp, qp, kIdescSS, 1u);
-                        mma_ss(d_p, v, go, kIdescSS, 0u);
-                        mma_ss(d_p, v + 2, go + 2, kIdescSS, 1u);
-                        mma_commit(bar(kSFull + h));
-                        if (u >= 2) mbar_arrive(bar(kSIssued));     // the gradient contractions of unit u - 2 may follow
-                    }
-                    __syncwarp();
-                    if (h == 1 && ++s_I == (uint32_t)nblk) { s_I = 0; ++s_nitem; }
+            for (uint32_t u = 0; u < total_units && ok; ++u) {
+                const uint32_t h = u & 1, g = u >> 1, st = g % kQStages, slot = nitem & 1;
+                if (u >= 2 && !wait_all(bar(kSFree + h), ((u - 2) >> 1) & 1)) { ok = false; break; }
+                if (h == 0 && I == 0) {
+                    if (!wait_all(bar(kKVFull + slot), (nitem >> 1) & 1)) { ok = false; break; }
+                    slot_base = base + slot * kContentBytes;
                 }
-                if (u >= 2) {
-                    // dV of unit u - 2 (tile v_I of item ordinal v_nitem, half h)
-                    const uint32_t g2 = (u - 2) >> 1, st2 = g2 % kQStages;
-                    const bool first = v_I == 0 && h == 0, last = v_I == (uint32_t)nblk - 1 && h == 1;
-                    if (first && v_nitem > 0 && !wait_all(bar(kAccFree), (v_nitem - 1) & 1)) { ok = false; break; }
-                    tc_fence_after();
-                    if (elect_one()) {
-                        const uint64_t go = smem_desc_at(kDesc64, base + kOffRing + st2 * kRingBytes + kRingDO + h * kPatchContent);
-                        const uint32_t a_p = tmem + kColP + h * (kHalfCols / 2);
-#pragma unroll
-                        for (int kk = 0; kk < kTile / 32; ++kk)     // 16 queries per step
-                            mma_ts(tmem + kColDV, a_p + 8 * kk, go + 64 * kk, kIdescT32, (kk || !first) ? 1u : 0u);
-                        mma_commit(bar(kPFree + h));
-                        if (h == 1) mma_commit(bar(kQEmpty + st2));
-                        if (last) mma_commit(bar(kAccFull));
-                    }
-                    __syncwarp();
-                    if (h == 1 && ++v_I == (uint32_t)nblk) { v_I = 0; ++v_nitem; }
+                if (h == 0 && !wait_all(bar(kQFull + st), (g / kQStages) & 1)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t ring = base + kOffRing + st * kRingBytes + h * kPatchContent;   // rows of patch h
+                if (elect_one()) {
+                    const uint64_t kc = smem_desc_at(kDesc64, slot_base + kOffKc), kp = smem_desc_at(kDesc64, slot_base + kOffKp);
+                    const uint64_t v = smem_desc_at(kDesc64, slot_base + kOffV);
+                    const uint64_t qc = smem_desc_at(kDesc64, ring + kRingQc), qp = smem_desc_at(kDesc64, ring + kRingQp);
+                    const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
+                    const uint32_t d_s = tmem + kColS + h * kHalfCols, d_p = tmem + kColDP + h * kHalfCols;
+                    mma_ss(d_s, kc, qc, kIdescSS, 0u);
+                    mma_ss(d_s, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
+                    mma_ss(d_s, kp, qp, kIdescSS, 1u);
+                    mma_ss(d_p, v, go, kIdescSS, 0u);
+                    mma_ss(d_p, v + 2, go + 2, kIdescSS, 1u);
+                    mma_commit(bar(kSFull + h));
                 }
+                __syncwarp();
+                if (h == 1 && ++I == (uint32_t)nblk) { I = 0; ++nitem; }
             }
         } else if (warp == 2) {
-            // ---- dK~_J += dS^T Q~_u (A from tensor memory, 16 queries per step)
+            // ---- dV_J += P^T dO_u and dK~_J += dS^T Q~_u (A from tensor memory, 16 queries per step)
             uint32_t nitem = 0, I = 0;
             for (uint32_t u = 0; u < total_units && ok; ++u) {
                 const uint32_t h = u & 1, g = u >> 1, st = g % kQStages;
                 const bool first = I == 0 && h == 0, last = I == (uint32_t)nblk - 1 && h == 1;
                 if (!wait_all(bar(kPReady + h), g & 1) ||
-                    (first && nitem > 0 && !wait_all(bar(kAccFree), (nitem - 1) & 1)) ||
-                    // let the scores of unit u + 2 into the tensor pipe first: an arithmetic group waits for them
-                    (u + 2 < total_units && !wait_all(bar(kSIssued), u & 1))) { ok = false; break; }
+                    (first && nitem > 0 && !wait_all(bar(kAccFree), (nitem - 1) & 1))) { ok = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint64_t q48 = smem_desc_at(kDescQ48, base + kOffRing + st * kRingBytes + kRingQc + h * kPatchContent);
-                    const uint32_t a_ds = tmem + kColDS + h * (kHalfCols / 2);
+                    const uint32_t ring = base + kOffRing + st * kRingBytes + h * kPatchContent;
+                    const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
+                    const uint64_t q48 = smem_desc_at(kDescQ48, ring + kRingQc);
+                    const uint32_t a_p = tmem + kColP + h * (kHalfCols / 2), a_ds = tmem + kColDS + h * (kHalfCols / 2);
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 32; ++kk)
+                        mma_ts(tmem + kColDV, a_p + 8 * kk, go + 64 * kk, kIdescT32, (kk || !first) ? 1u : 0u);
 #pragma unroll
                     for (int kk = 0; kk < kTile / 32; ++kk)
                         mma_ts(tmem + kColDK, a_ds + 8 * kk, q48 + 64 * kk, kIdescT48, (kk || !first) ? 1u : 0u);
                     mma_commit(bar(kPFree + h));
+                    // the tile's query-side rows may go: S^T, dP^T of both halves finished before P^T existed
                     if (h == 1) mma_commit(bar(kQEmpty + st));
                     if (last) mma_commit(bar(kAccFull));
                 }
@@ -279,8 +263,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             uint32_t nitem = 0, I = 0;
             for (uint32_t g = 0; g < total_tiles && ok; ++g) {
                 if (!wait_all(bar(kPReady), g & 1) || !wait_all(bar(kPReady + 1), g & 1) ||
-                    (g > 0 && !wait_all(bar(kDQFree), (g - 1) & 1)) ||
-                    (2 * g + 3 < total_units && !wait_all(bar(kSIssued), (2 * g + 1) & 1))) { ok = false; break; }
+                    (g > 0 && !wait_all(bar(kDQFree), (g - 1) & 1))) { ok = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t k48 = smem_desc_at(kDescK48, base + kOffKc + (nitem & 1) * kContentBytes);
@@ -323,14 +306,19 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tc_fence_after();
                 const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 32 * h + 16 * cg;
                 uint8_t* ds_row = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf + row * 128;
-                bool may_store = false;
+                uint32_t pp[2][8], dd[2][8];
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     uint32_t s[16], dp[16];
                     tmem_ld16(t_s + 16 * ch, s);
                     tmem_ld16(t_dp + 16 * ch, dp);
                     tmem_wait_ld();
-                    uint32_t pp[8], dd[8];
+                    if (ch == 1) {
+                        // S^T, dP^T of this half are in registers: the next unit's scores may overwrite them
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kSFree + h));
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float4 t = ld[8 * ch + i];        // (-lse2, -lse2', -D, -D') of two neighbouring queries
@@ -339,27 +327,26 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                         const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])),
                                                                  make_float2(t.z, t.w)));
-                        pp[i] = pack_bf16x2(e.x, e.y);
-                        dd[i] = pack_bf16x2(d.x, d.y);
+                        pp[ch][i] = pack_bf16x2(e.x, e.y);
+                        dd[ch][i] = pack_bf16x2(d.x, d.y);
                     }
-                    if (!may_store) {
-                        // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the
-                        // previous one still reads this dS buffer
-                        if (!__all_sync(0xffffffffu, (g == 0 || mbar_wait(bar(kPFree + h), (g - 1) & 1, abort_flag, p.status)) &&
-                                                         (g < 2 || mbar_wait(bar(kDSFree + (g & 1)), ((g >> 1) - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
-                        tc_fence_after();
-                        may_store = true;
-                    }
-                    tmem_st8(t_p + 8 * ch, pp);
-                    tmem_st8(t_ds + 8 * ch, dd);
+                }
+                // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
+                // still reads this dS buffer
+                if (!__all_sync(0xffffffffu, (g == 0 || mbar_wait(bar(kPFree + h), (g - 1) & 1, abort_flag, p.status)) &&
+                                                 (g < 2 || mbar_wait(bar(kDSFree + (g & 1)), ((g >> 1) - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ch = 0; ch < 2; ++ch) {
+                    tmem_st8(t_p + 8 * ch, pp[ch]);
+                    tmem_st8(t_ds + 8 * ch, dd[ch]);
 #pragma unroll
                     for (int q2 = 0; q2 < 2; ++q2) {
                         const int chunk = cg * 4 + ch * 2 + q2;
                         *reinterpret_cast<uint4*>(ds_row + ((chunk ^ sw) << 4)) =
-                            make_uint4(dd[4 * q2], dd[4 * q2 + 1], dd[4 * q2 + 2], dd[4 * q2 + 3]);
+                            make_uint4(dd[ch][4 * q2], dd[ch][4 * q2 + 1], dd[ch][4 * q2 + 2], dd[ch][4 * q2 + 3]);
                     }
                 }
-                if (!ok) break;
                 tmem_wait_st();
                 tc_fence_before();
                 fence_proxy_async();
