@@ -367,19 +367,16 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kDQFull), g & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
                 float* dst = p.dq_acc + (size_t)c.pair * kDk * p.n + (size_t)I * kTile + row;
+                // all 48 columns into registers first, so that the next tile's dQ~ may start while the adds drain
+                uint32_t a[3][16];
 #pragma unroll
-                for (int part = 0; part < 3; ++part) {       // 16 columns at a time keeps the register count low
-                    uint32_t a[16];
-                    tmem_ld16(tmem + lane_base + kColDQ + 16 * part, a);
-                    tmem_wait_ld();
-                    if (part == 2) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(kDQFree));
-                    }
+                for (int part = 0; part < 3; ++part) tmem_ld16(tmem + lane_base + kColDQ + 16 * part, a[part]);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kDQFree));
 #pragma unroll
-                    for (int col = 0; col < 16; ++col) red_add_f32(dst + (size_t)(16 * part + col) * p.n, __uint_as_float(a[col]));
-                }
+                for (int col = 0; col < kDk; ++col, dst += p.n) red_add_f32(dst, __uint_as_float(a[col >> 4][col & 15]));
             }
             if (!ok) break;
             if (!__all_sync(0xffffffffu, mbar_wait(bar(kAccFull), nitem & 1, abort_flag, p.status))) { ok = false; break; }
