@@ -42,7 +42,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kQStages = 3;           // ring of query-side tiles (Q content, Q RIB rows, dO, lse/D)
+constexpr int kQStages = 4;           // ring of query-side tiles (Q content, Q RIB rows, dO, lse/D)
 constexpr int kThreads = 768;
 constexpr int kDk = kD + kR;          // 48 columns of dQ~ / dK~
 
