@@ -57,9 +57,14 @@ constexpr uint32_t kRingBytes = kRingLD + kLdBytes;              // 25600
 constexpr uint32_t kOffDS = kOffRing + kQStages * kRingBytes;    // dS: [2 tiles][2 halves of 64 queries][128 keys][128 B], SWIZZLE_128B
 constexpr uint32_t kDSHalf = kTile * 128;
 constexpr uint32_t kOffBar = kOffDS + 4 * kDSHalf;
-// kSFull, kSFree, kPReady, kPFree: one per half h; kDSFree: one per dS tile buffer
+// kSFull, kSFree, kPFree: one per half h; kPReady: one per half and tile parity (index 2 h + parity); kDSFree: one per dS
+// tile buffer.  The rule behind the split: a barrier's next phase must not be able to complete before every waiter has seen
+// the current one, because a parity wait cannot tell "two phases ahead" from "not yet".  dQ~ of tile g waits for both halves'
+// P^T / dS^T, but nothing that the arithmetic warps need for tile g + 1 depends on dQ~ of tile g, so with one barrier per
+// half they could complete phase g + 1 before the dQ~ issuer has looked at phase g; with one per tile parity the next phase
+// belongs to tile g + 2, whose dS buffer is only released by dQ~ of tile g.
 enum Bar { kKVFull = 0, kKVEmpty = 2, kQFull = 4, kQEmpty = kQFull + kQStages, kSFull = kQEmpty + kQStages, kSFree = kSFull + 2,
-           kPReady = kSFree + 2, kPFree = kPReady + 2, kDSFree = kPFree + 2, kDQFull = kDSFree + 2, kDQFree, kAccFull, kAccFree, kDrain,
+           kPReady = kSFree + 2, kPFree = kPReady + 4, kDSFree = kPFree + 2, kDQFull = kDSFree + 2, kDQFree, kAccFull, kAccFree, kDrain,
            kNumBars = kDrain + 3 };
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;
 constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
@@ -123,7 +128,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int s = 0; s < 2; ++s) { mbar_init(bar(kKVFull + s), 1); mbar_init(bar(kKVEmpty + s), 1); }
         for (int s = 0; s < kQStages; ++s) { mbar_init(bar(kQFull + s), 1); mbar_init(bar(kQEmpty + s), 1); }
         for (int h = 0; h < 2; ++h) {
-            mbar_init(bar(kSFull + h), 1); mbar_init(bar(kSFree + h), 8); mbar_init(bar(kPReady + h), 8); mbar_init(bar(kPFree + h), 1);
+            mbar_init(bar(kSFull + h), 1); mbar_init(bar(kSFree + h), 8); mbar_init(bar(kPFree + h), 1);
+            mbar_init(bar(kPReady + 2 * h), 8); mbar_init(bar(kPReady + 2 * h + 1), 8);
             mbar_init(bar(kDSFree + h), 1);
         }
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
@@ -236,7 +242,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             for (uint32_t u = 0; u < total_units && ok; ++u) {
                 const uint32_t h = u & 1, g = u >> 1, st = g % kQStages;
                 const bool first = I == 0 && h == 0, last = I == (uint32_t)nblk - 1 && h == 1;
-                if (!wait_all(bar(kPReady + h), g & 1) ||
+                if (!wait_all(bar(kPReady + 2 * h + (g & 1)), (g >> 1) & 1) ||
                     (first && nitem > 0 && !wait_all(bar(kAccFree), (nitem - 1) & 1))) { ok = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
@@ -262,7 +268,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             // ---- dQ~_I = dS K~_J once both halves of dS are in shared memory (16 keys per step)
             uint32_t nitem = 0, I = 0;
             for (uint32_t g = 0; g < total_tiles && ok; ++g) {
-                if (!wait_all(bar(kPReady), g & 1) || !wait_all(bar(kPReady + 1), g & 1) ||
+                if (!wait_all(bar(kPReady + (g & 1)), (g >> 1) & 1) || !wait_all(bar(kPReady + 2 + (g & 1)), (g >> 1) & 1) ||
                     (g > 0 && !wait_all(bar(kDQFree), (g - 1) & 1))) { ok = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
@@ -351,7 +357,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tc_fence_before();
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kPReady + h));
+                if (lane == 0) mbar_arrive(bar(kPReady + 2 * h + (g & 1)));
             }
         }
     } else if (warp >= 20) {
