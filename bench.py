@@ -247,33 +247,65 @@ def main():
     # ------------------------------------------------ end to end: pinned host buffers, H2D + D2H inside
     e2e = None
     if not args.no_e2e:
-        s = sets[0]
         hout = {k: torch.empty_like(host["q"]).pin_memory() for k in ("out", "dq", "dk", "dv")}
         hdp = {k: torch.empty((wl.n, wl.r), dtype=torch.float32).pin_memory() for k in ("dpq", "dpk")}
         h2d = sum(host[k].numel() * host[k].element_size() for k in ("q", "k", "v", "pq", "pk", "dout"))
         d2h = sum(t.numel() * t.element_size() for t in list(hout.values()) + list(hdp.values()))
 
-        def e2e_step():
-            for k in ("q", "k", "v", "pq", "pk", "dout"):
-                s[k].copy_(host[k], non_blocking=True)
-            _, _, (dq, dk, dv, dpq, dpk) = step(s)
-            hout["out"].copy_(s["out"], non_blocking=True)
-            for k, t in (("dq", dq), ("dk", dk), ("dv", dv)):
-                hout[k].copy_(t, non_blocking=True)
-            hdp["dpq"].copy_(dpq, non_blocking=True)
-            hdp["dpk"].copy_(dpk, non_blocking=True)
+        # Three streams and two device buffer sets: while step i computes, the inputs of step i + 1 come in and the
+        # results of step i - 1 go out (PCIe is full duplex).  Every step's copies are inside the timed region.
+        st_in, st_run, st_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+        dsets = [sets[0], sets[1]]
+        ev_in = [torch.cuda.Event() for _ in range(2)]      # inputs of the set have arrived
+        ev_run = [torch.cuda.Event() for _ in range(2)]     # the set's step has finished (inputs may be overwritten)
+        ev_out = [torch.cuda.Event() for _ in range(2)]     # the set's results have left (outputs may be overwritten)
+        keep = []
 
-        for _ in range(3):
-            e2e_step()
+        def e2e_step(i):
+            b = i & 1
+            d = dsets[b]
+            with torch.cuda.stream(st_in):
+                st_in.wait_event(ev_run[b])
+                for k in ("q", "k", "v", "pq", "pk", "dout"):
+                    d[k].copy_(host[k], non_blocking=True)
+                ev_in[b].record(st_in)
+            with torch.cuda.stream(st_run):
+                st_run.wait_event(ev_in[b])
+                st_run.wait_event(ev_out[b])
+                binding.rib_window_attn_fwd(d["q"], d["k"], d["v"], d["pq"], d["pk"], wl.window, wl.shift,
+                                            out=d["out"], lse=d["lse"])
+                res = binding.rib_window_attn_bwd(d["q"], d["k"], d["v"], d["pq"], d["pk"], d["out"], d["lse"], d["dout"],
+                                                  wl.window, wl.shift, workspace=workspace)
+                ev_run[b].record(st_run)
+            with torch.cuda.stream(st_out):
+                st_out.wait_event(ev_run[b])
+                hout["out"].copy_(d["out"], non_blocking=True)
+                for k, t in zip(("dq", "dk", "dv"), res[:3]):
+                    t.record_stream(st_out)
+                    hout[k].copy_(t, non_blocking=True)
+                for k, t in zip(("dpq", "dpk"), res[3:]):
+                    t.record_stream(st_out)
+                    hdp[k].copy_(t, non_blocking=True)
+                ev_out[b].record(st_out)
+            keep.append(res)
+            del keep[:-4]
+
+        barrier()
+        for i in range(4):
+            e2e_step(i)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e2e_steps = max(3, min(args.steps, 10))
-        e0.record()
-        for _ in range(e2e_steps):
-            e2e_step()
-        e1.record()
+        e2e_steps = max(4, min(args.steps, 20))
+        e2e_steps += e2e_steps & 1
+        e0.record(st_in)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        st_out.wait_stream(st_run)
+        e1.record(st_out)
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
+        if binding.rib_query_status() != 0:
+            raise SystemExit("device status word set during the end-to-end steps")
     else:
         e2e_ms, h2d, d2h = None, 0, 0
 
@@ -357,7 +389,8 @@ def main():
         "kernels": kernels,
         "e2e": None if e2e_ms is None else {
             "value": flops_step / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_max,
-            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "overlap": "copies in, compute and copies out on three streams over two device buffer sets"},
         "gpu_launches": launches,
         "generator": gen,
         "clocks": sampler.summary(),
