@@ -37,20 +37,26 @@ using namespace sm100;
 constexpr int kStages = 4;            // K/V ring depth
 constexpr int kThreads = 640;
 
-// shared-memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQc = 0;                                        // [2 items][2 tiles] query content
-constexpr uint32_t kOffQp = kOffQc + 4 * kContentBytes;               // [2 items][2 tiles] query RIB rows (scaled)
-constexpr uint32_t kOffKc = kOffQp + 4 * kPosBytes;                   // [kStages] key content
-constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStages] key RIB rows
-constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
-constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
 // kPReady / kPFree: index 2 * tile + key half
 enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 14, kOFree = 18, kDrain = 20, kMerge = 22,
            kKFull = 30, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
            kNumBars = kVEmpty + kStages };
-constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
-constexpr uint32_t kOffMerge = kOffMisc + 16;                         // [2 tiles][2 halves][128 rows] (max, sum)
-constexpr uint32_t kSmemBytes = kOffMerge + 4 * kTile * 8 + 1024;     // + slack for manual alignment
+
+// shared-memory map (offsets from a 1024-byte aligned base) for RIB rank R = 16 (32-byte RIB rows, SWIZZLE_32B) or
+// R = 32 (64-byte RIB rows: the layout of the content rows)
+template <int R>
+struct Layout {
+    static constexpr uint32_t kPosBytes = kTile * R * 2, kPatchPos = kPosBytes / 2;
+    static constexpr uint32_t kOffQc = 0;                                        // [2 items][2 tiles] query content
+    static constexpr uint32_t kOffQp = kOffQc + 4 * kContentBytes;               // [2 items][2 tiles] query RIB rows (scaled)
+    static constexpr uint32_t kOffKc = kOffQp + 4 * kPosBytes;                   // [kStages] key content
+    static constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStages] key RIB rows
+    static constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
+    static constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
+    static constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
+    static constexpr uint32_t kOffMerge = kOffMisc + 16;                         // [2 tiles][2 halves][128 rows] (max, sum)
+    static constexpr uint32_t kSmemBytes = kOffMerge + 4 * kTile * 8 + 1024;     // + slack for manual alignment
+};
 
 // tensor-memory columns (fp32 accumulators; P is bf16x2, two keys per column)
 // O: [2 tiles][2 key halves][32]
@@ -93,11 +99,15 @@ __device__ __forceinline__ void patch_origin(const FwdParams& p, const ItemCoord
     sm100::patch_origin(WindowGeom{p.H, p.W, p.M, p.s}, c.wy, c.wx, sp, py, px, Y0, X0);
 }
 
+template <int R>
 __global__ void __launch_bounds__(kThreads, 1)
 rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_pk,
                      const FwdParams p)
 {
+    using L = Layout<R>;
+    constexpr uint32_t kOffQc = L::kOffQc, kOffQp = L::kOffQp, kOffKc = L::kOffKc, kOffKp = L::kOffKp, kOffV = L::kOffV, kOffBar = L::kOffBar,
+                       kOffMisc = L::kOffMisc, kOffMerge = L::kOffMerge, kPosBytes = L::kPosBytes, kPatchPos = L::kPatchPos;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -221,7 +231,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) &&
                                              mbar_wait(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status))) { ok = false; break; }
             const uint64_t qc = smem_desc_at(kDesc64, base + kOffQc + (2 * buf + qt) * kContentBytes);
-            const uint64_t qp = smem_desc_at(kDesc32, base + kOffQp + (2 * buf + qt) * kPosBytes);
+            const uint64_t qp = smem_desc_at(R == 16 ? kDesc32 : kDesc64, base + kOffQp + (2 * buf + qt) * kPosBytes);
             for (int j = 0; j < nblk; ++j, ++b) {
                 const uint32_t st = b % kStages;
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kKFull + st), (b / kStages) & 1, abort_flag, p.status) &&
@@ -229,10 +239,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
-                    const uint64_t kp = smem_desc_at(kDesc32, base + kOffKp + st * kPosBytes);
+                    const uint64_t kp = smem_desc_at(R == 16 ? kDesc32 : kDesc64, base + kOffKp + st * kPosBytes);
                     mma_ss(d_s, qc, kc, kIdescS, 0u);
                     mma_ss(d_s, qc + 2, kc + 2, kIdescS, 1u);          // + 32 bytes: second K16 step of the content rows
                     mma_ss(d_s, qp, kp, kIdescS, 1u);
+                    if (R == 32) mma_ss(d_s, qp + 2, kp + 2, kIdescS, 1u);
                     mma_commit(bar(kSFull + qt));
                     mma_commit(bar(kKEmpty + st));
                     if (j == nblk - 1) mma_commit(bar(kQEmpty + buf));
@@ -259,19 +270,22 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 int py, px, Y0, X0;
                 patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
                 const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
-                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * kR);
-                uint4 v[2] = {__ldg(src), __ldg(src + 1)};
+                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * R);
+                constexpr int kChunks = R / 8;                 // 16-byte chunks per row
+                uint4 v[kChunks];
+#pragma unroll
+                for (int ck = 0; ck < kChunks; ++ck) v[ck] = __ldg(src + ck);
                 uint32_t* w = reinterpret_cast<uint32_t*>(v);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < 4 * kChunks; ++i) {
                     const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
                     const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
                     w[i] = pack_bf16x2(lo, hi);
                 }
-                uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * 32;
-                const int sw = (row >> 2) & 1;
-                *reinterpret_cast<uint4*>(dst + ((0 ^ sw) << 4)) = v[0];
-                *reinterpret_cast<uint4*>(dst + ((1 ^ sw) << 4)) = v[1];
+                uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * (2 * R);
+                const int sw = R == 16 ? (row >> 2) & 1 : (row >> 1) & 3;      // SWIZZLE_32B / SWIZZLE_64B
+#pragma unroll
+                for (int ck = 0; ck < kChunks; ++ck) *reinterpret_cast<uint4*>(dst + ((ck ^ sw) << 4)) = v[ck];
             }
             fence_proxy_async();
             __syncwarp();
@@ -441,21 +455,23 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
 bool sm100_fwd_supported(const Problem& p)
 {
-    return p.d == kD && p.r == kR && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
+    return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
 }
 
-cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
+template <int R>
+cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
     CUtensorMap tm_q, tm_k, tm_v, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
         !encode_pos_map(&tm_pk, p.pk, p, pos_tables(p), p.pos_head_stride))
         return cudaErrorInvalidValue;
+    constexpr uint32_t kSmemBytes = Layout<R>::kSmemBytes;
     static int sm_count = 0;
     if (!sm_count) {
         cudaError_t e = sm_count_of_current_device(&sm_count);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rib_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            e = cudaFuncSetAttribute(rib_fwd_sm100_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) { sm_count = 0; return e; }
     }
     FwdParams fp{};
@@ -469,8 +485,13 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     const int grid = fp.items < sm_count ? fp.items : sm_count;
-    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
+    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<R><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
     return cudaGetLastError();
+}
+
+cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
+{
+    return p.r == 32 ? launch_fwd<32>(p, stream) : launch_fwd<16>(p, stream);
 }
 
 }  // namespace rib

@@ -79,15 +79,15 @@ inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// bf16 [tables][M][M][16] positional features (one table shared by all heads, or one per head), box = one
+// bf16 [tables][M][M][r] positional features (one table shared by all heads, or one per head; r = p.r), box = one
 // 8x8-token patch of one table.  `tables` = 1 or heads, `table_stride` elements apart (a multiple of 8,
 // at least M * M * 16); a kernel addresses table h * (tables > 1).
 inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
                                 cuuint32_t box_inner, CUtensorMapSwizzle swz)
 {
-    const cuuint64_t dims[4] = {(cuuint64_t)kR, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
-    const cuuint64_t one_table = (cuuint64_t)kR * 2 * p.M * p.M;
-    const cuuint64_t strides[3] = {(cuuint64_t)kR * 2, (cuuint64_t)kR * 2 * p.M,
+    const cuuint64_t dims[4] = {(cuuint64_t)p.r, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
+    const cuuint64_t one_table = (cuuint64_t)p.r * 2 * p.M * p.M;
+    const cuuint64_t strides[3] = {(cuuint64_t)p.r * 2, (cuuint64_t)p.r * 2 * p.M,
                                    tables > 1 ? (cuuint64_t)table_stride * 2 : one_table};
     const cuuint32_t box[4] = {box_inner, 8, 8, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -97,7 +97,7 @@ inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem
 }
 inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
 {
-    return encode_pos_map_impl(map, ptr, p, tables, table_stride, kR, CU_TENSOR_MAP_SWIZZLE_32B);
+    return encode_pos_map_impl(map, ptr, p, tables, table_stride, (cuuint32_t)p.r, p.r == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
 }
 // The same features fetched as 64-byte rows: the box is 32 elements wide on a 16-element dimension, so
 // TMA fills the upper half of every row with zeros.  A 64-byte-row RIB tile has the layout of a content
