@@ -209,7 +209,7 @@ size_t rib_window_attn_bwd_headwise_workspace(long long pos_head_stride, int B, 
     rib::Problem p{};
     fill_shape(p, B, H, W, heads, d, r, window, 0);
     if (rib::sm100_bwd_supported(p)) {   // whatever the shift: one size per shape
-        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1);
+        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1, r);
         if (fast > need) need = fast;
     }
     return need;

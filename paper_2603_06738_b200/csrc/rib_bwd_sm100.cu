@@ -1,7 +1,10 @@
 // Backward RIB window attention for B200 (sm_100a): the chain rule of Eq. 6 and the softmax as five
 // tcgen05 contractions per (query tile, key block) with TMEM accumulators and TMA loads.
 //
-// Shapes: d = 32, r = 16, window side M a multiple of 16, shift a multiple of 8 (as the forward).
+// Shapes: d = 32, r = 16 or 32 (template argument R), window side M a multiple of 16, shift a multiple of 8 (as
+// the forward).  The text below describes R = 16.  With R = 32 the RIB rows fill their 64-byte slots, dK~ and dQ~ are
+// 64 columns wide, and tensor memory has no room left for dS^T: dK~ then takes the dS tile in shared memory as a
+// K-major A operand (that tile's barrier counts two readers).
 //
 // Work item = one (batch, window, head) pair x one key block J of 128 tokens.  A persistent CTA keeps
 // K~_J = [k, Pk] and V_J in shared memory and dV_J, dK~_J in tensor memory, and walks the query tiles
@@ -44,7 +47,7 @@ using namespace sm100;
 
 constexpr int kQStages = 4;           // ring of query-side tiles (Q content, Q RIB rows, dO, lse/D)
 constexpr int kThreads = 768;
-constexpr int kDk = kD + kR;          // 48 columns of dQ~ / dK~
+// RIB rank R = 16 or 32 is a template argument of the kernels: dQ~ / dK~ have kD + R columns
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffKc = 0;                                   // [2] key content (one slot per item in flight)
@@ -71,14 +74,25 @@ constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
 static_assert(kOffRing % 1024 == 0 && kRingBytes % 1024 == 0 && kOffDS % 1024 == 0, "swizzle atoms need aligned tiles");
 
 // tensor-memory columns; S^T, dP^T (64 fp32 columns) and P^T, dS^T (32 columns of bf16 pairs) exist once per half h
-constexpr uint32_t kColS = 0, kColDP = 128, kColP = 256, kColDS = 320, kColDV = 384, kColDK = 416, kColDQ = 464;
+// R = 16: S 0, dP 128, P 256, dS 320, dV 384, dK~ 416 (48), dQ~ 464 (48).
+// R = 32: dK~ and dQ~ need 64 columns each, so dS^T is not kept in tensor memory (dK~ reads the dS tile in shared memory,
+//         K-major): S 0, dP 128, P 256, dV 320, dK~ 352 (64), dQ~ 416 (64).
+constexpr uint32_t kColS = 0, kColDP = 128, kColP = 256;
+template <int R> struct Cols {
+    static constexpr uint32_t kColDS = 320;                              // R = 16 only
+    static constexpr uint32_t kColDV = R == 16 ? 384 : 320, kColDK = kColDV + kD, kColDQ = kColDK + kD + R;
+    static_assert(kColDQ + kD + R <= 512, "tensor memory has 512 columns");
+};
 constexpr uint32_t kHalfCols = kTile / 2;
 constexpr uint32_t kTmemCols = 512;
 
 constexpr uint32_t kIdescSS = idesc_bf16_f32(kTile, kTile / 2, false);        // S^T, dP^T of a half-tile: both operands K-major
 constexpr uint32_t kIdescT32 = idesc_bf16_f32(kTile, kD, true);               // A in TMEM, B MN-major, N = 32
-constexpr uint32_t kIdescT48 = idesc_bf16_f32(kTile, kDk, true);              // A in TMEM, B MN-major, N = 48
-constexpr uint32_t kIdescQ48 = idesc_bf16_f32_ab(kTile, kDk, true, true);     // dQ~: A and B MN-major, N = 48
+// dK~ (A in TMEM or K-major in shared memory, B MN-major) and dQ~ (A and B MN-major), N = kD + R
+template <int R> struct Idesc {
+    static constexpr uint32_t kT = idesc_bf16_f32(kTile, kD + R, true);
+    static constexpr uint32_t kQ = idesc_bf16_f32_ab(kTile, kD + R, true, true);
+};
 
 struct BwdParams {
     const float2* ld;          // [pairs][n / 2] window order, per query pair: (-lse2, -lse2', -D, -D') as two float2
@@ -107,12 +121,16 @@ __device__ __forceinline__ ItemCoord decode_item(const BwdParams& p, int item)
     return c;
 }
 
+template <int R>
 __global__ void __launch_bounds__(kThreads, 1)
 rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                      const __grid_constant__ CUtensorMap tm_pqs, const __grid_constant__ CUtensorMap tm_pk,
                      const BwdParams p)
 {
+    constexpr int kDk = kD + R;
+    constexpr uint32_t kColDS = Cols<R>::kColDS, kColDV = Cols<R>::kColDV, kColDK = Cols<R>::kColDK, kColDQ = Cols<R>::kColDQ;
+    constexpr uint32_t kIdescT48 = Idesc<R>::kT, kIdescQ48 = Idesc<R>::kQ;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -130,7 +148,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int h = 0; h < 2; ++h) {
             mbar_init(bar(kSFull + h), 1); mbar_init(bar(kSFree + h), 8); mbar_init(bar(kPFree + h), 1);
             mbar_init(bar(kPReady + 2 * h), 8); mbar_init(bar(kPReady + 2 * h + 1), 8);
-            mbar_init(bar(kDSFree + h), 1);
+            mbar_init(bar(kDSFree + h), R == 16 ? 1 : 2);     // R = 32: dK~ reads the dS tile as well as dQ~
         }
         mbar_init(bar(kDQFull), 1); mbar_init(bar(kDQFree), 4);
         mbar_init(bar(kAccFull), 1); mbar_init(bar(kAccFree), 4);
@@ -199,7 +217,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         // MN-major operands of 48 columns: the content tile and, one leading-dimension step further, the RIB tile
         constexpr uint64_t kDescQ48 = smem_desc_const(kRingQp - kRingQc, 512, kSwizzle64B);
         constexpr uint64_t kDescK48 = smem_desc_const(kOffKp - kOffKc, 512, kSwizzle64B);
-        constexpr uint64_t kDescDS = smem_desc_const(kDSHalf, 1024, kSwizzle128B);
+        constexpr uint64_t kDescDS = smem_desc_const(kDSHalf, 1024, kSwizzle128B);    // MN-major: the two 64-query halves one leading step apart
+        constexpr uint64_t kDescDSk = smem_desc_const(16, 1024, kSwizzle128B);        // K-major view of one half (R = 32)
         const int nblk = p.nblk;
         const uint32_t total_tiles = (((uint32_t)p.items - blockIdx.x + gridDim.x - 1) / gridDim.x) * (uint32_t)nblk;
         const uint32_t total_units = 2 * total_tiles;       // half-tiles of this CTA, in order
@@ -229,6 +248,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     mma_ss(d_s, kc, qc, kIdescSS, 0u);
                     mma_ss(d_s, kc + 2, qc + 2, kIdescSS, 1u);     // + 32 bytes: second K16 step
                     mma_ss(d_s, kp, qp, kIdescSS, 1u);
+                    if (R == 32) mma_ss(d_s, kp + 2, qp + 2, kIdescSS, 1u);
                     mma_ss(d_p, v, go, kIdescSS, 0u);
                     mma_ss(d_p, v + 2, go + 2, kIdescSS, 1u);
                     mma_commit(bar(kSFull + h));
@@ -249,13 +269,24 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint32_t ring = base + kOffRing + st * kRingBytes + h * kPatchContent;
                     const uint64_t go = smem_desc_at(kDesc64, ring + kRingDO);
                     const uint64_t q48 = smem_desc_at(kDescQ48, ring + kRingQc);
-                    const uint32_t a_p = tmem + kColP + h * (kHalfCols / 2), a_ds = tmem + kColDS + h * (kHalfCols / 2);
+                    const uint32_t a_p = tmem + kColP + h * (kHalfCols / 2);
 #pragma unroll
                     for (int kk = 0; kk < kTile / 32; ++kk)
                         mma_ts(tmem + kColDV, a_p + 8 * kk, go + 64 * kk, kIdescT32, (kk || !first) ? 1u : 0u);
+                    if (R == 16) {
+                        const uint32_t a_ds = tmem + kColDS + h * (kHalfCols / 2);
 #pragma unroll
-                    for (int kk = 0; kk < kTile / 32; ++kk)
-                        mma_ts(tmem + kColDK, a_ds + 8 * kk, q48 + 64 * kk, kIdescT48, (kk || !first) ? 1u : 0u);
+                        for (int kk = 0; kk < kTile / 32; ++kk)
+                            mma_ts(tmem + kColDK, a_ds + 8 * kk, q48 + 64 * kk, kIdescT48, (kk || !first) ? 1u : 0u);
+                    } else {
+                        // A = this half of the dS tile in shared memory, read K-major: rows are keys, the 128-byte lines the
+                        // unit's 64 queries (32 bytes per K16 step)
+                        const uint64_t a_ds = smem_desc_at(kDescDSk, base + kOffDS + ((g & 1) * 2 + h) * kDSHalf);
+#pragma unroll
+                        for (int kk = 0; kk < kTile / 32; ++kk)
+                            mma_ss(tmem + kColDK, a_ds + 2 * kk, q48 + 64 * kk, kIdescT48, (kk || !first) ? 1u : 0u);
+                        if (h == 1) mma_commit(bar(kDSFree + (g & 1)));
+                    }
                     mma_commit(bar(kPFree + h));
                     // the tile's query-side rows may go: S^T, dP^T of both halves finished before P^T existed
                     if (h == 1) mma_commit(bar(kQEmpty + st));
@@ -345,7 +376,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     tmem_st8(t_p + 8 * ch, pp[ch]);
-                    tmem_st8(t_ds + 8 * ch, dd[ch]);
+                    if (R == 16) tmem_st8(t_ds + 8 * ch, dd[ch]);
 #pragma unroll
                     for (int q2 = 0; q2 < 2; ++q2) {
                         const int chunk = cg * 4 + ch * 2 + q2;
@@ -373,10 +404,10 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kDQFull), g & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
                 float* dst = p.dq_acc + (size_t)c.pair * kDk * p.n + (size_t)I * kTile + row;
-                // all 48 columns into registers first, so that the next tile's dQ~ may start while the adds drain
-                uint32_t a[3][16];
+                // all columns into registers first, so that the next tile's dQ~ may start while the adds drain
+                uint32_t a[kDk / 16][16];
 #pragma unroll
-                for (int part = 0; part < 3; ++part) tmem_ld16(tmem + lane_base + kColDQ + 16 * part, a[part]);
+                for (int part = 0; part < kDk / 16; ++part) tmem_ld16(tmem + lane_base + kColDQ + 16 * part, a[part]);
                 tmem_wait_ld();
                 tc_fence_before();
                 __syncwarp();
@@ -392,18 +423,21 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
             uint4* dst_v = reinterpret_cast<uint4*>(p.dv + tok * kD);
             uint4* dst_k = reinterpret_cast<uint4*>(p.dk + tok * kD);
-            float* dst_p = p.dkp + (size_t)c.pair * kR * p.n + (size_t)c.J * kTile + row;
+            float* dst_p = p.dkp + (size_t)c.pair * R * p.n + (size_t)c.J * kTile + row;
+            constexpr int kParts = 4 + R / 16;
 #pragma unroll
-            for (int part = 0; part < 5; ++part) {           // dV (2 x 16 columns), dK~ content (2 x 16), dK~ RIB (16)
+            for (int part = 0; part < kParts; ++part) {      // dV (2 x 16 columns), dK~ content (2 x 16), dK~ RIB (R / 16 x 16)
                 uint32_t a[16];
                 tmem_ld16(tmem + lane_base + kColDV + 16 * part, a);     // dV, dK~ are adjacent in tensor memory
                 tmem_wait_ld();
-                if (part == 4) {
+                if (part == kParts - 1) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kAccFree));
+                }
+                if (part >= 4) {
 #pragma unroll
-                    for (int col = 0; col < kR; ++col) dst_p[(size_t)col * p.n] = __uint_as_float(a[col]) * p.inv_sqrt_d;
+                    for (int col = 0; col < 16; ++col) dst_p[(size_t)(16 * (part - 4) + col) * p.n] = __uint_as_float(a[col]) * p.inv_sqrt_d;
                 } else {
                     const float f = part < 2 ? 1.f : p.inv_sqrt_d;
                     uint4* dst16 = (part < 2 ? dst_v : dst_k) + 2 * (part & 1);
@@ -460,12 +494,14 @@ __device__ __forceinline__ void decode_pair_token(const AuxParams& p, int pair, 
 // One thread per (pair, token in window order): D = dO . O and lse in the layout the main kernel
 // streams, zero of this token's dQ~ accumulators; the first threads also stage bf16(Pq sqrt(d/r))
 // and clear dPq, dPk.
+template <int R>
 __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
 {
+    constexpr int kDk = kD + R;
     const size_t total = (size_t)p.pairs * p.n;
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-    const size_t per_table = (size_t)p.n * kR;
+    const size_t per_table = (size_t)p.n * R;
     for (size_t e = t; e < per_table * p.tables; e += nthreads) {
         const size_t user = (e / per_table) * (size_t)p.pos_head_stride + e % per_table;
         p.pq_scaled[e] = __float2bfloat16_rn(__bfloat162float(p.pq[user]) * p.pos_scale);
@@ -505,8 +541,10 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
 // dQ~[:, :d] / sqrt(d) into the bf16 dq row of that token, and it keeps running sums of the 16 RIB
 // columns of dQ~ (-> dPq, times 1/sqrt(r)) and of dK~ (-> dPk); the group's partial sums go to the
 // zeroed results with one vector atomic per 4 columns.
+template <int R>
 __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_group)
 {
+    constexpr int kDk = kD + R;
     const int w = blockIdx.x * 128 + threadIdx.x;
     int pair0, pair1, step = 1;
     size_t table = 0;
@@ -520,9 +558,9 @@ __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, 
         pair1 = min(p.pairs, pair0 + pairs_per_group * step);
         table = (size_t)head * (size_t)p.pos_head_stride;
     }
-    float sq[kR], sk[kR];
+    float sq[R], sk[R];
 #pragma unroll
-    for (int c = 0; c < kR; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
+    for (int c = 0; c < R; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
     int i = 0;
     for (int pair = pair0; pair < pair1; pair += step) {
         size_t tok, scalar;
@@ -536,18 +574,18 @@ __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, 
             for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
             dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
         }
-        const float* srk = p.dkp + (size_t)pair * kR * p.n + w;
+        const float* srk = p.dkp + (size_t)pair * R * p.n + w;
 #pragma unroll
-        for (int c = 0; c < kR; ++c) {
+        for (int c = 0; c < R; ++c) {
             sq[c] += src[(size_t)(kD + c) * p.n];
             sk[c] += srk[(size_t)c * p.n];
         }
     }
     if (pair0 >= pair1) return;
-    float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * kR);
-    float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * kR);
+    float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R);
+    float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R);
 #pragma unroll
-    for (int c4 = 0; c4 < kR / 4; ++c4) {
+    for (int c4 = 0; c4 < R / 4; ++c4) {
         atomicAdd(out_q + c4, make_float4(sq[4 * c4] * p.inv_sqrt_r, sq[4 * c4 + 1] * p.inv_sqrt_r, sq[4 * c4 + 2] * p.inv_sqrt_r,
                                           sq[4 * c4 + 3] * p.inv_sqrt_r));
         atomicAdd(out_k + c4, make_float4(sk[4 * c4], sk[4 * c4 + 1], sk[4 * c4 + 2], sk[4 * c4 + 3]));
@@ -558,8 +596,9 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WorkspaceLayout { size_t ld, dq_acc, dkp, pq_scaled, total; };
 
-WorkspaceLayout workspace_layout(long long pairs, int n, int tables)
+WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
 {
+    const int kR = r, kDk = kD + r;
     WorkspaceLayout w;
     w.ld = 0;
     w.dq_acc = w.ld + align256((size_t)pairs * n * sizeof(float2));
@@ -573,16 +612,17 @@ WorkspaceLayout workspace_layout(long long pairs, int n, int tables)
 
 bool sm100_bwd_supported(const Problem& p)
 {
-    return p.d == sm100::kD && p.r == sm100::kR && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
+    return p.d == sm100::kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
 }
 
-size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables) { return workspace_layout(pairs, n, tables).total; }
+size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r) { return workspace_layout(pairs, n, tables, r).total; }
 
-cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
+template <int R>
+cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
     const int tables = pos_tables(p);
-    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n, tables);
+    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n, tables, R);
     if (p.workspace_bytes < wl.total) return cudaErrorInvalidValue;
     uint8_t* ws = static_cast<uint8_t*>(p.workspace);
     float2* ld = reinterpret_cast<float2*>(ws + wl.ld);
@@ -592,14 +632,14 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 
     CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
-        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * kR) ||
+        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * R) ||
         !encode_pos_map_padded(&tm_pk, p.pk, p, tables, p.pos_head_stride))
         return cudaErrorInvalidValue;
     static int sm_count = 0;
     if (!sm_count) {
         cudaError_t e = sm_count_of_current_device(&sm_count);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rib_bwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            e = cudaFuncSetAttribute(rib_bwd_sm100_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) { sm_count = 0; return e; }
     }
     AuxParams ap{};
@@ -615,7 +655,7 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     ap.inv_sqrt_r = 1.f / sqrtf((float)p.r);
     const size_t tokens = (size_t)p.pairs * p.n;
     const unsigned aux_blocks = (unsigned)((tokens + 255) / 256);
-    { ProfileScope scope(RIB_KERNEL_BWD_PREPARE, stream); rib_bwd_prepare_kernel<<<aux_blocks, 256, 0, stream>>>(ap); }
+    { ProfileScope scope(RIB_KERNEL_BWD_PREPARE, stream); rib_bwd_prepare_kernel<R><<<aux_blocks, 256, 0, stream>>>(ap); }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
@@ -628,7 +668,7 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
-    { ProfileScope scope(RIB_KERNEL_BWD_MAIN, stream); rib_bwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp); }
+    { ProfileScope scope(RIB_KERNEL_BWD_MAIN, stream); rib_bwd_sm100_kernel<R><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
@@ -637,8 +677,13 @@ cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
     const unsigned groups = tables == 1 ? (unsigned)((p.pairs + per_group - 1) / per_group)
                                         : (unsigned)(p.heads * ((windows + per_group - 1) / per_group));
     dim3 grid_fin((unsigned)(p.n / 128), groups);
-    { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<<<grid_fin, 128, 0, stream>>>(ap, per_group); }
+    { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<R><<<grid_fin, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();
+}
+
+cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
+{
+    return p.r == 32 ? launch_bwd<32>(p, stream) : launch_bwd<16>(p, stream);
 }
 
 }  // namespace rib

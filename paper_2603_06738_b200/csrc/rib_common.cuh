@@ -52,7 +52,7 @@ cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream);
 bool sm100_fwd_supported(const Problem& p);
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
 bool sm100_bwd_supported(const Problem& p);
-size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables);
+size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r);
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 3 kernels
 
 bool generator_supported(int window, int L, int dh, int r);

@@ -1,7 +1,8 @@
 // Forward RIB window attention for B200 (sm_100a): tcgen05 MMAs with TMEM accumulators, TMA loads
 // whose box coordinates do the window partition and the cyclic shift, online softmax in registers.
 //
-// Shapes: d = 32, r = 16, window side M a multiple of 16, shift a multiple of 8.
+// Shapes: d = 32, r = 16 or 32 (template argument R), window side M a multiple of 16, shift a multiple of 8.
+// The text below describes R = 16; with R = 32 the RIB rows are 64 bytes like the content rows and take two K16 steps.
 //
 // Work item = one (batch, window, head) pair x two query tiles of 128 tokens.  A persistent CTA
 // walks items; inside an item it streams the window's keys in blocks of 128:

@@ -25,7 +25,7 @@ SMALL = [
     Workload("w32_s16_fast_shape", 1, 64, 32, 3, 32, 16, 32, 16, seed=19),
     Workload("w48_s24_fast_shape", 1, 48, 96, 1, 32, 16, 48, 24, seed=20),
     Workload("w16_odd_shift", 1, 32, 32, 2, 32, 16, 16, 5, seed=21),       # fast shape but odd shift
-    Workload("w16_s8_rank32", 2, 32, 48, 2, 32, 32, 16, 8, seed=22),       # rank 32 (d + r = 64): tcgen05 forward
+    Workload("w16_s8_rank32", 2, 32, 48, 2, 32, 32, 16, 8, seed=22),       # rank 32 (d + r = 64) on the tcgen05 kernels
     Workload("w32_s16_rank32", 1, 64, 32, 3, 32, 32, 32, 16, seed=23),
 ]
 
@@ -124,19 +124,32 @@ def test_config5_full_forward_backward():
     compare("dpk", to_f64(dpk), rdpk, max_abs=1e-2 * scale)
 
 
-def test_rank32_forward_full_size_sampled_pairs():
-    """The paper's second window cycle uses rank 32 with 32-channel heads (d + r = 64): the forward runs on
-    the tcgen05 kernel (64-byte RIB rows), checked at the training-patch size on sampled pairs."""
+def test_rank32_full_size_forward_and_backward():
+    """The paper's second window cycle uses rank 32 with 32-channel heads (d + r = 64): both passes run on the
+    tcgen05 kernels (64-byte RIB rows; dK~ and dQ~ 64 columns wide), checked at the training-patch size: sampled
+    pairs for the image tensors, the complete reductions for dPq and dPk."""
     base = CONFIGS[1]
     wl = Workload("cfg2_rank32", base.B, base.H, base.W, base.heads, base.d, 32, base.window, base.shift, seed=34)
-    cpu, gpu = make(wl, with_dout=False)
+    cpu, gpu = make(wl, with_dout=True)
     out, lse = run_fwd(gpu, wl)
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    dq, dk, dv, dpq, dpk = run_bwd(gpu, wl, out, lse)
     assert binding.rib_last_path() == binding.RIB_PATH_SM100
     pairs = sample_pairs(wl, 6, seed=7)
     ref_out, ref_lse = oracle_fwd(cpu, wl, pairs=pairs)
-    compare("out", to_f64(out), ref_out, ~np.isnan(ref_out))
+    mask = ~np.isnan(ref_out)
+    compare("out", to_f64(out), ref_out, mask)
     compare("lse", to_f64(lse), ref_lse, ~np.isnan(ref_lse))
-    assert torch.isfinite(out.float()).all()
+    rdq, rdk, rdv, _, _ = oracle_bwd(cpu, wl, pairs=pairs)
+    compare("dq", to_f64(dq), rdq, mask)
+    compare("dk", to_f64(dk), rdk, mask)
+    compare("dv", to_f64(dv), rdv, mask)
+    _, _, _, rdpq, rdpk = oracle_bwd(cpu, wl)
+    scale = max(1.0, float(np.abs(rdpq).max()), float(np.abs(rdpk).max()))
+    compare("dpq", to_f64(dpq), rdpq, max_abs=1e-2 * scale)
+    compare("dpk", to_f64(dpk), rdpk, max_abs=1e-2 * scale)
+    for t in (out, dq, dk, dv):
+        assert torch.isfinite(t.float()).all()
 
 
 def test_largest_paper_window_96_forward_and_backward():
