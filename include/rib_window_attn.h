@@ -117,6 +117,22 @@ size_t rib_window_attn_bwd_headwise_workspace(long long pos_head_stride, int B, 
                                               int window);
 
 /*
+ * Forward pass on a feature map whose sides are not multiples of the window (Sec. 4 mentions padding the map up to
+ * the window; the paper does not say what the added positions do -- the reading taken here: they are not tokens).
+ * Windows, and the cyclic shift if any, are laid over the map extended at the bottom and the right to
+ * Hp = ceil(H / window) * window and Wp likewise; positions with Y >= H or X >= W are neither attended to nor
+ * written.  Every real token keeps the positional row i = y * window + x of its place in its window.  q, k, v, out
+ * and lse have the real sizes H and W: nothing is padded in memory.  With H and W multiples of the window this is
+ * rib_window_attn_fwd_headwise; other arguments, layouts and error codes as there.  H and W multiples of 8 (and
+ * the shape conditions above) take the tcgen05 kernel, where a patch of the extension costs a zero-filled TMA box;
+ * any other H, W take the any-shape kernel.  Forward only: there is no backward entry point for such maps.
+ */
+int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* out, float* lse, void* stream);
+
+/*
  * Backward pass for callers that cannot hand over scratch memory.  (The paper has no counterpart:
  * this entry point exists for the library's users, not for the method.)
  *

@@ -24,6 +24,7 @@ EXPORTS = (
     "rib_window_attn_bwd_noalloc", "rib_profile_begin", "rib_profile_end",
     "rib_generate_features", "rib_generate_features_bwd",
     "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
+    "rib_window_attn_fwd_padded",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
@@ -58,6 +59,8 @@ def library() -> ctypes.CDLL:
         ll = ctypes.c_longlong
         lib.rib_window_attn_fwd_headwise.restype = ci
         lib.rib_window_attn_fwd_headwise.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
+        lib.rib_window_attn_fwd_padded.restype = ci
+        lib.rib_window_attn_fwd_padded.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd_headwise.restype = ci
         lib.rib_window_attn_bwd_headwise.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
         lib.rib_window_attn_bwd_headwise_workspace.restype = ctypes.c_size_t
@@ -221,6 +224,31 @@ def rib_window_attn_fwd_headwise(q, k, v, pq, pk, window, shift=0, stream=None, 
     lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device) if want_lse else None
     rc = library().rib_window_attn_fwd_headwise(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r, B, H, W, heads,
                                                 d, r, window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return out, lse
+
+
+def rib_window_attn_fwd_padded(q, k, v, pq, pk, window, shift=0, stream=None, want_lse=True):
+    """Forward pass on a map whose sides need not be multiples of the window (positions of the extended map
+    beyond H x W are not tokens); pq, pk are [n, r] or [heads, n, r].  Returns (out, lse)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    _check_image("k", k, q.shape)
+    _check_image("v", v, q.shape)
+    n = window * window
+    headwise = pq.dim() == 3
+    if headwise:
+        _check_pos_headwise("pq", pq, heads, n)
+        _check_pos_headwise("pk", pk, heads, n)
+    else:
+        _check_pos("pq", pq, n)
+        _check_pos("pk", pk, n)
+    r = pq.shape[-1]
+    out = torch.empty_like(q)
+    lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device) if want_lse else None
+    rc = library().rib_window_attn_fwd_padded(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r if headwise else 0,
+                                              B, H, W, heads, d, r, window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
     if rc != RIB_OK:
         raise RibError(rc)
     return out, lse

@@ -17,13 +17,13 @@ std::atomic<long long> g_kernel_launches{0};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int check_shape(int B, int H, int W, int heads, int d, int r, int window, int shift)
+int check_shape(int B, int H, int W, int heads, int d, int r, int window, int shift, bool partial_windows = false)
 {
     if (B <= 0 || H <= 0 || W <= 0 || heads <= 0 || d <= 0 || r < 0 || window <= 0) return RIB_ERR_SHAPE;
-    if (H % window || W % window) return RIB_ERR_SHAPE;
+    if (!partial_windows && (H % window || W % window)) return RIB_ERR_SHAPE;
     if (shift < 0 || shift >= window) return RIB_ERR_SHAPE;
     if (d > 64 || r > 64 || (d % 8) || (r % 8)) return RIB_ERR_UNSUPPORTED;
-    const long long pairs = (long long)B * (H / window) * (W / window) * heads;
+    const long long pairs = (long long)B * ((H + window - 1) / window) * ((W + window - 1) / window) * heads;
     if (pairs > 0x7fffffffLL || (long long)window * window > (1 << 20)) return RIB_ERR_SHAPE;
     return RIB_OK;
 }
@@ -39,7 +39,9 @@ int device_status_ptr(int** out)
 void fill_shape(rib::Problem& p, int B, int H, int W, int heads, int d, int r, int window, int shift)
 {
     p.B = B; p.H = H; p.W = W; p.heads = heads; p.d = d; p.r = r; p.M = window; p.s = shift;
-    p.n = window * window; p.nWy = H / window; p.nWx = W / window;
+    p.nWy = (H + window - 1) / window; p.nWx = (W + window - 1) / window;   // exact in the plain calls (H, W multiples of window)
+    p.Hp = p.nWy * window; p.Wp = p.nWx * window;
+    p.n = window * window;
     p.pairs = B * p.nWy * p.nWx * heads;
 }
 
@@ -169,8 +171,17 @@ int rib_window_attn_fwd_headwise(const void* q, const void* k, const void* v, co
                                  int B, int H, int W, int heads, int d, int r, int window, int shift,
                                  void* out, float* lse, void* stream)
 {
+    if (H > 0 && W > 0 && window > 0 && (H % window || W % window)) return RIB_ERR_SHAPE;
+    return rib_window_attn_fwd_padded(q, k, v, pq, pk, pos_head_stride, B, H, W, heads, d, r, window, shift, out, lse, stream);
+}
+
+int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* out, float* lse, void* stream)
+{
     if (!q || !k || !v || !out || (r > 0 && (!pq || !pk))) return RIB_ERR_NULL;
-    if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    if (int rc = check_shape(B, H, W, heads, d, r, window, shift, true)) return rc;
     if (int rc = check_pos_stride(pos_head_stride, window, r)) return rc;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(pq) ||
         !aligned16(pk) || !aligned16(lse))

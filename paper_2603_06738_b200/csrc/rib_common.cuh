@@ -32,6 +32,8 @@ struct Problem {
     size_t workspace_bytes;
     long long pos_head_stride;        // elements between the heads' tables in pq/pk/dpq/dpk; 0 = one table for all heads
     int B, H, W, heads, d, r, M, s;   // M = window side, s = cyclic shift
+    int Hp, Wp;                       // sides of the map the windows are laid over: H, W rounded up to multiples of M
+                                      // (positions with Y >= H or X >= W are not tokens); equal to H, W in the plain calls
     int n, nWy, nWx, pairs;           // n = M*M, windows per image, B*nWy*nWx*heads
     int* status;                      // device status word (bounded waits report here)
 };

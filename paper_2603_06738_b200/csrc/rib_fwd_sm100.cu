@@ -72,6 +72,7 @@ struct FwdParams {
     float* lse;
     int* status;
     int H, W, heads, M, s, n, nWy, nWx;
+    int Hp, Wp;                // sides of the map the windows are laid over (H, W rounded up to multiples of M)
     int tiles_per_item_pair;   // n / 256: items per pair
     int items;
     float scale_log2;          // log2(e) / sqrt(d)
@@ -97,10 +98,13 @@ __device__ __forceinline__ ItemCoord decode_item(const FwdParams& p, int item)
 __device__ __forceinline__ void patch_origin(const FwdParams& p, const ItemCoord& c, int sp, int& py, int& px,
                                              int& Y0, int& X0)
 {
-    sm100::patch_origin(WindowGeom{p.H, p.W, p.M, p.s}, c.wy, c.wx, sp, py, px, Y0, X0);
+    sm100::patch_origin(WindowGeom{p.Hp, p.Wp, p.M, p.s}, c.wy, c.wx, sp, py, px, Y0, X0);
 }
 
-template <int R>
+// kPartial: H or W is not a multiple of the window (but of 8).  Windows are laid over the map extended to Hp x Wp;
+// an 8x8 patch of the extension holds no tokens: TMA fills it with zeros, the softmax warps give its keys the
+// probability 0, and nothing is stored for its queries.
+template <int R, bool kPartial>
 __global__ void __launch_bounds__(kThreads, 1)
 rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_pk,
@@ -325,11 +329,38 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
             const ItemCoord c = decode_item(p, item);
             float m_used = -INFINITY, l = 0.f;
+            bool have_ref = false;            // kPartial: a block with real keys has set the reference
             for (int j = 0; j < nblk; ++j, ++blk) {
                 // warp-uniform outcome: the TMEM loads below are warp-collective
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
                 bool p_free = blk == 0;       // P (and O) of this half are free once the previous block's PV has completed
+                if (kPartial) {
+                    // this thread's 64 keys are one 8x8 patch: beyond the image it holds no tokens
+                    int py, px, Y0, X0;
+                    patch_origin(p, c, 2 * j + half, py, px, Y0, X0);
+                    if (Y0 >= p.H || X0 >= p.W) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kSFree + qt));
+                        if (!p_free) {
+                            if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        uint32_t zero[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) zero[i] = 0u;
+                        tmem_st16(t_p, zero);
+                        tmem_st16(t_p + 16, zero);
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(b_ready);
+                        continue;
+                    }
+                }
+                const bool first_ref = kPartial ? !have_ref : j == 0;
+                have_ref = true;
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
                     uint32_t s[32];
@@ -342,7 +373,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
                     }
                     const float mx = fmaxf(mx0, mx1);
-                    if (j == 0 && ch == 0) {
+                    if (first_ref && ch == 0) {
                         m_used = mx;
                     } else {
                         // Move the reference (and rescale O, l) only when the maximum grew by more than
@@ -426,6 +457,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             int py, px, Y0, X0;
             patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
             const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
+            if (kPartial && (Y0 >= p.H || X0 >= p.W)) continue;        // a patch of the extension: no tokens, nothing to store
             const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
             uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD + half * 16);
 #pragma unroll
@@ -456,10 +488,10 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
 bool sm100_fwd_supported(const Problem& p)
 {
-    return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
+    return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
 }
 
-template <int R>
+template <int R, bool kPartial>
 cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
@@ -472,12 +504,13 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     if (!sm_count) {
         cudaError_t e = sm_count_of_current_device(&sm_count);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rib_fwd_sm100_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            e = cudaFuncSetAttribute(rib_fwd_sm100_kernel<R, kPartial>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) { sm_count = 0; return e; }
     }
     FwdParams fp{};
     fp.pq = p.pq; fp.out = p.out_w; fp.lse = p.lse_w; fp.status = p.status;
     fp.H = p.H; fp.W = p.W; fp.heads = p.heads; fp.M = p.M; fp.s = p.s; fp.n = p.n; fp.nWy = p.nWy; fp.nWx = p.nWx;
+    fp.Hp = p.Hp; fp.Wp = p.Wp;
     fp.tiles_per_item_pair = p.n / (2 * kTile);
     fp.items = p.pairs * fp.tiles_per_item_pair;
     fp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
@@ -486,13 +519,14 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     const int grid = fp.items < sm_count ? fp.items : sm_count;
-    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<R><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
+    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<R, kPartial><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
     return cudaGetLastError();
 }
 
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
 {
-    return p.r == 32 ? launch_fwd<32>(p, stream) : launch_fwd<16>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W) return p.r == 32 ? launch_fwd<32, true>(p, stream) : launch_fwd<16, true>(p, stream);
+    return p.r == 32 ? launch_fwd<32, false>(p, stream) : launch_fwd<16, false>(p, stream);
 }
 
 }  // namespace rib

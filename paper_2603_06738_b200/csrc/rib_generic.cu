@@ -30,18 +30,26 @@ __device__ inline PairCoord decode_pair(const Problem& p, int pid)
     return c;
 }
 
-// element offset of channel 0 of token i of the pair in a [B][H][W][heads][d] tensor
+// Position i of the pair's window is a token unless it lies in the part of the extended map beyond the image.
+__device__ inline bool token_exists(const Problem& p, const PairCoord& c, int i)
+{
+    int Y, X;
+    token_pixel(p.Hp, p.Wp, p.M, p.s, c.wy, c.wx, i, Y, X);
+    return Y < p.H && X < p.W;
+}
+
+// element offset of channel 0 of token i of the pair in a [B][H][W][heads][d] tensor (the token must exist)
 __device__ inline size_t token_offset(const Problem& p, const PairCoord& c, int i)
 {
     int Y, X;
-    token_pixel(p.H, p.W, p.M, p.s, c.wy, c.wx, i, Y, X);
+    token_pixel(p.Hp, p.Wp, p.M, p.s, c.wy, c.wx, i, Y, X);
     return ((((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h) * p.d;
 }
 
 __device__ inline size_t token_scalar_offset(const Problem& p, const PairCoord& c, int i)
 {
     int Y, X;
-    token_pixel(p.H, p.W, p.M, p.s, c.wy, c.wx, i, Y, X);
+    token_pixel(p.Hp, p.Wp, p.M, p.s, c.wy, c.wx, i, Y, X);
     return (((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X;
 }
 
@@ -67,7 +75,7 @@ __device__ inline void stage_concat(const Problem& p, const PairCoord& c, const 
         const int rr = idx / dk, col = idx - rr * dk;
         const int i = row0 + rr;
         float val = 0.f;
-        if (i < p.n) {
+        if (i < p.n && token_exists(p, c, i)) {
             val = col < p.d ? __bfloat162float(x[token_offset(p, c, i) + col]) * sx
                             : __bfloat162float(pos[(size_t)c.h * p.pos_head_stride + (size_t)i * p.r + (col - p.d)]) * sp;
         }
@@ -82,7 +90,7 @@ __device__ inline void stage_plain(const Problem& p, const PairCoord& c, const _
     for (int idx = threadIdx.x; idx < rows * p.d; idx += kThreads) {
         const int rr = idx / p.d, col = idx - rr * p.d;
         const int i = row0 + rr;
-        dst[rr * ld + col] = i < p.n ? __bfloat162float(x[token_offset(p, c, i) + col]) : 0.f;
+        dst[rr * ld + col] = i < p.n && token_exists(p, c, i) ? __bfloat162float(x[token_offset(p, c, i) + col]) : 0.f;
     }
 }
 
@@ -118,11 +126,13 @@ __global__ void __launch_bounds__(kThreads) generic_fwd_kernel(const Problem p)
                 s0 = fmaf(a, Kt[lane * ldk + col], s0);
                 s1 = fmaf(a, Kt[(lane + 32) * ldk + col], s1);
             }
-            if (j0 + lane >= p.n) s0 = -INFINITY;
-            if (j0 + lane + 32 >= p.n) s1 = -INFINITY;
-            const float m_new = fmaxf(m[rr], warp_max(fmaxf(s0, s1)));   // finite: key j0 exists
-            const float alpha = expf(m[rr] - m_new);
-            const float p0 = expf(s0 - m_new), p1 = expf(s1 - m_new);
+            if (j0 + lane >= p.n || !token_exists(p, c, j0 + lane)) s0 = -INFINITY;
+            if (j0 + lane + 32 >= p.n || !token_exists(p, c, j0 + lane + 32)) s1 = -INFINITY;
+            const float m_new = fmaxf(m[rr], warp_max(fmaxf(s0, s1)));
+            // -inf only while no key of the row's window has been seen yet (extended maps): nothing to add then
+            const bool none = m_new == -INFINITY;
+            const float alpha = none ? 1.f : expf(m[rr] - m_new);
+            const float p0 = none ? 0.f : expf(s0 - m_new), p1 = none ? 0.f : expf(s1 - m_new);
             l[rr] = l[rr] * alpha + warp_sum(p0 + p1);
             m[rr] = m_new;
             o[rr][0] *= alpha; o[rr][1] *= alpha;
@@ -143,7 +153,7 @@ __global__ void __launch_bounds__(kThreads) generic_fwd_kernel(const Problem p)
     }
     for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int i = row0 + warp * kRowsPerWarp + rr;
-        if (i >= p.n) continue;
+        if (i >= p.n || !token_exists(p, c, i)) continue;
         const size_t off = token_offset(p, c, i);
         const float inv = 1.f / l[rr];
         if (lane < p.d) p.out_w[off + lane] = __float2bfloat16_rn(o[rr][0] * inv);

@@ -1,0 +1,71 @@
+"""GPU parity for feature maps whose sides are not multiples of the window: rib_window_attn_fwd_padded against the
+numpy oracle of the same reading (positions of the extended map beyond the image are not tokens), on the tcgen05
+kernel (H, W multiples of 8) and on the any-shape kernel, every element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rib_padded_oracle as pad
+from paper_2603_06738_b200 import binding, synthetic
+from paper_2603_06738_b200.synthetic import Workload
+
+from parity_util import compare, to_f64
+
+pytestmark = pytest.mark.gpu
+
+# name, B, H, W, heads, d, r, window, shift
+CASES = [
+    Workload("p_6x10_w4", 2, 6, 10, 2, 16, 8, 4, 0, seed=61),
+    Workload("p_7x5_w4_s1", 1, 7, 5, 1, 8, 8, 4, 1, seed=62),
+    Workload("p_20x28_w8_s3", 1, 20, 28, 3, 32, 16, 8, 3, seed=63),
+    Workload("p_3x3_w4", 1, 3, 3, 2, 8, 8, 4, 0, seed=64),                       # one window, 9 of 16 positions real
+    Workload("p_40x56_w16", 2, 40, 56, 2, 32, 16, 16, 0, seed=65),               # tcgen05 shapes from here on
+    Workload("p_40x56_w16_s8", 1, 40, 56, 3, 32, 16, 16, 8, seed=66),
+    Workload("p_72x88_w32_s16", 1, 72, 88, 3, 32, 16, 32, 16, seed=67),
+    Workload("p_56x104_w48_s24_r32", 1, 56, 104, 2, 32, 32, 48, 24, seed=68),
+    Workload("p_40x24_w32_headwise", 1, 40, 24, 3, 32, 16, 32, 0, seed=69, headwise=True),
+    Workload("p_8x8_w16", 1, 8, 8, 1, 32, 16, 16, 0, seed=70),                    # a quarter of one window
+    Workload("p_120x200_w64", 1, 120, 200, 2, 32, 16, 64, 0, seed=71),            # 16:9-like frame, 64 x 64 windows
+]
+
+
+@pytest.mark.parametrize("wl", CASES, ids=lambda w: w.name)
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_padded_forward_every_element(wl, path):
+    cpu = synthetic.make_inputs(wl, with_dout=False)
+    gpu = {k: v.cuda() for k, v in cpu.items()}
+    binding.rib_set_path(binding.RIB_PATH_GENERIC if path == "generic" else binding.RIB_PATH_NONE)
+    try:
+        out, lse = binding.rib_window_attn_fwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+        used = binding.rib_last_path()
+    finally:
+        binding.rib_set_path(binding.RIB_PATH_NONE)
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0
+    fast = (path == "auto" and wl.d == 32 and wl.r in (16, 32) and wl.window % 16 == 0 and wl.shift % 8 == 0
+            and wl.H % 8 == 0 and wl.W % 8 == 0)
+    assert used == (binding.RIB_PATH_SM100 if fast else binding.RIB_PATH_GENERIC)
+    ref_out, ref_lse = pad.fwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk")), wl.window, wl.shift)
+    assert np.isfinite(ref_out).all() and np.isfinite(ref_lse).all()      # every real token belongs to one window
+    compare("out", to_f64(out), ref_out)
+    compare("lse", to_f64(lse), ref_lse)
+
+
+def test_divisible_map_through_the_padded_entry_point_is_the_plain_call():
+    wl = Workload("p_divisible", 2, 64, 32, 3, 32, 16, 32, 8, seed=72)
+    gpu = {k: v.cuda() for k, v in synthetic.make_inputs(wl, with_dout=False).items()}
+    a = binding.rib_window_attn_fwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+    b = binding.rib_window_attn_fwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+    torch.cuda.synchronize()
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_plain_entry_points_still_reject_partial_windows():
+    x = torch.zeros(40 * 56 * 32, dtype=torch.bfloat16, device="cuda")
+    pos = torch.zeros(256 * 16, dtype=torch.bfloat16, device="cuda")
+    lib = binding.library()
+    rc = lib.rib_window_attn_fwd(x.data_ptr(), x.data_ptr(), x.data_ptr(), pos.data_ptr(), pos.data_ptr(),
+                                 1, 40, 56, 1, 32, 16, 16, 0, x.data_ptr(), None, None)
+    assert rc == -2      # RIB_ERR_SHAPE
+    assert lib.rib_window_attn_bwd_workspace(1, 40, 56, 1, 32, 16, 16) == 0
