@@ -635,13 +635,9 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
         !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * R) ||
         !encode_pos_map_padded(&tm_pk, p.pk, p, tables, p.pos_head_stride))
         return cudaErrorInvalidValue;
-    static int sm_count = 0;
-    if (!sm_count) {
-        cudaError_t e = sm_count_of_current_device(&sm_count);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rib_bwd_sm100_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) { sm_count = 0; return e; }
-    }
+    static KernelSetup setup;       // one per instantiation of this launcher, i.e. per kernel
+    int sm_count = 0;
+    if (cudaError_t e = setup.prepare(rib_bwd_sm100_kernel<R>, kSmemBytes, &sm_count)) return e;
     AuxParams ap{};
     ap.out = p.out; ap.dout = p.dout; ap.pq = p.pq; ap.lse = p.lse_in;
     ap.ld = ld; ap.dq_acc = dq_acc; ap.dkp = dkp; ap.pq_scaled = pq_scaled;

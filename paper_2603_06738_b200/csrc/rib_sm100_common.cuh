@@ -115,5 +115,33 @@ inline cudaError_t sm_count_of_current_device(int* count)
     return e;
 }
 
+// Per-kernel, per-device launch set-up: the dynamic shared-memory limit of a kernel is an attribute of the kernel on
+// ONE device, so a process that drives several GPUs has to raise it on each of them.  One instance of this struct per
+// kernel (a function-local static); prepare() raises the limit on the current device the first time it is seen there
+// and returns that device's SM count.
+struct KernelSetup {
+    static constexpr int kMaxDevices = 64;
+    std::mutex mutex;
+    int sm_count[kMaxDevices] = {};
+    template <typename Kernel>
+    cudaError_t prepare(Kernel kernel, uint32_t smem_bytes, int* sms)
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mutex);
+        if (!sm_count[dev]) {
+            int count = 0;
+            e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+            if (e != cudaSuccess) return e;
+            sm_count[dev] = count;
+        }
+        *sms = sm_count[dev];
+        return cudaSuccess;
+    }
+};
+
 }  // namespace sm100
 }  // namespace rib

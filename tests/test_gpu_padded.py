@@ -26,6 +26,9 @@ CASES = [
     Workload("p_40x24_w32_headwise", 1, 40, 24, 3, 32, 16, 32, 0, seed=69, headwise=True),
     Workload("p_8x8_w16", 1, 8, 8, 1, 32, 16, 16, 0, seed=70),                    # a quarter of one window
     Workload("p_120x200_w64", 1, 120, 200, 2, 32, 16, 64, 0, seed=71),            # 16:9-like frame, 64 x 64 windows
+    Workload("p_8x24_w16", 2, 8, 24, 2, 32, 16, 16, 0, seed=73),                  # every item has one key block with tokens
+    Workload("p_8x24_w16_s8", 2, 8, 24, 2, 32, 16, 16, 8, seed=74),
+    Workload("p_88x40_w32_s8", 2, 88, 40, 2, 32, 16, 32, 8, seed=75),             # whole query tiles in the extension
 ]
 
 
