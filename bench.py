@@ -154,6 +154,7 @@ def main():
     ap.add_argument("--workload", default=None, help="prefix of a configuration name (default: cfg2 shape)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the timings of rank 32, head-wise tables and partial windows")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -334,6 +335,47 @@ def main():
                "algorithmic_bytes_fwd": 4 * ((2 + 4 * gL) * gdh + gdh + 2 * gdh * wl.r) + 2 * 2 * wl.n * wl.r,
                "algorithmic_flops_fwd": 2 * wl.n * ((2 + 4 * gL) * gdh + 2 * gdh * wl.r)}
 
+    # ------------------------------------------------ the path's variants beyond the benchmark shape (rank 0, device-timed)
+    variants = None
+    if rank == 0 and not args.no_variants:
+        variants = {"timing": "CUDA events, one buffer set per variant reused every iteration (inputs may stay in L2)"}
+
+        def timed(fn, reps=20):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        s0 = sets[0]
+        for name, r_v, headwise in (("rank32", 32, False), ("headwise", wl.r, True)):
+            shape = (wl.heads, wl.n, r_v) if headwise else (wl.n, r_v)
+            pq_v, pk_v = ((0.5 * torch.randn(shape, device=dev)).to(torch.bfloat16) for _ in range(2))
+            fwd_fn = binding.rib_window_attn_fwd_headwise if headwise else binding.rib_window_attn_fwd
+            bwd_fn = binding.rib_window_attn_bwd_headwise if headwise else binding.rib_window_attn_bwd
+            out_v, lse_v = fwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, wl.window, wl.shift)
+            f_ms = timed(lambda: fwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, wl.window, wl.shift))
+            b_ms = timed(lambda: bwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, out_v, lse_v, s0["dout"], wl.window, wl.shift))
+            ff = wl.pairs * 2 * wl.n * wl.n * (2 * wl.d + r_v)
+            bf = wl.pairs * 2 * wl.n * wl.n * (5 * wl.d + 3 * r_v)
+            variants[name] = {"r": r_v, "fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_tflops": ff / (f_ms * 1e-3) / 1e12,
+                              "bwd_tflops": bf / (b_ms * 1e-3) / 1e12, "paths": [binding.rib_last_path()]}
+        # the paper's inference frame: 360 x 640 tokens, not a multiple of the 64 x 64 window (forward only)
+        fh, fw, fwin = 360, 640, 64
+        fq, fk, fv = (torch.randn((1, fh, fw, wl.heads, wl.d), device=dev).to(torch.bfloat16) for _ in range(3))
+        fpq, fpk = ((0.5 * torch.randn((fwin * fwin, wl.r), device=dev)).to(torch.bfloat16) for _ in range(2))
+        f_ms = timed(lambda: binding.rib_window_attn_fwd_padded(fq, fk, fv, fpq, fpk, fwin, 0), reps=10)
+        variants["partial_windows_360x640_w64"] = {"fwd_ms": f_ms, "tokens_per_s": fh * fw / (f_ms * 1e-3),
+                                                   "paths": [binding.rib_last_path()]}
+        if binding.rib_query_status() != 0:
+            raise SystemExit("device status word set during the variant timings")
+        del fq, fk, fv
+
     # ------------------------------------------------ reduce over ranks (max time), compose the line
     total_ms, fwd_med, bwd_med, e2e_ms_max = multi.max_over_ranks(
         [total_ms, statistics.median(fwd_ms), statistics.median(bwd_ms), e2e_ms or 0.0], device=dev)
@@ -393,6 +435,7 @@ def main():
             "overlap": "copies in, compute and copies out on three streams over two device buffer sets"},
         "gpu_launches": launches,
         "generator": gen,
+        "variants": variants,
         "clocks": sampler.summary(),
         "wall_s": t_wall,
         "device_status": status,
