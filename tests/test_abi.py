@@ -57,6 +57,31 @@ def test_fwd_rejects_bad_arguments_without_launching(lib, over, code):
     assert lib.rib_window_attn_fwd(*fwd_args(**over)) == code
 
 
+def headwise_args(stride, **over):
+    a = fwd_args(**over)
+    return a[:5] + [stride] + a[5:]
+
+
+def test_headwise_and_padded_entry_points_validate_before_any_cuda_call(lib):
+    n_r = 16 * 16 * 16
+    # stride: 0 (shared table) or a multiple of 8 that is at least n * r
+    for stride, code in ((n_r - 8, -2), (n_r + 4, -2), (-8, -2)):
+        assert lib.rib_window_attn_fwd_headwise(*headwise_args(stride)) == code
+        assert lib.rib_window_attn_fwd_padded(*headwise_args(stride)) == code
+        assert lib.rib_window_attn_bwd_headwise_workspace(stride, 1, 32, 32, 2, 32, 16, 16) == 0
+    # only the padded entry point takes maps that are not multiples of the window; the other checks stay
+    assert lib.rib_window_attn_fwd_headwise(*headwise_args(0, H=40)) == -2
+    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, q=None)) == -1
+    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, shift=16)) == -2
+    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=0)) == -2
+    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, d=12)) == -3
+    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, v=770)) == -4
+    # rank 32 needs a larger backward workspace than rank 16 on the tcgen05 shapes
+    assert lib.rib_window_attn_bwd_workspace(1, 32, 32, 2, 32, 32, 16) > lib.rib_window_attn_bwd_workspace(1, 32, 32, 2, 32, 16, 16)
+    assert (lib.rib_window_attn_bwd_headwise_workspace(2 * n_r, 1, 32, 32, 2, 32, 16, 16)
+            > lib.rib_window_attn_bwd_headwise_workspace(0, 1, 32, 32, 2, 32, 16, 16))
+
+
 def test_bwd_rejects_bad_arguments(lib):
     base = dict(q=256, k=512, v=768, pq=1024, pk=1280, out=1536, lse=1792, dout=2048, B=1, H=32, W=32, heads=2,
                 d=32, r=16, window=16, shift=0, dq=4096, dk=8192, dv=12288, dpq=16384, dpk=20480,
