@@ -133,6 +133,29 @@ int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, cons
                                void* out, float* lse, void* stream);
 
 /*
+ * Convolutional Local Attention (paper: Sec. 3.2, Eq. 7, Eq. 8, Eq. 9): the step right after the attention.
+ *   G  = sigmoid(PWConv(DWConv3x3(X)))      X: the block's token features as an H x W map          (Eq. 8)
+ *   O' = O o G                              element-wise product with the attention output           (Eq. 9)
+ * rib_cla_gate computes G; rib_window_attn_fwd_gated is the forward pass with `out` = O o G, the product taken in
+ * the attention kernel's epilogue so that the ungated O never goes to memory.  Forward only (inference); for
+ * training, take the product outside and use the ungated entry points.
+ *   x     : bf16 [B][H][W][D], D = heads * d, the same channel order as `out` ([heads][d]).
+ *   w_dw  : fp32 [D][3][3] depth-wise filter, w_dw[c][dy][dx] multiplies x[y + dy - 1][x + dx - 1][c]; zero padding.
+ *   b_dw  : fp32 [D].   w_pw : fp32 [D][D], [output channel][input channel].   b_pw : fp32 [D].
+ *   gate  : bf16 [B][H][W][D], overwritten (rib_cla_gate) / read (rib_window_attn_fwd_gated).
+ * The paper does not state padding, stride or biases of the two convolutions; these are the readings taken.
+ * rib_cla_gate supports D = 64, 128 or 192 with H a multiple of 8 and W a multiple of 16 (RIB_ERR_UNSUPPORTED
+ * otherwise); all pointers 16-byte aligned.  rib_window_attn_fwd_gated takes the shapes of
+ * rib_window_attn_fwd_headwise (pos_head_stride = 0: one table for all heads).
+ */
+int rib_cla_gate(const void* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
+                 int B, int H, int W, int D, void* gate, void* stream);
+int rib_window_attn_fwd_gated(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                              long long pos_head_stride, const void* gate,
+                              int B, int H, int W, int heads, int d, int r, int window, int shift,
+                              void* out, float* lse, void* stream);
+
+/*
  * Backward pass for callers that cannot hand over scratch memory.  (The paper has no counterpart:
  * this entry point exists for the library's users, not for the method.)
  *
@@ -220,7 +243,8 @@ long long rib_kernel_launches(void);
  */
 enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH = 4,
        RIB_KERNEL_RESERVED = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
-       RIB_KERNEL_ANY_BWD_DKV = 9, RIB_KERNEL_GENERATOR_FWD = 10, RIB_KERNEL_GENERATOR_BWD = 11 };
+       RIB_KERNEL_ANY_BWD_DKV = 9, RIB_KERNEL_GENERATOR_FWD = 10, RIB_KERNEL_GENERATOR_BWD = 11,
+    RIB_KERNEL_CLA_GATE = 12 };
 int rib_profile_begin(int max_launches);
 int rib_profile_end(int* kernel_ids, float* ms, int capacity);
 

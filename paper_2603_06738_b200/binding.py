@@ -24,12 +24,12 @@ EXPORTS = (
     "rib_window_attn_bwd_noalloc", "rib_profile_begin", "rib_profile_end",
     "rib_generate_features", "rib_generate_features_bwd",
     "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
-    "rib_window_attn_fwd_padded",
+    "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
                 7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel",
-                10: "rib_generator_fwd_kernel", 11: "rib_generator_bwd_kernel"}
+                10: "rib_generator_fwd_kernel", 11: "rib_generator_bwd_kernel", 12: "rib_cla_gate_kernel"}
 RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
@@ -61,6 +61,10 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_fwd_headwise.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_fwd_padded.restype = ci
         lib.rib_window_attn_fwd_padded.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
+        lib.rib_cla_gate.restype = ci
+        lib.rib_cla_gate.argtypes = [vp] * 5 + [ci] * 4 + [vp, vp]
+        lib.rib_window_attn_fwd_gated.restype = ci
+        lib.rib_window_attn_fwd_gated.argtypes = [vp] * 5 + [ll, vp] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd_headwise.restype = ci
         lib.rib_window_attn_bwd_headwise.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
         lib.rib_window_attn_bwd_headwise_workspace.restype = ctypes.c_size_t
@@ -249,6 +253,49 @@ def rib_window_attn_fwd_padded(q, k, v, pq, pk, window, shift=0, stream=None, wa
     lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device) if want_lse else None
     rc = library().rib_window_attn_fwd_padded(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r if headwise else 0,
                                               B, H, W, heads, d, r, window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return out, lse
+
+
+def rib_cla_gate(x, w_dw, b_dw, w_pw, b_pw, stream=None):
+    """CLA gate (Eq. 8): x bf16 [B,H,W,D]; w_dw fp32 [D,3,3]; b_dw fp32 [D]; w_pw fp32 [D,D] (out, in); b_pw fp32 [D].
+    Returns the gate, bf16 [B,H,W,D]."""
+    if x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous() or x.dim() != 4:
+        raise ValueError("x must be a contiguous CUDA bfloat16 tensor [B,H,W,D]")
+    B, H, W, D = x.shape
+    for name, t, shape in (("w_dw", w_dw, (D, 3, 3)), ("b_dw", b_dw, (D,)), ("w_pw", w_pw, (D, D)), ("b_pw", b_pw, (D,))):
+        if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shape:
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor of shape {shape}")
+    gate = torch.empty_like(x)
+    rc = library().rib_cla_gate(_ptr(x), _ptr(w_dw), _ptr(b_dw), _ptr(w_pw), _ptr(b_pw), B, H, W, D, _ptr(gate), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return gate
+
+
+def rib_window_attn_fwd_gated(q, k, v, pq, pk, gate, window, shift=0, stream=None, want_lse=True):
+    """Forward pass whose output is multiplied by the CLA gate (Eq. 9); gate bf16 [B,H,W,heads*d]; pq, pk [n,r] or
+    [heads,n,r].  Returns (out, lse)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    _check_image("k", k, q.shape)
+    _check_image("v", v, q.shape)
+    if gate.dtype != torch.bfloat16 or not gate.is_cuda or not gate.is_contiguous() or tuple(gate.shape) != (B, H, W, heads * d):
+        raise ValueError("gate must be a contiguous CUDA bfloat16 tensor [B,H,W,heads*d]")
+    n = window * window
+    headwise = pq.dim() == 3
+    if headwise:
+        _check_pos_headwise("pq", pq, heads, n)
+        _check_pos_headwise("pk", pk, heads, n)
+    else:
+        _check_pos("pq", pq, n)
+        _check_pos("pk", pk, n)
+    r = pq.shape[-1]
+    out = torch.empty_like(q)
+    lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device) if want_lse else None
+    rc = library().rib_window_attn_fwd_gated(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r if headwise else 0, _ptr(gate),
+                                             B, H, W, heads, d, r, window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
     if rc != RIB_OK:
         raise RibError(rc)
     return out, lse

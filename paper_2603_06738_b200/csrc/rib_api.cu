@@ -45,6 +45,9 @@ void fill_shape(rib::Problem& p, int B, int H, int W, int heads, int d, int r, i
     p.pairs = B * p.nWy * p.nWx * heads;
 }
 
+int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk, long long pos_head_stride, const void* gate,
+             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream);
+
 int check_pos_stride(long long stride, int window, int r)
 {
     if (stride == 0) return RIB_OK;
@@ -180,6 +183,45 @@ int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, cons
                                int B, int H, int W, int heads, int d, int r, int window, int shift,
                                void* out, float* lse, void* stream)
 {
+    return fwd_impl(q, k, v, pq, pk, pos_head_stride, nullptr, B, H, W, heads, d, r, window, shift, out, lse, stream);
+}
+
+int rib_window_attn_fwd_gated(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                              long long pos_head_stride, const void* gate,
+                              int B, int H, int W, int heads, int d, int r, int window, int shift,
+                              void* out, float* lse, void* stream)
+{
+    if (!gate) return RIB_ERR_NULL;
+    if (H > 0 && W > 0 && window > 0 && (H % window || W % window)) return RIB_ERR_SHAPE;
+    if (!aligned16(gate)) return RIB_ERR_ALIGN;
+    return fwd_impl(q, k, v, pq, pk, pos_head_stride, gate, B, H, W, heads, d, r, window, shift, out, lse, stream);
+}
+
+int rib_cla_gate(const void* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
+                 int B, int H, int W, int D, void* gate, void* stream)
+{
+    if (!x || !w_dw || !b_dw || !w_pw || !b_pw || !gate) return RIB_ERR_NULL;
+    if (B <= 0 || H <= 0 || W <= 0 || D <= 0) return RIB_ERR_SHAPE;
+    if (!rib::cla_gate_supported(H, W, D)) return RIB_ERR_UNSUPPORTED;
+    const void* ptrs[] = {x, w_dw, b_dw, w_pw, b_pw, gate};
+    for (const void* ptr : ptrs)
+        if (!aligned16(ptr)) return RIB_ERR_ALIGN;
+    int* status = nullptr;
+    if (int rc = device_status_ptr(&status)) return rc;
+    const cudaError_t e = rib::cla_gate(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw, B, H, W, D,
+                                        static_cast<__nv_bfloat16*>(gate), status, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk, long long pos_head_stride, const void* gate,
+             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream)
+{
     if (!q || !k || !v || !out || (r > 0 && (!pq || !pk))) return RIB_ERR_NULL;
     if (int rc = check_shape(B, H, W, heads, d, r, window, shift, true)) return rc;
     if (int rc = check_pos_stride(pos_head_stride, window, r)) return rc;
@@ -196,6 +238,7 @@ int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, cons
     p.out_w = static_cast<__nv_bfloat16*>(out);
     p.lse_w = lse;
     p.pos_head_stride = pos_head_stride;
+    p.gate = static_cast<const __nv_bfloat16*>(gate);
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
@@ -205,6 +248,10 @@ int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, cons
     g_kernel_launches += 1;
     return RIB_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 size_t rib_window_attn_bwd_workspace(int B, int H, int W, int heads, int d, int r, int window)
 {

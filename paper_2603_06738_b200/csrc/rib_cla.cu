@@ -1,0 +1,225 @@
+// Convolutional Local Attention gate for B200 (sm_100a), Eq. 8 of the paper:
+//     G = sigmoid(PWConv(DWConv3x3(X)))        X, G: bf16 [B][H][W][D], D = heads * d channels
+// (3 x 3 depth-wise filter with zero padding and bias, then a D x D matrix over the channels with bias).
+// The attention kernels multiply their output by G in the epilogue (Eq. 9), so the gated output never makes a
+// round trip through HBM.
+//
+// One kernel.  A CTA walks tiles of 8 x 16 pixels: (1) the 10 x 18 halo of the tile goes to shared memory, (2) the
+// depth-wise filter runs on it in fp32 and its bf16 result becomes the A operand (128 pixels x D, K-major, SWIZZLE_128B),
+// (3) the point-wise matrix -- staged once per CTA as bf16, [out][in], the same layout -- is the B operand of D / 16
+// tcgen05 MMAs (M128, N = D, K16) that accumulate in tensor memory, (4) all warps read the accumulator back, add the
+// bias, apply the sigmoid and store bf16.  The step is small (a few GFLOP, tens of MB) and HBM-bound; the steps of a
+// tile are separated by CTA barriers, nothing is pipelined.
+#include "rib_sm100_common.cuh"
+
+namespace rib {
+namespace {
+
+using namespace sm100;
+
+constexpr int kTileH = 8, kTileW = 16, kPix = kTileH * kTileW;       // 128 pixels = the M of the MMA
+constexpr int kHaloH = kTileH + 2, kHaloW = kTileW + 2;
+constexpr int kThreads = 256;
+
+template <int D>
+struct Layout {
+    static_assert(D % 64 == 0 && D >= 64 && D <= 192, "channels come in SWIZZLE_128B atoms of 64");
+    static constexpr int kAtoms = D / 64;                                  // 128-byte K slices
+    static constexpr uint32_t kWAtom = D * 128, kAAtom = kPix * 128;       // bytes of one K slice of B and of A
+    static constexpr uint32_t kOffW = 0;                                   // [atoms][D rows][128 B]   point-wise matrix
+    static constexpr uint32_t kOffA = kOffW + kAtoms * kWAtom;             // [atoms][128 rows][128 B] depth-wise result
+    static constexpr uint32_t kOffHalo = kOffA + kAtoms * kAAtom;          // [10 * 18 pixels][D] bf16
+    static constexpr uint32_t kOffTaps = kOffHalo + kHaloH * kHaloW * D * 2;   // [9 taps][D] fp32
+    static constexpr uint32_t kOffBdw = kOffTaps + 9 * D * 4;
+    static constexpr uint32_t kOffBpw = kOffBdw + D * 4;
+    static constexpr uint32_t kOffBar = kOffBpw + D * 4;
+    static constexpr uint32_t kOffMisc = kOffBar + 8;
+    static constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
+    static_assert(kOffA % 1024 == 0 && kWAtom % 1024 == 0 && kAAtom % 1024 == 0, "swizzle atoms need aligned tiles");
+    static constexpr uint32_t kTmemCols = D <= 64 ? 64 : D <= 128 ? 128 : 256;
+};
+
+struct ClaParams {
+    const __nv_bfloat16* x;
+    const float* w_dw;     // [D][3][3]
+    const float* b_dw;     // [D]
+    const float* w_pw;     // [D out][D in]
+    const float* b_pw;     // [D]
+    __nv_bfloat16* gate;
+    int* status;
+    int B, H, W, tiles_y, tiles_x, tiles;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaParams p)
+{
+    using L = Layout<D>;
+    constexpr int kChunks = D / 8;                       // 16-byte channel chunks per pixel
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + L::kOffMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 4);
+    const uint32_t bar = base + L::kOffBar;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        abort_flag[0] = 0;
+        mbar_init(bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + L::kOffMisc, L::kTmemCols);
+        tmem_relinquish();
+    }
+    // the point-wise matrix as bf16, row = output channel, 64 input channels per 128-byte line, SWIZZLE_128B
+    for (int idx = threadIdx.x; idx < D * kChunks; idx += kThreads) {
+        const int n = idx / kChunks, c8 = idx - n * kChunks;
+        const float4 lo = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8));
+        const float4 hi = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8 + 4));
+        const uint4 v = make_uint4(pack_bf16x2(lo.x, lo.y), pack_bf16x2(lo.z, lo.w), pack_bf16x2(hi.x, hi.y), pack_bf16x2(hi.z, hi.w));
+        *reinterpret_cast<uint4*>(sm + L::kOffW + (c8 >> 3) * L::kWAtom + n * 128 + (((c8 & 7) ^ (n & 7)) << 4)) = v;
+    }
+    float* taps = reinterpret_cast<float*>(sm + L::kOffTaps);
+    float* bdw = reinterpret_cast<float*>(sm + L::kOffBdw);
+    float* bpw = reinterpret_cast<float*>(sm + L::kOffBpw);
+    for (int idx = threadIdx.x; idx < 9 * D; idx += kThreads) {
+        const int t = idx / D, c = idx - t * D;
+        taps[idx] = __ldg(p.w_dw + (size_t)c * 9 + t);      // tap-major: a thread's 8 channels of one tap are contiguous
+    }
+    for (int c = threadIdx.x; c < D; c += kThreads) { bdw[c] = __ldg(p.b_dw + c); bpw[c] = __ldg(p.b_pw + c); }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    constexpr uint64_t kDesc = smem_desc_const(16, 1024, kSwizzle128B);      // K-major, 8-row groups 1024 bytes apart
+    constexpr uint32_t kIdesc = idesc_bf16_f32(kPix, D, false);
+    bool ok = true;
+    uint32_t it = 0;
+    for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
+        const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, b = tile / (p.tiles_x * p.tiles_y);
+        const int y0 = ty * kTileH, x0 = tx * kTileW;
+        // (1) halo: zero outside the image
+        for (int idx = threadIdx.x; idx < kHaloH * kHaloW * kChunks; idx += kThreads) {
+            const int hp = idx / kChunks, c8 = idx - hp * kChunks;
+            const int Y = y0 + hp / kHaloW - 1, X = x0 + hp % kHaloW - 1;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (Y >= 0 && Y < p.H && X >= 0 && X < p.W)
+                v = __ldg(reinterpret_cast<const uint4*>(p.x + (((size_t)b * p.H + Y) * p.W + X) * D) + c8);
+            *reinterpret_cast<uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16) = v;
+        }
+        __syncthreads();
+        // (2) depth-wise 3 x 3 in fp32, result as the bf16 A operand
+        for (int idx = threadIdx.x; idx < kPix * kChunks; idx += kThreads) {
+            const int pix = idx / kChunks, c8 = idx - pix * kChunks;
+            const int py = pix / kTileW, px = pix - py * kTileW;
+            float acc[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] = bdw[8 * c8 + k];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                const int hp = (py + t / 3) * kHaloW + px + t % 3;
+                const uint4 v = *reinterpret_cast<const uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16);
+                const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
+                const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
+                const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+                const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    acc[2 * k] = fmaf(__uint_as_float(u[k] << 16), w[2 * k], acc[2 * k]);
+                    acc[2 * k + 1] = fmaf(__uint_as_float(u[k] & 0xffff0000u), w[2 * k + 1], acc[2 * k + 1]);
+                }
+            }
+            *reinterpret_cast<uint4*>(sm + L::kOffA + (c8 >> 3) * L::kAAtom + pix * 128 + (((c8 & 7) ^ (pix & 7)) << 4)) =
+                make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
+        }
+        fence_proxy_async();
+        __syncthreads();
+        // (3) point-wise matrix: D / 16 accumulating MMAs
+        if (warp == 0) {
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int a = 0; a < L::kAtoms; ++a) {
+                    const uint64_t da = smem_desc_at(kDesc, base + L::kOffA + a * L::kAAtom);
+                    const uint64_t db = smem_desc_at(kDesc, base + L::kOffW + a * L::kWAtom);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) mma_ss(tmem, da + 2 * kk, db + 2 * kk, kIdesc, (a | kk) ? 1u : 0u);   // + 32 bytes per K16 step
+                }
+                mma_commit(bar);
+            }
+            __syncwarp();
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(bar, it & 1, abort_flag, p.status))) { ok = false; break; }
+        tc_fence_after();
+        // (4) bias, sigmoid, store: a warp reads its 32 accumulator lanes (pixels) and one half of the channels
+        {
+            const int quarter = warp & 3, colhalf = warp >> 2;
+            const int pix = quarter * 32 + lane;
+            const int py = pix / kTileW, px = pix - py * kTileW;
+            const uint32_t t_acc = tmem + ((uint32_t)(quarter * 32) << 16) + colhalf * (D / 2);
+            __nv_bfloat16* dst = p.gate + (((size_t)b * p.H + y0 + py) * p.W + x0 + px) * D + colhalf * (D / 2);
+#pragma unroll
+            for (int part = 0; part < D / 32; ++part) {
+                uint32_t a[16];
+                tmem_ld16(t_acc + 16 * part, a);
+                tmem_wait_ld();
+                float g[16];
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const float z = __uint_as_float(a[k]) + bpw[colhalf * (D / 2) + 16 * part + k];
+                    g[k] = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z));
+                }
+                uint4* d16 = reinterpret_cast<uint4*>(dst + 16 * part);
+                d16[0] = make_uint4(pack_bf16x2(g[0], g[1]), pack_bf16x2(g[2], g[3]), pack_bf16x2(g[4], g[5]), pack_bf16x2(g[6], g[7]));
+                d16[1] = make_uint4(pack_bf16x2(g[8], g[9]), pack_bf16x2(g[10], g[11]), pack_bf16x2(g[12], g[13]), pack_bf16x2(g[14], g[15]));
+            }
+        }
+        tc_fence_before();
+        __syncthreads();       // accumulator, A tile and halo are free for the next tile
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, L::kTmemCols);
+    }
+}
+
+template <int D>
+cudaError_t launch(const ClaParams& p, cudaStream_t stream)
+{
+    static KernelSetup setup;
+    int sm_count = 0;
+    if (cudaError_t e = setup.prepare(rib_cla_gate_kernel<D>, Layout<D>::kSmemBytes, &sm_count)) return e;
+    const int grid = p.tiles < sm_count ? p.tiles : sm_count;
+    { ProfileScope scope(RIB_KERNEL_CLA_GATE, stream); rib_cla_gate_kernel<D><<<grid, kThreads, Layout<D>::kSmemBytes, stream>>>(p); }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool cla_gate_supported(int H, int W, int D)
+{
+    return (D == 64 || D == 128 || D == 192) && H % kTileH == 0 && W % kTileW == 0;
+}
+
+cudaError_t cla_gate(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw, int B, int H,
+                     int W, int D, __nv_bfloat16* gate, int* status, cudaStream_t stream)
+{
+    ClaParams p{};
+    p.x = x; p.w_dw = w_dw; p.b_dw = b_dw; p.w_pw = w_pw; p.b_pw = b_pw; p.gate = gate; p.status = status;
+    p.B = B; p.H = H; p.W = W;
+    p.tiles_y = H / kTileH; p.tiles_x = W / kTileW;
+    p.tiles = B * p.tiles_y * p.tiles_x;
+    switch (D) {
+        case 64: return launch<64>(p, stream);
+        case 128: return launch<128>(p, stream);
+        case 192: return launch<192>(p, stream);
+        default: return cudaErrorNotSupported;
+    }
+}
+
+}  // namespace rib

@@ -17,6 +17,7 @@ struct Problem {
     const __nv_bfloat16* v;
     const __nv_bfloat16* pq;
     const __nv_bfloat16* pk;
+    const __nv_bfloat16* gate;  // forward: optional CLA gate multiplied into the output (Eq. 9), layout of out
     const __nv_bfloat16* out;   // forward result (input of the backward pass)
     const __nv_bfloat16* dout;
     const float* lse_in;        // backward
@@ -56,6 +57,10 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
 bool sm100_bwd_supported(const Problem& p);
 size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r);
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 3 kernels
+
+bool cla_gate_supported(int H, int W, int D);
+cudaError_t cla_gate(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw, int B, int H,
+                     int W, int D, __nv_bfloat16* gate, int* status, cudaStream_t stream);
 
 bool generator_supported(int window, int L, int dh, int r);
 cudaError_t generator_fwd(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk, int window, int L, int dh, int r,

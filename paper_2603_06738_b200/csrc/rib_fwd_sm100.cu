@@ -68,6 +68,7 @@ constexpr uint32_t kIdescPV = idesc_bf16_f32(kTile, kD, true);
 
 struct FwdParams {
     const __nv_bfloat16* pq;
+    const __nv_bfloat16* gate; // kGated: the CLA gate, layout of out
     __nv_bfloat16* out;
     float* lse;
     int* status;
@@ -104,7 +105,8 @@ __device__ __forceinline__ void patch_origin(const FwdParams& p, const ItemCoord
 // kPartial: H or W is not a multiple of the window (but of 8).  Windows are laid over the map extended to Hp x Wp;
 // an 8x8 patch of the extension holds no tokens: TMA fills it with zeros, the softmax warps give its keys the
 // probability 0, and nothing is stored for its queries.
-template <int R, bool kPartial>
+// kGated: the output is multiplied by the CLA gate (Eq. 9) before it is stored.
+template <int R, bool kPartial, bool kGated>
 __global__ void __launch_bounds__(kThreads, 1)
 rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_pk,
@@ -460,14 +462,20 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (kPartial && (Y0 >= p.H || X0 >= p.W)) continue;        // a patch of the extension: no tokens, nothing to store
             const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
             uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD + half * 16);
+            const uint4* gsrc = reinterpret_cast<const uint4*>(p.gate + tok * kD + half * 16);
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
                 uint32_t w[4];
+                uint4 gv = make_uint4(0u, 0u, 0u, 0u);
+                if (kGated) gv = __ldg(gsrc + i);
+                const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const int e = 8 * i + 2 * k;
-                    w[k] = pack_bf16x2(__uint_as_float(oa[e]) * w_a + __uint_as_float(ob[e]) * w_b,
-                                       __uint_as_float(oa[e + 1]) * w_a + __uint_as_float(ob[e + 1]) * w_b);
+                    float lo = __uint_as_float(oa[e]) * w_a + __uint_as_float(ob[e]) * w_b;
+                    float hi = __uint_as_float(oa[e + 1]) * w_a + __uint_as_float(ob[e + 1]) * w_b;
+                    if (kGated) { lo *= __uint_as_float(gw[k] << 16); hi *= __uint_as_float(gw[k] & 0xffff0000u); }
+                    w[k] = pack_bf16x2(lo, hi);
                 }
                 dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
             }
@@ -488,10 +496,12 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
 bool sm100_fwd_supported(const Problem& p)
 {
-    return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
+    const bool partial = p.Hp != p.H || p.Wp != p.W;
+    return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0 &&
+           !(partial && p.gate);
 }
 
-template <int R, bool kPartial>
+template <int R, bool kPartial, bool kGated>
 cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
@@ -500,15 +510,11 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
         !encode_pos_map(&tm_pk, p.pk, p, pos_tables(p), p.pos_head_stride))
         return cudaErrorInvalidValue;
     constexpr uint32_t kSmemBytes = Layout<R>::kSmemBytes;
-    static int sm_count = 0;
-    if (!sm_count) {
-        cudaError_t e = sm_count_of_current_device(&sm_count);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rib_fwd_sm100_kernel<R, kPartial>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) { sm_count = 0; return e; }
-    }
+    static KernelSetup setup;       // one per instantiation of this launcher, i.e. per kernel
+    int sm_count = 0;
+    if (cudaError_t e = setup.prepare(rib_fwd_sm100_kernel<R, kPartial, kGated>, kSmemBytes, &sm_count)) return e;
     FwdParams fp{};
-    fp.pq = p.pq; fp.out = p.out_w; fp.lse = p.lse_w; fp.status = p.status;
+    fp.pq = p.pq; fp.gate = p.gate; fp.out = p.out_w; fp.lse = p.lse_w; fp.status = p.status;
     fp.H = p.H; fp.W = p.W; fp.heads = p.heads; fp.M = p.M; fp.s = p.s; fp.n = p.n; fp.nWy = p.nWy; fp.nWx = p.nWx;
     fp.Hp = p.Hp; fp.Wp = p.Wp;
     fp.tiles_per_item_pair = p.n / (2 * kTile);
@@ -519,14 +525,15 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     const int grid = fp.items < sm_count ? fp.items : sm_count;
-    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<R, kPartial><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
+    { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<R, kPartial, kGated><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
     return cudaGetLastError();
 }
 
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
 {
-    if (p.Hp != p.H || p.Wp != p.W) return p.r == 32 ? launch_fwd<32, true>(p, stream) : launch_fwd<16, true>(p, stream);
-    return p.r == 32 ? launch_fwd<32, false>(p, stream) : launch_fwd<16, false>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W) return p.r == 32 ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
+    if (p.gate) return p.r == 32 ? launch_fwd<32, false, true>(p, stream) : launch_fwd<16, false, true>(p, stream);
+    return p.r == 32 ? launch_fwd<32, false, false>(p, stream) : launch_fwd<16, false, false>(p, stream);
 }
 
 }  // namespace rib

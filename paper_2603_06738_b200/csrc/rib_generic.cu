@@ -156,8 +156,10 @@ __global__ void __launch_bounds__(kThreads) generic_fwd_kernel(const Problem p)
         if (i >= p.n || !token_exists(p, c, i)) continue;
         const size_t off = token_offset(p, c, i);
         const float inv = 1.f / l[rr];
-        if (lane < p.d) p.out_w[off + lane] = __float2bfloat16_rn(o[rr][0] * inv);
-        if (lane + 32 < p.d) p.out_w[off + lane + 32] = __float2bfloat16_rn(o[rr][1] * inv);
+        const float g0 = p.gate && lane < p.d ? __bfloat162float(p.gate[off + lane]) : 1.f;            // Eq. 9
+        const float g1 = p.gate && lane + 32 < p.d ? __bfloat162float(p.gate[off + lane + 32]) : 1.f;
+        if (lane < p.d) p.out_w[off + lane] = __float2bfloat16_rn(o[rr][0] * inv * g0);
+        if (lane + 32 < p.d) p.out_w[off + lane + 32] = __float2bfloat16_rn(o[rr][1] * inv * g1);
         if (p.lse_w && lane == 0) p.lse_w[token_scalar_offset(p, c, i)] = m[rr] + logf(l[rr]);
     }
 }

@@ -17,7 +17,7 @@ from dataclasses import dataclass
 import numpy as np
 import torch
 
-TENSOR_IDS = {"q": 0, "k": 1, "v": 2, "pq": 3, "pk": 4, "dout": 5}
+TENSOR_IDS = {"q": 0, "k": 1, "v": 2, "pq": 3, "pk": 4, "dout": 5, "x": 6, "gate": 7}
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
 
 
