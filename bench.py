@@ -372,6 +372,18 @@ def main():
         f_ms = timed(lambda: binding.rib_window_attn_fwd_padded(fq, fk, fv, fpq, fpk, fwin, 0), reps=10)
         variants["partial_windows_360x640_w64"] = {"fwd_ms": f_ms, "tokens_per_s": fh * fw / (f_ms * 1e-3),
                                                    "paths": [binding.rib_last_path()]}
+        # Convolutional Local Attention (Eq. 8, Eq. 9) on the benchmark shape: the gate kernel (HBM-bound: one read of the
+        # features and one write of the gate) and the forward pass with the gate multiplied into its output
+        D = wl.heads * wl.d
+        if D in (64, 128, 192) and wl.H % 8 == 0 and wl.W % 16 == 0:
+            cx = torch.randn((wl.B, wl.H, wl.W, D), device=dev).to(torch.bfloat16)
+            cw = [torch.randn(sz, device=dev) * sc for sz, sc in (((D, 3, 3), 0.3), ((D,), 0.2), ((D, D), 0.1), ((D,), 0.2))]
+            gate = binding.rib_cla_gate(cx, *cw)
+            g_ms = timed(lambda: binding.rib_cla_gate(cx, *cw))
+            gf_ms = timed(lambda: binding.rib_window_attn_fwd_gated(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], gate, wl.window, wl.shift))
+            gate_bytes = 2 * cx.numel() * 2
+            variants["cla"] = {"gate_ms": g_ms, "gate_algorithmic_bytes": gate_bytes, "gate_gbs": gate_bytes / (g_ms * 1e-3) / 1e9,
+                               "gate_flops": 2 * cx.numel() * (9 + D), "gated_fwd_ms": gf_ms, "paths": [binding.rib_last_path()]}
         if binding.rib_query_status() != 0:
             raise SystemExit("device status word set during the variant timings")
         del fq, fk, fv

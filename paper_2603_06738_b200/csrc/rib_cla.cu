@@ -19,7 +19,7 @@ using namespace sm100;
 
 constexpr int kTileH = 8, kTileW = 16, kPix = kTileH * kTileW;       // 128 pixels = the M of the MMA
 constexpr int kHaloH = kTileH + 2, kHaloW = kTileW + 2;
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 
 template <int D>
 struct Layout {
@@ -72,22 +72,50 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaPara
         tmem_alloc(base + L::kOffMisc, L::kTmemCols);
         tmem_relinquish();
     }
-    // the point-wise matrix as bf16, row = output channel, 64 input channels per 128-byte line, SWIZZLE_128B
-    for (int idx = threadIdx.x; idx < D * kChunks; idx += kThreads) {
-        const int n = idx / kChunks, c8 = idx - n * kChunks;
-        const float4 lo = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8));
-        const float4 hi = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8 + 4));
-        const uint4 v = make_uint4(pack_bf16x2(lo.x, lo.y), pack_bf16x2(lo.z, lo.w), pack_bf16x2(hi.x, hi.y), pack_bf16x2(hi.z, hi.w));
-        *reinterpret_cast<uint4*>(sm + L::kOffW + (c8 >> 3) * L::kWAtom + n * 128 + (((c8 & 7) ^ (n & 7)) << 4)) = v;
-    }
+    // Weights to shared memory.  Every load of a thread is issued before the first one is used: the prologue costs one
+    // memory latency, not one per item.
     float* taps = reinterpret_cast<float*>(sm + L::kOffTaps);
     float* bdw = reinterpret_cast<float*>(sm + L::kOffBdw);
     float* bpw = reinterpret_cast<float*>(sm + L::kOffBpw);
-    for (int idx = threadIdx.x; idx < 9 * D; idx += kThreads) {
-        const int t = idx / D, c = idx - t * D;
-        taps[idx] = __ldg(p.w_dw + (size_t)c * 9 + t);      // tap-major: a thread's 8 channels of one tap are contiguous
+    {
+        constexpr int kWItems = D * kChunks, kWIters = (kWItems + kThreads - 1) / kThreads;
+        constexpr int kTapIters = (9 * D + kThreads - 1) / kThreads;
+        float4 lo[kWIters], hi[kWIters];
+        float tp[kTapIters];
+#pragma unroll
+        for (int u = 0; u < kWIters; ++u) {
+            const int idx = threadIdx.x + u * kThreads;
+            if (idx < kWItems) {
+                const int n = idx / kChunks, c8 = idx - n * kChunks;
+                lo[u] = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8));
+                hi[u] = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8 + 4));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kTapIters; ++u) {
+            const int idx = threadIdx.x + u * kThreads;
+            if (idx < 9 * D) tp[u] = __ldg(p.w_dw + (size_t)(idx % D) * 9 + idx / D);
+        }
+        const float my_bdw = threadIdx.x < D ? __ldg(p.b_dw + threadIdx.x) : 0.f;
+        const float my_bpw = threadIdx.x < D ? __ldg(p.b_pw + threadIdx.x) : 0.f;
+        // the point-wise matrix as bf16, row = output channel, 64 input channels per 128-byte line, SWIZZLE_128B
+#pragma unroll
+        for (int u = 0; u < kWIters; ++u) {
+            const int idx = threadIdx.x + u * kThreads;
+            if (idx < kWItems) {
+                const int n = idx / kChunks, c8 = idx - n * kChunks;
+                *reinterpret_cast<uint4*>(sm + L::kOffW + (c8 >> 3) * L::kWAtom + n * 128 + (((c8 & 7) ^ (n & 7)) << 4)) =
+                    make_uint4(pack_bf16x2(lo[u].x, lo[u].y), pack_bf16x2(lo[u].z, lo[u].w), pack_bf16x2(hi[u].x, hi[u].y), pack_bf16x2(hi[u].z, hi[u].w));
+            }
+        }
+        // depth-wise taps, tap-major: the 8 channels of a chunk are contiguous for every tap
+#pragma unroll
+        for (int u = 0; u < kTapIters; ++u) {
+            const int idx = threadIdx.x + u * kThreads;
+            if (idx < 9 * D) taps[idx] = tp[u];
+        }
+        if (threadIdx.x < D) { bdw[threadIdx.x] = my_bdw; bpw[threadIdx.x] = my_bpw; }
     }
-    for (int c = threadIdx.x; c < D; c += kThreads) { bdw[c] = __ldg(p.b_dw + c); bpw[c] = __ldg(p.b_pw + c); }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -101,39 +129,64 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaPara
     for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
         const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, b = tile / (p.tiles_x * p.tiles_y);
         const int y0 = ty * kTileH, x0 = tx * kTileW;
-        // (1) halo: zero outside the image
-        for (int idx = threadIdx.x; idx < kHaloH * kHaloW * kChunks; idx += kThreads) {
+        // (1) halo: zero outside the image; the loads of a thread are issued together (their latency, not their number,
+        // is what a tile waits for)
+        constexpr int kHaloItems = kHaloH * kHaloW * kChunks;
+        constexpr int kHaloIters = (kHaloItems + kThreads - 1) / kThreads;
+        uint4 hv[kHaloIters];
+#pragma unroll
+        for (int u = 0; u < kHaloIters; ++u) {
+            const int idx = threadIdx.x + u * kThreads;
             const int hp = idx / kChunks, c8 = idx - hp * kChunks;
             const int Y = y0 + hp / kHaloW - 1, X = x0 + hp % kHaloW - 1;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (Y >= 0 && Y < p.H && X >= 0 && X < p.W)
-                v = __ldg(reinterpret_cast<const uint4*>(p.x + (((size_t)b * p.H + Y) * p.W + X) * D) + c8);
-            *reinterpret_cast<uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16) = v;
+            hv[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (idx < kHaloItems && Y >= 0 && Y < p.H && X >= 0 && X < p.W)
+                hv[u] = __ldg(reinterpret_cast<const uint4*>(p.x + (((size_t)b * p.H + Y) * p.W + X) * D) + c8);
+        }
+#pragma unroll
+        for (int u = 0; u < kHaloIters; ++u) {
+            const int idx = threadIdx.x + u * kThreads;
+            const int hp = idx / kChunks, c8 = idx - hp * kChunks;
+            if (idx < kHaloItems) *reinterpret_cast<uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16) = hv[u];
         }
         __syncthreads();
-        // (2) depth-wise 3 x 3 in fp32, result as the bf16 A operand
-        for (int idx = threadIdx.x; idx < kPix * kChunks; idx += kThreads) {
-            const int pix = idx / kChunks, c8 = idx - pix * kChunks;
-            const int py = pix / kTileW, px = pix - py * kTileW;
-            float acc[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) acc[k] = bdw[8 * c8 + k];
+        // (2) depth-wise 3 x 3 in fp32, result as the bf16 A operand.  A thread owns one chunk of 8 channels and a strip
+        // of 8 pixels of one tile row; its 9 x 8 taps sit in registers for the strip (the shared-memory pipe is what
+        // this phase is bound by: 9 halo reads per pixel remain).
+        if (threadIdx.x < 16 * kChunks) {
+            const int c8 = threadIdx.x % kChunks, strip = threadIdx.x / kChunks;
+            const int py = strip >> 1, px0 = (strip & 1) * 8;
+            float w[9][8];
 #pragma unroll
             for (int t = 0; t < 9; ++t) {
-                const int hp = (py + t / 3) * kHaloW + px + t % 3;
-                const uint4 v = *reinterpret_cast<const uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16);
                 const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
                 const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
-                const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-                const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    acc[2 * k] = fmaf(__uint_as_float(u[k] << 16), w[2 * k], acc[2 * k]);
-                    acc[2 * k + 1] = fmaf(__uint_as_float(u[k] & 0xffff0000u), w[2 * k + 1], acc[2 * k + 1]);
-                }
+                w[t][0] = w0.x; w[t][1] = w0.y; w[t][2] = w0.z; w[t][3] = w0.w;
+                w[t][4] = w1.x; w[t][5] = w1.y; w[t][6] = w1.z; w[t][7] = w1.w;
             }
-            *reinterpret_cast<uint4*>(sm + L::kOffA + (c8 >> 3) * L::kAAtom + pix * 128 + (((c8 & 7) ^ (pix & 7)) << 4)) =
-                make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
+            float bias[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) bias[k] = bdw[8 * c8 + k];
+#pragma unroll 2
+            for (int j = 0; j < 8; ++j) {
+                const int px = px0 + j, pix = py * kTileW + px;
+                float acc[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) acc[k] = bias[k];
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const int hp = (py + t / 3) * kHaloW + px + t % 3;
+                    const uint4 v = *reinterpret_cast<const uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16);
+                    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        acc[2 * k] = fmaf(__uint_as_float(u[k] << 16), w[t][2 * k], acc[2 * k]);
+                        acc[2 * k + 1] = fmaf(__uint_as_float(u[k] & 0xffff0000u), w[t][2 * k + 1], acc[2 * k + 1]);
+                    }
+                }
+                *reinterpret_cast<uint4*>(sm + L::kOffA + (c8 >> 3) * L::kAAtom + pix * 128 + (((c8 & 7) ^ (pix & 7)) << 4)) =
+                    make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
+            }
         }
         fence_proxy_async();
         __syncthreads();
@@ -154,22 +207,22 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaPara
         }
         if (!__all_sync(0xffffffffu, mbar_wait(bar, it & 1, abort_flag, p.status))) { ok = false; break; }
         tc_fence_after();
-        // (4) bias, sigmoid, store: a warp reads its 32 accumulator lanes (pixels) and one half of the channels
+        // (4) bias, sigmoid, store: a warp reads its 32 accumulator lanes (pixels) and one quarter of the channels
         {
-            const int quarter = warp & 3, colhalf = warp >> 2;
+            const int quarter = warp & 3, colpart = warp >> 2;
             const int pix = quarter * 32 + lane;
             const int py = pix / kTileW, px = pix - py * kTileW;
-            const uint32_t t_acc = tmem + ((uint32_t)(quarter * 32) << 16) + colhalf * (D / 2);
-            __nv_bfloat16* dst = p.gate + (((size_t)b * p.H + y0 + py) * p.W + x0 + px) * D + colhalf * (D / 2);
+            const uint32_t t_acc = tmem + ((uint32_t)(quarter * 32) << 16) + colpart * (D / 4);
+            __nv_bfloat16* dst = p.gate + (((size_t)b * p.H + y0 + py) * p.W + x0 + px) * D + colpart * (D / 4);
 #pragma unroll
-            for (int part = 0; part < D / 32; ++part) {
+            for (int part = 0; part < D / 64; ++part) {
                 uint32_t a[16];
                 tmem_ld16(t_acc + 16 * part, a);
                 tmem_wait_ld();
                 float g[16];
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    const float z = __uint_as_float(a[k]) + bpw[colhalf * (D / 2) + 16 * part + k];
+                    const float z = __uint_as_float(a[k]) + bpw[colpart * (D / 4) + 16 * part + k];
                     g[k] = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z));
                 }
                 uint4* d16 = reinterpret_cast<uint4*>(dst + 16 * part);
