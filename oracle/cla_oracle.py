@@ -7,8 +7,8 @@ Eq. 8:  G~ = sigmoid(PWConv(DWConv3x3(F^-1(X))))   on the H x W x D feature map 
 Eq. 9:  O' = O o G,  G = F(G~)                       (element-wise product with the attention output)
 
 F and F^-1 only reshape between the token list and the 2-D map (Eq. 7); with tensors kept as
-[B, H, W, D] they are the identity here.  Readings where the paper is silent (recorded in the
-design notes; parity unpinned against the paper, which prints no example):
+[B, H, W, D] they are the identity here.  Readings where the paper is silent (parity unpinned
+against the paper, which prints no example):
   * DWConv3x3: one 3 x 3 filter per channel, stride 1, zero padding 1, with a bias per channel;
     w_dw[c, dy, dx] multiplies X[y + dy - 1, x + dx - 1, c] (cross-correlation, as deep-learning
     libraries define convolution);

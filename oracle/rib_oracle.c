@@ -16,7 +16,7 @@
  * Attention is restricted to M x M windows (Sec. 2.2); Q_p and K_p depend only on the position
  * inside the window and are the same for every window (Sec. 3.1, last paragraph).
  *
- * Readings where the paper is silent (all listed in the design notes of the repository):
+ * Readings where the paper is silent:
  *   - token order inside a window is row-major, i = y*M + x, and row i of Q_p/K_p belongs to it;
  *   - the cyclic shift s reads window-frame token (wy, wx, y, x) from image pixel
  *     ((wy*M + y + s) mod H, (wx*M + x + s) mod W); the paper itself uses s = 0; wrapped

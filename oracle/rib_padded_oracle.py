@@ -5,10 +5,10 @@ the CUDA path nor with the C oracle of the divisible case (which serves as one o
 tests, the smoke check and the benchmark's CPU leg may import it.
 
 What it computes.  The paper cuts a feature map into M x M windows and, where the map is smaller
-than a multiple of the window, pads it up to one (Sec. 4, the remark on 96 x 96 windows and
-"substantial padding"); it does not say what the padded positions do inside the attention.
-Reading taken here (recorded in the design notes, parity unpinned against the paper for lack of
-a printed example): the map is extended at the bottom and the right to Hp = ceil(H / M) M and
+than a multiple of the window, pads it up to one (Sec. 4, the remark that a 96 x 96 window on
+64 x 64 training patches would need a lot of padding); it does not say what the padded positions
+do inside the attention.  Reading taken here (parity unpinned against the paper for lack of a
+printed example): the map is extended at the bottom and the right to Hp = ceil(H / M) M and
 Wp = ceil(W / M) M, windows (and the cyclic shift, if any) are laid over the extended map, and
 the added positions are not tokens: they are neither attended to nor produce an output.  Inside
 every window the logits of Eq. 6, SoftMax and O = P V (Sec. 2.2, Sec. 3.1) run over the real
