@@ -8,8 +8,9 @@
 // depth-wise filter runs on it in fp32 and its bf16 result becomes the A operand (128 pixels x D, K-major, SWIZZLE_128B),
 // (3) the point-wise matrix -- staged once per CTA as bf16, [out][in], the same layout -- is the B operand of D / 16
 // tcgen05 MMAs (M128, N = D, K16) that accumulate in tensor memory, (4) all warps read the accumulator back, add the
-// bias, apply the sigmoid and store bf16.  The step is small (a few GFLOP, tens of MB) and HBM-bound; the steps of a
-// tile are separated by CTA barriers, nothing is pipelined.
+// bias, apply the sigmoid and store bf16.  The step is small (a few GFLOP, tens of MB) and HBM-bound.  The halo is one
+// TMA box (out-of-range rows and columns arrive as zeros: the padding of the filter); the box of the next tile is
+// requested as soon as the depth-wise phase has read the current one, so it lands during the MMAs and the epilogue.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -33,7 +34,8 @@ struct Layout {
     static constexpr uint32_t kOffBdw = kOffTaps + 9 * D * 4;
     static constexpr uint32_t kOffBpw = kOffBdw + D * 4;
     static constexpr uint32_t kOffBar = kOffBpw + D * 4;
-    static constexpr uint32_t kOffMisc = kOffBar + 8;
+    static constexpr uint32_t kOffMisc = kOffBar + 16;                      // two barriers: MMAs done, halo landed
+    static constexpr uint32_t kHaloBytes = kHaloH * kHaloW * D * 2;
     static constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
     static_assert(kOffA % 1024 == 0 && kWAtom % 1024 == 0 && kAAtom % 1024 == 0, "swizzle atoms need aligned tiles");
     static constexpr uint32_t kTmemCols = D <= 64 ? 64 : D <= 128 ? 128 : 256;
@@ -51,7 +53,7 @@ struct ClaParams {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaParams p)
+__global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_constant__ CUtensorMap tm_x, const ClaParams p)
 {
     using L = Layout<D>;
     constexpr int kChunks = D / 8;                       // 16-byte channel chunks per pixel
@@ -60,13 +62,22 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaPara
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 4);
-    const uint32_t bar = base + L::kOffBar;
+    const uint32_t bar = base + L::kOffBar, bar_halo = bar + 8;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // requests the 10 x 18 halo of a tile: one box of the [B][H][W][D] map, starting one pixel up and to the left
+    auto request_halo = [&](int tile) {
+        const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, b = tile / (p.tiles_x * p.tiles_y);
+        mbar_arrive_expect_tx(bar_halo, L::kHaloBytes);
+        tma_load_4d(base + L::kOffHalo, &tm_x, bar_halo, 0, tx * kTileW - 1, ty * kTileH - 1, b);
+    };
 
     if (threadIdx.x == 0) {
         abort_flag[0] = 0;
         mbar_init(bar, 1);
+        mbar_init(bar_halo, 1);
         fence_barrier_init();
+        prefetch_tensormap(&tm_x);
+        if ((int)blockIdx.x < p.tiles) request_halo(blockIdx.x);
     }
     if (warp == 0) {
         tmem_alloc(base + L::kOffMisc, L::kTmemCols);
@@ -129,27 +140,8 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaPara
     for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
         const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, b = tile / (p.tiles_x * p.tiles_y);
         const int y0 = ty * kTileH, x0 = tx * kTileW;
-        // (1) halo: zero outside the image; the loads of a thread are issued together (their latency, not their number,
-        // is what a tile waits for)
-        constexpr int kHaloItems = kHaloH * kHaloW * kChunks;
-        constexpr int kHaloIters = (kHaloItems + kThreads - 1) / kThreads;
-        uint4 hv[kHaloIters];
-#pragma unroll
-        for (int u = 0; u < kHaloIters; ++u) {
-            const int idx = threadIdx.x + u * kThreads;
-            const int hp = idx / kChunks, c8 = idx - hp * kChunks;
-            const int Y = y0 + hp / kHaloW - 1, X = x0 + hp % kHaloW - 1;
-            hv[u] = make_uint4(0u, 0u, 0u, 0u);
-            if (idx < kHaloItems && Y >= 0 && Y < p.H && X >= 0 && X < p.W)
-                hv[u] = __ldg(reinterpret_cast<const uint4*>(p.x + (((size_t)b * p.H + Y) * p.W + X) * D) + c8);
-        }
-#pragma unroll
-        for (int u = 0; u < kHaloIters; ++u) {
-            const int idx = threadIdx.x + u * kThreads;
-            const int hp = idx / kChunks, c8 = idx - hp * kChunks;
-            if (idx < kHaloItems) *reinterpret_cast<uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16) = hv[u];
-        }
-        __syncthreads();
+        // (1) the halo of this tile (requested during the previous tile, or in the prologue)
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_halo, it & 1, abort_flag, p.status))) { ok = false; break; }
         // (2) depth-wise 3 x 3 in fp32, result as the bf16 A operand.  A thread owns one chunk of 8 channels and a strip
         // of 8 pixels of one tile row; its 9 x 8 taps sit in registers for the strip (the shared-memory pipe is what
         // this phase is bound by: 9 halo reads per pixel remain).
@@ -190,10 +182,11 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const ClaPara
         }
         fence_proxy_async();
         __syncthreads();
-        // (3) point-wise matrix: D / 16 accumulating MMAs
+        // (3) point-wise matrix: D / 16 accumulating MMAs; the halo buffer has been read, the next tile's box may land
         if (warp == 0) {
             tc_fence_after();
             if (elect_one()) {
+                if (tile + (int)gridDim.x < p.tiles) request_halo(tile + gridDim.x);
 #pragma unroll
                 for (int a = 0; a < L::kAtoms; ++a) {
                     const uint64_t da = smem_desc_at(kDesc, base + L::kOffA + a * L::kAAtom);
@@ -248,7 +241,19 @@ cudaError_t launch(const ClaParams& p, cudaStream_t stream)
     int sm_count = 0;
     if (cudaError_t e = setup.prepare(rib_cla_gate_kernel<D>, Layout<D>::kSmemBytes, &sm_count)) return e;
     const int grid = p.tiles < sm_count ? p.tiles : sm_count;
-    { ProfileScope scope(RIB_KERNEL_CLA_GATE, stream); rib_cla_gate_kernel<D><<<grid, kThreads, Layout<D>::kSmemBytes, stream>>>(p); }
+    if (!encode_fn()) return cudaErrorNotSupported;
+    CUtensorMap tm_x;
+    {
+        const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+        const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)D * 2 * p.W, (cuuint64_t)D * 2 * p.W * p.H};
+        const cuuint32_t box[4] = {(cuuint32_t)D, kHaloW, kHaloH, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (encode_fn()(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(p.x), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    { ProfileScope scope(RIB_KERNEL_CLA_GATE, stream); rib_cla_gate_kernel<D><<<grid, kThreads, Layout<D>::kSmemBytes, stream>>>(tm_x, p); }
     return cudaGetLastError();
 }
 
