@@ -558,34 +558,38 @@ __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, 
         pair1 = min(p.pairs, pair0 + pairs_per_group * step);
         table = (size_t)head * (size_t)p.pos_head_stride;
     }
-    float sq[R], sk[R];
+    // blockIdx.z picks 16 of the R RIB columns (grid.z = R / 16); the slice z = 0 also writes dq
+    const int col0 = 16 * blockIdx.z;
+    float sq[16], sk[16];
 #pragma unroll
-    for (int c = 0; c < R; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
+    for (int c = 0; c < 16; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
     int i = 0;
     for (int pair = pair0; pair < pair1; pair += step) {
         size_t tok, scalar;
         decode_pair_token(p, pair, w, i, tok, scalar);
         const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
-        uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
+        if (blockIdx.z == 0) {
+            uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-            float f[8];
+            for (int q4 = 0; q4 < 4; ++q4) {
+                float f[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
-            dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+                for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
+                dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+            }
         }
         const float* srk = p.dkp + (size_t)pair * R * p.n + w;
 #pragma unroll
-        for (int c = 0; c < R; ++c) {
-            sq[c] += src[(size_t)(kD + c) * p.n];
-            sk[c] += srk[(size_t)c * p.n];
+        for (int c = 0; c < 16; ++c) {
+            sq[c] += src[(size_t)(kD + col0 + c) * p.n];
+            sk[c] += srk[(size_t)(col0 + c) * p.n];
         }
     }
     if (pair0 >= pair1) return;
-    float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R);
-    float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R);
+    float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R + col0);
+    float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R + col0);
 #pragma unroll
-    for (int c4 = 0; c4 < R / 4; ++c4) {
+    for (int c4 = 0; c4 < 4; ++c4) {
         atomicAdd(out_q + c4, make_float4(sq[4 * c4] * p.inv_sqrt_r, sq[4 * c4 + 1] * p.inv_sqrt_r, sq[4 * c4 + 2] * p.inv_sqrt_r,
                                           sq[4 * c4 + 3] * p.inv_sqrt_r));
         atomicAdd(out_k + c4, make_float4(sk[4 * c4], sk[4 * c4 + 1], sk[4 * c4 + 2], sk[4 * c4 + 3]));
@@ -672,7 +676,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     const int windows = p.pairs / p.heads;   // pairs of one head
     const unsigned groups = tables == 1 ? (unsigned)((p.pairs + per_group - 1) / per_group)
                                         : (unsigned)(p.heads * ((windows + per_group - 1) / per_group));
-    dim3 grid_fin((unsigned)(p.n / 128), groups);
+    dim3 grid_fin((unsigned)(p.n / 128), groups, (unsigned)(R / 16));
     { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<R><<<grid_fin, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();
 }
