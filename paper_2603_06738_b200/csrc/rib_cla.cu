@@ -10,7 +10,9 @@
 // tcgen05 MMAs (M128, N = D, K16) that accumulate in tensor memory, (4) all warps read the accumulator back, add the
 // bias, apply the sigmoid and store bf16.  The step is small (a few GFLOP, tens of MB) and HBM-bound.  The halo is one
 // TMA box (out-of-range rows and columns arrive as zeros: the padding of the filter); the box of the next tile is
-// requested as soon as the depth-wise phase has read the current one, so it lands during the MMAs and the epilogue.
+// requested as soon as the depth-wise phase has read the current one.  Two groups of warps share the work: the filter
+// warps (which also request the halo and issue the MMAs) run one tile ahead of the four epilogue warps, so the
+// depth-wise phase of a tile overlaps the sigmoid and the stores of the one before.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
 
 namespace rib {
@@ -34,7 +36,7 @@ struct Layout {
     static constexpr uint32_t kOffBdw = kOffTaps + 9 * D * 4;
     static constexpr uint32_t kOffBpw = kOffBdw + D * 4;
     static constexpr uint32_t kOffBar = kOffBpw + D * 4;
-    static constexpr uint32_t kOffMisc = kOffBar + 16;                      // two barriers: MMAs done, halo landed
+    static constexpr uint32_t kOffMisc = kOffBar + 32;                      // barriers: MMAs done, halo landed, A written, accumulator read
     static constexpr uint32_t kHaloBytes = kHaloH * kHaloW * D * 2;
     static constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
     static_assert(kOffA % 1024 == 0 && kWAtom % 1024 == 0 && kAAtom % 1024 == 0, "swizzle atoms need aligned tiles");
@@ -62,7 +64,9 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 4);
-    const uint32_t bar = base + L::kOffBar, bar_halo = bar + 8;
+    const uint32_t bar = base + L::kOffBar, bar_halo = bar + 8, bar_afull = bar + 16, bar_accfree = bar + 24;
+    constexpr int kFilterWarps = 16 * (D / 8) / 32;       // one thread per (8-channel chunk, strip of 8 pixels)
+    constexpr int kEpilogueWarp0 = kThreads / 32 - 4;     // the last four warps, one per 32 accumulator lanes
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // requests the 10 x 18 halo of a tile: one box of the [B][H][W][D] map, starting one pixel up and to the left
     auto request_halo = [&](int tile) {
@@ -75,6 +79,8 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
         abort_flag[0] = 0;
         mbar_init(bar, 1);
         mbar_init(bar_halo, 1);
+        mbar_init(bar_afull, kFilterWarps);
+        mbar_init(bar_accfree, 4);
         fence_barrier_init();
         prefetch_tensormap(&tm_x);
         if ((int)blockIdx.x < p.tiles) request_halo(blockIdx.x);
@@ -137,17 +143,16 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
     constexpr uint32_t kIdesc = idesc_bf16_f32(kPix, D, false);
     bool ok = true;
     uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
-        const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, b = tile / (p.tiles_x * p.tiles_y);
-        const int y0 = ty * kTileH, x0 = tx * kTileW;
-        // (1) the halo of this tile (requested during the previous tile, or in the prologue)
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_halo, it & 1, abort_flag, p.status))) { ok = false; break; }
-        // (2) depth-wise 3 x 3 in fp32, result as the bf16 A operand.  A thread owns one chunk of 8 channels and a strip
-        // of 8 pixels of one tile row; its 9 x 8 taps sit in registers for the strip (the shared-memory pipe is what
-        // this phase is bound by: 9 halo reads per pixel remain).
-        if (threadIdx.x < 16 * kChunks) {
-            const int c8 = threadIdx.x % kChunks, strip = threadIdx.x / kChunks;
-            const int py = strip >> 1, px0 = (strip & 1) * 8;
+    if (warp < kFilterWarps) {
+        // ===================== filter warps: halo -> depth-wise 3 x 3 -> A operand; warp 0 also requests halos and issues MMAs
+        const int c8 = threadIdx.x % kChunks, strip = threadIdx.x / kChunks;
+        const int py = strip >> 1, px0 = (strip & 1) * 8;
+        for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
+            // the halo of this tile has landed, and the MMAs of the previous tile no longer read the A operand
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_halo, it & 1, abort_flag, p.status) &&
+                                             (it == 0 || mbar_wait(bar, (it - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+            // A thread owns one chunk of 8 channels and a strip of 8 pixels of one tile row; its 9 x 8 taps sit in
+            // registers for the strip (the shared-memory pipe is what this phase is bound by: 9 halo reads per pixel).
             float w[9][8];
 #pragma unroll
             for (int t = 0; t < 9; ++t) {
@@ -179,43 +184,57 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
                 *reinterpret_cast<uint4*>(sm + L::kOffA + (c8 >> 3) * L::kAAtom + pix * 128 + (((c8 & 7) ^ (pix & 7)) << 4)) =
                     make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
             }
-        }
-        fence_proxy_async();
-        __syncthreads();
-        // (3) point-wise matrix: D / 16 accumulating MMAs; the halo buffer has been read, the next tile's box may land
-        if (warp == 0) {
-            tc_fence_after();
-            if (elect_one()) {
-                if (tile + (int)gridDim.x < p.tiles) request_halo(tile + gridDim.x);
-#pragma unroll
-                for (int a = 0; a < L::kAtoms; ++a) {
-                    const uint64_t da = smem_desc_at(kDesc, base + L::kOffA + a * L::kAAtom);
-                    const uint64_t db = smem_desc_at(kDesc, base + L::kOffW + a * L::kWAtom);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_ss(tmem, da + 2 * kk, db + 2 * kk, kIdesc, (a | kk) ? 1u : 0u);   // + 32 bytes per K16 step
-                }
-                mma_commit(bar);
-            }
+            fence_proxy_async();
             __syncwarp();
-        }
-        if (!__all_sync(0xffffffffu, mbar_wait(bar, it & 1, abort_flag, p.status))) { ok = false; break; }
-        tc_fence_after();
-        // (4) bias, sigmoid, store: a warp reads its 32 accumulator lanes (pixels) and one quarter of the channels
-        {
-            const int quarter = warp & 3, colpart = warp >> 2;
-            const int pix = quarter * 32 + lane;
-            const int py = pix / kTileW, px = pix - py * kTileW;
-            const uint32_t t_acc = tmem + ((uint32_t)(quarter * 32) << 16) + colpart * (D / 4);
-            __nv_bfloat16* dst = p.gate + (((size_t)b * p.H + y0 + py) * p.W + x0 + px) * D + colpart * (D / 4);
+            if (lane == 0) mbar_arrive(bar_afull);
+            if (warp == 0) {
+                // every filter warp has written its part of A and is done with the halo buffer; the epilogue warps have
+                // read the previous tile's accumulator
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_afull, it & 1, abort_flag, p.status) &&
+                                                 (it == 0 || mbar_wait(bar_accfree, (it - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+                tc_fence_after();
+                if (elect_one()) {
+                    if (tile + (int)gridDim.x < p.tiles) request_halo(tile + gridDim.x);
 #pragma unroll
-            for (int part = 0; part < D / 64; ++part) {
+                    for (int a = 0; a < L::kAtoms; ++a) {
+                        const uint64_t da = smem_desc_at(kDesc, base + L::kOffA + a * L::kAAtom);
+                        const uint64_t db = smem_desc_at(kDesc, base + L::kOffW + a * L::kWAtom);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) mma_ss(tmem, da + 2 * kk, db + 2 * kk, kIdesc, (a | kk) ? 1u : 0u);   // + 32 bytes per K16 step
+                    }
+                    mma_commit(bar);
+                }
+                __syncwarp();
+            }
+        }
+        // the last MMAs must have finished before tensor memory is released
+        if (warp == 0 && ok && it > 0) mbar_wait(bar, (it - 1) & 1, abort_flag, p.status);
+    } else if (warp >= kEpilogueWarp0) {
+        // ===================== epilogue warps: bias, sigmoid, store; a warp reads its 32 accumulator lanes (pixels), all channels
+        const int quarter = warp & 3;
+        const int pix = quarter * 32 + lane;
+        const int py = pix / kTileW, px = pix - py * kTileW;
+        const uint32_t t_acc = tmem + ((uint32_t)(quarter * 32) << 16);
+        for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
+            const int tx = tile % p.tiles_x, ty = (tile / p.tiles_x) % p.tiles_y, b = tile / (p.tiles_x * p.tiles_y);
+            if (!__all_sync(0xffffffffu, mbar_wait(bar, it & 1, abort_flag, p.status))) { ok = false; break; }
+            tc_fence_after();
+            __nv_bfloat16* dst = p.gate + (((size_t)b * p.H + ty * kTileH + py) * p.W + tx * kTileW + px) * D;
+#pragma unroll 1
+            for (int part = 0; part < D / 16; ++part) {
                 uint32_t a[16];
                 tmem_ld16(t_acc + 16 * part, a);
                 tmem_wait_ld();
+                if (part == D / 16 - 1) {
+                    // the accumulator is in registers: the next tile's MMAs may overwrite it
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_accfree);
+                }
                 float g[16];
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    const float z = __uint_as_float(a[k]) + bpw[colpart * (D / 4) + 16 * part + k];
+                    const float z = __uint_as_float(a[k]) + bpw[16 * part + k];
                     g[k] = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z));
                 }
                 uint4* d16 = reinterpret_cast<uint4*>(dst + 16 * part);
@@ -223,8 +242,6 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
                 d16[1] = make_uint4(pack_bf16x2(g[8], g[9]), pack_bf16x2(g[10], g[11]), pack_bf16x2(g[12], g[13]), pack_bf16x2(g[14], g[15]));
             }
         }
-        tc_fence_before();
-        __syncthreads();       // accumulator, A tile and halo are free for the next tile
     }
     tc_fence_before();
     __syncthreads();
