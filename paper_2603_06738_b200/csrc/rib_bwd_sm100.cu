@@ -4,7 +4,8 @@
 // Shapes: d = 32, r = 16 or 32 (template argument R), window side M a multiple of 16, shift a multiple of 8 (as
 // the forward).  The text below describes R = 16.  With R = 32 the RIB rows fill their 64-byte slots, dK~ and dQ~ are
 // 64 columns wide, and tensor memory has no room left for dS^T: dK~ then takes the dS tile in shared memory as a
-// K-major A operand (that tile's barrier counts two readers).
+// K-major A operand (that tile's barrier counts two readers), and the arithmetic warps read the scores as 16-lane
+// fragments (4 key rows x 8 queries per thread), which quarters their reads of the per-query (-lse, -D) values.
 //
 // Work item = one (batch, window, head) pair x one key block J of 128 tokens.  A persistent CTA keeps
 // K~_J = [k, Pk] and V_J in shared memory and dV_J, dK~_J in tensor memory, and walks the query tiles
@@ -341,49 +342,108 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) &&
                                                  mbar_wait(bar(kSFull + h), g & 1, abort_flag, p.status))) { ok = false; break; }
                 tc_fence_after();
-                const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 32 * h + 16 * cg;
-                uint8_t* ds_row = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf + row * 128;
-                uint32_t pp[2][8], dd[2][8];
-#pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    uint32_t s[16], dp[16];
-                    tmem_ld16(t_s + 16 * ch, s);
-                    tmem_ld16(t_dp + 16 * ch, dp);
-                    tmem_wait_ld();
-                    if (ch == 1) {
-                        // S^T, dP^T of this half are in registers: the next unit's scores may overwrite them
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(kSFree + h));
+                if (R == 16) {
+                    // one thread per key row and 32 queries (measured faster than the fragment form below at this rank)
+                    const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 32 * h + 16 * cg;
+                    uint8_t* ds_row = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf + row * 128;
+                    uint32_t pp[2][8], dd[2][8];
+    #pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {
+                        uint32_t s[16], dp[16];
+                        tmem_ld16(t_s + 16 * ch, s);
+                        tmem_ld16(t_dp + 16 * ch, dp);
+                        tmem_wait_ld();
+                        if (ch == 1) {
+                            // S^T, dP^T of this half are in registers: the next unit's scores may overwrite them
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar(kSFree + h));
+                        }
+    #pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 t = ld[8 * ch + i];        // (-lse2, -lse2', -D, -D') of two neighbouring queries
+                            const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2,
+                                                        make_float2(t.x, t.y));
+                            const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                            const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])),
+                                                                     make_float2(t.z, t.w)));
+                            pp[ch][i] = pack_bf16x2(e.x, e.y);
+                            dd[ch][i] = pack_bf16x2(d.x, d.y);
+                        }
                     }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 t = ld[8 * ch + i];        // (-lse2, -lse2', -D, -D') of two neighbouring queries
-                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2,
-                                                    make_float2(t.x, t.y));
-                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-                        const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])),
-                                                                 make_float2(t.z, t.w)));
-                        pp[ch][i] = pack_bf16x2(e.x, e.y);
-                        dd[ch][i] = pack_bf16x2(d.x, d.y);
+                    // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
+                    // still reads this dS buffer
+                    if (!__all_sync(0xffffffffu, (g == 0 || mbar_wait(bar(kPFree + h), (g - 1) & 1, abort_flag, p.status)) &&
+                                                     (g < 2 || mbar_wait(bar(kDSFree + (g & 1)), ((g >> 1) - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+                    tc_fence_after();
+    #pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {
+                        tmem_st8(t_p + 8 * ch, pp[ch]);
+                        if (R == 16) tmem_st8(t_ds + 8 * ch, dd[ch]);
+    #pragma unroll
+                        for (int q2 = 0; q2 < 2; ++q2) {
+                            const int chunk = cg * 4 + ch * 2 + q2;
+                            *reinterpret_cast<uint4*>(ds_row + ((chunk ^ sw) << 4)) =
+                                make_uint4(dd[ch][4 * q2], dd[ch][4 * q2 + 1], dd[ch][4 * q2 + 2], dd[ch][4 * q2 + 3]);
+                        }
+                    }
+                } else {
+                    // The warp's 32 key rows x 32 queries are read as two 16-lane fragments: a thread then holds 4 key rows of
+                    // only 8 queries (4 neighbouring pairs), so the per-query (-lse2, -lse2', -D, -D') cost it 4 shared-memory
+                    // reads per tile instead of 16 -- those reads, not the arithmetic, load the shared-memory pipe.
+                    const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 32 * h + 16 * cg + (lane & 3);
+                    float4 t4[4];
+    #pragma unroll
+                    for (int gq = 0; gq < 4; ++gq) t4[gq] = ld[4 * gq];       // queries 8 gq + 2 (lane % 4), + 1 of this warp's 32
+                    uint8_t* ds_tile = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf;
+                    uint32_t pp[2][8], dd[2][8];
+    #pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {                          // lanes 16 ch .. 16 ch + 15 of the warp's quarter
+                        uint32_t s[16], dp[16];
+                        tmem_ld_16x256b_x4(t_s + ((uint32_t)(16 * ch) << 16), s);
+                        tmem_ld_16x256b_x4(t_dp + ((uint32_t)(16 * ch) << 16), dp);
+                        tmem_wait_ld();
+                        if (ch == 1) {
+                            // S^T, dP^T of this half are in registers: the next unit's scores may overwrite them
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar(kSFree + h));
+                        }
+    #pragma unroll
+                        for (int gq = 0; gq < 4; ++gq)
+    #pragma unroll
+                            for (int rr = 0; rr < 2; ++rr) {                  // key rows lane / 4 and lane / 4 + 8 of the fragment
+                                const int i = 4 * gq + 2 * rr;
+                                const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[i]), __uint_as_float(s[i + 1])), scale2,
+                                                            make_float2(t4[gq].x, t4[gq].y));
+                                const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                                const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])),
+                                                                         make_float2(t4[gq].z, t4[gq].w)));
+                                pp[ch][2 * gq + rr] = pack_bf16x2(e.x, e.y);
+                                dd[ch][2 * gq + rr] = pack_bf16x2(d.x, d.y);
+                            }
+                    }
+                    // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
+                    // still reads this dS buffer
+                    if (!__all_sync(0xffffffffu, (g == 0 || mbar_wait(bar(kPFree + h), (g - 1) & 1, abort_flag, p.status)) &&
+                                                     (g < 2 || mbar_wait(bar(kDSFree + (g & 1)), ((g >> 1) - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
+                    tc_fence_after();
+    #pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {
+                        tmem_st_16x128b_x4(t_p + ((uint32_t)(16 * ch) << 16), pp[ch]);
+                        if (R == 16) tmem_st_16x128b_x4(t_ds + ((uint32_t)(16 * ch) << 16), dd[ch]);
+                        // dS tile: row = key, 128-byte line = the unit's 64 queries, 16-byte chunks swizzled by the row
+    #pragma unroll
+                        for (int rr = 0; rr < 2; ++rr) {
+                            const int krow = quarter * 32 + 16 * ch + 8 * rr + (lane >> 2);
+                            uint8_t* line = ds_tile + krow * 128 + 4 * (lane & 3);
+    #pragma unroll
+                            for (int gq = 0; gq < 4; ++gq)
+                                *reinterpret_cast<uint32_t*>(line + (((cg * 4 + gq) ^ (krow & 7)) << 4)) = dd[ch][2 * gq + rr];
+                        }
                     }
                 }
-                // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
-                // still reads this dS buffer
-                if (!__all_sync(0xffffffffu, (g == 0 || mbar_wait(bar(kPFree + h), (g - 1) & 1, abort_flag, p.status)) &&
-                                                 (g < 2 || mbar_wait(bar(kDSFree + (g & 1)), ((g >> 1) - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    tmem_st8(t_p + 8 * ch, pp[ch]);
-                    if (R == 16) tmem_st8(t_ds + 8 * ch, dd[ch]);
-#pragma unroll
-                    for (int q2 = 0; q2 < 2; ++q2) {
-                        const int chunk = cg * 4 + ch * 2 + q2;
-                        *reinterpret_cast<uint4*>(ds_row + ((chunk ^ sw) << 4)) =
-                            make_uint4(dd[ch][4 * q2], dd[ch][4 * q2 + 1], dd[ch][4 * q2 + 2], dd[ch][4 * q2 + 3]);
-                    }
-                }
+                if (!ok) break;
                 tmem_wait_st();
                 tc_fence_before();
                 fence_proxy_async();
