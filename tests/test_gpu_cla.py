@@ -52,7 +52,8 @@ def test_gate_border_pixels_see_zero_padding():
 @pytest.mark.parametrize("path", ["auto", "generic"])
 @pytest.mark.parametrize("wl", [Workload("gated_w16_s8", 2, 32, 48, 2, 32, 16, 16, 8, seed=210),
                                 Workload("gated_w32_rank32", 1, 64, 32, 6, 32, 32, 32, 16, seed=211),
-                                Workload("gated_w8_generic", 1, 16, 24, 3, 16, 8, 8, 3, seed=212)], ids=lambda w: w.name)
+                                Workload("gated_w8_generic", 1, 16, 24, 3, 16, 8, 8, 3, seed=212),
+                                Workload("gated_w16_headwise", 1, 32, 32, 3, 32, 16, 16, 0, seed=215, headwise=True)], ids=lambda w: w.name)
 def test_gated_forward_is_attention_times_the_gate(wl, path):
     cpu, gpu = make(wl, with_dout=False)
     D = wl.heads * wl.d
