@@ -338,55 +338,60 @@ def main():
     # ------------------------------------------------ the path's variants beyond the benchmark shape (rank 0, device-timed)
     variants = None
     if rank == 0 and not args.no_variants:
-        variants = {"timing": "CUDA events, one buffer set per variant reused every iteration (inputs may stay in L2)"}
+        # extras: a failure here must not cost the benchmark line
+        try:
+            variants = {"timing": "CUDA events, one buffer set per variant reused every iteration (inputs may stay in L2)"}
 
-        def timed(fn, reps=20):
-            for _ in range(3):
-                fn()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(reps):
-                fn()
-            b.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) / reps
+            def timed(fn, reps=20):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(reps):
+                    fn()
+                b.record()
+                torch.cuda.synchronize()
+                return a.elapsed_time(b) / reps
 
-        s0 = sets[0]
-        for name, r_v, headwise in (("rank32", 32, False), ("headwise", wl.r, True)):
-            shape = (wl.heads, wl.n, r_v) if headwise else (wl.n, r_v)
-            pq_v, pk_v = ((0.5 * torch.randn(shape, device=dev)).to(torch.bfloat16) for _ in range(2))
-            fwd_fn = binding.rib_window_attn_fwd_headwise if headwise else binding.rib_window_attn_fwd
-            bwd_fn = binding.rib_window_attn_bwd_headwise if headwise else binding.rib_window_attn_bwd
-            out_v, lse_v = fwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, wl.window, wl.shift)
-            f_ms = timed(lambda: fwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, wl.window, wl.shift))
-            b_ms = timed(lambda: bwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, out_v, lse_v, s0["dout"], wl.window, wl.shift))
-            ff = wl.pairs * 2 * wl.n * wl.n * (2 * wl.d + r_v)
-            bf = wl.pairs * 2 * wl.n * wl.n * (5 * wl.d + 3 * r_v)
-            variants[name] = {"r": r_v, "fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_tflops": ff / (f_ms * 1e-3) / 1e12,
-                              "bwd_tflops": bf / (b_ms * 1e-3) / 1e12, "paths": [binding.rib_last_path()]}
-        # the paper's inference frame: 360 x 640 tokens, not a multiple of the 64 x 64 window (forward only)
-        fh, fw, fwin = 360, 640, 64
-        fq, fk, fv = (torch.randn((1, fh, fw, wl.heads, wl.d), device=dev).to(torch.bfloat16) for _ in range(3))
-        fpq, fpk = ((0.5 * torch.randn((fwin * fwin, wl.r), device=dev)).to(torch.bfloat16) for _ in range(2))
-        f_ms = timed(lambda: binding.rib_window_attn_fwd_padded(fq, fk, fv, fpq, fpk, fwin, 0), reps=10)
-        variants["partial_windows_360x640_w64"] = {"fwd_ms": f_ms, "tokens_per_s": fh * fw / (f_ms * 1e-3),
-                                                   "paths": [binding.rib_last_path()]}
-        # Convolutional Local Attention (Eq. 8, Eq. 9) on the benchmark shape: the gate kernel (HBM-bound: one read of the
-        # features and one write of the gate) and the forward pass with the gate multiplied into its output
-        D = wl.heads * wl.d
-        if D in (64, 128, 192) and wl.H % 8 == 0 and wl.W % 16 == 0:
-            cx = torch.randn((wl.B, wl.H, wl.W, D), device=dev).to(torch.bfloat16)
-            cw = [torch.randn(sz, device=dev) * sc for sz, sc in (((D, 3, 3), 0.3), ((D,), 0.2), ((D, D), 0.1), ((D,), 0.2))]
-            gate = binding.rib_cla_gate(cx, *cw)
-            g_ms = timed(lambda: binding.rib_cla_gate(cx, *cw))
-            gf_ms = timed(lambda: binding.rib_window_attn_fwd_gated(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], gate, wl.window, wl.shift))
-            gate_bytes = 2 * cx.numel() * 2
-            variants["cla"] = {"gate_ms": g_ms, "gate_algorithmic_bytes": gate_bytes, "gate_gbs": gate_bytes / (g_ms * 1e-3) / 1e9,
-                               "gate_flops": 2 * cx.numel() * (9 + D), "gated_fwd_ms": gf_ms, "paths": [binding.rib_last_path()]}
-        if binding.rib_query_status() != 0:
-            raise SystemExit("device status word set during the variant timings")
-        del fq, fk, fv
+            s0 = sets[0]
+            for name, r_v, headwise in (("rank32", 32, False), ("headwise", wl.r, True)):
+                shape = (wl.heads, wl.n, r_v) if headwise else (wl.n, r_v)
+                pq_v, pk_v = ((0.5 * torch.randn(shape, device=dev)).to(torch.bfloat16) for _ in range(2))
+                fwd_fn = binding.rib_window_attn_fwd_headwise if headwise else binding.rib_window_attn_fwd
+                bwd_fn = binding.rib_window_attn_bwd_headwise if headwise else binding.rib_window_attn_bwd
+                out_v, lse_v = fwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, wl.window, wl.shift)
+                f_ms = timed(lambda: fwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, wl.window, wl.shift))
+                b_ms = timed(lambda: bwd_fn(s0["q"], s0["k"], s0["v"], pq_v, pk_v, out_v, lse_v, s0["dout"], wl.window, wl.shift))
+                ff = wl.pairs * 2 * wl.n * wl.n * (2 * wl.d + r_v)
+                bf = wl.pairs * 2 * wl.n * wl.n * (5 * wl.d + 3 * r_v)
+                variants[name] = {"r": r_v, "fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_tflops": ff / (f_ms * 1e-3) / 1e12,
+                                  "bwd_tflops": bf / (b_ms * 1e-3) / 1e12, "paths": [binding.rib_last_path()]}
+            # the paper's inference frame: 360 x 640 tokens, not a multiple of the 64 x 64 window (forward only)
+            fh, fw, fwin = 360, 640, 64
+            fq, fk, fv = (torch.randn((1, fh, fw, wl.heads, wl.d), device=dev).to(torch.bfloat16) for _ in range(3))
+            fpq, fpk = ((0.5 * torch.randn((fwin * fwin, wl.r), device=dev)).to(torch.bfloat16) for _ in range(2))
+            f_ms = timed(lambda: binding.rib_window_attn_fwd_padded(fq, fk, fv, fpq, fpk, fwin, 0), reps=10)
+            variants["partial_windows_360x640_w64"] = {"fwd_ms": f_ms, "tokens_per_s": fh * fw / (f_ms * 1e-3),
+                                                       "paths": [binding.rib_last_path()]}
+            # Convolutional Local Attention (Eq. 8, Eq. 9) on the benchmark shape: the gate kernel (HBM-bound: one read of the
+            # features and one write of the gate) and the forward pass with the gate multiplied into its output
+            D = wl.heads * wl.d
+            if D in (64, 128, 192) and wl.H % 8 == 0 and wl.W % 16 == 0:
+                cx = torch.randn((wl.B, wl.H, wl.W, D), device=dev).to(torch.bfloat16)
+                cw = [torch.randn(sz, device=dev) * sc for sz, sc in (((D, 3, 3), 0.3), ((D,), 0.2), ((D, D), 0.1), ((D,), 0.2))]
+                gate = binding.rib_cla_gate(cx, *cw)
+                g_ms = timed(lambda: binding.rib_cla_gate(cx, *cw))
+                gf_ms = timed(lambda: binding.rib_window_attn_fwd_gated(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], gate, wl.window, wl.shift))
+                gate_bytes = 2 * cx.numel() * 2
+                variants["cla"] = {"gate_ms": g_ms, "gate_algorithmic_bytes": gate_bytes, "gate_gbs": gate_bytes / (g_ms * 1e-3) / 1e9,
+                                   "gate_flops": 2 * cx.numel() * (9 + D), "gated_fwd_ms": gf_ms, "paths": [binding.rib_last_path()]}
+            if binding.rib_query_status() != 0:
+                raise SystemExit("device status word set during the variant timings")
+            del fq, fk, fv
+
+        except Exception as exc:   # noqa: BLE001
+            variants = {"error": f"{type(exc).__name__}: {exc}"}
 
     # ------------------------------------------------ reduce over ranks (max time), compose the line
     total_ms, fwd_med, bwd_med, e2e_ms_max = multi.max_over_ranks(
