@@ -5,7 +5,8 @@
 // shared memory, so the concatenated rows of Eq. 5 exist only on chip.
 //
 // These kernels serve shapes outside the tcgen05 fast path (odd window sizes, shifts that are
-// not a multiple of 8, d != 32, r != 16) and the backward pass.  fp32 arithmetic throughout.
+// not a multiple of 8, d != 32, r other than 16 or 32, maps whose sides are not multiples of 8) and
+// are a second implementation of the addressing for the tests.  fp32 arithmetic throughout.
 #include "rib_common.cuh"
 
 namespace rib {
