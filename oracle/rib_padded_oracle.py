@@ -75,3 +75,52 @@ def fwd(q, k, v, pq, pk, window, shift=0):
                     out[b, ys, xs, h] = (e / den) @ vw
                     lse[b, h, ys, xs] = (mx + np.log(den))[:, 0]
     return out, lse
+
+
+def bwd(q, k, v, pq, pk, dout, window, shift=0):
+    """dq, dk, dv [B,H,W,heads,d] and dpq, dpk (shape of pq) in float64: the chain rule of `fwd`.
+
+    Per window and head, over the real tokens only (P, S as in `fwd`):
+        dV = P^T dO;  dP = dO V^T;  dS = P o (dP - rowsum(dP o P));
+        dq = dS k / sqrt(d);  dk = dS^T q / sqrt(d);
+        dPq[rows] += dS Pk[rows] / sqrt(r);  dPk[rows] += dS^T Pq[rows] / sqrt(r),
+    the last two summed over batch items and windows (and over heads when the table is shared).
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    dout = np.asarray(dout, dtype=np.float64)
+    pq = np.asarray(pq, dtype=np.float64)
+    pk = np.asarray(pk, dtype=np.float64)
+    B, H, W, heads, d = q.shape
+    r = pq.shape[-1]
+    if not 0 <= shift < window:
+        raise ValueError("shift must lie in [0, window)")
+    Hp, Wp = padded_size(H, W, window)
+    dq, dk, dv = (np.full(q.shape, np.nan) for _ in range(3))
+    dpq, dpk = np.zeros(pq.shape), np.zeros(pk.shape)
+    for wy in range(Hp // window):
+        for wx in range(Wp // window):
+            rows, ys, xs = window_tokens(H, W, window, shift, wy, wx)
+            if rows.size == 0:
+                continue
+            for h in range(heads):
+                pqh = pq[h] if pq.ndim == 3 else pq
+                pkh = pk[h] if pk.ndim == 3 else pk
+                gq = dpq[h] if pq.ndim == 3 else dpq
+                gk = dpk[h] if pk.ndim == 3 else dpk
+                bias = pqh[rows] @ pkh[rows].T / np.sqrt(r) if r else 0.0
+                for b in range(B):
+                    qw, kw, vw, go = q[b, ys, xs, h], k[b, ys, xs, h], v[b, ys, xs, h], dout[b, ys, xs, h]
+                    s = qw @ kw.T / np.sqrt(d) + bias
+                    e = np.exp(s - s.max(axis=1, keepdims=True))
+                    p = e / e.sum(axis=1, keepdims=True)
+                    dp = go @ vw.T
+                    ds = p * (dp - (dp * p).sum(axis=1, keepdims=True))
+                    dv[b, ys, xs, h] = p.T @ go
+                    dq[b, ys, xs, h] = ds @ kw / np.sqrt(d)
+                    dk[b, ys, xs, h] = ds.T @ qw / np.sqrt(d)
+                    if r:
+                        np.add.at(gq, rows, ds @ pkh[rows] / np.sqrt(r))
+                        np.add.at(gk, rows, ds.T @ pqh[rows] / np.sqrt(r))
+    return dq, dk, dv, dpq, dpk

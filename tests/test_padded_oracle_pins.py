@@ -111,3 +111,66 @@ def test_planted_mistakes_are_caught():
     rows_good = pad.window_tokens(6, 6, 4, 1, 1, 1)
     Y_wrong = (1 * 4 + np.arange(4) + 1) % 6
     assert not np.array_equal(np.unique(rows_good[1]), np.unique(Y_wrong[Y_wrong < 6]))
+
+
+# ------------------------------------------------------------------------------------------ backward
+@pytest.mark.parametrize("shift", [0, 3])
+@pytest.mark.parametrize("headwise", [False, True])
+def test_backward_on_divisible_maps_reproduces_the_c_oracle(shift, headwise):
+    q, k, v, pq, pk = rand_case(11, 2, 8, 12, 2, 8, 4, 4, headwise)
+    dout = np.random.default_rng(12).standard_normal(q.shape)
+    got = pad.bwd(q, k, v, pq, pk, dout, 4, shift)
+    ref = orc.bwd(q, k, v, pq, pk, dout, 4, shift)
+    for a, b in zip(got, ref):
+        np.testing.assert_allclose(a, b, rtol=0, atol=1e-11)
+
+
+@pytest.mark.parametrize("H,W,window,shift,headwise", [(6, 10, 4, 0, False), (7, 5, 4, 1, True), (3, 3, 4, 0, False)])
+def test_backward_by_central_differences_on_non_divisible_maps(H, W, window, shift, headwise):
+    q, k, v, pq, pk = rand_case(13, 1, H, W, 2, 4, 4, window, headwise)
+    dout = np.random.default_rng(14).standard_normal(q.shape)
+    grads = pad.bwd(q, k, v, pq, pk, dout, window, shift)
+    assert all(np.isfinite(g).all() for g in grads)
+
+    def loss(args):
+        return float((pad.fwd(*args, window, shift)[0] * dout).sum())
+
+    args = [q, k, v, pq, pk]
+    rng = np.random.default_rng(15)
+    eps = 1e-6
+    for which, grad in enumerate(grads):
+        x = args[which]
+        for _ in range(6):
+            idx = tuple(int(rng.integers(n)) for n in x.shape)
+            old = x[idx]
+            x[idx] = old + eps; up = loss(args)
+            x[idx] = old - eps; down = loss(args)
+            x[idx] = old
+            np.testing.assert_allclose(grad[idx], (up - down) / (2 * eps), rtol=2e-6, atol=2e-8)
+
+
+def test_backward_against_autograd_of_masked_library_attention():
+    H, W, window, shift = 6, 10, 4, 1
+    q, k, v, pq, pk = rand_case(16, 2, H, W, 2, 8, 4, window)
+    dout = np.random.default_rng(17).standard_normal(q.shape)
+    tq, tk, tv, tpq, tpk = (torch.tensor(x, requires_grad=True) for x in (q, k, v, pq, pk))
+    B, _, _, heads, d = q.shape
+    M, n, r = window, window * window, pq.shape[-1]
+    Hp, Wp = pad.padded_size(H, W, M)
+
+    def windows(x):
+        ext = torch.zeros((B, Hp, Wp) + tuple(x.shape[3:]), dtype=x.dtype)
+        ext[:, :H, :W] = x
+        ext = torch.roll(ext, (-shift, -shift), (1, 2))
+        c = x.shape[-1]
+        return ext.reshape(B, Hp // M, M, Wp // M, M, heads, c).permute(0, 1, 3, 5, 2, 4, 6).reshape(B, Hp // M, Wp // M, heads, n, c)
+
+    valid = windows(torch.ones((B, H, W, heads, 1), dtype=torch.float64))[..., 0] > 0.5
+    mask = torch.where(valid[..., None, :], 0.0, -float("inf")) + tpq @ tpk.T / np.sqrt(r)
+    o = torch.nn.functional.scaled_dot_product_attention(windows(tq), windows(tk), windows(tv), attn_mask=mask)
+    ext = o.reshape(B, Hp // M, Wp // M, heads, M, M, d).permute(0, 1, 4, 2, 5, 3, 6).reshape(B, Hp, Wp, heads, d)
+    out = torch.roll(ext, (shift, shift), (1, 2))[:, :H, :W]
+    (out * torch.tensor(dout)).sum().backward()
+    got = pad.bwd(q, k, v, pq, pk, dout, window, shift)
+    for g, t in zip(got, (tq, tk, tv, tpq, tpk)):
+        np.testing.assert_allclose(g, t.grad.numpy(), rtol=0, atol=1e-10)
