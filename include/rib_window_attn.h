@@ -125,12 +125,28 @@ size_t rib_window_attn_bwd_headwise_workspace(long long pos_head_stride, int B, 
  * and lse have the real sizes H and W: nothing is padded in memory.  With H and W multiples of the window this is
  * rib_window_attn_fwd_headwise; other arguments, layouts and error codes as there.  H and W multiples of 8 (and
  * the shape conditions above) take the tcgen05 kernel, where a patch of the extension costs a zero-filled TMA box;
- * any other H, W take the any-shape kernel.  Forward only: there is no backward entry point for such maps.
+ * any other H, W take the any-shape kernel.
  */
 int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
                                long long pos_head_stride,
                                int B, int H, int W, int heads, int d, int r, int window, int shift,
                                void* out, float* lse, void* stream);
+
+/*
+ * Backward pass of rib_window_attn_fwd_padded (same reading: positions of the extended map beyond H x W are not
+ * tokens, so they receive and contribute no gradient).  Arguments, results and workspace rules as
+ * rib_window_attn_bwd_headwise; the workspace size comes from rib_window_attn_bwd_padded_workspace.  Maps whose sides
+ * are multiples of the window are passed on to rib_window_attn_bwd_headwise; all others run on the any-shape CUDA
+ * kernels (the tcgen05 backward kernels take whole windows only), which is correct but slow.
+ */
+int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               const void* out, const float* lse, const void* dout,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                               void* workspace, size_t workspace_bytes, void* stream);
+size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, int H, int W, int heads, int d, int r,
+                                            int window);
 
 /*
  * Convolutional Local Attention (paper: Sec. 3.2, Eq. 7, Eq. 8, Eq. 9): the step right after the attention.

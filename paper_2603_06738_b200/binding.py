@@ -25,6 +25,7 @@ EXPORTS = (
     "rib_generate_features", "rib_generate_features_bwd",
     "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
     "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
+    "rib_window_attn_bwd_padded", "rib_window_attn_bwd_padded_workspace",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
@@ -61,6 +62,10 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_fwd_headwise.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_fwd_padded.restype = ci
         lib.rib_window_attn_fwd_padded.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
+        lib.rib_window_attn_bwd_padded.restype = ci
+        lib.rib_window_attn_bwd_padded.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_attn_bwd_padded_workspace.restype = ctypes.c_size_t
+        lib.rib_window_attn_bwd_padded_workspace.argtypes = [ll] + [ci] * 7
         lib.rib_cla_gate.restype = ci
         lib.rib_cla_gate.argtypes = [vp] * 5 + [ci] * 4 + [vp, vp]
         lib.rib_window_attn_fwd_gated.restype = ci
@@ -256,6 +261,39 @@ def rib_window_attn_fwd_padded(q, k, v, pq, pk, window, shift=0, stream=None, wa
     if rc != RIB_OK:
         raise RibError(rc)
     return out, lse
+
+
+def rib_window_attn_bwd_padded(q, k, v, pq, pk, out, lse, dout, window, shift=0, workspace=None, stream=None):
+    """Backward pass on a map whose sides need not be multiples of the window; pq, pk [n, r] or [heads, n, r].
+    Returns (dq, dk, dv bf16, dpq, dpk fp32 of the shape of pq)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    for name, t in (("k", k), ("v", v), ("out", out), ("dout", dout)):
+        _check_image(name, t, q.shape)
+    n = window * window
+    headwise = pq.dim() == 3
+    if headwise:
+        _check_pos_headwise("pq", pq, heads, n)
+        _check_pos_headwise("pk", pk, heads, n)
+    else:
+        _check_pos("pq", pq, n)
+        _check_pos("pk", pk, n)
+    r = pq.shape[-1]
+    stride = n * r if headwise else 0
+    if lse.dtype != torch.float32 or tuple(lse.shape) != (B, heads, H, W) or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous fp32 tensor [B,heads,H,W]")
+    need = int(library().rib_window_attn_bwd_padded_workspace(stride, B, H, W, heads, d, r, window))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dpq = torch.empty(tuple(pq.shape), dtype=torch.float32, device=q.device)
+    dpk = torch.empty(tuple(pk.shape), dtype=torch.float32, device=q.device)
+    rc = library().rib_window_attn_bwd_padded(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), stride, _ptr(out), _ptr(lse),
+                                              _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq), _ptr(dk), _ptr(dv),
+                                              _ptr(dpq), _ptr(dpk), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return dq, dk, dv, dpq, dpk
 
 
 def rib_cla_gate(x, w_dw, b_dw, w_pw, b_pw, stream=None):

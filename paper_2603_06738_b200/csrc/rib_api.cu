@@ -290,14 +290,35 @@ int rib_window_attn_bwd_headwise(const void* q, const void* k, const void* v, co
                                  void* dq, void* dk, void* dv, float* dpq, float* dpk,
                                  void* workspace, size_t workspace_bytes, void* stream)
 {
+    if (H > 0 && W > 0 && window > 0 && (H % window || W % window)) return RIB_ERR_SHAPE;
+    return rib_window_attn_bwd_padded(q, k, v, pq, pk, pos_head_stride, out, lse, dout, B, H, W, heads, d, r, window, shift, dq, dk,
+                                      dv, dpq, dpk, workspace, workspace_bytes, stream);
+}
+
+size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, int H, int W, int heads, int d, int r, int window)
+{
+    if (H > 0 && W > 0 && window > 0 && H % window == 0 && W % window == 0)
+        return rib_window_attn_bwd_headwise_workspace(pos_head_stride, B, H, W, heads, d, r, window);
+    if (check_shape(B, H, W, heads, d, r, window, 0, true) != RIB_OK) return 0;
+    if (check_pos_stride(pos_head_stride, window, r) != RIB_OK) return 0;
+    return rowdot_bytes(B, H, W, heads);      // such maps take the any-shape kernels
+}
+
+int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               const void* out, const float* lse, const void* dout,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                               void* workspace, size_t workspace_bytes, void* stream)
+{
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return RIB_ERR_NULL;
     if (r > 0 && (!pq || !pk || !dpq || !dpk)) return RIB_ERR_NULL;
-    if (int rc = check_shape(B, H, W, heads, d, r, window, shift)) return rc;
+    if (int rc = check_shape(B, H, W, heads, d, r, window, shift, true)) return rc;
     if (int rc = check_pos_stride(pos_head_stride, window, r)) return rc;
     const void* ptrs[] = {q, k, v, pq, pk, out, lse, dout, dq, dk, dv, dpq, dpk};
     for (const void* ptr : ptrs)
         if (!aligned16(ptr)) return RIB_ERR_ALIGN;
-    const size_t need = rib_window_attn_bwd_headwise_workspace(pos_head_stride, B, H, W, heads, d, r, window);
+    const size_t need = rib_window_attn_bwd_padded_workspace(pos_head_stride, B, H, W, heads, d, r, window);
     if (!workspace || workspace_bytes < need) return RIB_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return RIB_ERR_ALIGN;
     rib::Problem p{};
@@ -321,7 +342,8 @@ int rib_window_attn_bwd_headwise(const void* q, const void* k, const void* v, co
     p.pos_head_stride = pos_head_stride;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_bwd_supported(p);
+    const bool partial = p.Hp != p.H || p.Wp != p.W;      // the tcgen05 backward kernels take whole windows only
+    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && !partial && rib::sm100_bwd_supported(p);
     const cudaError_t e = fast ? rib::sm100_bwd(p, st) : rib::generic_bwd(p, st);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;

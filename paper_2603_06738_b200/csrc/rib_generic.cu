@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dq_kernel(const Problem 
     float lse[kRowsPerWarp], Di[kRowsPerWarp], acc[kRowsPerWarp][kMaxCols];
     for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int i = row0 + warp * kRowsPerWarp + rr;
-        const bool ok = i < p.n;
+        const bool ok = i < p.n && token_exists(p, c, i);
         lse[rr] = ok ? p.lse_in[token_scalar_offset(p, c, i)] : 0.f;
         Di[rr] = ok ? p.rowdot[token_scalar_offset(p, c, i)] : 0.f;
         for (int t = 0; t < kMaxCols; ++t) acc[rr][t] = 0.f;
@@ -228,8 +228,9 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dq_kernel(const Problem 
                 g0 = fmaf(a, Vt[lane * ldv + col], g0);
                 g1 = fmaf(a, Vt[(lane + 32) * ldv + col], g1);
             }
-            const float p0 = j0 + lane < p.n ? expf(s0 - lse[rr]) : 0.f;
-            const float p1 = j0 + lane + 32 < p.n ? expf(s1 - lse[rr]) : 0.f;
+            // keys beyond the window or, on an extended map, beyond the image have probability 0
+            const float p0 = j0 + lane < p.n && token_exists(p, c, j0 + lane) ? expf(s0 - lse[rr]) : 0.f;
+            const float p1 = j0 + lane + 32 < p.n && token_exists(p, c, j0 + lane + 32) ? expf(s1 - lse[rr]) : 0.f;
             float* srow = Ss + (warp * kRowsPerWarp + rr) * kTile;
             srow[lane] = p0 * (g0 - Di[rr]);
             srow[lane + 32] = p1 * (g1 - Di[rr]);
@@ -247,7 +248,7 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dq_kernel(const Problem 
     }
     for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int i = row0 + warp * kRowsPerWarp + rr;
-        if (i >= p.n) continue;
+        if (i >= p.n || !token_exists(p, c, i)) continue;
         const size_t off = token_offset(p, c, i);
         for (int t = 0; t < kMaxCols; ++t) {
             const int col = lane + 32 * t;
@@ -289,8 +290,8 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dkv_kernel(const Problem
         stage_concat(p, c, p.q, p.pq, isd, isr, i0, kTile, ldk, Qt);
         stage_plain(p, c, p.dout, i0, kTile, ldv, Gt);
         for (int t = threadIdx.x; t < kTile; t += kThreads) {
-            const bool ok = i0 + t < p.n;
-            Lt[t] = ok ? p.lse_in[token_scalar_offset(p, c, i0 + t)] : 0.f;
+            const bool ok = i0 + t < p.n && token_exists(p, c, i0 + t);
+            Lt[t] = ok ? p.lse_in[token_scalar_offset(p, c, i0 + t)] : INFINITY;      // +inf: probability 0 for a query that is no token
             Dt[t] = ok ? p.rowdot[token_scalar_offset(p, c, i0 + t)] : 0.f;
         }
         __syncthreads();
@@ -334,7 +335,7 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dkv_kernel(const Problem
     }
     for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int j = row0 + warp * kRowsPerWarp + rr;
-        if (j >= p.n) continue;
+        if (j >= p.n || !token_exists(p, c, j)) continue;
         const size_t off = token_offset(p, c, j);
         if (lane < p.d) p.dv[off + lane] = __float2bfloat16_rn(accV[rr][0]);
         if (lane + 32 < p.d) p.dv[off + lane + 32] = __float2bfloat16_rn(accV[rr][1]);

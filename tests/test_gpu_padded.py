@@ -54,6 +54,41 @@ def test_padded_forward_every_element(wl, path):
     compare("lse", to_f64(lse), ref_lse)
 
 
+BWD_CASES = [wl for wl in CASES if wl.H * wl.W <= 72 * 88]
+
+
+@pytest.mark.parametrize("wl", BWD_CASES, ids=lambda w: w.name)
+def test_padded_backward_every_element(wl):
+    """Backward on maps that are not multiples of the window (any-shape kernels), against the numpy oracle."""
+    cpu = synthetic.make_inputs(wl, with_dout=True)
+    gpu = {k: v.cuda() for k, v in cpu.items()}
+    out, lse = binding.rib_window_attn_fwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+    dq, dk, dv, dpq, dpk = binding.rib_window_attn_bwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse,
+                                                              gpu["dout"], wl.window, wl.shift)
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0
+    assert binding.rib_last_path() == binding.RIB_PATH_GENERIC
+    ref = pad.bwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk", "dout")), wl.window, wl.shift)
+    assert all(np.isfinite(r).all() for r in ref)
+    for name, got, want in zip(("dq", "dk", "dv"), (dq, dk, dv), ref[:3]):
+        compare(name, to_f64(got), want)
+    scale = max(1.0, float(np.abs(ref[3]).max()), float(np.abs(ref[4]).max()))
+    compare("dpq", to_f64(dpq), ref[3], max_abs=1e-2 * scale)
+    compare("dpk", to_f64(dpk), ref[4], max_abs=1e-2 * scale)
+
+
+def test_padded_backward_entry_point_on_a_divisible_map_is_the_plain_call():
+    wl = Workload("p_bwd_divisible", 1, 64, 32, 3, 32, 16, 32, 8, seed=76)
+    gpu = {k: v.cuda() for k, v in synthetic.make_inputs(wl, with_dout=True).items()}
+    out, lse = binding.rib_window_attn_fwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+    a = binding.rib_window_attn_bwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse, gpu["dout"], wl.window, wl.shift)
+    b = binding.rib_window_attn_bwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse, gpu["dout"], wl.window, wl.shift)
+    torch.cuda.synchronize()
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])     # dk, dv: bit-reproducible
+    compare("dq", to_f64(b[0]), to_f64(a[0]), max_abs=4e-3, rel_l2=1e-3)
+
+
 def test_divisible_map_through_the_padded_entry_point_is_the_plain_call():
     wl = Workload("p_divisible", 2, 64, 32, 3, 32, 16, 32, 8, seed=72)
     gpu = {k: v.cuda() for k, v in synthetic.make_inputs(wl, with_dout=False).items()}
