@@ -135,9 +135,8 @@ int rib_window_attn_fwd_padded(const void* q, const void* k, const void* v, cons
 /*
  * Backward pass of rib_window_attn_fwd_padded (same reading: positions of the extended map beyond H x W are not
  * tokens, so they receive and contribute no gradient).  Arguments, results and workspace rules as
- * rib_window_attn_bwd_headwise; the workspace size comes from rib_window_attn_bwd_padded_workspace.  Maps whose sides
- * are multiples of the window are passed on to rib_window_attn_bwd_headwise; all others run on the any-shape CUDA
- * kernels (the tcgen05 backward kernels take whole windows only), which is correct but slow.
+ * rib_window_attn_bwd_headwise; the workspace size comes from rib_window_attn_bwd_padded_workspace.  H and W multiples
+ * of 8 (and the shape conditions above) take the tcgen05 kernels, any other H, W the any-shape kernels.
  */
 int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
                                long long pos_head_stride,

@@ -301,7 +301,14 @@ size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, in
         return rib_window_attn_bwd_headwise_workspace(pos_head_stride, B, H, W, heads, d, r, window);
     if (check_shape(B, H, W, heads, d, r, window, 0, true) != RIB_OK) return 0;
     if (check_pos_stride(pos_head_stride, window, r) != RIB_OK) return 0;
-    return rowdot_bytes(B, H, W, heads);      // such maps take the any-shape kernels
+    size_t need = rowdot_bytes(B, H, W, heads);
+    rib::Problem p{};
+    fill_shape(p, B, H, W, heads, d, r, window, 0);
+    if (rib::sm100_bwd_supported(p)) {        // sized by the windows of the extended map
+        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1, r);
+        if (fast > need) need = fast;
+    }
+    return need;
 }
 
 int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
@@ -342,8 +349,7 @@ int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, cons
     p.pos_head_stride = pos_head_stride;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool partial = p.Hp != p.H || p.Wp != p.W;      // the tcgen05 backward kernels take whole windows only
-    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && !partial && rib::sm100_bwd_supported(p);
+    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_bwd_supported(p);
     const cudaError_t e = fast ? rib::sm100_bwd(p, st) : rib::generic_bwd(p, st);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;

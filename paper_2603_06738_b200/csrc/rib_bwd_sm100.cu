@@ -103,6 +103,7 @@ struct BwdParams {
     __nv_bfloat16* dv;
     int* status;
     int H, W, heads, M, s, n, nWy, nWx, nblk, items;
+    int Hp, Wp;                // sides of the map the windows are laid over (H, W rounded up to multiples of M)
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
     float scale_log2;          // log2(e) / sqrt(d)
     float inv_sqrt_d;
@@ -122,7 +123,12 @@ __device__ __forceinline__ ItemCoord decode_item(const BwdParams& p, int item)
     return c;
 }
 
-template <int R>
+// kPartial: H or W is not a multiple of the window (but of 8); windows are laid over the map extended to Hp x Wp and
+// an 8x8 patch of the extension holds no tokens.  TMA fills such patches with zeros; what is left to do: a key row that
+// is no token gets P^T = dS^T = 0 (a thread of the arithmetic warps is a key row, and the 64 rows of a patch share the
+// answer), a query that is no token reads -inf for -lse (written by the preparation kernel), i.e. probability 0,
+// and nothing is stored for either.
+template <int R, bool kPartial>
 __global__ void __launch_bounds__(kThreads, 1)
 rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -140,7 +146,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + kOffMisc + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const WindowGeom geom{p.H, p.W, p.M, p.s};
+    const WindowGeom geom{p.Hp, p.Wp, p.M, p.s};
 
     if (threadIdx.x == 0) {
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
@@ -336,6 +342,13 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         uint32_t g = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
+            bool key_real = true;         // kPartial: this warp's 32 key rows lie in one 8x8 patch of the key block
+            if (kPartial) {
+                const ItemCoord c = decode_item(p, item);
+                int py, px, Y0, X0;
+                patch_origin(geom, c.wy, c.wx, 2 * c.J + (quarter >> 1), py, px, Y0, X0);
+                key_real = Y0 < p.H && X0 < p.W;
+            }
             for (int I = 0; I < p.nblk; ++I, ++g) {
                 const uint32_t st = g % kQStages;
                 // warp-uniform outcome: the TMEM accesses below are warp-collective
@@ -367,8 +380,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                             const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])),
                                                                      make_float2(t.z, t.w)));
-                            pp[ch][i] = pack_bf16x2(e.x, e.y);
-                            dd[ch][i] = pack_bf16x2(d.x, d.y);
+                            pp[ch][i] = kPartial && !key_real ? 0u : pack_bf16x2(e.x, e.y);
+                            dd[ch][i] = kPartial && !key_real ? 0u : pack_bf16x2(d.x, d.y);
                         }
                     }
                     // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
@@ -419,8 +432,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                 const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                                 const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])),
                                                                          make_float2(t4[gq].z, t4[gq].w)));
-                                pp[ch][2 * gq + rr] = pack_bf16x2(e.x, e.y);
-                                dd[ch][2 * gq + rr] = pack_bf16x2(d.x, d.y);
+                                pp[ch][2 * gq + rr] = kPartial && !key_real ? 0u : pack_bf16x2(e.x, e.y);
+                                dd[ch][2 * gq + rr] = kPartial && !key_real ? 0u : pack_bf16x2(d.x, d.y);
                             }
                     }
                     // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
@@ -480,7 +493,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             tc_fence_after();
             int i, Y, X;
             window_order_token(geom, c.wy, c.wx, c.J * kTile + row, i, Y, X);
-            const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
+            const bool row_real = !kPartial || (Y < p.H && X < p.W);      // no dk / dv row for a position beyond the image
+            const size_t tok = row_real ? (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h : 0;
             uint4* dst_v = reinterpret_cast<uint4*>(p.dv + tok * kD);
             uint4* dst_k = reinterpret_cast<uint4*>(p.dk + tok * kD);
             float* dst_p = p.dkp + (size_t)c.pair * R * p.n + (size_t)c.J * kTile + row;
@@ -498,7 +512,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (part >= 4) {
 #pragma unroll
                     for (int col = 0; col < 16; ++col) dst_p[(size_t)(16 * (part - 4) + col) * p.n] = __uint_as_float(a[col]) * p.inv_sqrt_d;
-                } else {
+                } else if (row_real) {
                     const float f = part < 2 ? 1.f : p.inv_sqrt_d;
                     uint4* dst16 = (part < 2 ? dst_v : dst_k) + 2 * (part & 1);
 #pragma unroll
@@ -534,21 +548,24 @@ struct AuxParams {
     float* dpq;
     float* dpk;
     int H, W, heads, M, s, n, nWy, nWx, pairs;
+    int Hp, Wp;                  // sides of the extended map (equal to H, W when they are multiples of the window)
     int tables;                  // Pq/Pk tables: 1 (shared by the heads) or heads
     long long pos_head_stride;   // elements between the tables in pq, dpq, dpk (pq_scaled is packed: n * 16 apart)
     float pos_scale, inv_sqrt_d, inv_sqrt_r;
 };
 
-__device__ __forceinline__ void decode_pair_token(const AuxParams& p, int pair, int w, int& i, size_t& tok, size_t& scalar)
+// Returns false for a window position beyond the image (maps that are not multiples of the window): no token there.
+__device__ __forceinline__ bool decode_pair_token(const AuxParams& p, int pair, int w, int& i, size_t& tok, size_t& scalar)
 {
     const int h = pair % p.heads; pair /= p.heads;
     const int wx = pair % p.nWx; pair /= p.nWx;
     const int wy = pair % p.nWy; pair /= p.nWy;
     const int b = pair;
     int Y, X;
-    window_order_token(WindowGeom{p.H, p.W, p.M, p.s}, wy, wx, w, i, Y, X);
+    window_order_token(WindowGeom{p.Hp, p.Wp, p.M, p.s}, wy, wx, w, i, Y, X);
     tok = (((size_t)b * p.H + Y) * p.W + X) * p.heads + h;
     scalar = (((size_t)b * p.heads + h) * p.H + Y) * p.W + X;
+    return Y < p.H && X < p.W;
 }
 
 // One thread per (pair, token in window order): D = dO . O and lse in the layout the main kernel
@@ -571,7 +588,16 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     if (t >= total) return;
     const int pair = (int)(t / p.n), w = (int)(t % p.n);
     int i; size_t tok, scalar;
-    decode_pair_token(p, pair, w, i, tok, scalar);
+    float* z = p.dq_acc + (size_t)pair * kDk * p.n + w;
+    float* ldf = reinterpret_cast<float*>(p.ld) + ((t >> 1) << 2) + (t & 1);
+    if (!decode_pair_token(p, pair, w, i, tok, scalar)) {
+        // a position beyond the image: as a query it gets probability 0 (exp2(-inf)) and D = 0
+        ldf[0] = -INFINITY;
+        ldf[2] = 0.f;
+#pragma unroll 8
+        for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
+        return;
+    }
     const uint4* a = reinterpret_cast<const uint4*>(p.dout + tok * kD);
     const uint4* b = reinterpret_cast<const uint4*>(p.out + tok * kD);
     float acc = 0.f;
@@ -586,10 +612,8 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
         }
     }
     // per query pair (w even, w + 1): (-lse2, -lse2', -D, -D'), the operand order of the packed arithmetic
-    float* ldf = reinterpret_cast<float*>(p.ld) + ((t >> 1) << 2) + (t & 1);
     ldf[0] = -p.lse[scalar] * 1.4426950408889634f;
     ldf[2] = -acc;
-    float* z = p.dq_acc + (size_t)pair * kDk * p.n + w;
 #pragma unroll 8
     for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
 }
@@ -626,9 +650,9 @@ __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, 
     int i = 0;
     for (int pair = pair0; pair < pair1; pair += step) {
         size_t tok, scalar;
-        decode_pair_token(p, pair, w, i, tok, scalar);
+        const bool real = decode_pair_token(p, pair, w, i, tok, scalar);   // its sums are zero if not
         const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
-        if (blockIdx.z == 0) {
+        if (blockIdx.z == 0 && real) {
             uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
@@ -676,12 +700,12 @@ WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
 
 bool sm100_bwd_supported(const Problem& p)
 {
-    return p.d == sm100::kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256;
+    return p.d == sm100::kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
 }
 
 size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r) { return workspace_layout(pairs, n, tables, r).total; }
 
-template <int R>
+template <int R, bool kPartial>
 cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
@@ -701,12 +725,13 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
         return cudaErrorInvalidValue;
     static KernelSetup setup;       // one per instantiation of this launcher, i.e. per kernel
     int sm_count = 0;
-    if (cudaError_t e = setup.prepare(rib_bwd_sm100_kernel<R>, kSmemBytes, &sm_count)) return e;
+    if (cudaError_t e = setup.prepare(rib_bwd_sm100_kernel<R, kPartial>, kSmemBytes, &sm_count)) return e;
     AuxParams ap{};
     ap.out = p.out; ap.dout = p.dout; ap.pq = p.pq; ap.lse = p.lse_in;
     ap.ld = ld; ap.dq_acc = dq_acc; ap.dkp = dkp; ap.pq_scaled = pq_scaled;
     ap.dq = p.dq; ap.dpq = p.dpq; ap.dpk = p.dpk;
     ap.H = p.H; ap.W = p.W; ap.heads = p.heads; ap.M = p.M; ap.s = p.s; ap.n = p.n; ap.nWy = p.nWy; ap.nWx = p.nWx;
+    ap.Hp = p.Hp; ap.Wp = p.Wp;
     ap.pairs = p.pairs;
     ap.tables = tables;
     ap.pos_head_stride = p.pos_head_stride;
@@ -722,13 +747,14 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     BwdParams bp{};
     bp.ld = ld; bp.dq_acc = dq_acc; bp.dkp = dkp; bp.dk = p.dk; bp.dv = p.dv; bp.status = p.status;
     bp.H = p.H; bp.W = p.W; bp.heads = p.heads; bp.M = p.M; bp.s = p.s; bp.n = p.n; bp.nWy = p.nWy; bp.nWx = p.nWx;
+    bp.Hp = p.Hp; bp.Wp = p.Wp;
     bp.nblk = p.n / kTile;
     bp.items = p.pairs * bp.nblk;
     bp.pos_per_head = tables > 1 ? 1 : 0;
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
-    { ProfileScope scope(RIB_KERNEL_BWD_MAIN, stream); rib_bwd_sm100_kernel<R><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp); }
+    { ProfileScope scope(RIB_KERNEL_BWD_MAIN, stream); rib_bwd_sm100_kernel<R, kPartial><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
@@ -743,7 +769,8 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 {
-    return p.r == 32 ? launch_bwd<32>(p, stream) : launch_bwd<16>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W) return p.r == 32 ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
+    return p.r == 32 ? launch_bwd<32, false>(p, stream) : launch_bwd<16, false>(p, stream);
 }
 
 }  // namespace rib

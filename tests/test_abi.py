@@ -76,8 +76,10 @@ def test_headwise_and_padded_entry_points_validate_before_any_cuda_call(lib):
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=0)) == -2
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, d=12)) == -3
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, v=770)) == -4
-    # backward on maps that are not multiples of the window: any-shape kernels, which need one float per token-head
-    assert lib.rib_window_attn_bwd_padded_workspace(0, 1, 40, 56, 2, 32, 16, 16) == (4 * 40 * 56 * 2 + 255) // 256 * 256
+    # backward on maps that are not multiples of the window: sized by the windows of the extended map on the tcgen05
+    # shapes, one float per token-head on the any-shape kernels
+    assert lib.rib_window_attn_bwd_padded_workspace(0, 1, 40, 56, 2, 32, 16, 16) >= 264 * 48 * 64 * 2
+    assert lib.rib_window_attn_bwd_padded_workspace(0, 1, 41, 56, 2, 32, 16, 16) == (4 * 41 * 56 * 2 + 255) // 256 * 256
     assert lib.rib_window_attn_bwd_padded_workspace(0, 1, 32, 32, 2, 32, 16, 16) == lib.rib_window_attn_bwd_workspace(1, 32, 32, 2, 32, 16, 16)
     assert lib.rib_window_attn_bwd_padded_workspace(0, 1, 0, 56, 2, 32, 16, 16) == 0
     # rank 32 needs a larger backward workspace than rank 16 on the tcgen05 shapes

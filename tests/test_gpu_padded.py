@@ -58,16 +58,24 @@ BWD_CASES = [wl for wl in CASES if wl.H * wl.W <= 72 * 88]
 
 
 @pytest.mark.parametrize("wl", BWD_CASES, ids=lambda w: w.name)
-def test_padded_backward_every_element(wl):
-    """Backward on maps that are not multiples of the window (any-shape kernels), against the numpy oracle."""
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_padded_backward_every_element(wl, path):
+    """Backward on maps that are not multiples of the window, against the numpy oracle, on both kernel families."""
     cpu = synthetic.make_inputs(wl, with_dout=True)
     gpu = {k: v.cuda() for k, v in cpu.items()}
     out, lse = binding.rib_window_attn_fwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
-    dq, dk, dv, dpq, dpk = binding.rib_window_attn_bwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse,
-                                                              gpu["dout"], wl.window, wl.shift)
+    binding.rib_set_path(binding.RIB_PATH_GENERIC if path == "generic" else binding.RIB_PATH_NONE)
+    try:
+        dq, dk, dv, dpq, dpk = binding.rib_window_attn_bwd_padded(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse,
+                                                                  gpu["dout"], wl.window, wl.shift)
+        used = binding.rib_last_path()
+    finally:
+        binding.rib_set_path(binding.RIB_PATH_NONE)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
-    assert binding.rib_last_path() == binding.RIB_PATH_GENERIC
+    fast = (path == "auto" and wl.d == 32 and wl.r in (16, 32) and wl.window % 16 == 0 and wl.shift % 8 == 0
+            and wl.H % 8 == 0 and wl.W % 8 == 0)
+    assert used == (binding.RIB_PATH_SM100 if fast else binding.RIB_PATH_GENERIC)
     ref = pad.bwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk", "dout")), wl.window, wl.shift)
     assert all(np.isfinite(r).all() for r in ref)
     for name, got, want in zip(("dq", "dk", "dv"), (dq, dk, dv), ref[:3]):
