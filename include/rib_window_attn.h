@@ -152,8 +152,8 @@ size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, in
  *   G  = sigmoid(PWConv(DWConv3x3(X)))      X: the block's token features as an H x W map          (Eq. 8)
  *   O' = O o G                              element-wise product with the attention output           (Eq. 9)
  * rib_cla_gate computes G; rib_window_attn_fwd_gated is the forward pass with `out` = O o G, the product taken in
- * the attention kernel's epilogue so that the ungated O never goes to memory.  Forward only (inference); for
- * training, take the product outside and use the ungated entry points.
+ * the attention kernel's epilogue so that the ungated O never goes to memory (inference); for training, keep the
+ * ungated O of rib_window_attn_fwd for the attention backward and take the product with rib_cla_product (below).
  *   x     : bf16 [B][H][W][D], D = heads * d, the same channel order as `out` ([heads][d]).
  *   w_dw  : fp32 [D][3][3] depth-wise filter, w_dw[c][dy][dx] multiplies x[y + dy - 1][x + dx - 1][c]; zero padding.
  *   b_dw  : fp32 [D].   w_pw : fp32 [D][D], [output channel][input channel].   b_pw : fp32 [D].
@@ -169,6 +169,38 @@ int rib_window_attn_fwd_gated(const void* q, const void* k, const void* v, const
                               long long pos_head_stride, const void* gate,
                               int B, int H, int W, int heads, int d, int r, int window, int shift,
                               void* out, float* lse, void* stream);
+
+/*
+ * Backward pass of Convolutional Local Attention (paper: Sec. 3.2; the chain rule of Eq. 8 and Eq. 9) and the
+ * stand-alone product of Eq. 9 for training, where the ungated O has to stay in memory for the attention backward.
+ *
+ * rib_cla_product      out_gated = out o gate                                     (Eq. 9)
+ * rib_cla_product_bwd  dout = dout_gated o gate,  dgate = dout_gated o out         (its chain rule)
+ *   out, gate, dout_gated, out_gated, dout, dgate: bf16, `count` elements each in the same order ([B][H][W][D] with
+ *   D = heads * d); count a multiple of 8; products in fp32, rounded once.  One kernel each.
+ *
+ * rib_cla_gate_bwd     given dgate = dL/dG, with Y = DWConv3x3(X), Z = PWConv(Y), G = sigmoid(Z) recomputed in fp32:
+ *     dZ = dG o G o (1 - G);   db_pw[o] = sum dZ[o];   dw_pw[o][i] = sum dZ[o] Y[i];   dY = dZ W_pw;
+ *     db_dw[c] = sum dY[c];    dw_dw[c][dy][dx] = sum dY[y][x][c] X[y + dy - 1][x + dx - 1][c];
+ *     dX[y][x][c] = sum_{dy, dx} dY[y - dy + 1][x - dx + 1][c] w_dw[c][dy][dx]         (sums over pixels and batch items)
+ *   x, w_dw, b_dw, w_pw, b_pw: as for rib_cla_gate, read only.   dgate: bf16 [B][H][W][D], read only.
+ *   dx: bf16 [B][H][W][D];  dw_dw [D][3][3], db_dw [D], dw_pw [D][D], db_pw [D]: fp32; all five overwritten.
+ *   workspace: device scratch of at least rib_cla_gate_bwd_workspace(B, H, W, D) bytes (dY in fp32 and the
+ *   transposed matrix), 16-byte aligned, owned by the caller, contents undefined afterwards.
+ *   Any positive H and W; D = 64, 128 or 192 (RIB_ERR_UNSUPPORTED otherwise).  Four small memsets, one transpose and
+ *   two kernels on `stream`.  The weight gradients are fp32 sums in no fixed order (atomics): equal up to rounding
+ *   from call to call.
+ * All pointers are device pointers, 16-byte aligned, caller-owned; errors as for the other entry points
+ * (RIB_ERR_NULL, RIB_ERR_SHAPE, RIB_ERR_ALIGN, RIB_ERR_UNSUPPORTED, RIB_ERR_WORKSPACE, RIB_ERR_CUDA).
+ */
+int rib_cla_product(const void* out, const void* gate, long long count, void* out_gated, void* stream);
+int rib_cla_product_bwd(const void* out, const void* gate, const void* dout_gated, long long count, void* dout, void* dgate,
+                        void* stream);
+int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
+                     const void* dgate, int B, int H, int W, int D,
+                     void* dx, float* dw_dw, float* db_dw, float* dw_pw, float* db_pw,
+                     void* workspace, size_t workspace_bytes, void* stream);
+size_t rib_cla_gate_bwd_workspace(int B, int H, int W, int D);
 
 /*
  * Backward pass for callers that cannot hand over scratch memory.  (The paper has no counterpart:
@@ -259,7 +291,7 @@ long long rib_kernel_launches(void);
 enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH = 4,
        RIB_KERNEL_RESERVED = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
        RIB_KERNEL_ANY_BWD_DKV = 9, RIB_KERNEL_GENERATOR_FWD = 10, RIB_KERNEL_GENERATOR_BWD = 11,
-    RIB_KERNEL_CLA_GATE = 12 };
+    RIB_KERNEL_CLA_GATE = 12, RIB_KERNEL_CLA_BWD_PW = 13, RIB_KERNEL_CLA_BWD_DW = 14, RIB_KERNEL_CLA_PRODUCT = 15 };
 int rib_profile_begin(int max_launches);
 int rib_profile_end(int* kernel_ids, float* ms, int capacity);
 

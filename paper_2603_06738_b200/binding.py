@@ -26,11 +26,13 @@ EXPORTS = (
     "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
     "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
     "rib_window_attn_bwd_padded", "rib_window_attn_bwd_padded_workspace",
+    "rib_cla_product", "rib_cla_product_bwd", "rib_cla_gate_bwd", "rib_cla_gate_bwd_workspace",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
                 7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel",
-                10: "rib_generator_fwd_kernel", 11: "rib_generator_bwd_kernel", 12: "rib_cla_gate_kernel"}
+                10: "rib_generator_fwd_kernel", 11: "rib_generator_bwd_kernel", 12: "rib_cla_gate_kernel",
+                13: "rib_cla_bwd_pw_kernel", 14: "rib_cla_bwd_dw_kernel", 15: "rib_cla_product_kernel"}
 RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
@@ -68,6 +70,14 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_bwd_padded_workspace.argtypes = [ll] + [ci] * 7
         lib.rib_cla_gate.restype = ci
         lib.rib_cla_gate.argtypes = [vp] * 5 + [ci] * 4 + [vp, vp]
+        lib.rib_cla_product.restype = ci
+        lib.rib_cla_product.argtypes = [vp, vp, ll, vp, vp]
+        lib.rib_cla_product_bwd.restype = ci
+        lib.rib_cla_product_bwd.argtypes = [vp, vp, vp, ll, vp, vp, vp]
+        lib.rib_cla_gate_bwd.restype = ci
+        lib.rib_cla_gate_bwd.argtypes = [vp] * 6 + [ci] * 4 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_cla_gate_bwd_workspace.restype = ctypes.c_size_t
+        lib.rib_cla_gate_bwd_workspace.argtypes = [ci] * 4
         lib.rib_window_attn_fwd_gated.restype = ci
         lib.rib_window_attn_fwd_gated.argtypes = [vp] * 5 + [ll, vp] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd_headwise.restype = ci
@@ -310,6 +320,61 @@ def rib_cla_gate(x, w_dw, b_dw, w_pw, b_pw, stream=None):
     if rc != RIB_OK:
         raise RibError(rc)
     return gate
+
+
+def _check_bf16_like(name, t, like=None):
+    if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA bfloat16 tensor")
+    if like is not None and t.numel() != like.numel():
+        raise ValueError(f"{name} must have as many elements as out")
+
+
+def rib_cla_product(out, gate, stream=None):
+    """Eq. 9 on its own: out [B,H,W,heads,d] (or [B,H,W,D]) times gate [B,H,W,D], both bf16; returns out's shape."""
+    _check_bf16_like("out", out)
+    _check_bf16_like("gate", gate, out)
+    res = torch.empty_like(out)
+    rc = library().rib_cla_product(_ptr(out), _ptr(gate), out.numel(), _ptr(res), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return res
+
+
+def rib_cla_product_bwd(out, gate, dout_gated, stream=None):
+    """Chain rule of Eq. 9: returns (dout in out's shape, dgate in gate's shape), bf16."""
+    _check_bf16_like("out", out)
+    _check_bf16_like("gate", gate, out)
+    _check_bf16_like("dout_gated", dout_gated, out)
+    dout = torch.empty_like(out)
+    dgate = torch.empty_like(gate)
+    rc = library().rib_cla_product_bwd(_ptr(out), _ptr(gate), _ptr(dout_gated), out.numel(), _ptr(dout), _ptr(dgate),
+                                       _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return dout, dgate
+
+
+def rib_cla_gate_bwd(x, w_dw, b_dw, w_pw, b_pw, dgate, workspace=None, stream=None):
+    """Chain rule of Eq. 8: x, dgate bf16 [B,H,W,D]; weights as for rib_cla_gate.
+    Returns (dx bf16 [B,H,W,D], dw_dw [D,3,3], db_dw [D], dw_pw [D,D], db_pw [D] fp32)."""
+    if x.dtype != torch.bfloat16 or not x.is_cuda or not x.is_contiguous() or x.dim() != 4:
+        raise ValueError("x must be a contiguous CUDA bfloat16 tensor [B,H,W,D]")
+    B, H, W, D = x.shape
+    if dgate.dtype != torch.bfloat16 or not dgate.is_cuda or not dgate.is_contiguous() or dgate.shape != x.shape:
+        raise ValueError("dgate must be a contiguous CUDA bfloat16 tensor of x's shape")
+    for name, t, shape in (("w_dw", w_dw, (D, 3, 3)), ("b_dw", b_dw, (D,)), ("w_pw", w_pw, (D, D)), ("b_pw", b_pw, (D,))):
+        if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shape:
+            raise ValueError(f"{name} must be a contiguous CUDA fp32 tensor of shape {shape}")
+    need = library().rib_cla_gate_bwd_workspace(B, H, W, D)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=x.device)
+    dx = torch.empty_like(x)
+    grads = [torch.empty_like(t) for t in (w_dw, b_dw, w_pw, b_pw)]
+    rc = library().rib_cla_gate_bwd(_ptr(x), _ptr(w_dw), _ptr(b_dw), _ptr(w_pw), _ptr(b_pw), _ptr(dgate), B, H, W, D, _ptr(dx),
+                                    *[_ptr(g) for g in grads], _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return (dx, *grads)
 
 
 def rib_window_attn_fwd_gated(q, k, v, pq, pk, gate, window, shift=0, stream=None, want_lse=True):

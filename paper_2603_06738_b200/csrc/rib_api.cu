@@ -215,6 +215,62 @@ int rib_cla_gate(const void* x, const float* w_dw, const float* b_dw, const floa
     return RIB_OK;
 }
 
+int rib_cla_product(const void* out, const void* gate, long long count, void* out_gated, void* stream)
+{
+    if (!out || !gate || !out_gated) return RIB_ERR_NULL;
+    if (count < 0 || count % 8) return RIB_ERR_SHAPE;
+    if (!aligned16(out) || !aligned16(gate) || !aligned16(out_gated)) return RIB_ERR_ALIGN;
+    if (count == 0) return RIB_OK;
+    const cudaError_t e = rib::cla_product(static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(gate), nullptr,
+                                           count, static_cast<__nv_bfloat16*>(out_gated), nullptr, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
+int rib_cla_product_bwd(const void* out, const void* gate, const void* dout_gated, long long count, void* dout, void* dgate,
+                        void* stream)
+{
+    if (!out || !gate || !dout_gated || !dout || !dgate) return RIB_ERR_NULL;
+    if (count < 0 || count % 8) return RIB_ERR_SHAPE;
+    const void* ptrs[] = {out, gate, dout_gated, dout, dgate};
+    for (const void* ptr : ptrs)
+        if (!aligned16(ptr)) return RIB_ERR_ALIGN;
+    if (count == 0) return RIB_OK;
+    const cudaError_t e = rib::cla_product(static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(gate),
+                                           static_cast<const __nv_bfloat16*>(dout_gated), count, static_cast<__nv_bfloat16*>(dout),
+                                           static_cast<__nv_bfloat16*>(dgate), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
+size_t rib_cla_gate_bwd_workspace(int B, int H, int W, int D)
+{
+    if (B <= 0 || H <= 0 || W <= 0 || D <= 0) return 0;
+    return rib::cla_gate_bwd_workspace_bytes((long long)B * H * W, D);
+}
+
+int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
+                     const void* dgate, int B, int H, int W, int D,
+                     void* dx, float* dw_dw, float* db_dw, float* dw_pw, float* db_pw,
+                     void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!x || !w_dw || !b_dw || !w_pw || !b_pw || !dgate || !dx || !dw_dw || !db_dw || !dw_pw || !db_pw) return RIB_ERR_NULL;
+    if (B <= 0 || H <= 0 || W <= 0 || D <= 0) return RIB_ERR_SHAPE;
+    if (!rib::cla_gate_bwd_supported(D)) return RIB_ERR_UNSUPPORTED;
+    const void* ptrs[] = {x, w_dw, b_dw, w_pw, b_pw, dgate, dx, dw_dw, db_dw, dw_pw, db_pw, workspace};
+    for (const void* ptr : ptrs)
+        if (!aligned16(ptr)) return RIB_ERR_ALIGN;
+    if (!workspace || workspace_bytes < rib_cla_gate_bwd_workspace(B, H, W, D)) return RIB_ERR_WORKSPACE;
+    const cudaError_t e = rib::cla_gate_bwd(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw,
+                                            static_cast<const __nv_bfloat16*>(dgate), B, H, W, D, static_cast<__nv_bfloat16*>(dx),
+                                            dw_dw, db_dw, dw_pw, db_pw, workspace, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 3;
+    return RIB_OK;
+}
+
 }  // extern "C"
 
 namespace {

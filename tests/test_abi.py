@@ -116,3 +116,27 @@ def test_path_knob(lib):
     assert binding.rib_set_path(binding.RIB_PATH_GENERIC) in (0, 1)
     assert binding.rib_set_path(binding.RIB_PATH_NONE) == binding.RIB_PATH_GENERIC
     assert binding.rib_set_path(77) == binding.RIB_PATH_NONE   # invalid value: unchanged
+
+
+def test_cla_backward_entry_points_validate_before_any_cuda_call(lib):
+    a = [256, 512, 768, 1024, 1280, 1536]                       # x, w_dw, b_dw, w_pw, b_pw, dgate
+    outs = [2048, 4096, 8192, 12288, 16384]                     # dx, dw_dw, db_dw, dw_pw, db_pw
+    need = lib.rib_cla_gate_bwd_workspace(1, 5, 7, 64)
+    assert need == (5 * 7 * 64 + 64 * 64) * 4
+    assert lib.rib_cla_gate_bwd_workspace(1, 0, 7, 64) == 0
+    call = lambda **kw: lib.rib_cla_gate_bwd(*kw.get("ins", a), kw.get("B", 1), 5, 7, kw.get("D", 64), *kw.get("outs", outs),
+                                             kw.get("ws", 32768), kw.get("ws_bytes", need), None)
+    assert call(ins=[None] + a[1:]) == -1
+    assert call(outs=outs[:4] + [None]) == -1
+    assert call(B=0) == -2
+    assert call(D=96) == -3
+    assert call(outs=[2050] + outs[1:]) == -4
+    assert call(ws=None) == -5
+    assert call(ws_bytes=need - 1) == -5
+    assert lib.rib_cla_product(256, 512, 12, 768, None) == -2                      # count not a multiple of 8
+    assert lib.rib_cla_product(256, None, 16, 768, None) == -1
+    assert lib.rib_cla_product(256, 520, 16, 768, None) == -4
+    assert lib.rib_cla_product(256, 512, 0, 768, None) == 0                        # nothing to do
+    assert lib.rib_cla_product_bwd(256, 512, 768, -8, 1024, 1280, None) == -2
+    assert lib.rib_cla_product_bwd(256, 512, None, 16, 1024, 1280, None) == -1
+    assert lib.rib_cla_product_bwd(256, 512, 768, 16, 1024, 1284, None) == -4

@@ -98,3 +98,62 @@ def test_gate_rejects_unsupported_sizes():
     assert lib.rib_cla_gate(*ptrs, 0, 8, 16, 64, x.data_ptr(), None) == -2
     assert lib.rib_cla_gate(None, *ptrs[1:], 1, 8, 16, 64, x.data_ptr(), None) == -1
     assert binding.rib_kernel_launches() == launches
+
+
+# ---- backward of Eq. 8 and Eq. 9 ----
+
+def dgate_input(seed, shape):
+    return synthetic.bf16_tensor(seed, "gate", shape, 1.0)
+
+
+@pytest.mark.parametrize("B,H,W,D", [(1, 5, 7, 64), (2, 16, 32, 192), (1, 24, 47, 128), (3, 9, 16, 192), (1, 1, 1, 64),
+                                     (1, 96, 96, 192)])
+def test_gate_backward_matches_the_oracle(B, H, W, D):
+    x, ws = gate_inputs(300 + D + H, B, H, W, D)
+    dgate = dgate_input(301 + D + H, (B, H, W, D))
+    got = binding.rib_cla_gate_bwd(x.cuda(), *[torch.from_numpy(w).cuda() for w in ws], dgate.cuda())
+    torch.cuda.synchronize()
+    ref = cla.gate_bwd(to_f64(x), *ws, to_f64(dgate))
+    compare("dx", to_f64(got[0]), ref[0], max_abs=1e-2 * max(1.0, np.abs(ref[0]).max()))
+    # fp32 sums of fp32 products over the pixels, against float64
+    for name, g, r in zip(("dw_dw", "db_dw", "dw_pw", "db_pw"), got[1:], ref[1:]):
+        compare(name, to_f64(g), r, max_abs=1e-3 * max(1.0, np.abs(r).max()), rel_l2=1e-4)
+
+
+def test_gate_backward_overwrites_its_outputs_and_repeats():
+    B, H, W, D = 1, 16, 16, 64
+    x, ws = gate_inputs(310, B, H, W, D)
+    dgate = dgate_input(311, (B, H, W, D))
+    args = [x.cuda(), *[torch.from_numpy(w).cuda() for w in ws], dgate.cuda()]
+    first = [t.clone() for t in binding.rib_cla_gate_bwd(*args)]
+    second = binding.rib_cla_gate_bwd(*args)
+    torch.cuda.synchronize()
+    assert torch.equal(first[0], second[0])                                       # dx has a fixed summation order
+    for a, b in zip(first[1:], second[1:]):                                       # atomics: equal up to rounding
+        assert torch.allclose(a, b, rtol=1e-4, atol=1e-5)
+
+
+@pytest.mark.parametrize("shape", [(1, 8, 16, 2, 32), (2, 5, 7, 6, 32), (1, 96, 96, 6, 32)])
+def test_product_and_its_backward_match_the_oracle(shape):
+    B, H, W, heads, d = shape
+    out = synthetic.bf16_tensor(320, "x", shape, 1.0)
+    gate = synthetic.bf16_tensor(321, "gate", (B, H, W, heads * d), 0.3).abs().clamp(max=1.0).to(torch.bfloat16)
+    dgo = synthetic.bf16_tensor(322, "dout", shape, 1.0)
+    prod = binding.rib_cla_product(out.cuda(), gate.cuda())
+    dout, dgate = binding.rib_cla_product_bwd(out.cuda(), gate.cuda(), dgo.cuda())
+    torch.cuda.synchronize()
+    ref_dout, ref_dgate = cla.gated_output_bwd(to_f64(out), to_f64(gate), to_f64(dgo))
+    # one bf16 rounding of an exact fp32 product: the GPU result is the correctly rounded oracle value
+    for got, ref in ((prod, cla.gated_output(to_f64(out), to_f64(gate))), (dout, ref_dout), (dgate, ref_dgate)):
+        want = torch.from_numpy(ref).to(torch.bfloat16)
+        assert torch.equal(got.cpu().reshape(want.shape), want)
+
+
+def test_gate_backward_rejects_unsupported_channels_without_launching():
+    lib = binding.library()
+    x = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
+    launches = binding.rib_kernel_launches()
+    assert lib.rib_cla_gate_bwd(x.data_ptr(), *[w.data_ptr()] * 4, x.data_ptr(), 1, 4, 4, 96, x.data_ptr(), *[w.data_ptr()] * 4,
+                                w.data_ptr(), 1 << 18, None) == -3
+    assert binding.rib_kernel_launches() == launches
