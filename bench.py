@@ -386,6 +386,17 @@ def main():
                 gate_bytes = 2 * cx.numel() * 2
                 variants["cla"] = {"gate_ms": g_ms, "gate_algorithmic_bytes": gate_bytes, "gate_gbs": gate_bytes / (g_ms * 1e-3) / 1e9,
                                    "gate_flops": 2 * cx.numel() * (9 + D), "gated_fwd_ms": gf_ms, "paths": [binding.rib_last_path()]}
+                # training: the stand-alone product of Eq. 9, its chain rule, and the backward of the gate (fp32 kernels)
+                dgo = torch.randn_like(cx)
+                ws = torch.empty(binding.library().rib_cla_gate_bwd_workspace(wl.B, wl.H, wl.W, D), dtype=torch.uint8, device=dev)
+                p_ms = timed(lambda: binding.rib_cla_product(cx, gate))
+                pb_ms = timed(lambda: binding.rib_cla_product_bwd(cx, gate, dgo))
+                gb_ms = timed(lambda: binding.rib_cla_gate_bwd(cx, *cw, dgo, workspace=ws), reps=5)
+                variants["cla"].update({"product_ms": p_ms, "product_gbs": 3 * 2 * cx.numel() / (p_ms * 1e-3) / 1e9,
+                                        "product_bwd_ms": pb_ms, "product_bwd_gbs": 5 * 2 * cx.numel() / (pb_ms * 1e-3) / 1e9,
+                                        "gate_bwd_ms": gb_ms, "gate_bwd_flops": cx.numel() * (6 * D + 4 * 9),
+                                        "gate_bwd_tflops": cx.numel() * (6 * D + 4 * 9) / (gb_ms * 1e-3) / 1e12})
+                del dgo, ws
             if binding.rib_query_status() != 0:
                 raise SystemExit("device status word set during the variant timings")
             del fq, fk, fv
