@@ -291,7 +291,7 @@ long long rib_kernel_launches(void);
 enum { RIB_KERNEL_FWD_MAIN = 1, RIB_KERNEL_BWD_PREPARE = 2, RIB_KERNEL_BWD_MAIN = 3, RIB_KERNEL_BWD_FINISH = 4,
        RIB_KERNEL_RESERVED = 5, RIB_KERNEL_ANY_FWD = 6, RIB_KERNEL_ANY_ROWDOT = 7, RIB_KERNEL_ANY_BWD_DQ = 8,
        RIB_KERNEL_ANY_BWD_DKV = 9, RIB_KERNEL_GENERATOR_FWD = 10, RIB_KERNEL_GENERATOR_BWD = 11,
-    RIB_KERNEL_CLA_GATE = 12, RIB_KERNEL_CLA_BWD_PW = 13, RIB_KERNEL_CLA_BWD_DW = 14, RIB_KERNEL_CLA_PRODUCT = 15 };
+    RIB_KERNEL_CLA_GATE = 12, RIB_KERNEL_CLA_BWD_PW = 13, RIB_KERNEL_CLA_BWD_DW = 14, RIB_KERNEL_CLA_PRODUCT = 15, RIB_KERNEL_CLA_BWD_TC = 16 };
 int rib_profile_begin(int max_launches);
 int rib_profile_end(int* kernel_ids, float* ms, int capacity);
 

@@ -32,7 +32,7 @@ KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
                 7: "rowdot_kernel", 8: "generic_bwd_dq_kernel", 9: "generic_bwd_dkv_kernel",
                 10: "rib_generator_fwd_kernel", 11: "rib_generator_bwd_kernel", 12: "rib_cla_gate_kernel",
-                13: "rib_cla_bwd_pw_kernel", 14: "rib_cla_bwd_dw_kernel", 15: "rib_cla_product_kernel"}
+                13: "rib_cla_bwd_pw_kernel", 14: "rib_cla_bwd_dw_kernel", 15: "rib_cla_product_kernel", 16: "rib_cla_bwd_tc_kernel"}
 RIB_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 

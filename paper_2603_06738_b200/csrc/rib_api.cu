@@ -263,11 +263,15 @@ int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const 
     for (const void* ptr : ptrs)
         if (!aligned16(ptr)) return RIB_ERR_ALIGN;
     if (!workspace || workspace_bytes < rib_cla_gate_bwd_workspace(B, H, W, D)) return RIB_ERR_WORKSPACE;
+    int* status = nullptr;
+    if (int rc = device_status_ptr(&status)) return rc;
+    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC;
     const cudaError_t e = rib::cla_gate_bwd(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw,
                                             static_cast<const __nv_bfloat16*>(dgate), B, H, W, D, static_cast<__nv_bfloat16*>(dx),
-                                            dw_dw, db_dw, dw_pw, db_pw, workspace, static_cast<cudaStream_t>(stream));
+                                            dw_dw, db_dw, dw_pw, db_pw, workspace, fast, status, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return RIB_ERR_CUDA;
-    g_kernel_launches += 3;
+    t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
+    g_kernel_launches += fast ? 2 : 3;
     return RIB_OK;
 }
 

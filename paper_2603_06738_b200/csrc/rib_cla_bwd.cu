@@ -7,12 +7,14 @@
 //                               dZ = dG o G o (1 - G), writes dY = dZ W_pw to the workspace, and keeps the running sums
 //                               dW_pw += dZ^T Y, db_pw += dZ in registers over all its tiles (one atomic flush at the end).
 //   rib_cla_bwd_dw_kernel       dX from the 3 x 3 neighbourhood of dY, and dw_dw, db_dw summed over the pixels.
-// The matrix products run on the fp32 pipes from shared-memory tiles: a first, any-size path for this step (any H, W;
-// D = 64, 128 or 192); the gate is recomputed rather than read back, because G o (1 - G) from a bf16 G loses most of its
-// digits where the gate saturates.
-#include "rib_common.cuh"
-
-#include <mutex>
+//   rib_cla_bwd_tc_kernel       the point-wise part on the tensor cores (tcgen05, accumulators in tensor memory): per tile
+//                               of 128 pixels Y and dZ are bf16 shared-memory tiles, Z = Y W_pw^T, dY = dZ W_pw and
+//                               dW_pw += dZ^T Y are MMAs on those tiles and on the bf16 matrix staged once per CTA; dW_pw
+//                               stays in tensor memory over all tiles of the CTA.  The default; rib_cla_bwd_pw_kernel is the
+//                               fp32 form of the same step on the ordinary pipes (any-shape path).
+// Any H, W; D = 64, 128 or 192.  The gate is recomputed rather than read back, because G o (1 - G) from a bf16 G loses
+// most of its digits where the gate saturates.
+#include "rib_sm100_common.cuh"
 
 namespace rib {
 namespace {
@@ -71,6 +73,7 @@ struct ClaBwdParams {
     float* dw_dw; float* db_dw; float* dw_pw; float* db_pw;
     int B, H, W;
     long long pixels;
+    int* status;
 };
 
 __global__ void rib_cla_transpose_kernel(const float* __restrict__ w, float* __restrict__ wt, int D)
@@ -296,46 +299,300 @@ __global__ void __launch_bounds__(D * kDwLanes) rib_cla_bwd_dw_kernel(const ClaB
     }
 }
 
-// Per-kernel, per-device: shared-memory opt-in and the SM count.
-struct Setup {
-    std::mutex mutex;
-    int sm_count[64] = {};
-    template <typename Kernel>
-    cudaError_t prepare(Kernel kernel, size_t smem_bytes, int* sms)
-    {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-        std::lock_guard<std::mutex> lock(mutex);
-        if (!sm_count[dev]) {
-            int count = 0;
-            e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
-            if (e == cudaSuccess && smem_bytes) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-            if (e != cudaSuccess) return e;
-            sm_count[dev] = count;
-        }
-        *sms = sm_count[dev];
-        return cudaSuccess;
-    }
+// ------------------------------------------------------------------------------------------------------------------
+// Point-wise part on the tensor cores.
+// ------------------------------------------------------------------------------------------------------------------
+using namespace sm100;
+
+constexpr int kTcPix = 128;          // pixels per tile = the M of the MMAs
+constexpr int kTcThreads = 512;
+
+template <int D>
+struct TcLayout {
+    static_assert(D % 64 == 0 && D >= 64 && D <= 192, "channels come in SWIZZLE_128B atoms of 64");
+    static constexpr int kAtoms = D / 64;
+    static constexpr uint32_t kWAtom = D * 128, kTAtom = kTcPix * 128;     // bytes of a 64-channel slice of W, and of Y or dZ
+    static constexpr uint32_t kOffW = 0;                                   // [atoms of in][D out rows][128 B]
+    static constexpr uint32_t kOffZ = kOffW + kAtoms * kWAtom;             // dZ: [atoms of out][128 pixels][128 B]
+    static constexpr uint32_t kOffY = kOffZ + kAtoms * kTAtom;             // Y:  [atoms of in][128 pixels][128 B]
+    static constexpr uint32_t kOffTaps = kOffY + kAtoms * kTAtom;          // [9][D] fp32
+    static constexpr uint32_t kOffBdw = kOffTaps + 9 * D * 4;
+    static constexpr uint32_t kOffBpw = kOffBdw + D * 4;
+    static constexpr uint32_t kOffDb = kOffBpw + D * 4;                    // running db_pw of the CTA
+    static constexpr uint32_t kOffBar = kOffDb + D * 4;
+    static constexpr uint32_t kOffMisc = kOffBar + 16;
+    static constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
+    static_assert(kOffZ % 1024 == 0 && kOffY % 1024 == 0 && kWAtom % 1024 == 0, "swizzle atoms need aligned tiles");
+    // tensor memory: [0, 128) Z and dY, 128 columns at a time; then dW_pw as one or two blocks of 128 rows x D columns
+    static constexpr int kN1 = D < 128 ? D : 128, kN2 = D - kN1;           // column split of Z and dY
+    static constexpr int kBlocks = D > 128 ? 2 : 1;                        // dW_pw rows [0, 128) and [D - 128, D)
+    static constexpr uint32_t kColW = 128;
+    static constexpr uint32_t kTmemCols = kColW + kBlocks * D <= 256 ? 256 : 512;
 };
 
 template <int D>
-cudaError_t launch_gate_bwd(const ClaBwdParams& p, cudaStream_t stream)
+__global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const ClaBwdParams p)
 {
-    static Setup setup_pw, setup_dw;
+    using L = TcLayout<D>;
+    constexpr int kChunks = D / 8;                       // 16-byte channel chunks per pixel
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + L::kOffMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 4);
+    const uint32_t bar = base + L::kOffBar;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* taps = reinterpret_cast<float*>(sm + L::kOffTaps);
+    float* bdw = reinterpret_cast<float*>(sm + L::kOffBdw);
+    float* bpw = reinterpret_cast<float*>(sm + L::kOffBpw);
+    float* dbs = reinterpret_cast<float*>(sm + L::kOffDb);
+
+    if (threadIdx.x == 0) {
+        abort_flag[0] = 0;
+        mbar_init(bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(base + L::kOffMisc, L::kTmemCols);
+        tmem_relinquish();
+    }
+    // the point-wise matrix as bf16: row = output channel, 64 input channels per 128-byte line, SWIZZLE_128B
+    for (int idx = threadIdx.x; idx < D * kChunks; idx += kTcThreads) {
+        const int n = idx / kChunks, c8 = idx - n * kChunks;
+        const float4 lo = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8));
+        const float4 hi = __ldg(reinterpret_cast<const float4*>(p.w_pw + (size_t)n * D + 8 * c8 + 4));
+        *reinterpret_cast<uint4*>(sm + L::kOffW + (c8 >> 3) * L::kWAtom + n * 128 + (((c8 & 7) ^ (n & 7)) << 4)) =
+            make_uint4(pack_bf16x2(lo.x, lo.y), pack_bf16x2(lo.z, lo.w), pack_bf16x2(hi.x, hi.y), pack_bf16x2(hi.z, hi.w));
+    }
+    for (int idx = threadIdx.x; idx < 9 * D; idx += kTcThreads) taps[idx] = __ldg(p.w_dw + (size_t)(idx % D) * 9 + idx / D);   // tap-major
+    if (threadIdx.x < D) {
+        bdw[threadIdx.x] = __ldg(p.b_dw + threadIdx.x);
+        bpw[threadIdx.x] = __ldg(p.b_pw + threadIdx.x);
+        dbs[threadIdx.x] = 0.f;
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    constexpr uint64_t kDescK = smem_desc_const(16, 1024, kSwizzle128B);                // K-major: 8-row groups 1024 bytes apart
+    constexpr uint64_t kDescWmn = smem_desc_const(L::kWAtom, 1024, kSwizzle128B);       // W read with the input channel as N
+    constexpr uint64_t kDescTmn = smem_desc_const(L::kTAtom, 1024, kSwizzle128B);       // Y, dZ read with the channel as M or N
+    const int quarter = warp & 3, sub = warp >> 2;       // a warp reads accumulator lanes 32 quarter .., column groups sub, sub + 4, ...
+    const int row = quarter * 32 + lane;
+    const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
+    const long long hw = (long long)p.H * p.W;
+    const long long tiles = (p.pixels + kTcPix - 1) / kTcPix;
+    uint32_t ph = 0;                                     // commits waited for so far (all threads wait for every one)
+    // every thread waits for the MMAs committed last; the outcome is made uniform so that the CTA leaves the loop together
+    auto mma_done = [&]() -> bool {
+        const bool w = mbar_wait(bar, ph & 1, abort_flag, p.status);
+        ++ph;
+        const bool all = __syncthreads_and(w) != 0;
+        tc_fence_after();
+        return all;
+    };
+    // hand shared-memory tiles written by the threads and accumulator columns read by them over to the MMA issuer
+    auto hand_over = [&]() {
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    };
+    // dZ = dG o G o (1 - G) for output channels o0 + [0, ncols) from the accumulator columns [0, ncols)
+    auto z_epilogue = [&](long long pix, int o0, int ncols) {
+        for (int g = sub; g < ncols / 16; g += 4) {
+            uint32_t a[16];
+            tmem_ld16(t_lane + 16 * g, a);
+            const int o = o0 + 16 * g;
+            uint4 d0 = make_uint4(0, 0, 0, 0), d1 = d0;
+            if (pix < p.pixels) {
+                d0 = __ldg(reinterpret_cast<const uint4*>(p.dgate + pix * D + o));
+                d1 = __ldg(reinterpret_cast<const uint4*>(p.dgate + pix * D + o + 8));
+            }
+            tmem_wait_ld();
+            const uint32_t dg[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+            float dz[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float z = __uint_as_float(a[k]) + bpw[o + k];
+                const float gt = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z));
+                const float d = (k & 1) ? __uint_as_float(dg[k >> 1] & 0xffff0000u) : __uint_as_float(dg[k >> 1] << 16);
+                dz[k] = d * gt * (1.f - gt);           // zero for rows beyond the last pixel (d = 0)
+            }
+            const int c8 = o >> 3;
+            *reinterpret_cast<uint4*>(sm + L::kOffZ + (c8 >> 3) * L::kTAtom + row * 128 + (((c8 & 7) ^ (row & 7)) << 4)) =
+                make_uint4(pack_bf16x2(dz[0], dz[1]), pack_bf16x2(dz[2], dz[3]), pack_bf16x2(dz[4], dz[5]), pack_bf16x2(dz[6], dz[7]));
+            *reinterpret_cast<uint4*>(sm + L::kOffZ + ((c8 + 1) >> 3) * L::kTAtom + row * 128 + ((((c8 + 1) & 7) ^ (row & 7)) << 4)) =
+                make_uint4(pack_bf16x2(dz[8], dz[9]), pack_bf16x2(dz[10], dz[11]), pack_bf16x2(dz[12], dz[13]), pack_bf16x2(dz[14], dz[15]));
+            // db_pw: sum over the warp's 32 pixels, then one shared-memory add per column
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                float v = dz[k];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                if (lane == 0) atomicAdd(dbs + o + k, v);
+            }
+        }
+    };
+    // dY columns [0, ncols) of the accumulator -> input channels i0 + [0, ncols) of the workspace
+    auto dy_epilogue = [&](long long pix, int i0, int ncols) {
+        for (int g = sub; g < ncols / 16; g += 4) {
+            uint32_t a[16];
+            tmem_ld16(t_lane + 16 * g, a);
+            tmem_wait_ld();
+            if (pix < p.pixels) {
+                float4* dst = reinterpret_cast<float4*>(p.dy + pix * D + i0 + 16 * g);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    dst[k] = make_float4(__uint_as_float(a[4 * k]), __uint_as_float(a[4 * k + 1]), __uint_as_float(a[4 * k + 2]), __uint_as_float(a[4 * k + 3]));
+            }
+        }
+    };
+
+    uint32_t it = 0;
+    bool ok = true;
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
+        const long long pix0 = tile * kTcPix;
+        // ---- Y = DWConv3x3(X) + b_dw as the bf16 tile [pixel][channel]; rows beyond the last pixel are zero
+        for (int idx = threadIdx.x; idx < kTcPix * kChunks; idx += kTcThreads) {
+            const int r = idx / kChunks, c8 = idx - r * kChunks;
+            const long long pix = pix0 + r;
+            float acc[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+            if (pix < p.pixels) {
+                const long long b = pix / hw;
+                const int rem = (int)(pix - b * hw), Y = rem / p.W, X = rem - Y * p.W;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) acc[k] = bdw[8 * c8 + k];
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const int yy = Y + t / 3 - 1, xx = X + t % 3 - 1;
+                    if (yy < 0 || yy >= p.H || xx < 0 || xx >= p.W) continue;
+                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.x + ((b * p.H + yy) * p.W + xx) * D + 8 * c8));
+                    const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
+                    const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
+                    acc[0] = fmaf(__uint_as_float(v.x << 16), w0.x, acc[0]);
+                    acc[1] = fmaf(__uint_as_float(v.x & 0xffff0000u), w0.y, acc[1]);
+                    acc[2] = fmaf(__uint_as_float(v.y << 16), w0.z, acc[2]);
+                    acc[3] = fmaf(__uint_as_float(v.y & 0xffff0000u), w0.w, acc[3]);
+                    acc[4] = fmaf(__uint_as_float(v.z << 16), w1.x, acc[4]);
+                    acc[5] = fmaf(__uint_as_float(v.z & 0xffff0000u), w1.y, acc[5]);
+                    acc[6] = fmaf(__uint_as_float(v.w << 16), w1.z, acc[6]);
+                    acc[7] = fmaf(__uint_as_float(v.w & 0xffff0000u), w1.w, acc[7]);
+                }
+            }
+            *reinterpret_cast<uint4*>(sm + L::kOffY + (c8 >> 3) * L::kTAtom + r * 128 + (((c8 & 7) ^ (r & 7)) << 4)) =
+                make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
+        }
+        hand_over();
+        // ---- Z = Y W_pw^T, output channels [0, N1) then [N1, D), each followed by dZ into its slice of the dZ tile
+#pragma unroll
+        for (int part = 0; part < (L::kN2 ? 2 : 1); ++part) {
+            const int o0 = part ? L::kN1 : 0, ncols = part ? L::kN2 : L::kN1;
+            if (warp == 0 && elect_one()) {
+                const uint32_t idesc = idesc_bf16_f32(kTcPix, ncols, false);
+#pragma unroll
+                for (int a = 0; a < L::kAtoms; ++a) {
+                    const uint64_t da = smem_desc_at(kDescK, base + L::kOffY + a * L::kTAtom);
+                    const uint64_t db = smem_desc_at(kDescK, base + L::kOffW + a * L::kWAtom + o0 * 128);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) mma_ss(tmem, da + 2 * kk, db + 2 * kk, idesc, (a | kk) ? 1u : 0u);
+                }
+                mma_commit(bar);
+            }
+            __syncwarp();
+            if (!mma_done()) { ok = false; break; }
+            z_epilogue(pix0 + row, o0, ncols);
+            hand_over();
+        }
+        if (!ok) break;
+        // ---- dY = dZ W_pw, input channels [0, N1), together with dW_pw += dZ^T Y; then input channels [N1, D)
+#pragma unroll
+        for (int part = 0; part < (L::kN2 ? 2 : 1); ++part) {
+            const int i0 = part ? L::kN1 : 0, ncols = part ? L::kN2 : L::kN1;
+            if (warp == 0 && elect_one()) {
+                const uint32_t idesc = idesc_bf16_f32_ab(kTcPix, ncols, false, true);
+                const uint64_t db = smem_desc_at(kDescWmn, base + L::kOffW + (i0 / 64) * L::kWAtom);
+#pragma unroll
+                for (int a = 0; a < L::kAtoms; ++a) {
+                    const uint64_t da = smem_desc_at(kDescK, base + L::kOffZ + a * L::kTAtom);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)       // 16 output channels per step: 32 bytes along A's rows, 16 rows of W
+                        mma_ss(tmem, da + 2 * kk, db + 128 * (4 * a + kk), idesc, (a | kk) ? 1u : 0u);
+                }
+                if (part == 0) {
+                    constexpr uint32_t idesc_w = idesc_bf16_f32_ab(128, D, true, true);
+                    const uint64_t dy = smem_desc_at(kDescTmn, base + L::kOffY);
+#pragma unroll
+                    for (int blk = 0; blk < L::kBlocks; ++blk) {
+                        // rows of block 1 are the output channels [D - 128, D): it starts one 64-channel slice further
+                        const uint64_t dzm = smem_desc_at(kDescTmn, base + L::kOffZ + blk * (L::kAtoms - 2) * L::kTAtom);
+#pragma unroll
+                        for (int kk = 0; kk < kTcPix / 16; ++kk)     // 16 pixels per step
+                            mma_ss(tmem + L::kColW + blk * D, dzm + 128 * kk, dy + 128 * kk, idesc_w, (it | kk) ? 1u : 0u);
+                    }
+                }
+                mma_commit(bar);
+            }
+            __syncwarp();
+            if (!mma_done()) { ok = false; break; }
+            dy_epilogue(pix0 + row, i0, ncols);
+            hand_over();
+        }
+        if (!ok) break;
+    }
+    // ---- flush dW_pw (accumulated over the CTA's tiles) and db_pw
+    if (ok && it > 0) {
+#pragma unroll
+        for (int blk = 0; blk < L::kBlocks; ++blk) {
+            // block 0: rows are output channels 0 .. min(D, 128) - 1; block 1: channels D - 128 + row, of which the upper
+            // half (rows 64 .. 127) is new
+            const int o = blk ? D - 128 + row : row;
+            const bool mine = blk ? row >= 64 : row < D;
+            for (int g = sub; g < D / 16; g += 4) {
+                uint32_t a[16];
+                tmem_ld16(t_lane + L::kColW + blk * D + 16 * g, a);
+                tmem_wait_ld();
+                if (mine) {
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) atomicAdd(p.dw_pw + (size_t)o * D + 16 * g + k, __uint_as_float(a[k]));
+                }
+            }
+        }
+        if (threadIdx.x < D) atomicAdd(p.db_pw + threadIdx.x, dbs[threadIdx.x]);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, L::kTmemCols);
+    }
+}
+
+template <int D>
+cudaError_t launch_gate_bwd(const ClaBwdParams& p, bool tensor_cores, cudaStream_t stream)
+{
+    static sm100::KernelSetup setup_pw, setup_dw, setup_tc;
     constexpr size_t kSmem = (size_t)(2 * kTilePix * D + 10 * D) * sizeof(float);
     int sms = 0;
-    if (cudaError_t e = setup_pw.prepare(rib_cla_bwd_pw_kernel<D>, kSmem, &sms)) return e;
+    if (cudaError_t e = setup_pw.prepare(rib_cla_bwd_pw_kernel<D>, (uint32_t)kSmem, &sms)) return e;
     if (cudaError_t e = setup_dw.prepare(rib_cla_bwd_dw_kernel<D>, 0, &sms)) return e;
+    if (cudaError_t e = setup_tc.prepare(rib_cla_bwd_tc_kernel<D>, TcLayout<D>::kSmemBytes, &sms)) return e;
     cudaError_t e = cudaMemsetAsync(p.dw_dw, 0, sizeof(float) * 9 * D, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(p.db_dw, 0, sizeof(float) * D, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(p.dw_pw, 0, sizeof(float) * D * D, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(p.db_pw, 0, sizeof(float) * D, stream);
     if (e != cudaSuccess) return e;
-    rib_cla_transpose_kernel<<<(D * D + 255) / 256, 256, 0, stream>>>(p.w_pw, const_cast<float*>(p.w_pw_t), D);
-    const long long tiles = (p.pixels + kTilePix - 1) / kTilePix;
-    {
+    if (tensor_cores) {
+        const long long tiles = (p.pixels + kTcPix - 1) / kTcPix;
+        ProfileScope scope(RIB_KERNEL_CLA_BWD_TC, stream);
+        rib_cla_bwd_tc_kernel<D><<<(unsigned)(tiles < sms ? tiles : sms), kTcThreads, TcLayout<D>::kSmemBytes, stream>>>(p);
+    } else {
+        rib_cla_transpose_kernel<<<(D * D + 255) / 256, 256, 0, stream>>>(p.w_pw, const_cast<float*>(p.w_pw_t), D);
+        const long long tiles = (p.pixels + kTilePix - 1) / kTilePix;
         ProfileScope scope(RIB_KERNEL_CLA_BWD_PW, stream);
         rib_cla_bwd_pw_kernel<D><<<(unsigned)(tiles < sms ? tiles : sms), kPwThreads, kSmem, stream>>>(p);
     }
@@ -359,9 +616,10 @@ size_t cla_gate_bwd_workspace_bytes(long long pixels, int D)
 
 cudaError_t cla_gate_bwd(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
                          const __nv_bfloat16* dgate, int B, int H, int W, int D, __nv_bfloat16* dx, float* dw_dw, float* db_dw,
-                         float* dw_pw, float* db_pw, void* workspace, cudaStream_t stream)
+                         float* dw_pw, float* db_pw, void* workspace, bool tensor_cores, int* status, cudaStream_t stream)
 {
     ClaBwdParams p{};
+    p.status = status;
     p.x = x; p.w_dw = w_dw; p.b_dw = b_dw; p.w_pw = w_pw; p.b_pw = b_pw; p.dgate = dgate;
     p.dx = dx; p.dw_dw = dw_dw; p.db_dw = db_dw; p.dw_pw = dw_pw; p.db_pw = db_pw;
     p.B = B; p.H = H; p.W = W;
@@ -369,9 +627,9 @@ cudaError_t cla_gate_bwd(const __nv_bfloat16* x, const float* w_dw, const float*
     p.dy = static_cast<float*>(workspace);
     p.w_pw_t = p.dy + (size_t)p.pixels * D;
     switch (D) {
-        case 64: return launch_gate_bwd<64>(p, stream);
-        case 128: return launch_gate_bwd<128>(p, stream);
-        case 192: return launch_gate_bwd<192>(p, stream);
+        case 64: return launch_gate_bwd<64>(p, tensor_cores, stream);
+        case 128: return launch_gate_bwd<128>(p, tensor_cores, stream);
+        case 192: return launch_gate_bwd<192>(p, tensor_cores, stream);
         default: return cudaErrorNotSupported;
     }
 }

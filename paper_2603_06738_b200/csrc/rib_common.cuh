@@ -67,7 +67,7 @@ bool cla_gate_bwd_supported(int D);
 size_t cla_gate_bwd_workspace_bytes(long long pixels, int D);
 cudaError_t cla_gate_bwd(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
                          const __nv_bfloat16* dgate, int B, int H, int W, int D, __nv_bfloat16* dx, float* dw_dw, float* db_dw,
-                         float* dw_pw, float* db_pw, void* workspace, cudaStream_t stream);
+                         float* dw_pw, float* db_pw, void* workspace, bool tensor_cores, int* status, cudaStream_t stream);
 cudaError_t cla_product(const __nv_bfloat16* out, const __nv_bfloat16* gate, const __nv_bfloat16* dout_gated, long long count,
                         __nv_bfloat16* res0, __nv_bfloat16* res1, cudaStream_t stream);
 

@@ -106,18 +106,30 @@ def dgate_input(seed, shape):
     return synthetic.bf16_tensor(seed, "gate", shape, 1.0)
 
 
+@pytest.mark.parametrize("path", ["auto", "generic"])
 @pytest.mark.parametrize("B,H,W,D", [(1, 5, 7, 64), (2, 16, 32, 192), (1, 24, 47, 128), (3, 9, 16, 192), (1, 1, 1, 64),
-                                     (1, 96, 96, 192)])
-def test_gate_backward_matches_the_oracle(B, H, W, D):
+                                     (1, 96, 96, 192), (2, 40, 56, 64)])
+def test_gate_backward_matches_the_oracle(B, H, W, D, path):
     x, ws = gate_inputs(300 + D + H, B, H, W, D)
     dgate = dgate_input(301 + D + H, (B, H, W, D))
-    got = binding.rib_cla_gate_bwd(x.cuda(), *[torch.from_numpy(w).cuda() for w in ws], dgate.cuda())
+    binding.rib_set_path(binding.RIB_PATH_GENERIC if path == "generic" else binding.RIB_PATH_NONE)
+    try:
+        got = binding.rib_cla_gate_bwd(x.cuda(), *[torch.from_numpy(w).cuda() for w in ws], dgate.cuda())
+        used = binding.rib_last_path()
+    finally:
+        binding.rib_set_path(binding.RIB_PATH_NONE)
     torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0
+    assert used == (binding.RIB_PATH_GENERIC if path == "generic" else binding.RIB_PATH_SM100)
     ref = cla.gate_bwd(to_f64(x), *ws, to_f64(dgate))
     compare("dx", to_f64(got[0]), ref[0], max_abs=1e-2 * max(1.0, np.abs(ref[0]).max()))
-    # fp32 sums of fp32 products over the pixels, against float64
     for name, g, r in zip(("dw_dw", "db_dw", "dw_pw", "db_pw"), got[1:], ref[1:]):
-        compare(name, to_f64(g), r, max_abs=1e-3 * max(1.0, np.abs(r).max()), rel_l2=1e-4)
+        if path == "generic":
+            # fp32 products and fp32 sums over the pixels, against float64
+            compare(name, to_f64(g), r, max_abs=1e-3 * max(1.0, np.abs(r).max()), rel_l2=1e-4)
+        else:
+            # Y, dZ and the point-wise matrix enter the MMAs as bf16 (fp32 accumulation): the bar of the attention outputs
+            compare(name, to_f64(g), r, max_abs=1e-2 * max(1.0, np.abs(r).max()), rel_l2=5e-3)
 
 
 def test_gate_backward_overwrites_its_outputs_and_repeats():
