@@ -246,56 +246,83 @@ __global__ void __launch_bounds__(kPwThreads, 1) rib_cla_bwd_pw_kernel(const Cla
 }
 
 // ------------------------------------------------------------------------------------------------------------------
-// Depth-wise part: thread (c, lane) walks pixels lane, lane + stride, ...; channel c.
+// Depth-wise part.  A block takes a tile of 8 x 16 pixels and 64 channels: the 10 x 18 halo of dY (fp32) and of X (bf16)
+// goes to shared memory (zero outside the map), thread (channel, lane) walks 16 pixels of the tile.
 // ------------------------------------------------------------------------------------------------------------------
-constexpr int kDwLanes = 4;
+constexpr int kDwTileH = 8, kDwTileW = 16, kDwHaloH = kDwTileH + 2, kDwHaloW = kDwTileW + 2, kDwHalo = kDwHaloH * kDwHaloW;
+constexpr int kDwCh = 64, kDwLanes = 8;
+constexpr int kDwSmemBytes = kDwHalo * kDwCh * 6 + kDwLanes * 10 * kDwCh * 4;
 
 template <int D>
-__global__ void __launch_bounds__(D * kDwLanes) rib_cla_bwd_dw_kernel(const ClaBwdParams p)
+__global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const ClaBwdParams p, int tiles_y, int tiles_x)
 {
-    __shared__ float red[kDwLanes][10][D];
-    const int c = threadIdx.x, lane = threadIdx.y;
+    extern __shared__ __align__(16) uint8_t dw_smem[];
+    float* dys = reinterpret_cast<float*>(dw_smem);                                        // [180][64]
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(dw_smem + kDwHalo * kDwCh * 4);   // [180][64]
+    float* red = reinterpret_cast<float*>(dw_smem + kDwHalo * kDwCh * 6);                  // [8 lanes][10][64]
+    const int c = threadIdx.x, lane = threadIdx.y, tid = lane * kDwCh + c;
+    constexpr int kGroups = D / kDwCh;
+    int tile = blockIdx.x;
+    const int cg = tile % kGroups; tile /= kGroups;
+    const int tx = tile % tiles_x; tile /= tiles_x;
+    const int ty = tile % tiles_y, b = tile / tiles_y;
+    const int y0 = ty * kDwTileH, x0 = tx * kDwTileW, ch0 = cg * kDwCh;
+    // halo: 16 threads per pixel (4 channels each), 32 pixels per pass
+    for (int idx = tid; idx < kDwHalo * 16; idx += kDwCh * kDwLanes) {
+        const int hp = idx >> 4, c4 = (idx & 15) * 4;
+        const int yy = y0 + hp / kDwHaloW - 1, xx = x0 + hp % kDwHaloW - 1;
+        float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);
+        uint2 xv = make_uint2(0, 0);
+        if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W) {
+            const size_t g = (((size_t)b * p.H + yy) * p.W + xx) * D + ch0 + c4;
+            dv = __ldg(reinterpret_cast<const float4*>(p.dy + g));
+            xv = __ldg(reinterpret_cast<const uint2*>(p.x + g));
+        }
+        *reinterpret_cast<float4*>(dys + hp * kDwCh + c4) = dv;
+        *reinterpret_cast<uint2*>(xs + hp * kDwCh + c4) = xv;
+    }
     float w[9];
 #pragma unroll
-    for (int t = 0; t < 9; ++t) w[t] = p.w_dw[c * 9 + t];
+    for (int t = 0; t < 9; ++t) w[t] = p.w_dw[(ch0 + c) * 9 + t];
     float gw[9], gb = 0.f;
 #pragma unroll
     for (int t = 0; t < 9; ++t) gw[t] = 0.f;
-    const long long hw = (long long)p.H * p.W;
-    for (long long pix = (long long)blockIdx.x * kDwLanes + lane; pix < p.pixels; pix += (long long)gridDim.x * kDwLanes) {
-        const long long b = pix / hw;
-        const int rem = (int)(pix - b * hw), Y = rem / p.W, X = rem - Y * p.W;
-        const float dy_here = p.dy[pix * D + c];
-        gb += dy_here;
-        float dx = 0.f;
+    __syncthreads();
+    // lane l takes tile row l: 16 pixels
+    const int py = lane;
+    if (y0 + py < p.H) {
+#pragma unroll 4
+        for (int px = 0; px < kDwTileW; ++px) {
+            if (x0 + px >= p.W) break;
+            const int hc = (py + 1) * kDwHaloW + px + 1;                  // this pixel in the halo
+            const float dy_here = dys[hc * kDwCh + c];
+            gb += dy_here;
+            float dx = 0.f;
 #pragma unroll
-        for (int ky = 0; ky < 3; ++ky) {
+            for (int ky = 0; ky < 3; ++ky) {
 #pragma unroll
-            for (int kx = 0; kx < 3; ++kx) {
-                // forward: Y[y, x] reads X[y + ky - 1, x + kx - 1] through tap (ky, kx)
-                const int yf = Y + ky - 1, xf = X + kx - 1;          // the input this output pixel read
-                if (yf >= 0 && yf < p.H && xf >= 0 && xf < p.W)
-                    gw[ky * 3 + kx] = fmaf(dy_here, __bfloat162float(p.x[((b * p.H + yf) * p.W + xf) * D + c]), gw[ky * 3 + kx]);
-                const int yb = Y - ky + 1, xb = X - kx + 1;          // the output pixel that read this input
-                if (yb >= 0 && yb < p.H && xb >= 0 && xb < p.W)
-                    dx = fmaf(p.dy[((b * p.H + yb) * p.W + xb) * D + c], w[ky * 3 + kx], dx);
+                for (int kx = 0; kx < 3; ++kx) {
+                    // forward: Y[y, x] reads X[y + ky - 1, x + kx - 1] through tap (ky, kx); X is zero outside the map
+                    gw[ky * 3 + kx] = fmaf(dy_here, __bfloat162float(xs[(hc + (ky - 1) * kDwHaloW + kx - 1) * kDwCh + c]), gw[ky * 3 + kx]);
+                    // so X[y, x] was read by the output pixel (y - ky + 1, x - kx + 1); dY is zero outside the map
+                    dx = fmaf(dys[(hc - (ky - 1) * kDwHaloW - (kx - 1)) * kDwCh + c], w[ky * 3 + kx], dx);
+                }
             }
+            p.dx[(((size_t)b * p.H + y0 + py) * p.W + x0 + px) * D + ch0 + c] = __float2bfloat16_rn(dx);
         }
-        p.dx[pix * D + c] = __float2bfloat16_rn(dx);
     }
 #pragma unroll
-    for (int t = 0; t < 9; ++t) red[lane][t][c] = gw[t];
-    red[lane][9][c] = gb;
+    for (int t = 0; t < 9; ++t) red[(lane * 10 + t) * kDwCh + c] = gw[t];
+    red[(lane * 10 + 9) * kDwCh + c] = gb;
     __syncthreads();
-    if (lane == 0) {
+    // 640 sums of 8 lanes
+    for (int idx = tid; idx < 10 * kDwCh; idx += kDwCh * kDwLanes) {
+        const int t = idx / kDwCh, cc = idx - t * kDwCh;
+        float sum = 0.f;
 #pragma unroll
-        for (int t = 0; t < 10; ++t) {
-            float s = 0.f;
-#pragma unroll
-            for (int l = 0; l < kDwLanes; ++l) s += red[l][t][c];
-            if (t < 9) atomicAdd(p.dw_dw + c * 9 + t, s);
-            else atomicAdd(p.db_dw + c, s);
-        }
+        for (int l = 0; l < kDwLanes; ++l) sum += red[(l * 10 + t) * kDwCh + cc];
+        if (t < 9) atomicAdd(p.dw_dw + (ch0 + cc) * 9 + t, sum);
+        else atomicAdd(p.db_dw + ch0 + cc, sum);
     }
 }
 
@@ -579,7 +606,7 @@ cudaError_t launch_gate_bwd(const ClaBwdParams& p, bool tensor_cores, cudaStream
     constexpr size_t kSmem = (size_t)(2 * kTilePix * D + 10 * D) * sizeof(float);
     int sms = 0;
     if (cudaError_t e = setup_pw.prepare(rib_cla_bwd_pw_kernel<D>, (uint32_t)kSmem, &sms)) return e;
-    if (cudaError_t e = setup_dw.prepare(rib_cla_bwd_dw_kernel<D>, 0, &sms)) return e;
+    if (cudaError_t e = setup_dw.prepare(rib_cla_bwd_dw_kernel<D>, kDwSmemBytes, &sms)) return e;
     if (cudaError_t e = setup_tc.prepare(rib_cla_bwd_tc_kernel<D>, TcLayout<D>::kSmemBytes, &sms)) return e;
     cudaError_t e = cudaMemsetAsync(p.dw_dw, 0, sizeof(float) * 9 * D, stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(p.db_dw, 0, sizeof(float) * D, stream);
@@ -598,9 +625,10 @@ cudaError_t launch_gate_bwd(const ClaBwdParams& p, bool tensor_cores, cudaStream
     }
     {
         ProfileScope scope(RIB_KERNEL_CLA_BWD_DW, stream);
-        const long long want = (p.pixels + kDwLanes - 1) / kDwLanes;
-        const long long cap = (long long)sms * (D <= 64 ? 8 : D <= 128 ? 4 : 2);
-        rib_cla_bwd_dw_kernel<D><<<(unsigned)(want < cap ? want : cap), dim3(D, kDwLanes), 0, stream>>>(p);
+        const int tiles_y = (p.H + kDwTileH - 1) / kDwTileH, tiles_x = (p.W + kDwTileW - 1) / kDwTileW;
+        const long long blocks = (long long)p.B * tiles_y * tiles_x * (D / kDwCh);
+        if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+        rib_cla_bwd_dw_kernel<D><<<(unsigned)blocks, dim3(kDwCh, kDwLanes), kDwSmemBytes, stream>>>(p, tiles_y, tiles_x);
     }
     return cudaGetLastError();
 }
