@@ -350,6 +350,8 @@ struct TcLayout {
     static constexpr uint32_t kOffMisc = kOffBar + 16;
     static constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;
     static_assert(kOffZ % 1024 == 0 && kOffY % 1024 == 0 && kWAtom % 1024 == 0, "swizzle atoms need aligned tiles");
+    // the final flush stages 128 rows of D + 4 floats over the dZ and Y tiles and the first bytes of the taps
+    static_assert(kTcPix * (D + 4) * 4 <= 2 * kAtoms * kTAtom + 9 * D * 4, "flush staging must end before the biases and sums");
     // tensor memory: [0, 128) Z and dY, 128 columns at a time; then dW_pw as one or two blocks of 128 rows x D columns
     static constexpr int kN1 = D < 128 ? D : 128, kN2 = D - kN1;           // column split of Z and dY
     static constexpr int kBlocks = D > 128 ? 2 : 1;                        // dW_pw rows [0, 128) and [D - 128, D)
@@ -492,23 +494,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
             if (pix < p.pixels) {
                 const long long b = pix / hw;
                 const int rem = (int)(pix - b * hw), Y = rem / p.W, X = rem - Y * p.W;
+                const __nv_bfloat16* centre = p.x + pix * D + 8 * c8;
+                uint4 v[9];                              // all nine loads are in flight before the first is used
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const int dyy = t / 3 - 1, dxx = t % 3 - 1;
+                    const bool in = Y + dyy >= 0 && Y + dyy < p.H && X + dxx >= 0 && X + dxx < p.W;
+                    v[t] = in ? __ldg(reinterpret_cast<const uint4*>(centre + ((long long)dyy * p.W + dxx) * D)) : make_uint4(0, 0, 0, 0);
+                }
 #pragma unroll
                 for (int k = 0; k < 8; ++k) acc[k] = bdw[8 * c8 + k];
 #pragma unroll
                 for (int t = 0; t < 9; ++t) {
-                    const int yy = Y + t / 3 - 1, xx = X + t % 3 - 1;
-                    if (yy < 0 || yy >= p.H || xx < 0 || xx >= p.W) continue;
-                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.x + ((b * p.H + yy) * p.W + xx) * D + 8 * c8));
                     const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
                     const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
-                    acc[0] = fmaf(__uint_as_float(v.x << 16), w0.x, acc[0]);
-                    acc[1] = fmaf(__uint_as_float(v.x & 0xffff0000u), w0.y, acc[1]);
-                    acc[2] = fmaf(__uint_as_float(v.y << 16), w0.z, acc[2]);
-                    acc[3] = fmaf(__uint_as_float(v.y & 0xffff0000u), w0.w, acc[3]);
-                    acc[4] = fmaf(__uint_as_float(v.z << 16), w1.x, acc[4]);
-                    acc[5] = fmaf(__uint_as_float(v.z & 0xffff0000u), w1.y, acc[5]);
-                    acc[6] = fmaf(__uint_as_float(v.w << 16), w1.z, acc[6]);
-                    acc[7] = fmaf(__uint_as_float(v.w & 0xffff0000u), w1.w, acc[7]);
+                    acc[0] = fmaf(__uint_as_float(v[t].x << 16), w0.x, acc[0]);
+                    acc[1] = fmaf(__uint_as_float(v[t].x & 0xffff0000u), w0.y, acc[1]);
+                    acc[2] = fmaf(__uint_as_float(v[t].y << 16), w0.z, acc[2]);
+                    acc[3] = fmaf(__uint_as_float(v[t].y & 0xffff0000u), w0.w, acc[3]);
+                    acc[4] = fmaf(__uint_as_float(v[t].z << 16), w1.x, acc[4]);
+                    acc[5] = fmaf(__uint_as_float(v[t].z & 0xffff0000u), w1.y, acc[5]);
+                    acc[6] = fmaf(__uint_as_float(v[t].w << 16), w1.z, acc[6]);
+                    acc[7] = fmaf(__uint_as_float(v[t].w & 0xffff0000u), w1.w, acc[7]);
                 }
             }
             *reinterpret_cast<uint4*>(sm + L::kOffY + (c8 >> 3) * L::kTAtom + r * 128 + (((c8 & 7) ^ (r & 7)) << 4)) =
@@ -573,21 +580,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
     }
     // ---- flush dW_pw (accumulated over the CTA's tiles) and db_pw
     if (ok && it > 0) {
+        // through shared memory (the dZ and Y tiles are free now; rows padded by 4 floats), so that a warp adds 32
+        // consecutive columns of one row: one 128-byte request instead of 32 scattered ones
+        float* stage = reinterpret_cast<float*>(sm + L::kOffZ);
+        constexpr int kStride = D + 4;
 #pragma unroll
         for (int blk = 0; blk < L::kBlocks; ++blk) {
-            // block 0: rows are output channels 0 .. min(D, 128) - 1; block 1: channels D - 128 + row, of which the upper
-            // half (rows 64 .. 127) is new
-            const int o = blk ? D - 128 + row : row;
-            const bool mine = blk ? row >= 64 : row < D;
             for (int g = sub; g < D / 16; g += 4) {
                 uint32_t a[16];
                 tmem_ld16(t_lane + L::kColW + blk * D + 16 * g, a);
                 tmem_wait_ld();
-                if (mine) {
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) atomicAdd(p.dw_pw + (size_t)o * D + 16 * g + k, __uint_as_float(a[k]));
-                }
+                for (int k = 0; k < 4; ++k)
+                    *reinterpret_cast<float4*>(stage + row * kStride + 16 * g + 4 * k) =
+                        make_float4(__uint_as_float(a[4 * k]), __uint_as_float(a[4 * k + 1]), __uint_as_float(a[4 * k + 2]), __uint_as_float(a[4 * k + 3]));
             }
+            __syncthreads();
+            // block 0: rows are output channels 0 .. min(D, 128) - 1; block 1: channels D - 128 + row, of which the upper
+            // half (rows 64 .. 127) is new
+            constexpr int kRow0 = 0;
+            const int first = blk ? 64 : kRow0, count = blk ? 64 : (D < 128 ? D : 128), o0 = blk ? D - 128 : 0;
+            for (int idx = threadIdx.x; idx < count * D; idx += kTcThreads) {
+                const int r = first + idx / D, col = idx % D;
+                atomicAdd(p.dw_pw + (size_t)(o0 + r) * D + col, stage[r * kStride + col]);
+            }
+            __syncthreads();
         }
         if (threadIdx.x < D) atomicAdd(p.db_pw + threadIdx.x, dbs[threadIdx.x]);
     }
