@@ -455,14 +455,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
                 make_uint4(pack_bf16x2(dz[0], dz[1]), pack_bf16x2(dz[2], dz[3]), pack_bf16x2(dz[4], dz[5]), pack_bf16x2(dz[6], dz[7]));
             *reinterpret_cast<uint4*>(sm + L::kOffZ + ((c8 + 1) >> 3) * L::kTAtom + row * 128 + ((((c8 + 1) & 7) ^ (row & 7)) << 4)) =
                 make_uint4(pack_bf16x2(dz[8], dz[9]), pack_bf16x2(dz[10], dz[11]), pack_bf16x2(dz[12], dz[13]), pack_bf16x2(dz[14], dz[15]));
-            // db_pw: sum over the warp's 32 pixels, then one shared-memory add per column
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                float v = dz[k];
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-                if (lane == 0) atomicAdd(dbs + o + k, v);
-            }
         }
     };
     // dY columns [0, ncols) of the accumulator -> input channels i0 + [0, ncols) of the workspace
@@ -485,6 +477,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
         const long long pix0 = tile * kTcPix;
         // ---- Y = DWConv3x3(X) + b_dw as the bf16 tile [pixel][channel]; rows beyond the last pixel are zero
+#pragma unroll 2
         for (int idx = threadIdx.x; idx < kTcPix * kChunks; idx += kTcThreads) {
             const int r = idx / kChunks, c8 = idx - r * kChunks;
             const long long pix = pix0 + r;
@@ -572,6 +565,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
                 mma_commit(bar);
             }
             __syncwarp();
+            if (part == 0 && threadIdx.x < 2 * D) {
+                // db_pw while the MMAs run: thread (column, half) sums 64 rows of the dZ tile (rows beyond the last pixel
+                // hold zeros)
+                const int col = threadIdx.x % D, r0 = (threadIdx.x / D) * (kTcPix / 2), c8 = col >> 3;
+                const uint8_t* src = sm + L::kOffZ + (c8 >> 3) * L::kTAtom + (col & 7) * 2;
+                float sum = 0.f;
+#pragma unroll 8
+                for (int r = r0; r < r0 + kTcPix / 2; ++r)
+                    sum += __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(src + r * 128 + (((c8 & 7) ^ (r & 7)) << 4)));
+                atomicAdd(dbs + col, sum);
+            }
             if (!mma_done()) { ok = false; break; }
             dy_epilogue(pix0 + row, i0, ncols);
             hand_over();
