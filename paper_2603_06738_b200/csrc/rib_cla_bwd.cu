@@ -267,19 +267,34 @@ __global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const 
     const int tx = tile % tiles_x; tile /= tiles_x;
     const int ty = tile % tiles_y, b = tile / tiles_y;
     const int y0 = ty * kDwTileH, x0 = tx * kDwTileW, ch0 = cg * kDwCh;
-    // halo: 16 threads per pixel (4 channels each), 32 pixels per pass
-    for (int idx = tid; idx < kDwHalo * 16; idx += kDwCh * kDwLanes) {
-        const int hp = idx >> 4, c4 = (idx & 15) * 4;
-        const int yy = y0 + hp / kDwHaloW - 1, xx = x0 + hp % kDwHaloW - 1;
-        float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);
-        uint2 xv = make_uint2(0, 0);
-        if (yy >= 0 && yy < p.H && xx >= 0 && xx < p.W) {
-            const size_t g = (((size_t)b * p.H + yy) * p.W + xx) * D + ch0 + c4;
-            dv = __ldg(reinterpret_cast<const float4*>(p.dy + g));
-            xv = __ldg(reinterpret_cast<const uint2*>(p.x + g));
+    // halo: 16 threads per pixel (4 channels each), 32 pixels per pass; all loads of a thread are issued before the
+    // first store, so the prologue costs one memory latency
+    {
+        constexpr int kItems = kDwHalo * 16, kIters = (kItems + kDwCh * kDwLanes - 1) / (kDwCh * kDwLanes);
+        float4 dv[kIters];
+        uint2 xv[kIters];
+#pragma unroll
+        for (int u = 0; u < kIters; ++u) {
+            const int idx = tid + u * kDwCh * kDwLanes;
+            const int hp = idx >> 4, c4 = (idx & 15) * 4;
+            const int yy = y0 + hp / kDwHaloW - 1, xx = x0 + hp % kDwHaloW - 1;
+            dv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            xv[u] = make_uint2(0, 0);
+            if (idx < kItems && yy >= 0 && yy < p.H && xx >= 0 && xx < p.W) {
+                const size_t g = (((size_t)b * p.H + yy) * p.W + xx) * D + ch0 + c4;
+                dv[u] = __ldg(reinterpret_cast<const float4*>(p.dy + g));
+                xv[u] = __ldg(reinterpret_cast<const uint2*>(p.x + g));
+            }
         }
-        *reinterpret_cast<float4*>(dys + hp * kDwCh + c4) = dv;
-        *reinterpret_cast<uint2*>(xs + hp * kDwCh + c4) = xv;
+#pragma unroll
+        for (int u = 0; u < kIters; ++u) {
+            const int idx = tid + u * kDwCh * kDwLanes;
+            if (idx < kItems) {
+                const int hp = idx >> 4, c4 = (idx & 15) * 4;
+                *reinterpret_cast<float4*>(dys + hp * kDwCh + c4) = dv[u];
+                *reinterpret_cast<uint2*>(xs + hp * kDwCh + c4) = xv[u];
+            }
+        }
     }
     float w[9];
 #pragma unroll
