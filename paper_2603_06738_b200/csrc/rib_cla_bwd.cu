@@ -1,7 +1,7 @@
 // Backward pass of Convolutional Local Attention (Sec. 3.2): the chain rule of
 //     G = sigmoid(PWConv(DWConv3x3(X)))   (Eq. 8)        and        O' = O o G   (Eq. 9).
 //
-// Three kinds of kernel, all fp32 arithmetic on bf16 activations:
+// Four kernels on bf16 activations (fp32 arithmetic except for the bf16 operands of the MMAs):
 //   rib_cla_product_kernel      O' = O o G, or (dO, dG) = (dO' o G, dO' o O): element-wise, HBM-bound.
 //   rib_cla_bwd_pw_kernel       per tile of 64 pixels: recomputes Y = DWConv3x3(X) and Z = PWConv(Y), forms
 //                               dZ = dG o G o (1 - G), writes dY = dZ W_pw to the workspace, and keeps the running sums
