@@ -368,7 +368,7 @@ struct TcLayout {
     // the final flush stages 128 rows of D + 4 floats over the dZ and Y tiles and the first bytes of the taps
     static_assert(kTcPix * (D + 4) * 4 <= 2 * kAtoms * kTAtom + 9 * D * 4, "flush staging must end before the biases and sums");
     // tensor memory: [0, 128) Z and dY, 128 columns at a time; then dW_pw as one or two blocks of 128 rows x D columns
-    static constexpr int kN1 = D < 128 ? D : 128, kN2 = D - kN1;           // column split of Z and dY
+    static constexpr int kN1 = D < 128 ? D : 128, kN2 = D - kN1;           // column split of Z and dY (at most 8 groups of 16 per part)
     static constexpr int kBlocks = D > 128 ? 2 : 1;                        // dW_pw rows [0, 128) and [D - 128, D)
     static constexpr uint32_t kColW = 128;
     static constexpr uint32_t kTmemCols = kColW + kBlocks * D <= 256 ? 256 : 512;
@@ -445,16 +445,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
         tc_fence_after();
     };
     // dZ = dG o G o (1 - G) for output channels o0 + [0, ncols) from the accumulator columns [0, ncols)
-    auto z_epilogue = [&](long long pix, int o0, int ncols) {
-        for (int g = sub; g < ncols / 16; g += 4) {
+    // the thread's dG values of one column part (at most two groups of 16), requested before the wait for the MMAs
+    auto dg_load = [&](long long pix, int o0, int ncols, uint4 (&dgv)[4]) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int g = sub + 4 * j;
+            dgv[2 * j] = dgv[2 * j + 1] = make_uint4(0, 0, 0, 0);
+            if (g < ncols / 16 && pix < p.pixels) {
+                dgv[2 * j] = __ldg(reinterpret_cast<const uint4*>(p.dgate + pix * D + o0 + 16 * g));
+                dgv[2 * j + 1] = __ldg(reinterpret_cast<const uint4*>(p.dgate + pix * D + o0 + 16 * g + 8));
+            }
+        }
+    };
+    auto z_epilogue = [&](int o0, int ncols, const uint4 (&dgv)[4]) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int g = sub + 4 * j;
+            if (g >= ncols / 16) break;
             uint32_t a[16];
             tmem_ld16(t_lane + 16 * g, a);
             const int o = o0 + 16 * g;
-            uint4 d0 = make_uint4(0, 0, 0, 0), d1 = d0;
-            if (pix < p.pixels) {
-                d0 = __ldg(reinterpret_cast<const uint4*>(p.dgate + pix * D + o));
-                d1 = __ldg(reinterpret_cast<const uint4*>(p.dgate + pix * D + o + 8));
-            }
+            const uint4 d0 = dgv[2 * j], d1 = dgv[2 * j + 1];
             tmem_wait_ld();
             const uint32_t dg[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
             float dz[16];
@@ -546,8 +557,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
                 mma_commit(bar);
             }
             __syncwarp();
+            uint4 dgv[4];
+            dg_load(pix0 + row, o0, ncols, dgv);
             if (!mma_done()) { ok = false; break; }
-            z_epilogue(pix0 + row, o0, ncols);
+            z_epilogue(o0, ncols, dgv);
             hand_over();
         }
         if (!ok) break;

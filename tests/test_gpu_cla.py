@@ -169,3 +169,33 @@ def test_gate_backward_rejects_unsupported_channels_without_launching():
     assert lib.rib_cla_gate_bwd(x.data_ptr(), *[w.data_ptr()] * 4, x.data_ptr(), 1, 4, 4, 96, x.data_ptr(), *[w.data_ptr()] * 4,
                                 w.data_ptr(), 1 << 18, None) == -3
     assert binding.rib_kernel_launches() == launches
+
+
+def test_training_chain_matches_the_oracles_chained():
+    """Features -> gate, attention -> out, out o gate, and the whole way back on the GPU, against the oracles chained in
+    float64 (no intermediate rounded to bf16 on the oracle's side)."""
+    from oracle import rib_oracle as orc
+    wl = Workload("cla_train_chain", 2, 32, 48, 2, 32, 16, 16, 8, seed=330)
+    cpu, gpu = make(wl)
+    D = wl.heads * wl.d
+    x, ws = gate_inputs(331, wl.B, wl.H, wl.W, D)
+    wg = [torch.from_numpy(w).cuda() for w in ws]
+    gate = binding.rib_cla_gate(x.cuda(), *wg)
+    out, lse = binding.rib_window_attn_fwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], wl.window, wl.shift)
+    out_gated = binding.rib_cla_product(out, gate)
+    dout_attn, dgate = binding.rib_cla_product_bwd(out, gate, gpu["dout"])            # dout: the gradient of out_gated
+    grads_gate = binding.rib_cla_gate_bwd(x.cuda(), *wg, dgate)
+    grads_attn = binding.rib_window_attn_bwd(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse, dout_attn, wl.window, wl.shift)
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0
+
+    ref_out, _ = oracle_fwd(cpu, wl)
+    ref_gate = cla.gate(to_f64(x), *ws)
+    compare("gated out", to_f64(out_gated), cla.gated_output(ref_out, ref_gate))
+    ref_dout, ref_dgate = cla.gated_output_bwd(ref_out, ref_gate, to_f64(cpu["dout"]))
+    ref_gate_grads = cla.gate_bwd(to_f64(x), *ws, ref_dgate)
+    ref_attn_grads = orc.bwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk")), ref_dout, wl.window, wl.shift)
+    for name, g, r in zip(("dx", "dw_dw", "db_dw", "dw_pw", "db_pw"), grads_gate, ref_gate_grads):
+        compare(name, to_f64(g), r, max_abs=1e-2 * max(1.0, np.abs(r).max()))
+    for name, g, r in zip(("dq", "dk", "dv", "dpq", "dpk"), grads_attn, ref_attn_grads):
+        compare(name, to_f64(g), r, max_abs=1e-2 * max(1.0, np.abs(r).max()))
