@@ -374,6 +374,13 @@ struct TcLayout {
     static constexpr uint32_t kTmemCols = kColW + kBlocks * D <= 256 ? 256 : 512;
 };
 
+// 32-byte store of eight 32-bit words; the address must be 32-byte aligned
+__device__ __forceinline__ void st_global_v8(float* dst, const uint32_t* v)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]),
+                 "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
+
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const ClaBwdParams p)
 {
@@ -483,6 +490,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
                 make_uint4(pack_bf16x2(dz[8], dz[9]), pack_bf16x2(dz[10], dz[11]), pack_bf16x2(dz[12], dz[13]), pack_bf16x2(dz[14], dz[15]));
         }
     };
+    const bool wide_stores = (reinterpret_cast<uintptr_t>(p.dy) & 31u) == 0;      // the workspace is only promised 16-byte alignment
     // dY columns [0, ncols) of the accumulator -> input channels i0 + [0, ncols) of the workspace
     auto dy_epilogue = [&](long long pix, int i0, int ncols) {
         for (int g = sub; g < ncols / 16; g += 4) {
@@ -490,10 +498,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
             tmem_ld16(t_lane + 16 * g, a);
             tmem_wait_ld();
             if (pix < p.pixels) {
-                float4* dst = reinterpret_cast<float4*>(p.dy + pix * D + i0 + 16 * g);
+                float* dst = p.dy + pix * D + i0 + 16 * g;
+                if (wide_stores) {
+                    // a thread owns 64 contiguous bytes of its pixel's row: two 32-byte stores fill whole sectors
+                    st_global_v8(dst, a);
+                    st_global_v8(dst + 8, a + 8);
+                } else {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    dst[k] = make_float4(__uint_as_float(a[4 * k]), __uint_as_float(a[4 * k + 1]), __uint_as_float(a[4 * k + 2]), __uint_as_float(a[4 * k + 3]));
+                    for (int k = 0; k < 4; ++k)
+                        reinterpret_cast<float4*>(dst)[k] =
+                            make_float4(__uint_as_float(a[4 * k]), __uint_as_float(a[4 * k + 1]), __uint_as_float(a[4 * k + 2]), __uint_as_float(a[4 * k + 3]));
+                }
             }
         }
     };

@@ -199,3 +199,22 @@ def test_training_chain_matches_the_oracles_chained():
         compare(name, to_f64(g), r, max_abs=1e-2 * max(1.0, np.abs(r).max()))
     for name, g, r in zip(("dq", "dk", "dv", "dpq", "dpk"), grads_attn, ref_attn_grads):
         compare(name, to_f64(g), r, max_abs=1e-2 * max(1.0, np.abs(r).max()))
+
+
+def test_gate_backward_with_a_workspace_that_is_only_16_byte_aligned():
+    """The workspace is promised 16-byte alignment only; the kernel's 32-byte stores must then not be used."""
+    B, H, W, D = 1, 16, 24, 192
+    x, ws = gate_inputs(340, B, H, W, D)
+    dgate = dgate_input(341, (B, H, W, D))
+    args = [x.cuda(), *[torch.from_numpy(w).cuda() for w in ws], dgate.cuda()]
+    need = binding.library().rib_cla_gate_bwd_workspace(B, H, W, D)
+    buf = torch.empty(need + 64, dtype=torch.uint8, device="cuda")
+    off = 16 if buf.data_ptr() % 32 == 0 else 0
+    assert (buf.data_ptr() + off) % 32 == 16
+    plain = [t.clone() for t in binding.rib_cla_gate_bwd(*args)]
+    shifted = binding.rib_cla_gate_bwd(*args, workspace=buf[off:])
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0
+    assert torch.equal(plain[0], shifted[0])
+    for a, b in zip(plain[1:], shifted[1:]):
+        assert torch.allclose(a, b, rtol=1e-4, atol=1e-5)
