@@ -517,43 +517,90 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
     bool ok = true;
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
         const long long pix0 = tile * kTcPix;
-        // ---- Y = DWConv3x3(X) + b_dw as the bf16 tile [pixel][channel]; rows beyond the last pixel are zero
-#pragma unroll 2
-        for (int idx = threadIdx.x; idx < kTcPix * kChunks; idx += kTcThreads) {
-            const int r = idx / kChunks, c8 = idx - r * kChunks;
+        // ---- Y = DWConv3x3(X) + b_dw as the bf16 tile [pixel][channel]; rows beyond the last pixel are zero.
+        // A thread takes an 8-channel chunk of two neighbouring pixels: when both lie in one image row they share the
+        // 3 x 4 patch of X (12 loads instead of 18, every tap read once); otherwise each pixel is filtered on its own.
+        for (int idx = threadIdx.x; idx < (kTcPix / 2) * kChunks; idx += kTcThreads) {
+            const int pr = idx / kChunks, c8 = idx - pr * kChunks, r = 2 * pr;
             const long long pix = pix0 + r;
-            float acc[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-            if (pix < p.pixels) {
-                const long long b = pix / hw;
-                const int rem = (int)(pix - b * hw), Y = rem / p.W, X = rem - Y * p.W;
+            const long long b = pix / hw;
+            const int rem = (int)(pix - b * hw), Y = rem / p.W, X = rem - Y * p.W;
+            float acc0[8], acc1[8];
+            if (pix + 1 < p.pixels && X + 1 < p.W) {
                 const __nv_bfloat16* centre = p.x + pix * D + 8 * c8;
-                uint4 v[9];                              // all nine loads are in flight before the first is used
+                uint4 v[3][4];                           // all twelve loads are in flight before the first is used
 #pragma unroll
-                for (int t = 0; t < 9; ++t) {
-                    const int dyy = t / 3 - 1, dxx = t % 3 - 1;
-                    const bool in = Y + dyy >= 0 && Y + dyy < p.H && X + dxx >= 0 && X + dxx < p.W;
-                    v[t] = in ? __ldg(reinterpret_cast<const uint4*>(centre + ((long long)dyy * p.W + dxx) * D)) : make_uint4(0, 0, 0, 0);
+                for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+                    for (int cx = 0; cx < 4; ++cx) {
+                        const bool in = Y + ky - 1 >= 0 && Y + ky - 1 < p.H && X + cx - 1 >= 0 && X + cx - 1 < p.W;
+                        v[ky][cx] = in ? __ldg(reinterpret_cast<const uint4*>(centre + ((long long)(ky - 1) * p.W + cx - 1) * D))
+                                       : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) acc0[k] = acc1[k] = bdw[8 * c8 + k];
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky) {
+                    float w[3][8];
+#pragma unroll
+                    for (int kx = 0; kx < 3; ++kx) {
+                        const float4 w0 = *reinterpret_cast<const float4*>(taps + (ky * 3 + kx) * D + 8 * c8);
+                        const float4 w1 = *reinterpret_cast<const float4*>(taps + (ky * 3 + kx) * D + 8 * c8 + 4);
+                        w[kx][0] = w0.x; w[kx][1] = w0.y; w[kx][2] = w0.z; w[kx][3] = w0.w;
+                        w[kx][4] = w1.x; w[kx][5] = w1.y; w[kx][6] = w1.z; w[kx][7] = w1.w;
+                    }
+#pragma unroll
+                    for (int cx = 0; cx < 4; ++cx) {
+                        const uint32_t u[4] = {v[ky][cx].x, v[ky][cx].y, v[ky][cx].z, v[ky][cx].w};
+                        float f[8];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) { f[2 * k] = __uint_as_float(u[k] << 16); f[2 * k + 1] = __uint_as_float(u[k] & 0xffff0000u); }
+                        if (cx < 3) {                    // column X - 1 + cx is tap kx = cx of the left pixel
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) acc0[k] = fmaf(f[k], w[cx][k], acc0[k]);
+                        }
+                        if (cx > 0) {                    // and tap kx = cx - 1 of the right pixel
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) acc1[k] = fmaf(f[k], w[cx - 1][k], acc1[k]);
+                        }
+                    }
                 }
+            } else {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) acc[k] = bdw[8 * c8 + k];
+                for (int which = 0; which < 2; ++which) {
+                    float* acc = which ? acc1 : acc0;
+                    const long long px = pix + which;
 #pragma unroll
-                for (int t = 0; t < 9; ++t) {
-                    const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
-                    const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
-                    acc[0] = fmaf(__uint_as_float(v[t].x << 16), w0.x, acc[0]);
-                    acc[1] = fmaf(__uint_as_float(v[t].x & 0xffff0000u), w0.y, acc[1]);
-                    acc[2] = fmaf(__uint_as_float(v[t].y << 16), w0.z, acc[2]);
-                    acc[3] = fmaf(__uint_as_float(v[t].y & 0xffff0000u), w0.w, acc[3]);
-                    acc[4] = fmaf(__uint_as_float(v[t].z << 16), w1.x, acc[4]);
-                    acc[5] = fmaf(__uint_as_float(v[t].z & 0xffff0000u), w1.y, acc[5]);
-                    acc[6] = fmaf(__uint_as_float(v[t].w << 16), w1.z, acc[6]);
-                    acc[7] = fmaf(__uint_as_float(v[t].w & 0xffff0000u), w1.w, acc[7]);
+                    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+                    if (px < p.pixels) {
+                        const long long bb = px / hw;
+                        const int rm = (int)(px - bb * hw), Yp = rm / p.W, Xp = rm - Yp * p.W;
+                        const __nv_bfloat16* centre = p.x + px * D + 8 * c8;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) acc[k] = bdw[8 * c8 + k];
+#pragma unroll
+                        for (int t = 0; t < 9; ++t) {
+                            const int dyy = t / 3 - 1, dxx = t % 3 - 1;
+                            if (Yp + dyy < 0 || Yp + dyy >= p.H || Xp + dxx < 0 || Xp + dxx >= p.W) continue;
+                            const uint4 vv = __ldg(reinterpret_cast<const uint4*>(centre + ((long long)dyy * p.W + dxx) * D));
+                            const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
+                            const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
+                            acc[0] = fmaf(__uint_as_float(vv.x << 16), w0.x, acc[0]);
+                            acc[1] = fmaf(__uint_as_float(vv.x & 0xffff0000u), w0.y, acc[1]);
+                            acc[2] = fmaf(__uint_as_float(vv.y << 16), w0.z, acc[2]);
+                            acc[3] = fmaf(__uint_as_float(vv.y & 0xffff0000u), w0.w, acc[3]);
+                            acc[4] = fmaf(__uint_as_float(vv.z << 16), w1.x, acc[4]);
+                            acc[5] = fmaf(__uint_as_float(vv.z & 0xffff0000u), w1.y, acc[5]);
+                            acc[6] = fmaf(__uint_as_float(vv.w << 16), w1.z, acc[6]);
+                            acc[7] = fmaf(__uint_as_float(vv.w & 0xffff0000u), w1.w, acc[7]);
+                        }
+                    }
                 }
             }
             *reinterpret_cast<uint4*>(sm + L::kOffY + (c8 >> 3) * L::kTAtom + r * 128 + (((c8 & 7) ^ (r & 7)) << 4)) =
-                make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
+                make_uint4(pack_bf16x2(acc0[0], acc0[1]), pack_bf16x2(acc0[2], acc0[3]), pack_bf16x2(acc0[4], acc0[5]), pack_bf16x2(acc0[6], acc0[7]));
+            *reinterpret_cast<uint4*>(sm + L::kOffY + (c8 >> 3) * L::kTAtom + (r + 1) * 128 + (((c8 & 7) ^ ((r + 1) & 7)) << 4)) =
+                make_uint4(pack_bf16x2(acc1[0], acc1[1]), pack_bf16x2(acc1[2], acc1[3]), pack_bf16x2(acc1[4], acc1[5]), pack_bf16x2(acc1[6], acc1[7]));
         }
         hand_over();
         // ---- Z = Y W_pw^T, output channels [0, N1) then [N1, D), each followed by dZ into its slice of the dZ tile
