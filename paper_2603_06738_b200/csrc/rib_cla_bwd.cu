@@ -303,14 +303,30 @@ __global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const 
 #pragma unroll
     for (int t = 0; t < 9; ++t) gw[t] = 0.f;
     __syncthreads();
-    // lane l takes tile row l: 16 pixels
+    // lane l takes tile row l: 16 pixels, walked left to right with the 3 x 3 windows of dY and X in registers, so each
+    // pixel costs one new halo column (6 shared-memory reads) instead of 18.  Pixels to the right of the map need no
+    // test for the sums: dY is zero there.
     const int py = lane;
     if (y0 + py < p.H) {
-#pragma unroll 4
+        float dwin[3][3], xwin[3][3];                    // [halo row py + i][halo column px + j]
+#pragma unroll
+        for (int i = 0; i < 3; ++i)
+#pragma unroll
+            for (int j = 1; j < 3; ++j) {
+                dwin[i][j] = dys[((py + i) * kDwHaloW + j - 1) * kDwCh + c];
+                xwin[i][j] = __bfloat162float(xs[((py + i) * kDwHaloW + j - 1) * kDwCh + c]);
+            }
+        __nv_bfloat16* dst = p.dx + (((size_t)b * p.H + y0 + py) * p.W + x0) * D + ch0 + c;
+#pragma unroll
         for (int px = 0; px < kDwTileW; ++px) {
-            if (x0 + px >= p.W) break;
-            const int hc = (py + 1) * kDwHaloW + px + 1;                  // this pixel in the halo
-            const float dy_here = dys[hc * kDwCh + c];
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                dwin[i][0] = dwin[i][1]; dwin[i][1] = dwin[i][2];
+                xwin[i][0] = xwin[i][1]; xwin[i][1] = xwin[i][2];
+                dwin[i][2] = dys[((py + i) * kDwHaloW + px + 2) * kDwCh + c];
+                xwin[i][2] = __bfloat162float(xs[((py + i) * kDwHaloW + px + 2) * kDwCh + c]);
+            }
+            const float dy_here = dwin[1][1];
             gb += dy_here;
             float dx = 0.f;
 #pragma unroll
@@ -318,12 +334,12 @@ __global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const 
 #pragma unroll
                 for (int kx = 0; kx < 3; ++kx) {
                     // forward: Y[y, x] reads X[y + ky - 1, x + kx - 1] through tap (ky, kx); X is zero outside the map
-                    gw[ky * 3 + kx] = fmaf(dy_here, __bfloat162float(xs[(hc + (ky - 1) * kDwHaloW + kx - 1) * kDwCh + c]), gw[ky * 3 + kx]);
+                    gw[ky * 3 + kx] = fmaf(dy_here, xwin[ky][kx], gw[ky * 3 + kx]);
                     // so X[y, x] was read by the output pixel (y - ky + 1, x - kx + 1); dY is zero outside the map
-                    dx = fmaf(dys[(hc - (ky - 1) * kDwHaloW - (kx - 1)) * kDwCh + c], w[ky * 3 + kx], dx);
+                    dx = fmaf(dwin[2 - ky][2 - kx], w[ky * 3 + kx], dx);
                 }
             }
-            p.dx[(((size_t)b * p.H + y0 + py) * p.W + x0 + px) * D + ch0 + c] = __float2bfloat16_rn(dx);
+            if (x0 + px < p.W) dst[(size_t)px * D] = __float2bfloat16_rn(dx);
         }
     }
 #pragma unroll
