@@ -246,37 +246,44 @@ __global__ void __launch_bounds__(kPwThreads, 1) rib_cla_bwd_pw_kernel(const Cla
 }
 
 // ------------------------------------------------------------------------------------------------------------------
-// Depth-wise part.  A block takes a tile of 8 x 16 pixels and 64 channels: the 10 x 18 halo of dY (fp32) and of X (bf16)
+// Depth-wise part.  A block takes a tile of 8 x 16 pixels and 32 channels: the 10 x 18 halo of dY (fp32) and of X (bf16)
 // goes to shared memory (zero outside the map), thread (channel, lane) walks 16 pixels of the tile.
 // ------------------------------------------------------------------------------------------------------------------
 constexpr int kDwTileH = 8, kDwTileW = 16, kDwHaloH = kDwTileH + 2, kDwHaloW = kDwTileW + 2, kDwHalo = kDwHaloH * kDwHaloW;
-constexpr int kDwCh = 64, kDwLanes = 8;
+constexpr int kDwCh = 32, kDwLanes = 8;
 constexpr int kDwSmemBytes = kDwHalo * kDwCh * 6 + kDwLanes * 10 * kDwCh * 4;
 
 template <int D>
 __global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const ClaBwdParams p, int tiles_y, int tiles_x)
 {
     extern __shared__ __align__(16) uint8_t dw_smem[];
-    float* dys = reinterpret_cast<float*>(dw_smem);                                        // [180][64]
-    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(dw_smem + kDwHalo * kDwCh * 4);   // [180][64]
-    float* red = reinterpret_cast<float*>(dw_smem + kDwHalo * kDwCh * 6);                  // [8 lanes][10][64]
+    float* dys = reinterpret_cast<float*>(dw_smem);                                        // [180][channels]
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(dw_smem + kDwHalo * kDwCh * 4);   // [180][channels]
+    float* red = reinterpret_cast<float*>(dw_smem + kDwHalo * kDwCh * 6);                  // [8 lanes][10][channels]
     const int c = threadIdx.x, lane = threadIdx.y, tid = lane * kDwCh + c;
     constexpr int kGroups = D / kDwCh;
-    int tile = blockIdx.x;
-    const int cg = tile % kGroups; tile /= kGroups;
-    const int tx = tile % tiles_x; tile /= tiles_x;
-    const int ty = tile % tiles_y, b = tile / tiles_y;
-    const int y0 = ty * kDwTileH, x0 = tx * kDwTileW, ch0 = cg * kDwCh;
-    // halo: 16 threads per pixel (4 channels each), 32 pixels per pass; all loads of a thread are issued before the
+    // a block keeps one channel group and walks spatial tiles, so its ten sums per channel reach global memory once
+    const int cg = blockIdx.x % kGroups, ch0 = cg * kDwCh;
+    const int spatial = p.B * tiles_y * tiles_x, step = gridDim.x / kGroups;      // the grid is a multiple of kGroups
+    float w[9];
+#pragma unroll
+    for (int t = 0; t < 9; ++t) w[t] = p.w_dw[(ch0 + c) * 9 + t];
+    float gw[9], gb = 0.f;
+#pragma unroll
+    for (int t = 0; t < 9; ++t) gw[t] = 0.f;
+    for (int st = blockIdx.x / kGroups; st < spatial; st += step) {
+    const int tx = st % tiles_x, ty = (st / tiles_x) % tiles_y, b = st / (tiles_x * tiles_y);
+    const int y0 = ty * kDwTileH, x0 = tx * kDwTileW;
+    // halo: a thread moves 4 channels of a pixel; all loads of a thread are issued before the
     // first store, so the prologue costs one memory latency
     {
-        constexpr int kItems = kDwHalo * 16, kIters = (kItems + kDwCh * kDwLanes - 1) / (kDwCh * kDwLanes);
+        constexpr int kPer = kDwCh / 4, kItems = kDwHalo * kPer, kIters = (kItems + kDwCh * kDwLanes - 1) / (kDwCh * kDwLanes);
         float4 dv[kIters];
         uint2 xv[kIters];
 #pragma unroll
         for (int u = 0; u < kIters; ++u) {
             const int idx = tid + u * kDwCh * kDwLanes;
-            const int hp = idx >> 4, c4 = (idx & 15) * 4;
+            const int hp = idx / kPer, c4 = (idx % kPer) * 4;
             const int yy = y0 + hp / kDwHaloW - 1, xx = x0 + hp % kDwHaloW - 1;
             dv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
             xv[u] = make_uint2(0, 0);
@@ -290,18 +297,12 @@ __global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const 
         for (int u = 0; u < kIters; ++u) {
             const int idx = tid + u * kDwCh * kDwLanes;
             if (idx < kItems) {
-                const int hp = idx >> 4, c4 = (idx & 15) * 4;
+                const int hp = idx / kPer, c4 = (idx % kPer) * 4;
                 *reinterpret_cast<float4*>(dys + hp * kDwCh + c4) = dv[u];
                 *reinterpret_cast<uint2*>(xs + hp * kDwCh + c4) = xv[u];
             }
         }
     }
-    float w[9];
-#pragma unroll
-    for (int t = 0; t < 9; ++t) w[t] = p.w_dw[(ch0 + c) * 9 + t];
-    float gw[9], gb = 0.f;
-#pragma unroll
-    for (int t = 0; t < 9; ++t) gw[t] = 0.f;
     __syncthreads();
     // lane l takes tile row l: 16 pixels, walked left to right with the 3 x 3 windows of dY and X in registers, so each
     // pixel costs one new halo column (6 shared-memory reads) instead of 18.  Pixels to the right of the map need no
@@ -342,11 +343,13 @@ __global__ void __launch_bounds__(kDwCh * kDwLanes) rib_cla_bwd_dw_kernel(const 
             if (x0 + px < p.W) dst[(size_t)px * D] = __float2bfloat16_rn(dx);
         }
     }
+    __syncthreads();                                     // the next tile overwrites the halos
+    }
 #pragma unroll
     for (int t = 0; t < 9; ++t) red[(lane * 10 + t) * kDwCh + c] = gw[t];
     red[(lane * 10 + 9) * kDwCh + c] = gb;
     __syncthreads();
-    // 640 sums of 8 lanes
+    // 10 sums of 8 lanes per channel
     for (int idx = tid; idx < 10 * kDwCh; idx += kDwCh * kDwLanes) {
         const int t = idx / kDwCh, cc = idx - t * kDwCh;
         float sum = 0.f;
@@ -753,9 +756,11 @@ cudaError_t launch_gate_bwd(const ClaBwdParams& p, bool tensor_cores, cudaStream
     {
         ProfileScope scope(RIB_KERNEL_CLA_BWD_DW, stream);
         const int tiles_y = (p.H + kDwTileH - 1) / kDwTileH, tiles_x = (p.W + kDwTileW - 1) / kDwTileW;
-        const long long blocks = (long long)p.B * tiles_y * tiles_x * (D / kDwCh);
-        if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-        rib_cla_bwd_dw_kernel<D><<<(unsigned)blocks, dim3(kDwCh, kDwLanes), kDwSmemBytes, stream>>>(p, tiles_y, tiles_x);
+        const long long spatial = (long long)p.B * tiles_y * tiles_x;
+        if (spatial > 0x7fffffffLL) return cudaErrorInvalidValue;
+        constexpr int kGroups = D / kDwCh;
+        const long long per_group = spatial < (long long)sms * 4 / kGroups ? spatial : (long long)sms * 4 / kGroups;   // four blocks fit on an SM
+        rib_cla_bwd_dw_kernel<D><<<(unsigned)(per_group * kGroups), dim3(kDwCh, kDwLanes), kDwSmemBytes, stream>>>(p, tiles_y, tiles_x);
     }
     return cudaGetLastError();
 }
