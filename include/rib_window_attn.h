@@ -57,7 +57,7 @@ enum {
 };
 
 /* Which kernel family a call used (see rib_last_path). */
-enum { RIB_PATH_NONE = 0, RIB_PATH_GENERIC = 1, RIB_PATH_SM100 = 2 };
+enum { RIB_PATH_NONE = 0, RIB_PATH_GENERIC = 1, RIB_PATH_SM100 = 2, RIB_PATH_SM100_EXACT = 3 };
 
 /*
  * Forward (Eq. 5, Eq. 6, O = SoftMax(S) V).
@@ -270,7 +270,11 @@ const char* rib_status_string(int status);
 
 /*
  * Debugging knobs, per process.  rib_set_path(RIB_PATH_GENERIC) forces the any-shape kernels,
- * rib_set_path(RIB_PATH_NONE) restores automatic selection; returns the previous setting.
+ * rib_set_path(RIB_PATH_SM100_EXACT) keeps automatic selection but makes the tcgen05 forward kernel
+ * take its exact softmax form (running maximum, rescaling) for every item instead of only for the
+ * items whose scores leave the range of the fast form (Sec. 3.1: the steps after Eq. 6 are those of
+ * standard attention; both forms compute the same SoftMax), rib_set_path(RIB_PATH_NONE) restores
+ * automatic selection; returns the previous setting (other values: nothing changes).
  * rib_last_path() tells which family the last successful fwd/bwd call of this thread launched.
  */
 int rib_set_path(int path);

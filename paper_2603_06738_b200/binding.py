@@ -16,7 +16,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "librib_window_attn.so"
 _lib = None
 
 RIB_OK = 0
-RIB_PATH_NONE, RIB_PATH_GENERIC, RIB_PATH_SM100 = 0, 1, 2
+RIB_PATH_NONE, RIB_PATH_GENERIC, RIB_PATH_SM100, RIB_PATH_SM100_EXACT = 0, 1, 2, 3
 
 EXPORTS = (
     "rib_window_attn_fwd", "rib_window_attn_bwd", "rib_window_attn_bwd_workspace",

@@ -301,7 +301,9 @@ int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const 
     p.gate = static_cast<const __nv_bfloat16*>(gate);
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
+    const int forced = g_forced_path.load();
+    const bool fast = forced != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
+    p.exact_softmax = forced == RIB_PATH_SM100_EXACT;
     const cudaError_t e = fast ? rib::sm100_fwd(p, st) : rib::generic_fwd(p, st);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
@@ -499,7 +501,7 @@ const char* rib_status_string(int status)
 
 int rib_set_path(int path)
 {
-    if (path != RIB_PATH_NONE && path != RIB_PATH_GENERIC) return g_forced_path.load();
+    if (path != RIB_PATH_NONE && path != RIB_PATH_GENERIC && path != RIB_PATH_SM100_EXACT) return g_forced_path.load();
     return g_forced_path.exchange(path);
 }
 

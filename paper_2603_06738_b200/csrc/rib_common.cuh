@@ -37,6 +37,7 @@ struct Problem {
                                       // (positions with Y >= H or X >= W are not tokens); equal to H, W in the plain calls
     int n, nWy, nWx, pairs;           // n = M*M, windows per image, B*nWy*nWx*heads
     int* status;                      // device status word (bounded waits report here)
+    bool exact_softmax;               // tcgen05 forward: every item takes the exact (running-maximum) softmax form
 };
 
 // Pq/Pk tables: one shared by the heads, or one per head (Sec. 3.1, after Eq. 3: head-wise projections of the shared h).

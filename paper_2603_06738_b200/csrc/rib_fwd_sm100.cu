@@ -1,5 +1,5 @@
 // Forward RIB window attention for B200 (sm_100a): tcgen05 MMAs with TMEM accumulators, TMA loads
-// whose box coordinates do the window partition and the cyclic shift, online softmax in registers.
+// whose box coordinates do the window partition and the cyclic shift, softmax in registers.
 //
 // Shapes: d = 32, r = 16 or 32 (template argument R), window side M a multiple of 16, shift a multiple of 8.
 // The text below describes R = 16; with R = 32 the RIB rows are 64 bytes like the content rows and take two K16 steps.
@@ -10,25 +10,47 @@
 //                        32-byte RIB rows -- the concatenation of Eq. 5 exists only as three
 //                        accumulating MMAs on separately staged shared-memory slabs)
 //     P_q = exp2((S_q - m) * log2e / sqrt(d))      softmax warps, fp32 -> bf16 written back to TMEM
-//     O_q += P_q V      (M128 N32 K128, A operand from TMEM, V as an MN-major shared-memory tile)
-// for the two query tiles q = 0, 1.  The two tiles run as independent pipelines, each with its own
-// MMA-issuing warp; the S accumulator is released as soon as the scores are in registers, so the
-// next block's S_q is computed while the exponentials of this one are still being evaluated.
+//     O_q += P_q V      (A operand from TMEM, V as an MN-major shared-memory tile)
+// for the two query tiles q = 0, 1.  The two tiles run as independent pipelines; the S accumulator is
+// released as soon as the scores are in registers, so the next block's S_q is computed while the
+// exponentials of this one are being evaluated.
 //
-// The softmax of a query tile is split over the keys: two threads own a query row, one takes keys
-// 0-63 of every block and the other keys 64-127.  Each keeps its own running maximum and sum and
-// its own O accumulator in tensor memory (PV of a block is two K64 contractions), and the two
-// partial results are merged in the epilogue with the usual log-sum-exp combination.  This puts
-// four softmax warps on every SM sub-partition, which is what keeps the exp (XU) pipe fed: with one
-// thread per row the tensor-memory and barrier latencies of a block were exposed.
+// Two threads own a query row: one takes keys 0-63 of every block and the other keys 64-127, which
+// puts four softmax warps on every SM sub-partition.
+//
+// The softmax has two forms.
+//   Fast form (first pass over the items; maps that are multiples of the window): the exp (MUFU)
+//   and issue pipes are what this kernel runs out of, so the per-score work is cut to one scale-and-
+//   subtract, one exponential and one conversion.  The reference m of a row is fixed once per item (the
+//   maximum over the first 32 keys, read by both threads of the row, so they agree without talking to
+//   each other), no running maximum is kept and nothing is ever rescaled: fp32 and bf16 carry 8
+//   exponent bits, so probabilities up to 2^100 relative to the reference are as exact as those below 1.
+//   The row sum comes from the tensor core: V is followed by a second shared-memory tile whose first
+//   column is 1, the PV contraction is N = 48 wide and column 32 of the accumulator is
+//   l = sum_j bf16(P_ij) -- the sum of exactly the probabilities that were contracted with V.  Both
+//   key halves accumulate into ONE accumulator per query tile (same reference), so there is nothing to
+//   merge.  A row whose scores leave the representable range (a key more than ~69 nat above the
+//   reference, or a polynomial-path key more than ~83 nat below) shows up as l >= 2^100 or not finite:
+//   the item is then noted in shared memory and redone by the exact form in a second pass of the
+//   same launch.  Every third or fourth pair of exponentials (kPolyMask) is evaluated on the FMA and
+//   integer pipes instead of the MUFU.
+//   Exact form (second pass, and maps with partial windows): classic online softmax per key half
+//   with a running maximum, lazy rescaling of O, separate accumulators and a log-sum-exp merge.
 //
 // Tiles are two 8x8-token patches (see rib_sm100_common.cuh), fetched by one TMA box each.
 //
-// Roles (640 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers of query tile 0 and 1, warp 2
-// stages the scaled query RIB rows of the next item (and owns the TMEM allocation), warps 4-11
-// softmax/epilogue of query tile 0 (4-7 first half of the keys, 8-11 second half), warps 12-19 of
-// query tile 1.  Every wait is bounded.
+// Roles (640 threads): warp 0 TMA producer (one lane) that also stages the scaled query RIB rows of the item
+// it is about to fetch; warp 1 issues S for both query tiles, warps 2 and 3 issue PV for tile 0 and 1 (three
+// issuers, because what bounds the bare pipeline is the serial time of an issuing warp: a group of MMAs holds
+// its issuer for several hundred cycles, and with S and PV in one warp the two dependency loops
+// scores -> S free -> next scores  and  P ready -> PV -> P free  went through the same instruction stream);
+// warp 2 owns the TMEM allocation; warps 4-11 softmax/epilogue of query tile 0 (4-7 first half of the keys,
+// 8-11 second half), warps 12-19 of query tile 1.  Every wait is bounded.
 #include "rib_sm100_common.cuh"
+
+#ifndef RIB_FWD_POLY_MASK
+#define RIB_FWD_POLY_MASK 0x88u         // of every 8 score pairs: which go to the FMA pipe
+#endif
 
 namespace rib {
 namespace {
@@ -37,10 +59,12 @@ using namespace sm100;
 
 constexpr int kStages = 4;            // K/V ring depth
 constexpr int kThreads = 640;
+constexpr int kMaxRedo = 64;          // items a CTA can note for the exact pass (more: all of its items are redone)
+constexpr uint32_t kPolyMask = RIB_FWD_POLY_MASK;
 
-// kPReady / kPFree: index 2 * tile + key half
-enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 14, kOFree = 18, kDrain = 20, kMerge = 22,
-           kKFull = 30, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
+// kSFull .. kOFree: one per query tile; kDrain: one per issuing warp; kMerge: 4 * tile + quarter of the rows
+enum Bar { kQFull = 0, kQEmpty = 2, kQPos = 4, kSFull = 6, kSFree = 8, kPReady = 10, kPFree = 12, kOFree = 14, kDrain = 16, kMerge = 20,
+           kKFull = 28, kKEmpty = kKFull + kStages, kVFull = kKEmpty + kStages, kVEmpty = kVFull + kStages,
            kNumBars = kVEmpty + kStages };
 
 // shared-memory map (offsets from a 1024-byte aligned base) for RIB rank R = 16 (32-byte RIB rows, SWIZZLE_32B) or
@@ -53,18 +77,23 @@ struct Layout {
     static constexpr uint32_t kOffKc = kOffQp + 4 * kPosBytes;                   // [kStages] key content
     static constexpr uint32_t kOffKp = kOffKc + kStages * kContentBytes;         // [kStages] key RIB rows
     static constexpr uint32_t kOffV = kOffKp + kStages * kPosBytes;              // [kStages] values
-    static constexpr uint32_t kOffBar = kOffV + kStages * kContentBytes;
-    static constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flag
-    static constexpr uint32_t kOffMerge = kOffMisc + 16;                         // [2 tiles][2 halves][128 rows] (max, sum)
+    static constexpr uint32_t kOffOnes = kOffV + kStages * kContentBytes;        // [128 keys][32] column 0 = 1: second atom of V
+    static constexpr uint32_t kOffBar = kOffOnes + kContentBytes;
+    static constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flags, redo count
+    static constexpr uint32_t kOffRedo = kOffMisc + 16;                          // [kMaxRedo] item ordinals of the exact pass
+    static constexpr uint32_t kOffMerge = kOffRedo + kMaxRedo * 4;               // [2 tiles][2 halves][128 rows] (max, sum)
     static constexpr uint32_t kSmemBytes = kOffMerge + 4 * kTile * 8 + 1024;     // + slack for manual alignment
+    static_assert(kOffV % 1024 == 0 && kOffOnes % 1024 == 0, "swizzle atoms need aligned tiles");
 };
 
 // tensor-memory columns (fp32 accumulators; P is bf16x2, two keys per column)
-// O: [2 tiles][2 key halves][32]
+// O, exact form: [2 tiles][2 key halves][32];  fast form: [2 tiles][48] (32 value columns, the row sum, 15 unused)
 constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
+constexpr uint32_t kFastOCols = kD + 16;
 
 constexpr uint32_t kIdescS = idesc_bf16_f32(kTile, kTile, false);
 constexpr uint32_t kIdescPV = idesc_bf16_f32(kTile, kD, true);
+constexpr uint32_t kIdescPV1 = idesc_bf16_f32(kTile, kFastOCols, true);
 
 struct FwdParams {
     const __nv_bfloat16* pq;
@@ -81,6 +110,8 @@ struct FwdParams {
     float pos_scale;           // sqrt(d / r): folds 1/sqrt(r) into the content scale
     long long pos_head_stride; // elements between the heads' Pq tables (0: one table for all heads)
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
+    int exact_only;            // 1: skip the fast form (every item takes the exact softmax)
+    FastDiv div_tp, div_heads, div_nwx, div_nwy, div_per_row;   // tiles_per_item_pair, heads, nWx, nWy, M / 8
 };
 
 struct ItemCoord { int b, wy, wx, h, tp; };
@@ -88,18 +119,38 @@ struct ItemCoord { int b, wy, wx, h, tp; };
 __device__ __forceinline__ ItemCoord decode_item(const FwdParams& p, int item)
 {
     ItemCoord c;
-    c.tp = item % p.tiles_per_item_pair; item /= p.tiles_per_item_pair;
-    c.h = item % p.heads; item /= p.heads;
-    c.wx = item % p.nWx; item /= p.nWx;
-    c.wy = item % p.nWy; item /= p.nWy;
-    c.b = item;
+    p.div_tp.divmod(item, item, c.tp);
+    p.div_heads.divmod(item, item, c.h);
+    p.div_nwx.divmod(item, item, c.wx);
+    p.div_nwy.divmod(item, c.b, c.wy);
     return c;
 }
 
 __device__ __forceinline__ void patch_origin(const FwdParams& p, const ItemCoord& c, int sp, int& py, int& px,
                                              int& Y0, int& X0)
 {
-    sm100::patch_origin(WindowGeom{p.Hp, p.Wp, p.M, p.s}, c.wy, c.wx, sp, py, px, Y0, X0);
+    sm100::patch_origin(WindowGeom{p.Hp, p.Wp, p.M, p.s}, p.div_per_row, c.wy, c.wx, sp, py, px, Y0, X0);
+}
+
+// 2^x for a pair of arguments on the FMA and integer pipes, for the fast softmax form.  x = n + f with
+// n = round(x), |f| <= 1/2.  The cubic (relative error 7.5e-5) is evaluated with coefficients scaled by
+// 2^-120, so its result carries the exponent field 6 or 7 and 2^n is applied by adding (n + 120) to that
+// field.  ONE unsigned add-and-min bounds n + 120 to [0, 248]: below -120.5 the unsigned value wraps and
+// is bounded to 248 as well, so an argument outside [-120.5, 128.5) always yields a value of at least 2^126,
+// which the epilogue of the fast form sees in the row sum and answers by redoing the item exactly.
+__device__ __forceinline__ float2 ex2_poly2_ranged(float2 x)
+{
+    constexpr float kS = 7.52316384526264005e-37f;      // 2^-120
+    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
+    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+    float2 q = __ffma2_rn(make_float2(0.05517084f * kS, 0.05517084f * kS), f, make_float2(0.24260935f * kS, 0.24260935f * kS));
+    q = __ffma2_rn(q, f, make_float2(0.69326097f * kS, 0.69326097f * kS));
+    q = __ffma2_rn(q, f, make_float2(0.99992818f * kS, 0.99992818f * kS));
+    // bits(t) = 0x4B400000 + n for |x| < 2^22
+    const uint32_t vx = min(__float_as_uint(t.x) + (120u - 0x4B400000u), 248u);
+    const uint32_t vy = min(__float_as_uint(t.y) + (120u - 0x4B400000u), 248u);
+    return make_float2(__uint_as_float(__float_as_uint(q.x) + (vx << 23)), __uint_as_float(__float_as_uint(q.y) + (vy << 23)));
 }
 
 // kPartial: H or W is not a multiple of the window (but of 8).  Windows are laid over the map extended to Hp x Wp;
@@ -113,29 +164,34 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                      const FwdParams p)
 {
     using L = Layout<R>;
-    constexpr uint32_t kOffQc = L::kOffQc, kOffQp = L::kOffQp, kOffKc = L::kOffKc, kOffKp = L::kOffKp, kOffV = L::kOffV, kOffBar = L::kOffBar,
-                       kOffMisc = L::kOffMisc, kOffMerge = L::kOffMerge, kPosBytes = L::kPosBytes, kPatchPos = L::kPatchPos;
+    constexpr uint32_t kOffQc = L::kOffQc, kOffQp = L::kOffQp, kOffKc = L::kOffKc, kOffKp = L::kOffKp, kOffV = L::kOffV, kOffOnes = L::kOffOnes,
+                       kOffBar = L::kOffBar, kOffMisc = L::kOffMisc, kOffRedo = L::kOffRedo, kOffMerge = L::kOffMerge, kPosBytes = L::kPosBytes,
+                       kPatchPos = L::kPatchPos;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     auto bar = [&](int i) { return base + kOffBar + 8u * i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + kOffMisc + 4);
+    int* redo_count = reinterpret_cast<int*>(base_ptr + kOffMisc + 12);      // notes taken (duplicates included)
+    volatile int* redo_list = reinterpret_cast<volatile int*>(base_ptr + kOffRedo);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nblk = p.n / kTile;
+    const int my_items = (int)blockIdx.x < p.items ? (p.items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
     if (threadIdx.x == 0) {
         abort_flag[0] = 0; abort_flag[1] = 0;   // [1] stays 0: used by the drain waits
+        *redo_count = 0;
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(kQFull + i), 1); mbar_init(bar(kQEmpty + i), 2); mbar_init(bar(kQPos + i), 1);
-            mbar_init(bar(kDrain + i), 1);
+            mbar_init(bar(kQFull + i), 1); mbar_init(bar(kQEmpty + i), 1); mbar_init(bar(kQPos + i), 1);
             mbar_init(bar(kSFull + i), 1); mbar_init(bar(kSFree + i), 8); mbar_init(bar(kOFree + i), 8);
-            for (int h = 0; h < 2; ++h) { mbar_init(bar(kPReady + 2 * i + h), 4); mbar_init(bar(kPFree + 2 * i + h), 1); }
+            mbar_init(bar(kPReady + i), 8); mbar_init(bar(kPFree + i), 1);
             for (int q4 = 0; q4 < 4; ++q4) mbar_init(bar(kMerge + 4 * i + q4), 2);
         }
-        for (int s = 0; s < kStages; ++s) {     // the "empty" barriers take one commit from each MMA issuer
-            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 2);
+        for (int i = 0; i < 3; ++i) mbar_init(bar(kDrain + i), 1);
+        for (int s = 0; s < kStages; ++s) {     // keys: one commit of the S issuer; values: one commit of each PV issuer
+            mbar_init(bar(kKFull + s), 1); mbar_init(bar(kKEmpty + s), 1);
             mbar_init(bar(kVFull + s), 1); mbar_init(bar(kVEmpty + s), 2);
         }
         fence_barrier_init();
@@ -145,51 +201,101 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tmem_alloc(base + kOffMisc, kTmemCols);
         tmem_relinquish();
     }
+    if (!kPartial && warp >= 4 && warp < 8) {
+        // the tile behind V: 128 key rows of 64 bytes, SWIZZLE_64B like V, element 0 of every row = 1
+        const int row = (warp - 4) * 32 + lane;
+        uint4* dst = reinterpret_cast<uint4*>(base_ptr + kOffOnes + row * 64);
+        const int sw = (row >> 1) & 3;
+#pragma unroll
+        for (int ck = 0; ck < 4; ++ck) dst[ck] = make_uint4(ck == sw ? 0x00003F80u : 0u, 0u, 0u, 0u);
+        fence_proxy_async();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 0) {
-        // ============================================================ TMA producer (one thread)
-        if (lane == 0) {
-            uint32_t blk = 0, io = 0, q_armed = 0, k_armed = 0, v_armed = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
-                const ItemCoord c = decode_item(p, item);
+    // Role state that carries over from the first pass to the exact pass: block and item counters give the barrier phases.
+    uint32_t blk = 0, io = 0, nmerge = 0;
+    uint32_t q_armed = 0, k_armed = 0, v_armed = 0;
+    bool ok = true;
+
+    for (int pass = 0; pass < 2; ++pass) {
+        const bool fast = !kPartial && pass == 0 && !p.exact_only;
+        // pass 0: every item of this CTA; pass 1: the items noted by the fast form (all of them when the notes overflowed)
+        const int noted = pass == 0 ? 0 : *redo_count;
+        const bool all_items = pass == 0 || noted > kMaxRedo;
+        const int count = all_items ? my_items : noted;
+        auto item_at = [&](int i) { return (int)blockIdx.x + (all_items ? i : redo_list[i]) * (int)gridDim.x; };
+
+        if (warp == 0) {
+            // ===================== TMA producer (lane 0) and query RIB rows bf16(Pq * sqrt(d/r)) of the same item (whole warp)
+            for (int i = 0; i < count && ok; ++i, ++io) {
+                const ItemCoord c = decode_item(p, item_at(i));
                 const uint32_t buf = io & 1;
-                if (io >= 2 && !mbar_wait(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                mbar_arrive_expect_tx(bar(kQFull + buf), 2 * kContentBytes);
-                ++q_armed;
-                for (int qt = 0; qt < 2; ++qt)
-                    for (int sub = 0; sub < 2; ++sub) {
-                        int py, px, Y0, X0;
-                        patch_origin(p, c, 2 * (2 * c.tp + qt) + sub, py, px, Y0, X0);
-                        tma_load_5d(base + kOffQc + (2 * buf + qt) * kContentBytes + sub * kPatchContent, &tm_q,
-                                    bar(kQFull + buf), 0, c.h, X0, Y0, c.b);
-                    }
-                for (int j = 0; j < nblk; ++j, ++blk) {
-                    const uint32_t st = blk % kStages, use = blk / kStages;
-                    if (use > 0 && !mbar_wait(bar(kKEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                    mbar_arrive_expect_tx(bar(kKFull + st), kContentBytes + kPosBytes);
-                    ++k_armed;
-                    int py[2], px[2], Y0[2], X0[2];
-                    for (int sub = 0; sub < 2; ++sub) {
-                        patch_origin(p, c, 2 * j + sub, py[sub], px[sub], Y0[sub], X0[sub]);
-                        tma_load_5d(base + kOffKc + st * kContentBytes + sub * kPatchContent, &tm_k, bar(kKFull + st),
-                                    0, c.h, X0[sub], Y0[sub], c.b);
-                        tma_load_4d(base + kOffKp + st * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKFull + st),
-                                    0, px[sub], py[sub], c.h * p.pos_per_head);
-                    }
-                    if (use > 0 && !mbar_wait(bar(kVEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                    mbar_arrive_expect_tx(bar(kVFull + st), kContentBytes);
-                    ++v_armed;
-                    for (int sub = 0; sub < 2; ++sub)
-                        tma_load_5d(base + kOffV + st * kContentBytes + sub * kPatchContent, &tm_v, bar(kVFull + st),
-                                    0, c.h, X0[sub], Y0[sub], c.b);
+                if (io >= 2 && !mbar_wait_warp(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(kQFull + buf), 2 * kContentBytes);
+                    ++q_armed;
+                    for (int qt = 0; qt < 2; ++qt)
+                        for (int sub = 0; sub < 2; ++sub) {
+                            int py, px, Y0, X0;
+                            patch_origin(p, c, 2 * (2 * c.tp + qt) + sub, py, px, Y0, X0);
+                            tma_load_5d(base + kOffQc + (2 * buf + qt) * kContentBytes + sub * kPatchContent, &tm_q,
+                                        bar(kQFull + buf), 0, c.h, X0, Y0, c.b);
+                        }
                 }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int r256 = lane + 32 * k, qt = r256 >> 7, row = r256 & 127;
+                    int py, px, Y0, X0;
+                    patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+                    const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
+                    const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * R);
+                    constexpr int kChunks = R / 8;                 // 16-byte chunks per row
+                    uint4 v[kChunks];
+#pragma unroll
+                    for (int ck = 0; ck < kChunks; ++ck) v[ck] = __ldg(src + ck);
+                    uint32_t* w = reinterpret_cast<uint32_t*>(v);
+#pragma unroll
+                    for (int e = 0; e < 4 * kChunks; ++e) {
+                        const float lo = __uint_as_float(w[e] << 16) * p.pos_scale;
+                        const float hi = __uint_as_float(w[e] & 0xffff0000u) * p.pos_scale;
+                        w[e] = pack_bf16x2(lo, hi);
+                    }
+                    uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * (2 * R);
+                    const int sw = R == 16 ? (row >> 2) & 1 : (row >> 1) & 3;      // SWIZZLE_32B / SWIZZLE_64B
+#pragma unroll
+                    for (int ck = 0; ck < kChunks; ++ck) *reinterpret_cast<uint4*>(dst + ((ck ^ sw) << 4)) = v[ck];
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar(kQPos + buf));
+                    for (int j = 0; j < nblk; ++j, ++blk) {
+                        const uint32_t st = blk % kStages, use = blk / kStages;
+                        if (use > 0 && !mbar_wait(bar(kKEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                        mbar_arrive_expect_tx(bar(kKFull + st), kContentBytes + kPosBytes);
+                        ++k_armed;
+                        int py[2], px[2], Y0[2], X0[2];
+                        for (int sub = 0; sub < 2; ++sub) {
+                            patch_origin(p, c, 2 * j + sub, py[sub], px[sub], Y0[sub], X0[sub]);
+                            tma_load_5d(base + kOffKc + st * kContentBytes + sub * kPatchContent, &tm_k, bar(kKFull + st),
+                                        0, c.h, X0[sub], Y0[sub], c.b);
+                            tma_load_4d(base + kOffKp + st * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKFull + st),
+                                        0, px[sub], py[sub], c.h * p.pos_per_head);
+                        }
+                        if (use > 0 && !mbar_wait(bar(kVEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                        mbar_arrive_expect_tx(bar(kVFull + st), kContentBytes);
+                        ++v_armed;
+                        for (int sub = 0; sub < 2; ++sub)
+                            tma_load_5d(base + kOffV + st * kContentBytes + sub * kPatchContent, &tm_v, bar(kVFull + st),
+                                        0, c.h, X0[sub], Y0[sub], c.b);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 // Gave up: let the copies already in flight land before the CTA may exit.
                 for (uint32_t b2 = q_armed > 2u ? q_armed - 2 : 0; b2 < q_armed; ++b2)
                     mbar_wait(bar(kQFull + (b2 & 1)), (b2 >> 1) & 1, abort_flag + 1, p.status);
@@ -198,290 +304,408 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 for (uint32_t b2 = v_armed > (uint32_t)kStages ? v_armed - kStages : 0; b2 < v_armed; ++b2)
                     mbar_wait(bar(kVFull + b2 % kStages), (b2 / kStages) & 1, abort_flag + 1, p.status);
             }
-        }
-    } else if (warp == 1 || warp == 3) {
-        // ===================================== MMA issuers: warp 1 drives query tile 0, warp 3 tile 1
-        // Per block b of this CTA's items: S(b) as soon as the softmax warps have taken S(b-1) out
-        // of tensor memory, then PV(b-1) once P(b-1) is there.  The whole warp walks the loop and
-        // waits; one elected lane issues (this keeps descriptors in uniform registers).
-        const int qt = warp >> 1;
-        constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
-        const uint32_t d_s = tmem + kColS + qt * kTile, d_o = tmem + kColO + qt * 2 * kD, a_p = tmem + kColP + qt * (kTile / 2);
-        uint32_t b = 0, io = 0;
-        bool ok = true;
-        // O_q[half] += P_q[:, half] V[half] for block `pb` (first: the first block of item ordinal `pio`)
-        auto do_pv = [&](uint32_t pb, bool first, uint32_t pio) -> bool {
-            const uint32_t st = pb % kStages;
-            // warp-uniform outcomes, so that the warp stays converged
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kVFull + st), (pb / kStages) & 1, abort_flag, p.status) &&
-                                             (!first || pio == 0 || mbar_wait(bar(kOFree + qt), (pio - 1) & 1, abort_flag, p.status))))
-                return false;
-            const uint64_t v = smem_desc_at(kDesc64, base + kOffV + st * kContentBytes);
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(kPReady + 2 * qt + half), pb & 1, abort_flag, p.status))) return false;
-                tc_fence_after();
-                if (elect_one()) {
-                    mma_ts(d_o + half * kD, a_p + 32 * half, v + 256 * half, kIdescPV, first ? 0u : 1u);
-#pragma unroll
-                    for (int kk = 1; kk < 4; ++kk)
-                        mma_ts(d_o + half * kD, a_p + 32 * half + 8 * kk, v + 256 * half + 64 * kk, kIdescPV, 1u);
-                    mma_commit(bar(kPFree + 2 * qt + half));
-                    if (half == 1) mma_commit(bar(kVEmpty + st));
-                }
-                __syncwarp();
-            }
-            return true;
-        };
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++io) {
-            const uint32_t buf = io & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) &&
-                                             mbar_wait(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status))) { ok = false; break; }
-            const uint64_t qc = smem_desc_at(kDesc64, base + kOffQc + (2 * buf + qt) * kContentBytes);
-            const uint64_t qp = smem_desc_at(R == 16 ? kDesc32 : kDesc64, base + kOffQp + (2 * buf + qt) * kPosBytes);
-            for (int j = 0; j < nblk; ++j, ++b) {
-                const uint32_t st = b % kStages;
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(kKFull + st), (b / kStages) & 1, abort_flag, p.status) &&
-                                                 (b == 0 || mbar_wait(bar(kSFree + qt), (b - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
-                tc_fence_after();
-                if (elect_one()) {
+        } else if (warp == 1) {
+            // ===================================== issuer of S = Q~ K~^T for both query tiles
+            // Three issuing warps (this one and one per tile for PV): a warp that is held in the issue of one group of
+            // MMAs, or waits for the softmax warps, keeps nobody else from issuing.  The whole warp walks the loop
+            // and waits; one elected lane issues (this keeps descriptors in uniform registers).
+            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
+            for (int i = 0; i < count && ok; ++i, ++io) {
+                const uint32_t buf = io & 1;
+                if (!mbar_wait_warp(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) ||
+                    !mbar_wait_warp(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                for (int j = 0; j < nblk && ok; ++j, ++blk) {
+                    const uint32_t st = blk % kStages;
+                    if (!mbar_wait_warp(bar(kKFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
                     const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
                     const uint64_t kp = smem_desc_at(R == 16 ? kDesc32 : kDesc64, base + kOffKp + st * kPosBytes);
-                    mma_ss(d_s, qc, kc, kIdescS, 0u);
-                    mma_ss(d_s, qc + 2, kc + 2, kIdescS, 1u);          // + 32 bytes: second K16 step of the content rows
-                    mma_ss(d_s, qp, kp, kIdescS, 1u);
-                    if (R == 32) mma_ss(d_s, qp + 2, kp + 2, kIdescS, 1u);
-                    mma_commit(bar(kSFull + qt));
-                    mma_commit(bar(kKEmpty + st));
-                    if (j == nblk - 1) mma_commit(bar(kQEmpty + buf));
+#pragma unroll
+                    for (int qt = 0; qt < 2; ++qt) {
+                        // the softmax warps have taken S(b-1) of this tile out of tensor memory
+                        if (blk > 0 && !mbar_wait_warp(bar(kSFree + qt), (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint64_t qc = smem_desc_at(kDesc64, base + kOffQc + (2 * buf + qt) * kContentBytes);
+                            const uint64_t qp = smem_desc_at(R == 16 ? kDesc32 : kDesc64, base + kOffQp + (2 * buf + qt) * kPosBytes);
+                            const uint32_t d_s = tmem + kColS + qt * kTile;
+                            mma_ss(d_s, qc, kc, kIdescS, 0u);
+                            mma_ss(d_s, qc + 2, kc + 2, kIdescS, 1u);          // + 32 bytes: second K16 step of the content rows
+                            mma_ss(d_s, qp, kp, kIdescS, 1u);
+                            if (R == 32) mma_ss(d_s, qp + 2, kp + 2, kIdescS, 1u);
+                            mma_commit(bar(kSFull + qt));
+                            if (qt == 1) {
+                                mma_commit(bar(kKEmpty + st));
+                                if (j == nblk - 1) mma_commit(bar(kQEmpty + buf));
+                            }
+                        }
+                        __syncwarp();
+                    }
                 }
-                __syncwarp();
-                if (b > 0 && !do_pv(b - 1, j == 1, io)) { ok = false; break; }
             }
-        }
-        if (ok && b > 0) do_pv(b - 1, false, io);
-        // everything issued by this warp's leader must have finished before TMEM is released
-        if (elect_one()) mma_commit(bar(kDrain + qt));
-        __syncwarp();
-        mbar_wait(bar(kDrain + qt), 0, abort_flag + 1, p.status);
-    } else if (warp == 2) {
-        // ====================== query RIB rows of the coming items: bf16(Pq * sqrt(d/r)), SWIZZLE_32B
-        uint32_t io = 0;
-        for (int item = blockIdx.x; item < p.items; item += gridDim.x, ++io) {
-            const ItemCoord c = decode_item(p, item);
-            const uint32_t buf = io & 1;
-            if (io >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status))) break;
+        } else if (warp < 4) {
+            // ===================================== issuers of O_q (+)= P_q V: warp 2 for query tile 0, warp 3 for tile 1
+            const int qt = warp - 2;
+            constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B);
+            const uint32_t a_p = tmem + kColP + qt * (kTile / 2);
+            const uint32_t d_o = tmem + kColO + qt * 2 * kD;              // exact form: one accumulator per key half
+            const uint32_t d_o1 = tmem + kColO + qt * kFastOCols;         // fast form: one accumulator
+            for (int i = 0; i < count && ok; ++i, ++io) {
+                for (int j = 0; j < nblk; ++j, ++blk) {
+                    const uint32_t st = blk % kStages;
+                    // warp-uniform outcomes, so that the warp stays converged.  The first block of an item overwrites the
+                    // accumulator: the epilogue of the item before must have read it.
+                    if (!mbar_wait_warp(bar(kVFull + st), (blk / kStages) & 1, abort_flag, p.status) ||
+                        !(j > 0 || io == 0 || mbar_wait_warp(bar(kOFree + qt), (io - 1) & 1, abort_flag, p.status)) ||
+                        !mbar_wait_warp(bar(kPReady + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint32_t v_addr = base + kOffV + st * kContentBytes;
+                        if (fast) {
+                            // [V | ones] as one MN-major operand of 48 columns, the second 32-column atom `lbo` bytes behind the first
+                            const uint64_t v = smem_desc(v_addr, kOffOnes - (kOffV + st * kContentBytes), 512, kSwizzle64B);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int r256 = lane + 32 * k, qt = r256 >> 7, row = r256 & 127;
-                int py, px, Y0, X0;
-                patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
-                const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
-                const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * R);
-                constexpr int kChunks = R / 8;                 // 16-byte chunks per row
-                uint4 v[kChunks];
+                            for (int kk = 0; kk < 8; ++kk)
+                                mma_ts(d_o1, a_p + 8 * kk, v + 64 * kk, kIdescPV1, (j == 0 && kk == 0) ? 0u : 1u);
+                        } else {
+                            const uint64_t v = smem_desc_at(kDesc64, v_addr);
 #pragma unroll
-                for (int ck = 0; ck < kChunks; ++ck) v[ck] = __ldg(src + ck);
-                uint32_t* w = reinterpret_cast<uint32_t*>(v);
-#pragma unroll
-                for (int i = 0; i < 4 * kChunks; ++i) {
-                    const float lo = __uint_as_float(w[i] << 16) * p.pos_scale;
-                    const float hi = __uint_as_float(w[i] & 0xffff0000u) * p.pos_scale;
-                    w[i] = pack_bf16x2(lo, hi);
+                            for (int kk = 0; kk < 8; ++kk)     // keys 16 kk ..: key half kk / 4 has its own accumulator
+                                mma_ts(d_o + (kk >> 2) * kD, a_p + 8 * kk, v + 64 * kk, kIdescPV, (j == 0 && (kk & 3) == 0) ? 0u : 1u);
+                        }
+                        mma_commit(bar(kPFree + qt));
+                        mma_commit(bar(kVEmpty + st));
+                    }
+                    __syncwarp();
                 }
-                uint8_t* dst = base_ptr + kOffQp + (2 * buf + qt) * kPosBytes + row * (2 * R);
-                const int sw = R == 16 ? (row >> 2) & 1 : (row >> 1) & 3;      // SWIZZLE_32B / SWIZZLE_64B
-#pragma unroll
-                for (int ck = 0; ck < kChunks; ++ck) *reinterpret_cast<uint4*>(dst + ((ck ^ sw) << 4)) = v[ck];
             }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kQPos + buf));
-        }
-    } else {
-        // ================ softmax + epilogue: two threads per query row, one per half of the keys
-        const int qt = (warp - 4) >> 3;
-        const int half = ((warp - 4) >> 2) & 1;
-        const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;                 // row of the tile == TMEM lane
-        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + kColS + qt * kTile + half * 64;
-        const uint32_t t_o = tmem + lane_base + kColO + qt * 2 * kD;        // both halves' accumulators
-        const uint32_t t_p = tmem + lane_base + kColP + qt * (kTile / 2) + half * 32;
-        const uint32_t b_ready = bar(kPReady + 2 * qt + half), b_free = bar(kPFree + 2 * qt + half);
-        float2* merge = reinterpret_cast<float2*>(base_ptr + kOffMerge) + qt * 2 * kTile;   // [half][row]
-        const float rescale_threshold = 8.0f / p.scale_log2;    // raw-logit units: p stays <= 2^8
-        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
-        uint32_t blk = 0, nitem = 0;
-        bool ok = true;
-        // exp2 of 32 scores against the reference -m * log2e/sqrt(d); returns their sum
-        auto exp_chunk = [&](const uint32_t (&s)[32], float neg_ms, uint32_t (&packed)[16]) -> float {
-            const float2 neg2 = make_float2(neg_ms, neg_ms);
-            float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+        } else {
+            // ================ softmax + epilogue: two threads per query row, one per half of the keys
+            const int qt = (warp - 4) >> 3;
+            const int half = ((warp - 4) >> 2) & 1;
+            const int quarter = warp & 3;
+            const int row = quarter * 32 + lane;                 // row of the tile == TMEM lane
+            const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+            const uint32_t t_s = tmem + lane_base + kColS + qt * kTile + half * 64;
+            const uint32_t t_p = tmem + lane_base + kColP + qt * (kTile / 2) + half * 32;
+            const uint32_t b_ready = bar(kPReady + qt), b_free = bar(kPFree + qt);   // P of the tile: both key halves
+            const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+
+            if (fast) {
+                // ------------------------------------------------------------------ fast form
+                const uint32_t t_o1 = tmem + lane_base + kColO + qt * kFastOCols;
+                // exp2 of 32 scores against the fixed reference, packed to bf16 pairs
+                auto exp_chunk1 = [&](const uint32_t (&s)[32], float2 neg2, uint32_t (&packed)[16]) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg2);
-                // the exp (MUFU) pipe is the busiest unit of this kernel: every fourth pair goes to the FMA pipe instead
-                const float2 e = (i & 3) == 3 ? ex2_poly2(x) : make_float2(ex2_approx(x.x), ex2_approx(x.y));
-                if (i & 1) sum_b = __fadd2_rn(sum_b, e); else sum_a = __fadd2_rn(sum_a, e);
-                packed[i] = pack_bf16x2(e.x, e.y);
-            }
-            return (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
-        };
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++nitem) {
-            const ItemCoord c = decode_item(p, item);
-            float m_used = -INFINITY, l = 0.f;
-            bool have_ref = false;            // kPartial: a block with real keys has set the reference
-            for (int j = 0; j < nblk; ++j, ++blk) {
-                // warp-uniform outcome: the TMEM loads below are warp-collective
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(kSFull + qt), blk & 1, abort_flag, p.status))) { ok = false; break; }
-                tc_fence_after();
-                bool p_free = blk == 0;       // P (and O) of this half are free once the previous block's PV has completed
-                if (kPartial) {
-                    // this thread's 64 keys are one 8x8 patch: beyond the image it holds no tokens
+                    for (int i = 0; i < 16; ++i) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg2);
+                        const float2 e = ((kPolyMask >> (i & 7)) & 1u) ? ex2_poly2_ranged(x) : make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        packed[i] = pack_bf16x2(e.x, e.y);
+                    }
+                };
+                // The epilogue of an item is run inside the first block of the NEXT item, between its exponentials and its
+                // P store: by then the last PV of the item has completed long ago (it is the very completion the P store
+                // has to wait for anyway), so nobody waits for the tensor pipe at an item boundary.
+                __nv_bfloat16* pend_out = nullptr;          // this thread's half row of the pending item
+                const __nv_bfloat16* pend_gate = nullptr;
+                float* pend_lse = nullptr;
+                float pend_ref = 0.f;
+                int pend_ordinal = -1;                      // -1: nothing pending
+                // O and l of the pending item are complete (the caller has waited for its last PV): normalise, store, note overflow
+                auto epilogue = [&]() {
+                    uint32_t o[16], lsum[1];
+                    tmem_ld16(t_o1 + half * 16, o);
+                    tmem_ld1(t_o1 + kD, lsum);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kOFree + qt));
+                    const float l_all = __uint_as_float(lsum[0]);
+                    // a score left the range the fixed reference covers: the exact form redoes the item
+                    const bool bad = !(l_all > 0.f && l_all < 1.2676506e30f);     // 2^100
+                    if (__any_sync(0xffffffffu, bad) && lane == 0) {
+                        const int slot = atomicAdd(redo_count, 1);
+                        if (slot < kMaxRedo) redo_list[slot] = pend_ordinal;
+                    }
+                    const float w_o = 1.f / l_all;
+                    uint4* dst = reinterpret_cast<uint4*>(pend_out);
+                    const uint4* gsrc = reinterpret_cast<const uint4*>(pend_gate);
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t w[4];
+                        uint4 gv = make_uint4(0u, 0u, 0u, 0u);
+                        if (kGated) gv = __ldg(gsrc + g);
+                        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int e = 8 * g + 2 * k;
+                            float lo = __uint_as_float(o[e]) * w_o, hi = __uint_as_float(o[e + 1]) * w_o;
+                            if (kGated) { lo *= __uint_as_float(gw[k] << 16); hi *= __uint_as_float(gw[k] & 0xffff0000u); }
+                            w[k] = pack_bf16x2(lo, hi);
+                        }
+                        dst[g] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    if (pend_lse) *pend_lse = pend_ref * p.inv_sqrt_d + logf(l_all);
+                    pend_ordinal = -1;
+                };
+                for (int i = 0; i < count && ok; ++i, ++io) {
+                    const int item = item_at(i);
+                    const ItemCoord c = decode_item(p, item);
+                    // where this thread's half row of the item goes
                     int py, px, Y0, X0;
-                    patch_origin(p, c, 2 * j + half, py, px, Y0, X0);
-                    if (Y0 >= p.H || X0 >= p.W) {
+                    patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+                    const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
+                    const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
+                    __nv_bfloat16* const out_row = p.out + tok * kD + half * 16;
+                    const __nv_bfloat16* const gate_row = kGated ? p.gate + tok * kD + half * 16 : nullptr;
+                    float* const lse_row = (p.lse && half == 0) ? p.lse + (((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X : nullptr;
+                    float m_ref = 0.f;
+                    float2 neg2 = make_float2(0.f, 0.f);
+                    for (int j = 0; j < nblk; ++j, ++blk) {
+                        // warp-uniform outcome: the TMEM loads below are warp-collective
+                        if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        uint32_t sa[32], sb[32];
+                        if (j == 0) {
+                            // the row's reference: the maximum over keys 0-31 of the window, the same for both key halves
+                            tmem_ld32(tmem + lane_base + kColS + qt * kTile, sa);
+                            tmem_wait_ld();
+                            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4) {
+                                mx0 = max3(mx0, __uint_as_float(sa[e]), __uint_as_float(sa[e + 1]));
+                                mx1 = max3(mx1, __uint_as_float(sa[e + 2]), __uint_as_float(sa[e + 3]));
+                            }
+                            m_ref = fmaxf(mx0, mx1);
+                            const float neg = -m_ref * p.scale_log2;
+                            neg2 = make_float2(neg, neg);
+                        }
+                        // all 64 scores of this thread at once: the accumulator goes back to the MMA warp before any exponential
+                        tmem_ld32(t_s, sa);
+                        tmem_ld32(t_s + 32, sb);
+                        tmem_wait_ld();
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(kSFree + qt));
-                        if (!p_free) {
-                            if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                        if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
+                        uint32_t pa[16], pb[16];
+                        exp_chunk1(sa, neg2, pa);
+                        exp_chunk1(sb, neg2, pb);
+                        // P of the tile is free once the previous block's PV has completed (long ago, as a rule)
+                        if (blk > 0) {
+                            if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                             tc_fence_after();
                         }
-                        uint32_t zero[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) zero[i] = 0u;
-                        tmem_st16(t_p, zero);
-                        tmem_st16(t_p + 16, zero);
+                        if (j == 0 && pend_ordinal >= 0) epilogue();      // that PV was the last one of the item before
+                        tmem_st16(t_p, pa);
+                        tmem_st16(t_p + 16, pb);
                         tmem_wait_st();
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(b_ready);
-                        continue;
                     }
+                    if (!ok) break;
+                    pend_out = out_row; pend_gate = gate_row; pend_lse = lse_row; pend_ref = m_ref; pend_ordinal = i;
                 }
-                const bool first_ref = kPartial ? !have_ref : j == 0;
-                have_ref = true;
+                if (ok && pend_ordinal >= 0) {
+                    // the last item of the pass
+                    if (mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { tc_fence_after(); epilogue(); } else ok = false;
+                }
+            } else {
+                // ------------------------------------------------------------------ exact form
+                const uint32_t t_o = tmem + lane_base + kColO + qt * 2 * kD;        // both halves' accumulators
+                float2* merge = reinterpret_cast<float2*>(base_ptr + kOffMerge) + qt * 2 * kTile;   // [half][row]
+                const float rescale_threshold = 8.0f / p.scale_log2;    // raw-logit units: p stays <= 2^8
+                // exp2 of 32 scores against the reference -m * log2e/sqrt(d); returns their sum
+                auto exp_chunk = [&](const uint32_t (&s)[32], float neg_ms, uint32_t (&packed)[16]) -> float {
+                    const float2 neg2 = make_float2(neg_ms, neg_ms);
+                    float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    uint32_t s[32];
-                    tmem_ld32(t_s + 32 * ch, s);
-                    tmem_wait_ld();
-                    float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
-                        mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+                    for (int i = 0; i < 16; ++i) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg2);
+                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        if (i & 1) sum_b = __fadd2_rn(sum_b, e); else sum_a = __fadd2_rn(sum_a, e);
+                        packed[i] = pack_bf16x2(e.x, e.y);
                     }
-                    const float mx = fmaxf(mx0, mx1);
-                    if (first_ref && ch == 0) {
-                        m_used = mx;
-                    } else {
-                        // Move the reference (and rescale O, l) only when the maximum grew by more than
-                        // the threshold; the result is exact after the final normalisation because l
-                        // carries the same reference.
-                        const bool need = mx > m_used + rescale_threshold;
-                        if (__any_sync(0xffffffffu, need)) {
+                    return (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+                };
+                for (int i = 0; i < count && ok; ++i, ++io, ++nmerge) {
+                    const int item = item_at(i);
+                    const ItemCoord c = decode_item(p, item);
+                    float m_used = -INFINITY, l = 0.f;
+                    bool have_ref = false;            // kPartial: a block with real keys has set the reference
+                    for (int j = 0; j < nblk; ++j, ++blk) {
+                        // warp-uniform outcome: the TMEM loads below are warp-collective
+                        if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        bool p_free = blk == 0;       // P (and O) of this half are free once the previous block's PV has completed
+                        if (kPartial) {
+                            // this thread's 64 keys are one 8x8 patch: beyond the image it holds no tokens
+                            int py, px, Y0, X0;
+                            patch_origin(p, c, 2 * j + half, py, px, Y0, X0);
+                            if (Y0 >= p.H || X0 >= p.W) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(bar(kSFree + qt));
+                                if (!p_free) {
+                                    if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                                    tc_fence_after();
+                                }
+                                uint32_t zero[16];
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) zero[e] = 0u;
+                                tmem_st16(t_p, zero);
+                                tmem_st16(t_p + 16, zero);
+                                tmem_wait_st();
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(b_ready);
+                                continue;
+                            }
+                        }
+                        const bool first_ref = kPartial ? !have_ref : j == 0;
+                        have_ref = true;
+#pragma unroll
+                        for (int ch = 0; ch < 2; ++ch) {
+                            uint32_t s[32];
+                            tmem_ld32(t_s + 32 * ch, s);
+                            tmem_wait_ld();
+                            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4) {
+                                mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+                                mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+                            }
+                            const float mx = fmaxf(mx0, mx1);
+                            if (first_ref && ch == 0) {
+                                m_used = mx;
+                            } else {
+                                // Move the reference (and rescale O, l) only when the maximum grew by more than
+                                // the threshold; the result is exact after the final normalisation because l
+                                // carries the same reference.
+                                const bool need = mx > m_used + rescale_threshold;
+                                if (__any_sync(0xffffffffu, need)) {
+                                    if (!p_free) {
+                                        if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                                        tc_fence_after();
+                                        p_free = true;
+                                    }
+                                    const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
+                                    if (need) { l *= factor; m_used = mx; }
+                                    if (j > 0) {
+                                        uint32_t o[32];
+                                        tmem_ld32(t_o + half * kD, o);
+                                        tmem_wait_ld();
+#pragma unroll
+                                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                                        tmem_st32(t_o + half * kD, o);
+                                    }
+                                    if (ch == 1) {
+                                        // the first 32 keys of this block were exponentiated against the old
+                                        // reference: redo them (their sum is already in l, rescaled above)
+                                        uint32_t s0[32], packed0[16];
+                                        tmem_ld32(t_s, s0);
+                                        tmem_wait_ld();
+                                        exp_chunk(s0, -m_used * p.scale_log2, packed0);
+                                        tmem_st16(t_p, packed0);
+                                    }
+                                    tmem_wait_st();
+                                }
+                            }
+                            if (ch == 1) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
+                            }
+                            uint32_t packed[16];
+                            l += exp_chunk(s, -m_used * p.scale_log2, packed);
                             if (!p_free) {
-                                if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
+                                if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                                 tc_fence_after();
                                 p_free = true;
                             }
-                            const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
-                            if (need) { l *= factor; m_used = mx; }
-                            if (j > 0) {
-                                uint32_t o[32];
-                                tmem_ld32(t_o + half * kD, o);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                                tmem_st32(t_o + half * kD, o);
-                            }
-                            if (ch == 1) {
-                                // the first 32 keys of this block were exponentiated against the old
-                                // reference: redo them (their sum is already in l, rescaled above)
-                                uint32_t s0[32], packed0[16];
-                                tmem_ld32(t_s, s0);
-                                tmem_wait_ld();
-                                exp_chunk(s0, -m_used * p.scale_log2, packed0);
-                                tmem_st16(t_p, packed0);
-                            }
-                            tmem_wait_st();
+                            tmem_st16(t_p + 16 * ch, packed);
                         }
-                    }
-                    if (ch == 1) {
+                        if (!ok) break;
+                        tmem_wait_st();
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
+                        if (lane == 0) mbar_arrive(b_ready);
                     }
-                    uint32_t packed[16];
-                    l += exp_chunk(s, -m_used * p.scale_log2, packed);
-                    if (!p_free) {
-                        if (!__all_sync(0xffffffffu, mbar_wait(b_free, (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
-                        tc_fence_after();
-                        p_free = true;
+                    if (!ok) break;
+                    // ---- merge the two key halves and write this thread's 16 output columns
+                    merge[half * kTile + row] = make_float2(m_used, l);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kMerge + 4 * qt + quarter));
+                    // The partner's (m, l) must be there and the item's last PV must have completed.
+                    if (!mbar_wait_warp(bar(kMerge + 4 * qt + quarter), nmerge & 1, abort_flag, p.status) ||
+                        !mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    uint32_t oa[16], ob[16];
+                    tmem_ld16(t_o + half * 16, oa);
+                    tmem_ld16(t_o + kD + half * 16, ob);
+                    tmem_wait_ld();
+                    const float2 other = merge[(half ^ 1) * kTile + row];
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kOFree + qt));
+                    const float m_a = half ? other.x : m_used, l_a = half ? other.y : l;
+                    const float m_b = half ? m_used : other.x, l_b = half ? l : other.y;
+                    const float m = fmaxf(m_a, m_b);
+                    const float f_a = ex2_approx((m_a - m) * p.scale_log2), f_b = ex2_approx((m_b - m) * p.scale_log2);
+                    const float l_all = l_a * f_a + l_b * f_b;
+                    const float w_a = f_a / l_all, w_b = f_b / l_all;
+                    int py, px, Y0, X0;
+                    patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
+                    const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
+                    if (kPartial && (Y0 >= p.H || X0 >= p.W)) continue;        // a patch of the extension: no tokens, nothing to store
+                    const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD + half * 16);
+                    const uint4* gsrc = reinterpret_cast<const uint4*>(p.gate + tok * kD + half * 16);
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t w[4];
+                        uint4 gv = make_uint4(0u, 0u, 0u, 0u);
+                        if (kGated) gv = __ldg(gsrc + g);
+                        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int e = 8 * g + 2 * k;
+                            float lo = __uint_as_float(oa[e]) * w_a + __uint_as_float(ob[e]) * w_b;
+                            float hi = __uint_as_float(oa[e + 1]) * w_a + __uint_as_float(ob[e + 1]) * w_b;
+                            if (kGated) { lo *= __uint_as_float(gw[k] << 16); hi *= __uint_as_float(gw[k] & 0xffff0000u); }
+                            w[k] = pack_bf16x2(lo, hi);
+                        }
+                        dst[g] = make_uint4(w[0], w[1], w[2], w[3]);
                     }
-                    tmem_st16(t_p + 16 * ch, packed);
+                    if (p.lse && half == 0)
+                        p.lse[(((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X] = m * p.inv_sqrt_d + logf(l_all);
                 }
-                if (!ok) break;
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(b_ready);
             }
-            if (!ok) break;
-            // ---- merge the two key halves and write this thread's 16 output columns
-            merge[half * kTile + row] = make_float2(m_used, l);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kMerge + 4 * qt + quarter));
-            // The partner's (m, l) must be there and both halves' last PV must have completed.  The
-            // merge barrier comes first: a parity wait on the partner's PV barrier is only meaningful once
-            // the partner has passed its own last block (otherwise an older phase of equal parity answers).
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(kMerge + 4 * qt + quarter), nitem & 1, abort_flag, p.status) &&
-                                             mbar_wait(bar(kPFree + 2 * qt + half), (blk - 1) & 1, abort_flag, p.status) &&
-                                             mbar_wait(bar(kPFree + 2 * qt + (half ^ 1)), (blk - 1) & 1, abort_flag, p.status))) { ok = false; break; }
-            tc_fence_after();
-            uint32_t oa[16], ob[16];
-            tmem_ld16(t_o + half * 16, oa);
-            tmem_ld16(t_o + kD + half * 16, ob);
-            tmem_wait_ld();
-            const float2 other = merge[(half ^ 1) * kTile + row];
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kOFree + qt));
-            const float m_a = half ? other.x : m_used, l_a = half ? other.y : l;
-            const float m_b = half ? m_used : other.x, l_b = half ? l : other.y;
-            const float m = fmaxf(m_a, m_b);
-            const float f_a = ex2_approx((m_a - m) * p.scale_log2), f_b = ex2_approx((m_b - m) * p.scale_log2);
-            const float l_all = l_a * f_a + l_b * f_b;
-            const float w_a = f_a / l_all, w_b = f_b / l_all;
-            int py, px, Y0, X0;
-            patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
-            const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
-            if (kPartial && (Y0 >= p.H || X0 >= p.W)) continue;        // a patch of the extension: no tokens, nothing to store
-            const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD + half * 16);
-            const uint4* gsrc = reinterpret_cast<const uint4*>(p.gate + tok * kD + half * 16);
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                uint32_t w[4];
-                uint4 gv = make_uint4(0u, 0u, 0u, 0u);
-                if (kGated) gv = __ldg(gsrc + i);
-                const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int e = 8 * i + 2 * k;
-                    float lo = __uint_as_float(oa[e]) * w_a + __uint_as_float(ob[e]) * w_b;
-                    float hi = __uint_as_float(oa[e + 1]) * w_a + __uint_as_float(ob[e + 1]) * w_b;
-                    if (kGated) { lo *= __uint_as_float(gw[k] << 16); hi *= __uint_as_float(gw[k] & 0xffff0000u); }
-                    w[k] = pack_bf16x2(lo, hi);
-                }
-                dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            if (p.lse && half == 0)
-                p.lse[(((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X] = m * p.inv_sqrt_d + logf(l_all);
         }
+        if (pass == 1 || !fast) break;                   // CTA-uniform: `fast` depends on the kernel arguments only
+        // ---- between the passes: every role has finished its items; has the fast form noted any?
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        const int notes = *redo_count;
+        if (notes == 0 || abort_flag[0]) break;          // CTA-uniform: shared memory read after the barrier
+        if (threadIdx.x == 0 && notes <= kMaxRedo) {
+            // several warps may have noted the same item: keep each ordinal once
+            int kept = 0;
+            for (int a = 0; a < notes; ++a) {
+                const int v = redo_list[a];
+                bool seen = false;
+                for (int b2 = 0; b2 < kept; ++b2) seen = seen || redo_list[b2] == v;
+                if (!seen) redo_list[kept++] = v;
+            }
+            *redo_count = kept;
+        }
+        __syncthreads();
+    }
+    if (warp >= 1 && warp < 4) {
+        // everything issued by this warp's leader must have finished before TMEM is released
+        if (elect_one()) mma_commit(bar(kDrain + warp - 1));
+        __syncwarp();
+        mbar_wait(bar(kDrain + warp - 1), 0, abort_flag + 1, p.status);
     }
     // ================================================================================ common tail
     tc_fence_before();
@@ -524,6 +748,9 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_scale = sqrtf((float)p.d / (float)p.r);
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
+    fp.exact_only = p.exact_softmax ? 1 : 0;
+    fp.div_tp = make_fast_div(fp.tiles_per_item_pair); fp.div_heads = make_fast_div(p.heads);
+    fp.div_nwx = make_fast_div(p.nWx); fp.div_nwy = make_fast_div(p.nWy); fp.div_per_row = make_fast_div(p.M >> 3);
     const int grid = fp.items < sm_count ? fp.items : sm_count;
     { ProfileScope scope(RIB_KERNEL_FWD_MAIN, stream); rib_fwd_sm100_kernel<R, kPartial, kGated><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_pk, fp); }
     return cudaGetLastError();

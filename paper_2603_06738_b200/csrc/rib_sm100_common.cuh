@@ -23,6 +23,25 @@ constexpr uint32_t kPatchContent = kContentBytes / 2, kPatchPos = kPosBytes / 2;
 // row-major over the window), at row (w / 8) % 8 and column w % 8 of the patch.
 struct WindowGeom { int H, W, M, s; };
 
+// Division of a non-negative int below 2^31 by a constant set on the host: q = (n * mul) >> shr, exact for every
+// such n (mul = floor(2^shr / d) + 1 with shr = 31 + ceil(log2 d), so the error term n * (mul * d - 2^shr) stays
+// below 2^shr).  The kernels decode work items with it instead of the emulated 32-bit division.
+struct FastDiv {
+    uint32_t mul, shr, d;
+    __host__ __device__ __forceinline__ int div(int n) const { return (int)(((unsigned long long)(uint32_t)n * mul) >> shr); }
+    __host__ __device__ __forceinline__ void divmod(int n, int& q, int& r) const { q = div(n); r = n - q * (int)d; }
+};
+inline FastDiv make_fast_div(int d)
+{
+    uint32_t l = 0;
+    while ((1u << l) < (uint32_t)d) ++l;
+    FastDiv f;
+    f.shr = 31 + l;
+    f.mul = (uint32_t)(((1ull << f.shr) / (uint32_t)d) + 1ull);
+    f.d = (uint32_t)d;
+    return f;
+}
+
 // Patch `sp` of window (wy, wx): top-left token in window coordinates (py, px) and in shifted,
 // wrapped image coordinates (Y0, X0).
 __host__ __device__ __forceinline__ void patch_origin(const WindowGeom& g, int wy, int wx, int sp, int& py, int& px,
@@ -31,6 +50,18 @@ __host__ __device__ __forceinline__ void patch_origin(const WindowGeom& g, int w
     const int per_row = g.M >> 3;
     py = (sp / per_row) << 3;
     px = (sp % per_row) << 3;
+    Y0 = wy * g.M + py + g.s; if (Y0 >= g.H) Y0 -= g.H;
+    X0 = wx * g.M + px + g.s; if (X0 >= g.W) X0 -= g.W;
+}
+
+// The same with the division by the patches per window row prepared on the host.
+__device__ __forceinline__ void patch_origin(const WindowGeom& g, const FastDiv& per_row, int wy, int wx, int sp, int& py, int& px,
+                                             int& Y0, int& X0)
+{
+    int q, r;
+    per_row.divmod(sp, q, r);
+    py = q << 3;
+    px = r << 3;
     Y0 = wy * g.M + py + g.s; if (Y0 >= g.H) Y0 -= g.H;
     X0 = wx * g.M + px + g.s; if (X0 >= g.W) X0 -= g.W;
 }
