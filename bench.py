@@ -5,10 +5,13 @@
 
 One step = one forward and one backward pass of the whole path (window partition + cyclic shift,
 RIB concat, logits, softmax, PV, lse; D pre-pass, the five backward contractions, dPq/dPk
-reduction) over one synthetic batch of the training-patch configuration (B8, 96x96, 6 heads,
-d=32, r=16, window 32, shift 16).  Rank 0 prints ONE JSON line.  With N > 1 every rank runs its
-own batch (pairs are independent: no data-path collective) and the value is the sum over ranks
-divided by the slowest rank's device time.
+reduction) over one synthetic batch of the training configuration (B16, 96x96, 6 heads,
+d=32, r=16, window 32, shift 16: the largest of the five benchmark configurations and the only
+one with a backward pass).  Rank 0 prints ONE JSON line; its `configs` key times each of the five
+configurations in the same run, `exp_ceiling` is the measured exp-pipe roof of the forward pass and
+`parity` compares the timed workload's results with the CPU oracle on every pair.  With N > 1
+every rank runs its own batch (pairs are independent: no data-path collective) and the value is
+the sum over ranks divided by the slowest rank's device time.
 
 `--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
 """
@@ -30,6 +33,7 @@ sys.path.insert(0, str(ROOT))
 METRIC = "rib_window_attn_fwd_bwd_tflops_bf16"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0        # dense bf16, data sheet
 L2_BYTES = 126 * 1000 * 1000
 
 
@@ -46,7 +50,7 @@ def load_peaks():
 def pick_workload(name):
     from paper_2603_06738_b200 import synthetic
     if name is None:
-        base = synthetic.CONFIGS[1]
+        base = synthetic.CONFIGS[4]
         return synthetic.Workload(base.name, base.B, base.H, base.W, base.heads, base.d, base.r, base.window,
                                   base.shift, base.seed, backward=True)
     for wl in synthetic.CONFIGS:
@@ -88,7 +92,7 @@ class ClockSampler(threading.Thread):
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.01)
+            time.sleep(0.001)
 
     def summary(self):
         if not self.sm:
@@ -97,13 +101,14 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.sm)}
 
 
-def cpu_oracle_sample(wl, budget_pairs=None):
-    """Times the CPU oracle, as it stands, on the first pairs of the workload (forward + backward)."""
+def cpu_oracle_sample(wl, budget_pairs=None, keep=None):
+    """Times the CPU oracle, as it stands, on the first pairs of the workload (forward + backward).  With a dict as
+    `keep` and a sample that covers every pair, the oracle's results are left there for the parity check."""
     import numpy as np
     from oracle import rib_oracle as orc
     from paper_2603_06738_b200 import synthetic
     cores = orc.threads()
-    npairs = min(wl.pairs, budget_pairs or 48 * cores)
+    npairs = min(wl.pairs, budget_pairs or 64 * cores)
     # the sampled pairs live in the first images only: generate just those
     per_image = wl.pairs // wl.B
     nb = min(wl.B, -(-npairs // per_image))
@@ -111,10 +116,12 @@ def cpu_oracle_sample(wl, budget_pairs=None):
     t = {k: v.to(dtype=__import__("torch").float64).numpy() for k, v in synthetic.make_inputs(sub, True).items()}
     pairs = list(range(npairs))
     t0 = time.perf_counter()
-    orc.fwd(t["q"], t["k"], t["v"], t["pq"], t["pk"], wl.window, wl.shift, pairs=pairs)
+    f = orc.fwd(t["q"], t["k"], t["v"], t["pq"], t["pk"], wl.window, wl.shift, pairs=pairs)
     t1 = time.perf_counter()
-    orc.bwd(t["q"], t["k"], t["v"], t["pq"], t["pk"], t["dout"], wl.window, wl.shift, pairs=pairs)
+    b = orc.bwd(t["q"], t["k"], t["v"], t["pq"], t["pk"], t["dout"], wl.window, wl.shift, pairs=pairs)
     t2 = time.perf_counter()
+    if keep is not None and npairs == wl.pairs:
+        keep.update(zip(("out", "lse", "dq", "dk", "dv", "dpq", "dpk"), list(f) + list(b)))
     flops = npairs * 2 * wl.n * wl.n * ((2 * wl.d + wl.r) + (5 * wl.d + 3 * wl.r))
     return {"value": flops / (t2 - t0) / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {npairs} of {wl.pairs} pairs of {wl.name}, forward {t1 - t0:.2f} s + backward "
@@ -155,6 +162,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the timings of rank 32, head-wise tables and partial windows")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration timings and the exp-pipe measurement")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -241,6 +249,14 @@ def main():
     for kid, ms in binding.rib_profile_end(prof_capacity):
         per_kernel.setdefault(binding.KERNEL_NAMES.get(kid, str(kid)), []).append(ms)
     status = binding.rib_query_status()
+    # results on the seeded batch (set 0 holds the generator's tensors unrotated), kept for the parity check
+    parity_got = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        res0 = step(sets[0])[2]
+        torch.cuda.synchronize()
+        parity_got = {k: t.detach().to("cpu", torch.float64).numpy()
+                      for k, t in zip(("out", "lse", "dq", "dk", "dv", "dpq", "dpk"), (sets[0]["out"], sets[0]["lse"]) + tuple(res0))}
+        del res0
     fwd_ms = [e[0].elapsed_time(e[1]) for e in ev]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in ev]
     total_ms = ev[0][0].elapsed_time(ev[-1][2])          # device time of exactly K steps
@@ -334,6 +350,86 @@ def main():
                "bwd_us": g1.elapsed_time(g2) * 1e3 / reps, "bound": "launch latency",
                "algorithmic_bytes_fwd": 4 * ((2 + 4 * gL) * gdh + gdh + 2 * gdh * wl.r) + 2 * 2 * wl.n * wl.r,
                "algorithmic_flops_fwd": 2 * wl.n * ((2 + 4 * gL) * gdh + 2 * gdh * wl.r)}
+
+    # ------------------------------------------------ the five benchmark configurations, one by one (rank 0, device-timed)
+    configs, exp_ceiling = None, None
+    if rank == 0 and not args.no_configs:
+        peaks_c, _ = load_peaks()
+        denoms = {"burst": float(peaks_c["bf16_tflops"]), "sustained": float(peaks_c.get("bf16_tflops_sustained", peaks_c["bf16_tflops"])),
+                  "nominal": NOMINAL_BF16_TFLOPS}
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)      # writing it evicts the 126 MB L2
+
+        def launch_times(fn, reps, flushed):
+            """Device time of every launch on its own (CUDA events); optionally with the L2 flushed before each."""
+            for _ in range(10):
+                fn()
+            torch.cuda.synchronize()
+            pairs = []
+            for _ in range(reps):
+                if flushed:
+                    flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                pairs.append((a, b))
+            torch.cuda.synchronize()
+            return [a.elapsed_time(b) for a, b in pairs]
+
+        def figures(ms_list, flops, tokens):
+            med, mn = statistics.median(ms_list), min(ms_list)
+            tf = flops / (med * 1e-3) / 1e12
+            return {"median_ms": med, "min_ms": mn, "tflops": tf, "tflops_at_min": flops / (mn * 1e-3) / 1e12,
+                    "frac_of_peak": {k: tf / v for k, v in denoms.items()}, "tokens_per_s": tokens / (med * 1e-3)}
+
+        configs = {"timing": "50 launches each, one CUDA-event pair per launch, inputs resident and reused (steady state); "
+                             "`l2_flushed`: the same with a 252 MB fill before every launch", "denominators_tflops": denoms}
+        try:
+            for ci, cw in enumerate(synthetic.CONFIGS):
+                shape = (cw.B, cw.H, cw.W, cw.heads, cw.d)
+                cq, ck, cv, cdo = (torch.randn(shape, device=dev).to(torch.bfloat16) for _ in range(4))
+                cpq, cpk = ((0.5 * torch.randn((cw.n, cw.r), device=dev)).to(torch.bfloat16) for _ in range(2))
+                cout = torch.empty_like(cq)
+                clse = torch.empty((cw.B, cw.heads, cw.H, cw.W), dtype=torch.float32, device=dev)
+                f = lambda: binding.rib_window_attn_fwd(cq, ck, cv, cpq, cpk, cw.window, cw.shift, out=cout, lse=clse)
+                entry = {"shape": f"B{cw.B} {cw.H}x{cw.W} h{cw.heads} d{cw.d} r{cw.r} w{cw.window} s{cw.shift}",
+                         "fwd": figures(launch_times(f, 50, False), cw.fwd_flops, cw.tokens)}
+                entry["fwd"]["l2_flushed"] = {k: v for k, v in figures(launch_times(f, 20, True), cw.fwd_flops, cw.tokens).items()
+                                              if k in ("median_ms", "min_ms", "tflops")}
+                entry["fwd"]["path"] = binding.rib_last_path()
+                if cw.fwd_flops < 1e9:
+                    entry["fwd"]["note"] = "launch-bound: the time is the figure, not the TFLOP/s"
+                if ci == 4:
+                    cws = torch.empty(max(binding.rib_window_attn_bwd_workspace(cw.B, cw.H, cw.W, cw.heads, cw.d, cw.r, cw.window), 256),
+                                      dtype=torch.uint8, device=dev)
+                    bfn = lambda: binding.rib_window_attn_bwd(cq, ck, cv, cpq, cpk, cout, clse, cdo, cw.window, cw.shift, workspace=cws)
+                    entry["bwd"] = figures(launch_times(bfn, 50, False), cw.bwd_flops, cw.tokens)
+                    entry["bwd"]["l2_flushed"] = {k: v for k, v in figures(launch_times(bfn, 20, True), cw.bwd_flops, cw.tokens).items()
+                                                  if k in ("median_ms", "min_ms", "tflops")}
+                    del cws
+                configs[f"cfg{ci + 1}"] = entry
+                del cq, ck, cv, cdo, cout, clse
+            # the exp pipe's roof over the forward pass: exponentials per second x 160 flops per score (d = 32, r = 16)
+            sink = torch.zeros(4, device=dev)
+            blocks, iters = 148 * 8, 4096
+            for _ in range(2):
+                n_exp = binding.rib_exp_probe(sink, blocks, iters)
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); n_exp = binding.rib_exp_probe(sink, blocks, iters); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            exps_per_s = n_exp / (min(ts) * 1e-3)
+            ceiling = exps_per_s * 160 / 1e12
+            exp_ceiling = {"exp_per_s": exps_per_s, "flops_per_exp": 160, "tflops": ceiling, "frac_of_burst_peak": ceiling / denoms["burst"],
+                           "kernel": "rib_exp_probe (ex2.approx.f32, 8 independent chains per thread)",
+                           "note": "a forward pass that evaluates every exponential on the MUFU pipe cannot exceed this; the kernel sends "
+                                   "one pair in four to the FMA pipe instead, which moves the roof to 4/3 of it"}
+        except Exception as exc:   # noqa: BLE001
+            configs["error"] = f"{type(exc).__name__}: {exc}"
+        del flush
+        if binding.rib_query_status() != 0:
+            raise SystemExit("device status word set during the per-configuration timings")
 
     # ------------------------------------------------ the path's variants beyond the benchmark shape (rank 0, device-timed)
     variants = None
@@ -429,17 +525,36 @@ def main():
     algo_flops = {"rib_fwd_sm100_kernel": wl.fwd_flops, "generic_fwd_kernel": wl.fwd_flops,
                   "rib_bwd_sm100_kernel": wl.bwd_flops}.get(dominant)
     dom_tf = None if algo_flops is None else algo_flops / (kernels[dominant]["avg_ms"] * 1e-3) / 1e12
-    traffic = None
-    traffic_file = ROOT / "profiles" / "traffic.json"
-    if traffic_file.exists():
+    def recorded_traffic(kernel):
+        """dram bytes per launch from the committed ncu summary, or None when the kernel has changed since (or the
+        capture was taken on another workload and no per-unit scaling is recorded)."""
+        traffic_file = ROOT / "profiles" / "traffic.json"
+        if not traffic_file.exists():
+            return None
         try:
-            rec = json.loads(traffic_file.read_text()).get(dominant)
+            rec = json.loads(traffic_file.read_text()).get(kernel)
             src = ROOT / "paper_2603_06738_b200" / "csrc" / rec["source"]
             # counters taken on an older version of the kernel say nothing about this one
-            if rec["workload"] == wl.name and hashlib.sha256(src.read_bytes()).hexdigest() == rec["source_sha256"]:
-                traffic = rec["dram_bytes_per_launch"]
+            if hashlib.sha256(src.read_bytes()).hexdigest() != rec["source_sha256"]:
+                return None
+            if rec["workload"] == wl.name:
+                return rec["dram_bytes_per_launch"]
+            if rec.get("units"):        # traffic grows with the token-heads a launch processes: scale the smaller capture
+                return rec["dram_bytes_per_launch"] * (wl.tokens * wl.heads) / rec["units"]
         except Exception:
-            traffic = None
+            pass
+        return None
+
+    traffic = recorded_traffic(dominant)
+    fwd_kernel = "rib_fwd_sm100_kernel" if "rib_fwd_sm100_kernel" in kernels else None
+    roofline_fwd = None
+    if fwd_kernel:
+        f_tf = wl.fwd_flops / (kernels[fwd_kernel]["avg_ms"] * 1e-3) / 1e12
+        roofline_fwd = {"bound": "tensor", "kernel": fwd_kernel, "achieved": f_tf, "peak": peak, "unit": "TFLOP/s", "frac": f_tf / peak,
+                        "traffic": recorded_traffic(fwd_kernel), "peak_source": f"bf16_tflops burst, {peak_kind}",
+                        "algorithmic_flops_per_launch": wl.fwd_flops, "avg_launch_ms": kernels[fwd_kernel]["avg_ms"],
+                        "frac_of_exp_ceiling": None if not exp_ceiling else f_tf / exp_ceiling["tflops"],
+                        "target": "0.60 of the dense bf16 peak at windows >= 32 x 32; the measured exp-pipe roof is `exp_ceiling`"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -456,6 +571,9 @@ def main():
                      "frac": None if dom_tf is None else dom_tf / peak, "traffic": traffic,
                      "peak_source": f"bf16_tflops burst, {peak_kind}",
                      "algorithmic_flops_per_launch": algo_flops, "avg_launch_ms": kernels[dominant]["avg_ms"]},
+        "roofline_fwd": roofline_fwd,
+        "exp_ceiling": exp_ceiling,
+        "configs": configs,
         "kernels": kernels,
         "e2e": None if e2e_ms is None else {
             "value": flops_step / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms_max,
@@ -469,7 +587,25 @@ def main():
         "device_status": status,
     }
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = {k: v for k, v in cpu_oracle_sample(wl).items() if k != "seconds"}
+        import numpy as np
+        want = {}
+        # the oracle on every pair of the timed workload (about 10-20 s of host time): the CPU baseline and the parity reference
+        line["cpu_baseline"] = {k: v for k, v in cpu_oracle_sample(wl, budget_pairs=wl.pairs, keep=want).items() if k != "seconds"}
+        if want and parity_got:
+            parity = {"against": "CPU oracle (fp64) on the same seeded bf16 inputs, every pair of the timed workload",
+                      "bounds": {"max_abs": 1e-2, "rel_l2": 5e-3, "dpq_dpk_max_abs": "1e-2 x max|reference| (sums over all pairs)"}}
+            ok_all = True
+            for name, ref in want.items():
+                got = parity_got[name]
+                err = float(np.abs(got - ref).max())
+                rl2 = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+                mref = float(np.abs(ref).max())
+                bound = 1e-2 * max(1.0, mref) if name in ("dpq", "dpk") else 1e-2
+                good = bool(np.isfinite(got).all()) and err <= bound and rl2 <= 5e-3
+                ok_all = ok_all and good
+                parity[name] = {"max_abs": err, "rel_l2": rl2, "max_ref": mref, "ok": good}
+            parity["ok"] = ok_all
+            line["parity"] = parity
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -265,6 +265,28 @@ int rib_generate_features_bwd(const float* w_h, const float* b_h, const float* w
  */
 int rib_query_status(void* stream);
 
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Enqueues one small kernel that allocates
+ * tensor memory and waits for an mbarrier phase that never completes, with a limit of `limit_ns` nanoseconds
+ * (1 .. 100 000 000) instead of the 2 s of the real kernels; when the limit runs out it records the status
+ * word, every warp leaves through the common tail and the tensor memory is freed: the way every tcgen05
+ * kernel of this library gives up.  Afterwards rib_query_status() returns RIB_ERR_DEVICE_WAIT once, then
+ * RIB_OK, and the device is as usable as before.  Returns RIB_OK, RIB_ERR_SHAPE (limit out of range) or
+ * RIB_ERR_CUDA.
+ */
+int rib_wait_probe(unsigned long long limit_ns, void* stream);
+
+/*
+ * Measurement aid for the roofline of the forward pass (Sec. 3.1, Eq. 6: one exponential per score): enqueues a
+ * kernel of `blocks` thread blocks in which every thread evaluates `iters` rounds of 8 independent
+ * ex2.approx.f32, and returns the number of exponentials evaluated (a positive count) or a negative RIB_ERR_*
+ * code.  Timed by the caller (CUDA events around the call), count / time is the exp throughput of the
+ * device; times 2 (2d + r) = 160 flops per score at d = 32, r = 16 it is the TFLOP/s at which a forward pass
+ * that sends every exponential to that pipe stops.  `sink` is a device pointer to at least one float (never
+ * written in practice).  blocks <= 2^20, iters <= 2^24.
+ */
+long long rib_exp_probe(float* sink, int blocks, int iters, void* stream);
+
 /* Human-readable name of a status code; never NULL; static storage. */
 const char* rib_status_string(int status);
 
@@ -282,6 +304,14 @@ int rib_last_path(void);
 
 /* Number of CUDA kernels this library has launched in this process so far (memsets excluded). */
 long long rib_kernel_launches(void);
+
+/*
+ * The tcgen05 kernels address their operands through TMA tensor maps, which depend on the base pointer and the
+ * shape only; the library keeps the last 64 distinct ones, so a call that repeats an earlier call's buffers and
+ * shape encodes none.  Writes how many maps were served from that cache (`hits`) and how many had to be encoded
+ * (`misses`) in this process so far; either pointer may be NULL.
+ */
+void rib_tensor_map_cache_counts(long long* hits, long long* misses);
 
 /*
  * Per-kernel device timing, for benchmarks (not part of the method).  Between rib_profile_begin and

@@ -16,6 +16,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "librib_window_attn.so"
 _lib = None
 
 RIB_OK = 0
+RIB_ERR_DEVICE_WAIT = -7
 RIB_PATH_NONE, RIB_PATH_GENERIC, RIB_PATH_SM100, RIB_PATH_SM100_EXACT = 0, 1, 2, 3
 
 EXPORTS = (
@@ -27,6 +28,7 @@ EXPORTS = (
     "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
     "rib_window_attn_bwd_padded", "rib_window_attn_bwd_padded_workspace",
     "rib_cla_product", "rib_cla_product_bwd", "rib_cla_gate_bwd", "rib_cla_gate_bwd_workspace",
+    "rib_wait_probe", "rib_exp_probe", "rib_tensor_map_cache_counts",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
@@ -106,6 +108,12 @@ def library() -> ctypes.CDLL:
         lib.rib_last_path.argtypes = []
         lib.rib_kernel_launches.restype = ctypes.c_longlong
         lib.rib_kernel_launches.argtypes = []
+        lib.rib_tensor_map_cache_counts.restype = None
+        lib.rib_tensor_map_cache_counts.argtypes = [ctypes.POINTER(ctypes.c_longlong)] * 2
+        lib.rib_wait_probe.restype = ci
+        lib.rib_wait_probe.argtypes = [ctypes.c_ulonglong, vp]
+        lib.rib_exp_probe.restype = ctypes.c_longlong
+        lib.rib_exp_probe.argtypes = [vp, ci, ci, vp]
         _lib = lib
     return _lib
 
@@ -171,6 +179,28 @@ def rib_profile_end(capacity: int) -> list[tuple[int, float]]:
 
 def rib_query_status(stream=None) -> int:
     return int(library().rib_query_status(_stream_ptr(stream)))
+
+
+def rib_tensor_map_cache_counts() -> tuple[int, int]:
+    """(hits, misses) of the library's tensor-map cache in this process."""
+    h, m = ctypes.c_longlong(0), ctypes.c_longlong(0)
+    library().rib_tensor_map_cache_counts(ctypes.byref(h), ctypes.byref(m))
+    return int(h.value), int(m.value)
+
+
+def rib_wait_probe(limit_ns: int, stream=None) -> None:
+    """Enqueue the self-test kernel whose bounded wait runs out after `limit_ns` nanoseconds."""
+    rc = int(library().rib_wait_probe(int(limit_ns), _stream_ptr(stream)))
+    if rc != RIB_OK:
+        raise RibError(rc)
+
+
+def rib_exp_probe(sink, blocks: int, iters: int, stream=None) -> int:
+    """Enqueue the exp-throughput kernel; returns the number of exponentials it evaluates."""
+    n = int(library().rib_exp_probe(_ptr(sink), int(blocks), int(iters), _stream_ptr(stream)))
+    if n < 0:
+        raise RibError(n)
+    return n
 
 
 def rib_window_attn_bwd_workspace(B, H, W, heads, d, r, window) -> int:

@@ -25,14 +25,29 @@ int check_shape(int B, int H, int W, int heads, int d, int r, int window, int sh
     if (d > 64 || r > 64 || (d % 8) || (r % 8)) return RIB_ERR_UNSUPPORTED;
     const long long pairs = (long long)B * ((H + window - 1) / window) * ((W + window - 1) / window) * heads;
     if (pairs > 0x7fffffffLL || (long long)window * window > (1 << 20)) return RIB_ERR_SHAPE;
+    // launch limits of the kernels: the any-shape kernels put n / 16 row groups on grid.y, the tcgen05 kernels count
+    // pairs * key blocks in an int
+    const long long n = (long long)window * window;
+    if (n > 65535LL * 16 || pairs * ((n + 127) / 128) > 0x7fffffffLL) return RIB_ERR_UNSUPPORTED;
     return RIB_OK;
 }
 
+// Device address of the status word on the current device; looked up once per device.
+constexpr int kMaxStatusDevices = 64;
+std::mutex g_status_mutex;
+int* g_status_ptr[kMaxStatusDevices] = {};
+
 int device_status_ptr(int** out)
 {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_status_word) != cudaSuccess) return RIB_ERR_CUDA;
-    *out = static_cast<int*>(ptr);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxStatusDevices) return RIB_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_status_mutex);
+    if (!g_status_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_status_word) != cudaSuccess || !ptr) return RIB_ERR_CUDA;
+        g_status_ptr[dev] = static_cast<int*>(ptr);
+    }
+    *out = g_status_ptr[dev];
     return RIB_OK;
 }
 
@@ -466,6 +481,25 @@ int rib_generate_features_bwd(const float* w_h, const float* b_h, const float* w
     return RIB_OK;
 }
 
+long long rib_exp_probe(float* sink, int blocks, int iters, void* stream)
+{
+    if (!sink) return RIB_ERR_NULL;
+    if (blocks <= 0 || iters <= 0 || blocks > (1 << 20) || iters > (1 << 24)) return RIB_ERR_SHAPE;
+    if (rib::exp_probe(sink, blocks, iters, static_cast<cudaStream_t>(stream)) != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return rib::exp_probe_count(blocks, iters);
+}
+
+int rib_wait_probe(unsigned long long limit_ns, void* stream)
+{
+    if (limit_ns == 0 || limit_ns > 100000000ull) return RIB_ERR_SHAPE;      // at most 0.1 s
+    int* status = nullptr;
+    if (int rc = device_status_ptr(&status)) return rc;
+    if (rib::wait_probe(status, limit_ns, static_cast<cudaStream_t>(stream)) != cudaSuccess) return RIB_ERR_CUDA;
+    g_kernel_launches += 1;
+    return RIB_OK;
+}
+
 int rib_query_status(void* stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -508,5 +542,13 @@ int rib_set_path(int path)
 int rib_last_path(void) { return t_last_path; }
 
 long long rib_kernel_launches(void) { return g_kernel_launches.load(); }
+
+void rib_tensor_map_cache_counts(long long* hits, long long* misses)
+{
+    long long h = 0, m = 0;
+    rib::tensor_map_cache_counts(&h, &m);
+    if (hits) *hits = h;
+    if (misses) *misses = m;
+}
 
 }  // extern "C"

@@ -78,6 +78,14 @@ cudaError_t generator_fwd(const float* w_h, const float* b_h, const float* w_pq,
 cudaError_t generator_bwd(const float* w_h, const float* b_h, const float* w_pq, const float* w_pk, const float* dpq, const float* dpk,
                           int window, int L, int dh, int r, float* dw_h, float* db_h, float* dw_pq, float* dw_pk, cudaStream_t stream);
 
+// Hits and misses of the host-side tensor-map cache (rib_fwd_sm100.cu).
+void tensor_map_cache_counts(long long* hits, long long* misses);
+
+// Measurement / self-test kernels (rib_probe.cu).
+cudaError_t exp_probe(float* sink, int blocks, int iters, cudaStream_t stream);
+long long exp_probe_count(int blocks, int iters);
+cudaError_t wait_probe(int* status, unsigned long long limit_ns, cudaStream_t stream);
+
 // Per-kernel device timing (off unless rib_profile_begin was called): records a CUDA event on
 // `stream` before (phase 0) and after (phase 1) the launch of kernel `kernel_id` (RIB_KERNEL_*).
 void profile_mark(int kernel_id, int phase, cudaStream_t stream);

@@ -718,6 +718,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
 }  // namespace
 
+void tensor_map_cache_counts(long long* hits, long long* misses) { sm100::map_cache_counts(hits, misses); }
+
 bool sm100_fwd_supported(const Problem& p)
 {
     const bool partial = p.Hp != p.H || p.Wp != p.W;

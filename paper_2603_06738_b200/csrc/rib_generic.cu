@@ -378,11 +378,14 @@ cudaError_t rowdot_prepass(const Problem& p, cudaStream_t stream)
 cudaError_t generic_bwd(const Problem& p, cudaStream_t stream)
 {
     const int dk = p.d + p.r;
-    const size_t pos_floats = pos_extent(p);
-    cudaError_t e = cudaMemsetAsync(p.dpq, 0, sizeof(float) * pos_floats, stream);
-    if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(p.dpk, 0, sizeof(float) * pos_floats, stream);
-    if (e != cudaSuccess) return e;
+    const size_t pos_floats = p.r > 0 ? pos_extent(p) : 0;      // rank 0: there are no positional gradients (dpq, dpk may be null)
+    cudaError_t e = cudaSuccess;
+    if (pos_floats) {
+        e = cudaMemsetAsync(p.dpq, 0, sizeof(float) * pos_floats, stream);
+        if (e != cudaSuccess) return e;
+        e = cudaMemsetAsync(p.dpk, 0, sizeof(float) * pos_floats, stream);
+        if (e != cudaSuccess) return e;
+    }
     e = rowdot_prepass(p, stream);
     if (e != cudaSuccess) return e;
     dim3 grid(p.pairs, (p.n + kRows - 1) / kRows);

@@ -97,8 +97,52 @@ inline EncodeTiledFn encode_fn()
     return fn;
 }
 
+// Tensor maps depend on the base pointer and the shape only, and a training loop calls with the same few buffers
+// over and over: the last kMapCacheSlots distinct maps of the process are kept (round-robin replacement, one
+// mutex), so a repeated call encodes nothing.  The key holds every argument of the encoding.
+struct MapKey {
+    const void* ptr; long long a, b; int kind, c, d, e, f, g;
+    bool operator==(const MapKey& o) const
+    {
+        return ptr == o.ptr && a == o.a && b == o.b && kind == o.kind && c == o.c && d == o.d && e == o.e && f == o.f && g == o.g;
+    }
+};
+constexpr int kMapCacheSlots = 64;
+struct MapCache {
+    std::mutex mutex;
+    MapKey keys[kMapCacheSlots];
+    CUtensorMap maps[kMapCacheSlots];
+    int used = 0, next = 0;
+    long long hits = 0, misses = 0;
+};
+inline MapCache& map_cache()
+{
+    static MapCache cache;
+    return cache;
+}
+template <typename Encode>
+inline bool cached_map(CUtensorMap* map, const MapKey& key, Encode encode)
+{
+    MapCache& c = map_cache();
+    std::lock_guard<std::mutex> lock(c.mutex);
+    for (int i = 0; i < c.used; ++i)
+        if (c.keys[i] == key) { *map = c.maps[i]; ++c.hits; return true; }
+    if (!encode(map)) return false;
+    ++c.misses;
+    const int slot = c.used < kMapCacheSlots ? c.used++ : (c.next = (c.next + 1) % kMapCacheSlots);
+    c.keys[slot] = key;
+    c.maps[slot] = *map;
+    return true;
+}
+inline void map_cache_counts(long long* hits, long long* misses)
+{
+    MapCache& c = map_cache();
+    std::lock_guard<std::mutex> lock(c.mutex);
+    *hits = c.hits; *misses = c.misses;
+}
+
 // bf16 [B][H][W][heads][32] image tensor, box = one 8x8-token patch of one head.
-inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p)
+inline bool encode_image_map_now(CUtensorMap* map, const void* ptr, const Problem& p)
 {
     const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)p.heads, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
     const cuuint64_t row = (cuuint64_t)kD * 2;
@@ -113,8 +157,14 @@ inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p
 // bf16 [tables][M][M][r] positional features (one table shared by all heads, or one per head; r = p.r), box = one
 // 8x8-token patch of one table.  `tables` = 1 or heads, `table_stride` elements apart (a multiple of 8,
 // at least M * M * 16); a kernel addresses table h * (tables > 1).
-inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
-                                cuuint32_t box_inner, CUtensorMapSwizzle swz)
+inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p)
+{
+    const MapKey key{ptr, 0, 0, 1, p.B, p.H, p.W, p.heads, 0};
+    return cached_map(map, key, [&](CUtensorMap* m) { return encode_image_map_now(m, ptr, p); });
+}
+
+inline bool encode_pos_map_now(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
+                               cuuint32_t box_inner, CUtensorMapSwizzle swz)
 {
     const cuuint64_t dims[4] = {(cuuint64_t)p.r, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
     const cuuint64_t one_table = (cuuint64_t)p.r * 2 * p.M * p.M;
@@ -125,6 +175,12 @@ inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem
     return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
+                                cuuint32_t box_inner, CUtensorMapSwizzle swz)
+{
+    const MapKey key{ptr, table_stride, 0, 2, p.r, p.M, tables, (int)box_inner, (int)swz};
+    return cached_map(map, key, [&](CUtensorMap* m) { return encode_pos_map_now(m, ptr, p, tables, table_stride, box_inner, swz); });
 }
 inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
 {

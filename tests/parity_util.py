@@ -26,6 +26,8 @@ def compare(name, got, ref, mask=None, max_abs=MAX_ABS, rel_l2=REL_L2):
     assert np.isfinite(got).all(), f"{name}: non-finite values in the GPU result"
     err = np.abs(got - ref).max()
     rl2 = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    # shown with `pytest -s` / `-rP`: how much of each bound is used
+    print(f"parity {name}: max|d|={err:.3e} (bound {max_abs:.1e}), rel-L2={rl2:.3e} (bound {rel_l2:.1e}), max|ref|={np.abs(ref).max():.3e}, n={got.size}")
     assert err <= max_abs and rl2 <= rel_l2, f"{name}: max|d|={err:.3e} (<= {max_abs}), rel-L2={rl2:.3e} (<= {rel_l2})"
     return err, rl2
 
@@ -58,13 +60,3 @@ def oracle_fwd(cpu, wl, pairs=None):
 
 def oracle_bwd(cpu, wl, pairs=None):
     return orc.bwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk", "dout")), wl.window, wl.shift, pairs=pairs)
-
-
-def sample_pairs(wl: synthetic.Workload, count: int, seed: int = 0):
-    """Pair ids spread over batch, heads and windows, always including the first and the last
-    window (the last one wraps around the image border when shift > 0)."""
-    rng = np.random.default_rng(seed)
-    ids = {0, wl.pairs - 1}
-    while len(ids) < min(count, wl.pairs):
-        ids.add(int(rng.integers(wl.pairs)))
-    return sorted(ids)

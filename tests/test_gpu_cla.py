@@ -23,7 +23,9 @@ def gate_inputs(seed, B, H, W, D):
     return x, [w_dw, b_dw, w_pw, b_pw]
 
 
-@pytest.mark.parametrize("B,H,W,D", [(1, 8, 16, 64), (2, 16, 32, 192), (1, 24, 48, 128), (3, 40, 16, 192), (1, 96, 96, 192)])
+# the last three shapes give every persistent CTA several tiles (the benchmark shape: 576 tiles on 148 CTAs)
+@pytest.mark.parametrize("B,H,W,D", [(1, 8, 16, 64), (2, 16, 32, 192), (1, 24, 48, 128), (3, 40, 16, 192), (1, 96, 96, 192),
+                                     (8, 96, 96, 192), (2, 160, 160, 64), (4, 88, 96, 128)])
 def test_gate_matches_the_oracle(B, H, W, D):
     x, ws = gate_inputs(200 + D + H, B, H, W, D)
     g = binding.rib_cla_gate(x.cuda(), *[torch.from_numpy(w).cuda() for w in ws])
@@ -108,7 +110,9 @@ def dgate_input(seed, shape):
 
 @pytest.mark.parametrize("path", ["auto", "generic"])
 @pytest.mark.parametrize("B,H,W,D", [(1, 5, 7, 64), (2, 16, 32, 192), (1, 24, 47, 128), (3, 9, 16, 192), (1, 1, 1, 64),
-                                     (1, 96, 96, 192), (2, 40, 56, 64)])
+                                     (1, 96, 96, 192), (2, 40, 56, 64),
+                                     # several tiles per persistent CTA / block, the last one with ragged H and W
+                                     (8, 96, 96, 192), (2, 160, 160, 64), (4, 90, 100, 128)])
 def test_gate_backward_matches_the_oracle(B, H, W, D, path):
     x, ws = gate_inputs(300 + D + H, B, H, W, D)
     dgate = dgate_input(301 + D + H, (B, H, W, D))

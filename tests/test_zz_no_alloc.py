@@ -11,7 +11,7 @@ import torch
 from paper_2603_06738_b200 import binding
 from paper_2603_06738_b200.synthetic import Workload
 
-from parity_util import make, run_bwd, run_fwd
+from parity_util import compare, make, oracle_bwd, run_bwd, run_fwd, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -36,6 +36,7 @@ def test_noalloc_backward_matches_workspace_backward_twice(wl):
     out, lse = run_fwd(gpu, wl)
     ref = run_bwd(gpu, wl, out, lse)
     ref_path = binding.rib_last_path()
+    want = oracle_bwd(cpu, wl)        # the gradients the paper's definition gives (CPU oracle)
     for attempt in range(2):      # the second call finds the first call's leftovers in the scratch
         got = _noalloc_bwd(gpu, wl, out, lse)
         assert binding.rib_last_path() == ref_path
@@ -43,6 +44,9 @@ def test_noalloc_backward_matches_workspace_backward_twice(wl):
             assert torch.isfinite(x.float()).all(), f"{name} (call {attempt}) has unwritten or non-finite values"
             # same kernels on the same inputs: only the order of the fp32 atomic sums may differ
             torch.testing.assert_close(x.float(), y.float(), rtol=2e-2, atol=1e-3, msg=lambda m: f"{name}: {m}")
+        for name, x, r in zip(("dq", "dk", "dv", "dpq", "dpk"), got, want):
+            scale = max(1.0, float(abs(r).max())) if name in ("dpq", "dpk") else 1.0      # sums over all pairs: bound relative to their size
+            compare(f"{name} (call {attempt}, against the oracle)", to_f64(x), r, max_abs=1e-2 * scale)
 
 
 def test_noalloc_rejects_shapes_beyond_the_builtin_scratch():
