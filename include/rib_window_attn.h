@@ -31,7 +31,8 @@
  * fallback: every step runs in CUDA kernels of this library.
  *
  * Supported shapes: H and W multiples of `window`, 0 <= shift < window, 1 <= d <= 64,
- * 0 <= r <= 64, d and r multiples of 8 (16-byte rows).  Shapes with d = 32, r = 16 or 32, window a
+ * 0 <= r <= 64 (any widths in that range: the SST rows of the paper's network table use d = 30 with
+ * r = 18 or 34, the light-weight ones d = 16 with r = 16 or 24).  Shapes with d = 32, r = 16 or 32, window a
  * multiple of 16 and shift a multiple of 8 take the tcgen05 / TMEM / TMA kernels; every other
  * supported shape takes a slower any-shape CUDA kernel.
  */

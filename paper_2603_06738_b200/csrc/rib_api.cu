@@ -22,7 +22,7 @@ int check_shape(int B, int H, int W, int heads, int d, int r, int window, int sh
     if (B <= 0 || H <= 0 || W <= 0 || heads <= 0 || d <= 0 || r < 0 || window <= 0) return RIB_ERR_SHAPE;
     if (!partial_windows && (H % window || W % window)) return RIB_ERR_SHAPE;
     if (shift < 0 || shift >= window) return RIB_ERR_SHAPE;
-    if (d > 64 || r > 64 || (d % 8) || (r % 8)) return RIB_ERR_UNSUPPORTED;
+    if (d > 64 || r > 64) return RIB_ERR_UNSUPPORTED;      // any width up to 64: the any-shape kernels read element by element
     const long long pairs = (long long)B * ((H + window - 1) / window) * ((W + window - 1) / window) * heads;
     if (pairs > 0x7fffffffLL || (long long)window * window > (1 << 20)) return RIB_ERR_SHAPE;
     // launch limits of the kernels: the any-shape kernels put n / 16 row groups on grid.y, the tcgen05 kernels count

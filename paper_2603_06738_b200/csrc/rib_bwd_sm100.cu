@@ -618,28 +618,33 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
 }
 
-// Finishing pass over the fp32 accumulators.  grid (n / 128, groups of pairs), 128 threads: a thread
-// owns one token position w of the window and walks the pairs of its group.  With one table for all
+// Finishing pass over the fp32 accumulators.  grid (n / 32, groups of pairs), 32 x 4 threads: a thread
+// owns one token position w of the window and walks a quarter of the pairs of its group; the four
+// quarters' partial sums meet in shared memory, so that one atomic per element and GROUP reaches the
+// results (these adds all land on the same n x r addresses: their number, not the traffic, set the
+// time of this kernel).  With one table for all
 // heads a group is a run of consecutive pairs; with head-wise tables it is a run of windows of one
 // head (pair = head + heads * window), so that its sums belong to one table.  Per pair it turns
 // dQ~[:, :d] / sqrt(d) into the bf16 dq row of that token, and it keeps running sums of the 16 RIB
 // columns of dQ~ (-> dPq, times 1/sqrt(r)) and of dK~ (-> dPk); the group's partial sums go to the
 // zeroed results with one vector atomic per 4 columns.
 template <int R>
-__global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_group)
+__global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_thread)
 {
     constexpr int kDk = kD + R;
-    const int w = blockIdx.x * 128 + threadIdx.x;
+    __shared__ float red[3][2][16][32];          // quarters 1-3: [dPq | dPk][column][token]
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int w = blockIdx.x * 32 + tx;
     int pair0, pair1, step = 1;
     size_t table = 0;
     if (p.tables == 1) {
-        pair0 = blockIdx.y * pairs_per_group;
-        pair1 = min(p.pairs, pair0 + pairs_per_group);
+        pair0 = (blockIdx.y * 4 + ty) * pairs_per_thread;
+        pair1 = min(p.pairs, pair0 + pairs_per_thread);
     } else {
-        const int head = blockIdx.y % p.heads, first = (blockIdx.y / p.heads) * pairs_per_group;
+        const int head = blockIdx.y % p.heads, first = ((blockIdx.y / p.heads) * 4 + ty) * pairs_per_thread;
         step = p.heads;
         pair0 = head + first * step;
-        pair1 = min(p.pairs, pair0 + pairs_per_group * step);
+        pair1 = min(p.pairs, pair0 + pairs_per_thread * step);
         table = (size_t)head * (size_t)p.pos_head_stride;
     }
     // blockIdx.z picks 16 of the R RIB columns (grid.z = R / 16); the slice z = 0 also writes dq
@@ -669,7 +674,18 @@ __global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, 
             sk[c] += srk[(size_t)(col0 + c) * p.n];
         }
     }
-    if (pair0 >= pair1) return;
+    // (quarter 0 always has pairs: the grid is sized by the groups; later quarters may be empty and then add zeros)
+    if (ty > 0) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) { red[ty - 1][0][c][tx] = sq[c]; red[ty - 1][1][c][tx] = sk[c]; }
+    }
+    __syncthreads();
+    if (ty > 0) return;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        sq[c] += red[0][0][c][tx] + red[1][0][c][tx] + red[2][0][c][tx];
+        sk[c] += red[0][1][c][tx] + red[1][1][c][tx] + red[2][1][c][tx];
+    }
     float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R + col0);
     float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R + col0);
 #pragma unroll
@@ -760,9 +776,10 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
     const int per_group = p.pairs < 8 ? 1 : 4;
     const int windows = p.pairs / p.heads;   // pairs of one head
-    const unsigned groups = tables == 1 ? (unsigned)((p.pairs + per_group - 1) / per_group)
-                                        : (unsigned)(p.heads * ((windows + per_group - 1) / per_group));
-    dim3 grid_fin((unsigned)(p.n / 128), groups, (unsigned)(R / 16));
+    // a block takes four runs of per_group pairs (of one head, with head-wise tables)
+    const unsigned runs = (unsigned)(((tables == 1 ? p.pairs : windows) + per_group - 1) / per_group);
+    const unsigned groups = (tables == 1 ? 1u : (unsigned)p.heads) * ((runs + 3) / 4);
+    dim3 grid_fin((unsigned)(p.n / 32), groups, (unsigned)(R / 16));
     { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<R><<<grid_fin, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();
 }

@@ -49,7 +49,7 @@ def fwd_args(**over):
 @pytest.mark.parametrize("over,code", [
     (dict(q=None), -1), (dict(out=None), -1), (dict(pq=None), -1),
     (dict(H=40), -2), (dict(shift=16), -2), (dict(shift=-1), -2), (dict(B=0), -2), (dict(window=0), -2),
-    (dict(d=128), -3), (dict(r=20), -3), (dict(d=12), -3),
+    (dict(d=128), -3), (dict(r=72), -3), (dict(d=65), -3),
     (dict(k=516), -4), (dict(lse=4100), -4),
 ])
 def test_fwd_rejects_bad_arguments_without_launching(lib, over, code):
@@ -74,7 +74,7 @@ def test_headwise_and_padded_entry_points_validate_before_any_cuda_call(lib):
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, q=None)) == -1
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, shift=16)) == -2
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=0)) == -2
-    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, d=12)) == -3
+    assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, d=72)) == -3
     assert lib.rib_window_attn_fwd_padded(*headwise_args(0, H=40, v=770)) == -4
     # backward on maps that are not multiples of the window: sized by the windows of the extended map on the tcgen05
     # shapes, one float per token-head on the any-shape kernels

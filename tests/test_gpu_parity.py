@@ -27,6 +27,11 @@ SMALL = [
     Workload("w16_odd_shift", 1, 32, 32, 2, 32, 16, 16, 5, seed=21),       # fast shape but odd shift
     Workload("w16_s8_rank32", 2, 32, 48, 2, 32, 32, 16, 8, seed=22),       # rank 32 (d + r = 64) on the tcgen05 kernels
     Workload("w32_s16_rank32", 1, 64, 32, 3, 32, 32, 32, 16, seed=23),
+    # the head widths of the paper's other network rows (appendix table of network implementations): 60-byte rows
+    Workload("sst_d30_r18_w16", 1, 32, 32, 6, 30, 18, 16, 0, seed=24),
+    Workload("sst_d30_r34_w32", 1, 32, 64, 3, 30, 34, 32, 16, seed=25),
+    Workload("light_d16_r24_w16", 2, 32, 32, 3, 16, 24, 16, 8, seed=26),       # d + r = 40: not a multiple of 16
+    Workload("odd_d15_r7_w8", 1, 16, 16, 2, 15, 7, 8, 3, seed=27),
 ]
 
 
