@@ -470,6 +470,11 @@ def main():
             f_ms = timed(lambda: binding.rib_window_attn_fwd_padded(fq, fk, fv, fpq, fpk, fwin, 0), reps=10)
             variants["partial_windows_360x640_w64"] = {"fwd_ms": f_ms, "tokens_per_s": fh * fw / (f_ms * 1e-3),
                                                        "paths": [binding.rib_last_path()]}
+            # the next larger map that the window divides, for comparison: 384 x 640 (the frame holds 93.75 % of its tokens)
+            gq, gk, gv = (torch.randn((1, 384, fw, wl.heads, wl.d), device=dev).to(torch.bfloat16) for _ in range(3))
+            g_ms = timed(lambda: binding.rib_window_attn_fwd(gq, gk, gv, fpq, fpk, fwin, 0), reps=10)
+            variants["partial_windows_360x640_w64"].update({"divisible_384x640_fwd_ms": g_ms, "ratio_to_divisible": f_ms / g_ms})
+            del gq, gk, gv
             # Convolutional Local Attention (Eq. 8, Eq. 9) on the benchmark shape: the gate kernel (HBM-bound: one read of the
             # features and one write of the gate) and the forward pass with the gate multiplied into its output
             D = wl.heads * wl.d

@@ -149,6 +149,23 @@ size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, in
                                             int window);
 
 /*
+ * The cyclic window strategy (Sec. 3.3: the window size cycles over the attention layers of a block, e.g.
+ * {16, 32, 64, 16, 32, 64}, instead of shifting windows): one call that enqueues the forward pass of `layers`
+ * attention layers over maps of one size, layer l with window windows[l] (and cyclic shift shifts[l]; shifts
+ * may be NULL = no shift, the paper's setting).  q, k, v, pq, pk, out, lse are HOST arrays of `layers` device
+ * pointers: layer l reads q[l], k[l], v[l] (bf16 [B][H][W][heads][d]) and its own tables pq[l], pk[l]
+ * (bf16 [windows[l]^2][r], shared by the heads) and writes out[l] (and lse[l]; lse itself or single entries may
+ * be NULL).  Layers may share buffers where that makes sense (the same pointer in several entries).  A window
+ * that does not divide H or W is laid over the extended map as in rib_window_attn_fwd_padded.  Every layer's
+ * arguments are checked before the first launch: on an error (codes as for rib_window_attn_fwd_padded, plus
+ * RIB_ERR_SHAPE for layers outside 1..64) nothing has been launched.  The tensor maps of repeated calls on the
+ * same buffers come from the library's cache (rib_tensor_map_cache_counts), so a block's steady state encodes none.
+ */
+int rib_window_cycle_fwd(const void* const* q, const void* const* k, const void* const* v, const void* const* pq, const void* const* pk,
+                         const int* windows, const int* shifts, int layers,
+                         int B, int H, int W, int heads, int d, int r, void* const* out, float* const* lse, void* stream);
+
+/*
  * Convolutional Local Attention (paper: Sec. 3.2, Eq. 7, Eq. 8, Eq. 9): the step right after the attention.
  *   G  = sigmoid(PWConv(DWConv3x3(X)))      X: the block's token features as an H x W map          (Eq. 8)
  *   O' = O o G                              element-wise product with the attention output           (Eq. 9)

@@ -28,7 +28,7 @@ EXPORTS = (
     "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
     "rib_window_attn_bwd_padded", "rib_window_attn_bwd_padded_workspace",
     "rib_cla_product", "rib_cla_product_bwd", "rib_cla_gate_bwd", "rib_cla_gate_bwd_workspace",
-    "rib_wait_probe", "rib_exp_probe", "rib_tensor_map_cache_counts",
+    "rib_wait_probe", "rib_exp_probe", "rib_tensor_map_cache_counts", "rib_window_cycle_fwd",
 )
 KERNEL_NAMES = {1: "rib_fwd_sm100_kernel", 2: "rib_bwd_prepare_kernel", 3: "rib_bwd_sm100_kernel",
                 4: "rib_bwd_finish_kernel", 6: "generic_fwd_kernel",
@@ -108,6 +108,8 @@ def library() -> ctypes.CDLL:
         lib.rib_last_path.argtypes = []
         lib.rib_kernel_launches.restype = ctypes.c_longlong
         lib.rib_kernel_launches.argtypes = []
+        lib.rib_window_cycle_fwd.restype = ci
+        lib.rib_window_cycle_fwd.argtypes = [ctypes.POINTER(vp)] * 5 + [ctypes.POINTER(ci)] * 2 + [ci] * 7 + [ctypes.POINTER(vp)] * 2 + [vp]
         lib.rib_tensor_map_cache_counts.restype = None
         lib.rib_tensor_map_cache_counts.argtypes = [ctypes.POINTER(ctypes.c_longlong)] * 2
         lib.rib_wait_probe.restype = ci
@@ -301,6 +303,34 @@ def rib_window_attn_fwd_padded(q, k, v, pq, pk, window, shift=0, stream=None, wa
     if rc != RIB_OK:
         raise RibError(rc)
     return out, lse
+
+
+def rib_window_cycle_fwd(qs, ks, vs, pqs, pks, windows, shifts=None, stream=None, want_lse=True):
+    """The cyclic window strategy in one call: layer l attends qs[l], ks[l], vs[l] in windows of side windows[l] with the tables
+    pqs[l], pks[l] ([windows[l]^2, r]).  Returns (outs, lses), one tensor per layer."""
+    layers = len(windows)
+    if not (len(qs) == len(ks) == len(vs) == len(pqs) == len(pks) == layers) or (shifts is not None and len(shifts) != layers):
+        raise ValueError("one q, k, v, pq, pk (and shift) per layer")
+    _check_image("q", qs[0])
+    B, H, W, heads, d = qs[0].shape
+    r = pqs[0].shape[1]
+    for l in range(layers):
+        for name, t in (("q", qs[l]), ("k", ks[l]), ("v", vs[l])):
+            _check_image(name, t, qs[0].shape)
+        _check_pos("pq", pqs[l], windows[l] * windows[l])
+        _check_pos("pk", pks[l], windows[l] * windows[l])
+        if pqs[l].shape[1] != r or pks[l].shape[1] != r:
+            raise ValueError("every layer uses the same rank")
+    outs = [torch.empty_like(qs[0]) for _ in range(layers)]
+    lses = [torch.empty((B, heads, H, W), dtype=torch.float32, device=qs[0].device) if want_lse else None for _ in range(layers)]
+    arr = lambda ts: (ctypes.c_void_p * layers)(*[_ptr(t) for t in ts])
+    ints = lambda xs: (ctypes.c_int * layers)(*[int(x) for x in xs])
+    rc = library().rib_window_cycle_fwd(arr(qs), arr(ks), arr(vs), arr(pqs), arr(pks), ints(windows),
+                                        ints(shifts) if shifts is not None else None, layers, B, H, W, heads, d, r,
+                                        arr(outs), arr(lses) if want_lse else None, _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return outs, lses
 
 
 def rib_window_attn_bwd_padded(q, k, v, pq, pk, out, lse, dout, window, shift=0, workspace=None, stream=None):

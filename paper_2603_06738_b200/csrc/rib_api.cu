@@ -61,7 +61,8 @@ void fill_shape(rib::Problem& p, int B, int H, int W, int heads, int d, int r, i
 }
 
 int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk, long long pos_head_stride, const void* gate,
-             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream);
+             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream,
+             bool validate_only = false);
 
 int check_pos_stride(long long stride, int window, int r)
 {
@@ -212,6 +213,22 @@ int rib_window_attn_fwd_gated(const void* q, const void* k, const void* v, const
     return fwd_impl(q, k, v, pq, pk, pos_head_stride, gate, B, H, W, heads, d, r, window, shift, out, lse, stream);
 }
 
+int rib_window_cycle_fwd(const void* const* q, const void* const* k, const void* const* v, const void* const* pq, const void* const* pk,
+                         const int* windows, const int* shifts, int layers,
+                         int B, int H, int W, int heads, int d, int r, void* const* out, float* const* lse, void* stream)
+{
+    if (!q || !k || !v || !pq || !pk || !windows || !out) return RIB_ERR_NULL;
+    if (layers <= 0 || layers > 64) return RIB_ERR_SHAPE;
+    // every layer is checked before the first one is launched
+    for (int pass = 0; pass < 2; ++pass)
+        for (int l = 0; l < layers; ++l) {
+            const int rc = fwd_impl(q[l], k[l], v[l], pq[l], pk[l], 0, nullptr, B, H, W, heads, d, r, windows[l], shifts ? shifts[l] : 0,
+                                    out[l], lse ? lse[l] : nullptr, stream, pass == 0);
+            if (rc != RIB_OK) return rc;
+        }
+    return RIB_OK;
+}
+
 int rib_cla_gate(const void* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
                  int B, int H, int W, int D, void* gate, void* stream)
 {
@@ -295,7 +312,7 @@ int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const 
 namespace {
 
 int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk, long long pos_head_stride, const void* gate,
-             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream)
+             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream, bool validate_only)
 {
     if (!q || !k || !v || !out || (r > 0 && (!pq || !pk))) return RIB_ERR_NULL;
     if (int rc = check_shape(B, H, W, heads, d, r, window, shift, true)) return rc;
@@ -303,6 +320,7 @@ int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const 
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(pq) ||
         !aligned16(pk) || !aligned16(lse))
         return RIB_ERR_ALIGN;
+    if (validate_only) return RIB_OK;
     rib::Problem p{};
     fill_shape(p, B, H, W, heads, d, r, window, shift);
     p.q = static_cast<const __nv_bfloat16*>(q);

@@ -19,7 +19,7 @@
 // puts four softmax warps on every SM sub-partition.
 //
 // The softmax has two forms.
-//   Fast form (first pass over the items; maps that are multiples of the window): the exp (MUFU)
+//   Fast form (first pass over the items): the exp (MUFU)
 //   and issue pipes are what this kernel runs out of, so the per-score work is cut to one scale-and-
 //   subtract, one exponential and one conversion.  The reference m of a row is fixed once per item (the
 //   maximum over the first 32 keys, read by both threads of the row, so they agree without talking to
@@ -34,8 +34,11 @@
 //   the item is then noted in shared memory and redone by the exact form in a second pass of the
 //   same launch.  Every third or fourth pair of exponentials (kPolyMask) is evaluated on the FMA and
 //   integer pipes instead of the MUFU.
-//   Exact form (second pass, and maps with partial windows): classic online softmax per key half
+//   Exact form (second pass): classic online softmax per key half
 //   with a running maximum, lazy rescaling of O, separate accumulators and a log-sum-exp merge.
+//   On maps with partial windows (kPartial) key patches in the extension of the map contribute probability 0 in
+//   both forms, the fast form takes its reference from the first block that holds real keys, and items whose query
+//   patches all lie in the extension are skipped by every role alike.
 //
 // Tiles are two 8x8-token patches (see rib_sm100_common.cuh), fetched by one TMA box each.
 //
@@ -201,7 +204,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tmem_alloc(base + kOffMisc, kTmemCols);
         tmem_relinquish();
     }
-    if (!kPartial && warp >= 4 && warp < 8) {
+    if (warp >= 4 && warp < 8) {
         // the tile behind V: 128 key rows of 64 bytes, SWIZZLE_64B like V, element 0 of every row = 1
         const int row = (warp - 4) * 32 + lane;
         uint4* dst = reinterpret_cast<uint4*>(base_ptr + kOffOnes + row * 64);
@@ -221,16 +224,31 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     bool ok = true;
 
     for (int pass = 0; pass < 2; ++pass) {
-        const bool fast = !kPartial && pass == 0 && !p.exact_only;
+        const bool fast = pass == 0 && !p.exact_only;
         // pass 0: every item of this CTA; pass 1: the items noted by the fast form (all of them when the notes overflowed)
         const int noted = pass == 0 ? 0 : *redo_count;
         const bool all_items = pass == 0 || noted > kMaxRedo;
         const int count = all_items ? my_items : noted;
         auto item_at = [&](int i) { return (int)blockIdx.x + (all_items ? i : redo_list[i]) * (int)gridDim.x; };
+        // kPartial: an item whose four query patches all lie in the extension of the map has nothing to compute; every role
+        // skips it by the same test, so the item and block counters that give the barrier phases stay in step
+        auto item_live = [&](int item) {
+            if (!kPartial) return true;
+            const ItemCoord c = decode_item(p, item);
+            bool live = false;
+#pragma unroll
+            for (int sp = 0; sp < 4; ++sp) {
+                int py, px, Y0, X0;
+                patch_origin(p, c, 4 * c.tp + sp, py, px, Y0, X0);
+                live = live || (Y0 < p.H && X0 < p.W);
+            }
+            return live;
+        };
 
         if (warp == 0) {
             // ===================== TMA producer (lane 0) and query RIB rows bf16(Pq * sqrt(d/r)) of the same item (whole warp)
             for (int i = 0; i < count && ok; ++i, ++io) {
+                if (!item_live(item_at(i))) { --io; continue; }
                 const ItemCoord c = decode_item(p, item_at(i));
                 const uint32_t buf = io & 1;
                 if (io >= 2 && !mbar_wait_warp(bar(kQEmpty + buf), ((io >> 1) - 1) & 1, abort_flag, p.status)) { ok = false; break; }
@@ -311,6 +329,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             // and waits; one elected lane issues (this keeps descriptors in uniform registers).
             constexpr uint64_t kDesc64 = smem_desc_const(16, 512, kSwizzle64B), kDesc32 = smem_desc_const(16, 256, kSwizzle32B);
             for (int i = 0; i < count && ok; ++i, ++io) {
+                if (!item_live(item_at(i))) { --io; continue; }
                 const uint32_t buf = io & 1;
                 if (!mbar_wait_warp(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) ||
                     !mbar_wait_warp(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
@@ -350,6 +369,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const uint32_t d_o = tmem + kColO + qt * 2 * kD;              // exact form: one accumulator per key half
             const uint32_t d_o1 = tmem + kColO + qt * kFastOCols;         // fast form: one accumulator
             for (int i = 0; i < count && ok; ++i, ++io) {
+                if (!item_live(item_at(i))) { --io; continue; }
                 for (int j = 0; j < nblk; ++j, ++blk) {
                     const uint32_t st = blk % kStages;
                     // warp-uniform outcomes, so that the warp stays converged.  The first block of an item overwrites the
@@ -421,11 +441,12 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     if (lane == 0) mbar_arrive(bar(kOFree + qt));
                     const float l_all = __uint_as_float(lsum[0]);
                     // a score left the range the fixed reference covers: the exact form redoes the item
-                    const bool bad = !(l_all > 0.f && l_all < 1.2676506e30f);     // 2^100
+                    const bool bad = pend_out != nullptr && !(l_all > 0.f && l_all < 1.2676506e30f);     // 2^100
                     if (__any_sync(0xffffffffu, bad) && lane == 0) {
                         const int slot = atomicAdd(redo_count, 1);
                         if (slot < kMaxRedo) redo_list[slot] = pend_ordinal;
                     }
+                    if (kPartial && pend_out == nullptr) { pend_ordinal = -1; return; }
                     const float w_o = 1.f / l_all;
                     uint4* dst = reinterpret_cast<uint4*>(pend_out);
                     const uint4* gsrc = reinterpret_cast<const uint4*>(pend_gate);
@@ -449,15 +470,17 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 };
                 for (int i = 0; i < count && ok; ++i, ++io) {
                     const int item = item_at(i);
+                    if (!item_live(item)) { --io; continue; }
                     const ItemCoord c = decode_item(p, item);
                     // where this thread's half row of the item goes
                     int py, px, Y0, X0;
                     patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
                     const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
+                    const bool no_query = kPartial && (Y0 >= p.H || X0 >= p.W);   // a patch of the extension: no tokens, nothing to store
                     const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
-                    __nv_bfloat16* const out_row = p.out + tok * kD + half * 16;
+                    __nv_bfloat16* const out_row = no_query ? nullptr : p.out + tok * kD + half * 16;
                     const __nv_bfloat16* const gate_row = kGated ? p.gate + tok * kD + half * 16 : nullptr;
-                    float* const lse_row = (p.lse && half == 0) ? p.lse + (((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X : nullptr;
+                    float* const lse_row = (p.lse && half == 0 && !no_query) ? p.lse + (((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X : nullptr;
                     float m_ref = 0.f;
                     float2 neg2 = make_float2(0.f, 0.f);
                     for (int j = 0; j < nblk; ++j, ++blk) {
@@ -478,6 +501,32 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             m_ref = fmaxf(mx0, mx1);
                             const float neg = -m_ref * p.scale_log2;
                             neg2 = make_float2(neg, neg);
+                        }
+                        if (kPartial) {
+                            // this thread's 64 keys are one 8x8 patch: beyond the image it holds no tokens (the reference above may
+                            // come from such keys: any finite score near the row's scores serves as a reference)
+                            int kpy, kpx, kY0, kX0;
+                            patch_origin(p, c, 2 * j + half, kpy, kpx, kY0, kX0);
+                            if (kY0 >= p.H || kX0 >= p.W) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(bar(kSFree + qt));
+                                if (blk > 0) {
+                                    if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                                    tc_fence_after();
+                                }
+                                if (j == 0 && pend_ordinal >= 0) epilogue();
+                                uint32_t zero[16];
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) zero[e] = 0u;
+                                tmem_st16(t_p, zero);
+                                tmem_st16(t_p + 16, zero);
+                                tmem_wait_st();
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(b_ready);
+                                continue;
+                            }
                         }
                         // all 64 scores of this thread at once: the accumulator goes back to the MMA warp before any exponential
                         tmem_ld32(t_s, sa);
@@ -529,6 +578,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 };
                 for (int i = 0; i < count && ok; ++i, ++io, ++nmerge) {
                     const int item = item_at(i);
+                    if (!item_live(item)) { --io; --nmerge; continue; }
                     const ItemCoord c = decode_item(p, item);
                     float m_used = -INFINITY, l = 0.f;
                     bool have_ref = false;            // kPartial: a block with real keys has set the reference

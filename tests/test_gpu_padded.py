@@ -115,3 +115,33 @@ def test_plain_entry_points_still_reject_partial_windows():
                                  1, 40, 56, 1, 32, 16, 16, 0, x.data_ptr(), None, None)
     assert rc == -2      # RIB_ERR_SHAPE
     assert lib.rib_window_attn_bwd_workspace(1, 40, 56, 1, 32, 16, 16) == 0
+
+
+def test_window_cycle_driver_runs_the_six_layers_of_a_block():
+    """Sec. 3.3: the window size cycles over the layers of a block.  One call enqueues all six layers; every layer is
+    compared with the oracle (64 does not divide the 96-row map: that layer runs on partial windows), and a repeated
+    call encodes no tensor map."""
+    B, H, W, heads, d, r = 1, 96, 64, 2, 32, 16
+    windows = [16, 32, 64, 16, 32, 64]
+    layers = []
+    for l, win in enumerate(windows):
+        wl = Workload(f"cycle_l{l}", B, H, W, heads, d, r, win, 0, seed=300 + l)
+        cpu = synthetic.make_inputs(Workload(wl.name, B, win, win, heads, d, r, win, 0, seed=300 + l), False)   # tables of n = win^2 rows
+        img = synthetic.make_inputs(Workload(wl.name, B, 96, 96, heads, d, r, 96, 0, seed=310 + l), False)
+        layers.append({"q": img["q"][:, :H, :W].contiguous(), "k": img["k"][:, :H, :W].contiguous(), "v": img["v"][:, :H, :W].contiguous(),
+                       "pq": cpu["pq"], "pk": cpu["pk"]})
+    dev = [{k: v.cuda() for k, v in layer.items()} for layer in layers]
+    args = [[layer[k] for layer in dev] for k in ("q", "k", "v", "pq", "pk")]
+    launches = binding.rib_kernel_launches()
+    outs, lses = binding.rib_window_cycle_fwd(*args, windows)
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0 and binding.rib_kernel_launches() == launches + 6
+    for l, win in enumerate(windows):
+        f64 = {k: to_f64(v) for k, v in layers[l].items()}
+        ref_out, ref_lse = pad.fwd(f64["q"], f64["k"], f64["v"], f64["pq"], f64["pk"], win, 0)
+        compare(f"layer {l} (window {win}) out", to_f64(outs[l]), ref_out)
+        compare(f"layer {l} (window {win}) lse", to_f64(lses[l]), ref_lse)
+    _, misses = binding.rib_tensor_map_cache_counts()
+    binding.rib_window_cycle_fwd(*args, windows)
+    torch.cuda.synchronize()
+    assert binding.rib_tensor_map_cache_counts()[1] == misses      # q, k, v and Pk of every layer were mapped by the first call

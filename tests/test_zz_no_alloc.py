@@ -38,6 +38,16 @@ def test_noalloc_backward_matches_workspace_backward_twice(wl):
     ref_path = binding.rib_last_path()
     want = oracle_bwd(cpu, wl)        # the gradients the paper's definition gives (CPU oracle)
     for attempt in range(2):      # the second call finds the first call's leftovers in the scratch
+        if attempt == 1:
+            # what the entry point is for: once its scratch address is known (first call), a call takes no device memory
+            dq, dk, dv = (torch.empty_like(gpu["q"]) for _ in range(3))
+            dpq, dpk = (torch.empty((wl.n, wl.r), dtype=torch.float32, device="cuda") for _ in range(2))
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
+            binding.rib_window_attn_bwd_noalloc(gpu["q"], gpu["k"], gpu["v"], gpu["pq"], gpu["pk"], out, lse, gpu["dout"],
+                                                dq, dk, dv, dpq, dpk, wl.window, wl.shift)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
         got = _noalloc_bwd(gpu, wl, out, lse)
         assert binding.rib_last_path() == ref_path
         for name, x, y in zip(("dq", "dk", "dv", "dpq", "dpk"), got, ref):
