@@ -244,6 +244,19 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
             return live;
         };
+        // kPartial: which patch rows / patch columns of the item's window lie in the extension of the map, one bit each
+        // (lane l votes for row and column l; a window has at most 32 of either).  Warp-collective.
+        auto dead_masks = [&](const ItemCoord& c, uint32_t& row_dead, uint32_t& col_dead) {
+            int y = c.wy * p.M + 8 * lane + p.s; if (y >= p.Hp) y -= p.Hp;
+            int x = c.wx * p.M + 8 * lane + p.s; if (x >= p.Wp) x -= p.Wp;
+            row_dead = __ballot_sync(0xffffffffu, y >= p.H);
+            col_dead = __ballot_sync(0xffffffffu, x >= p.W);
+        };
+        auto patch_dead = [&](int sp, uint32_t row_dead, uint32_t col_dead) {
+            int pr, pc;
+            p.div_per_row.divmod(sp, pr, pc);
+            return (((row_dead >> pr) | (col_dead >> pc)) & 1u) != 0u;
+        };
 
         if (warp == 0) {
             // ===================== TMA producer (lane 0) and query RIB rows bf16(Pq * sqrt(d/r)) of the same item (whole warp)
@@ -414,10 +427,10 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 // ------------------------------------------------------------------ fast form
                 const uint32_t t_o1 = tmem + lane_base + kColO + qt * kFastOCols;
                 // exp2 of 32 scores against the fixed reference, packed to bf16 pairs
-                auto exp_chunk1 = [&](const uint32_t (&s)[32], float2 neg2, uint32_t (&packed)[16]) {
+                auto exp_chunk1 = [&](const uint32_t (&s)[32], float2 sc2, float2 neg2, uint32_t (&packed)[16]) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg2);
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), sc2, neg2);
                         const float2 e = ((kPolyMask >> (i & 7)) & 1u) ? ex2_poly2_ranged(x) : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                         packed[i] = pack_bf16x2(e.x, e.y);
                     }
@@ -441,7 +454,9 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     if (lane == 0) mbar_arrive(bar(kOFree + qt));
                     const float l_all = __uint_as_float(lsum[0]);
                     // a score left the range the fixed reference covers: the exact form redoes the item
-                    const bool bad = pend_out != nullptr && !(l_all > 0.f && l_all < 1.2676506e30f);     // 2^100
+                    // (kPartial: or the row sum is so small that the weights of keys beyond the map could show in it)
+                    const float l_min = kPartial ? 8.6736174e-19f : 0.f;                                   // 2^-60
+                    const bool bad = pend_out != nullptr && !(l_all > l_min && l_all < 1.2676506e30f);     // 2^100
                     if (__any_sync(0xffffffffu, bad) && lane == 0) {
                         const int slot = atomicAdd(redo_count, 1);
                         if (slot < kMaxRedo) redo_list[slot] = pend_ordinal;
@@ -483,6 +498,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     float* const lse_row = (p.lse && half == 0 && !no_query) ? p.lse + (((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X : nullptr;
                     float m_ref = 0.f;
                     float2 neg2 = make_float2(0.f, 0.f);
+                    uint32_t row_dead = 0u, col_dead = 0u;
+                    if (kPartial) dead_masks(c, row_dead, col_dead);
                     for (int j = 0; j < nblk; ++j, ++blk) {
                         // warp-uniform outcome: the TMEM loads below are warp-collective
                         if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
@@ -502,32 +519,6 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             const float neg = -m_ref * p.scale_log2;
                             neg2 = make_float2(neg, neg);
                         }
-                        if (kPartial) {
-                            // this thread's 64 keys are one 8x8 patch: beyond the image it holds no tokens (the reference above may
-                            // come from such keys: any finite score near the row's scores serves as a reference)
-                            int kpy, kpx, kY0, kX0;
-                            patch_origin(p, c, 2 * j + half, kpy, kpx, kY0, kX0);
-                            if (kY0 >= p.H || kX0 >= p.W) {
-                                tc_fence_before();
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(bar(kSFree + qt));
-                                if (blk > 0) {
-                                    if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                                    tc_fence_after();
-                                }
-                                if (j == 0 && pend_ordinal >= 0) epilogue();
-                                uint32_t zero[16];
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) zero[e] = 0u;
-                                tmem_st16(t_p, zero);
-                                tmem_st16(t_p + 16, zero);
-                                tmem_wait_st();
-                                tc_fence_before();
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(b_ready);
-                                continue;
-                            }
-                        }
                         // all 64 scores of this thread at once: the accumulator goes back to the MMA warp before any exponential
                         tmem_ld32(t_s, sa);
                         tmem_ld32(t_s + 32, sb);
@@ -536,8 +527,18 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
                         uint32_t pa[16], pb[16];
-                        exp_chunk1(sa, neg2, pa);
-                        exp_chunk1(sb, neg2, pb);
+                        float2 sc2 = scale2, ng2 = neg2;
+                        if (kPartial && patch_dead(2 * j + half, row_dead, col_dead)) {
+                            // This thread's 64 keys are one 8x8 patch; in the extension of the map it holds no tokens.  The block
+                            // runs through the same instructions with scale 0 and offset -119: each such key gets the weight
+                            // 2^-119 (the smallest both exponential paths deliver), its zero-filled value row adds nothing to
+                            // O, and the at most 2^16 such keys add less than 2^-103 to a row sum that the epilogue accepts
+                            // only from 2^-60 upwards.  The reference above may come from such keys: any finite score serves.
+                            sc2 = make_float2(0.f, 0.f);
+                            ng2 = make_float2(-119.f, -119.f);
+                        }
+                        exp_chunk1(sa, sc2, ng2, pa);
+                        exp_chunk1(sb, sc2, ng2, pb);
                         // P of the tile is free once the previous block's PV has completed (long ago, as a rule)
                         if (blk > 0) {
                             if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
@@ -582,6 +583,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const ItemCoord c = decode_item(p, item);
                     float m_used = -INFINITY, l = 0.f;
                     bool have_ref = false;            // kPartial: a block with real keys has set the reference
+                    uint32_t row_dead = 0u, col_dead = 0u;
+                    if (kPartial) dead_masks(c, row_dead, col_dead);
                     for (int j = 0; j < nblk; ++j, ++blk) {
                         // warp-uniform outcome: the TMEM loads below are warp-collective
                         if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
@@ -589,9 +592,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         bool p_free = blk == 0;       // P (and O) of this half are free once the previous block's PV has completed
                         if (kPartial) {
                             // this thread's 64 keys are one 8x8 patch: beyond the image it holds no tokens
-                            int py, px, Y0, X0;
-                            patch_origin(p, c, 2 * j + half, py, px, Y0, X0);
-                            if (Y0 >= p.H || X0 >= p.W) {
+                            if (patch_dead(2 * j + half, row_dead, col_dead)) {
                                 tc_fence_before();
                                 __syncwarp();
                                 if (lane == 0) mbar_arrive(bar(kSFree + qt));
