@@ -114,6 +114,7 @@ struct FwdParams {
     long long pos_head_stride; // elements between the heads' Pq tables (0: one table for all heads)
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
     int exact_only;            // 1: skip the fast form (every item takes the exact softmax)
+    int skip_dead;             // kPartial: 1 = items and key blocks without tokens are skipped, 0 = walked with probability 0
     FastDiv div_tp, div_heads, div_nwx, div_nwy, div_per_row;   // tiles_per_item_pair, heads, nWx, nWy, M / 8
 };
 
@@ -231,9 +232,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const int count = all_items ? my_items : noted;
         auto item_at = [&](int i) { return (int)blockIdx.x + (all_items ? i : redo_list[i]) * (int)gridDim.x; };
         // kPartial: an item whose four query patches all lie in the extension of the map has nothing to compute; every role
-        // skips it by the same test, so the item and block counters that give the barrier phases stay in step
+        // skips it by the same test, so the item and block counters that give the barrier phases stay in step.  The tests cost
+        // every role some hundred cycles per item, which pays from windows of 32 x 32 tokens on (skip_dead); in smaller
+        // windows an item is a block or two long and everything is walked.
         auto item_live = [&](int item) {
-            if (!kPartial) return true;
+            if (!kPartial || !p.skip_dead) return true;
             const ItemCoord c = decode_item(p, item);
             bool live = false;
 #pragma unroll
@@ -256,6 +259,23 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             int pr, pc;
             p.div_per_row.divmod(sp, pr, pc);
             return (((row_dead >> pr) | (col_dead >> pc)) & 1u) != 0u;
+        };
+        // kPartial: a key block is two neighbouring patches of one patch row (a window row holds an even number of patches); it
+        // holds no token when its row is dead or both of its columns are.  Every role walks the blocks jf .. jl of an item
+        // (its first and last block with tokens; a live item has some: its own query patches) and skips the dead ones in
+        // between by the same test, so the block counters that give the barrier phases stay in step.
+        auto block_dead = [&](int j, uint32_t row_dead, uint32_t col_dead) {
+            int pr, pc;
+            p.div_per_row.divmod(2 * j, pr, pc);
+            return (((row_dead >> pr) | ((col_dead & (col_dead >> 1)) >> pc)) & 1u) != 0u;
+        };
+        auto live_range = [&](uint32_t row_dead, uint32_t col_dead, int& jf, int& jl) {
+            const int per_row = p.M >> 3;
+            const uint32_t in_window = per_row == 32 ? 0xffffffffu : (1u << per_row) - 1u;
+            const uint32_t rows = ~row_dead & in_window;
+            const uint32_t pairs = ~(col_dead & (col_dead >> 1)) & 0x55555555u & in_window;     // bit 2c: columns 2c, 2c + 1
+            jf = (__ffs(rows) - 1) * (per_row >> 1) + ((__ffs(pairs) - 1) >> 1);
+            jl = (31 - __clz(rows)) * (per_row >> 1) + ((31 - __clz(pairs)) >> 1);
         };
 
         if (warp == 0) {
@@ -301,9 +321,13 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 }
                 fence_proxy_async();
                 __syncwarp();
+                uint32_t row_dead = 0u, col_dead = 0u;
+                int jf = 0, jl = nblk - 1;
+                if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
                 if (lane == 0) {
                     mbar_arrive(bar(kQPos + buf));
-                    for (int j = 0; j < nblk; ++j, ++blk) {
+                    for (int j = jf; j <= jl; ++j, ++blk) {
+                        if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         const uint32_t st = blk % kStages, use = blk / kStages;
                         if (use > 0 && !mbar_wait(bar(kKEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                         mbar_arrive_expect_tx(bar(kKFull + st), kContentBytes + kPosBytes);
@@ -346,7 +370,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint32_t buf = io & 1;
                 if (!mbar_wait_warp(bar(kQFull + buf), (io >> 1) & 1, abort_flag, p.status) ||
                     !mbar_wait_warp(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
-                for (int j = 0; j < nblk && ok; ++j, ++blk) {
+                uint32_t row_dead = 0u, col_dead = 0u;
+                int jf = 0, jl = nblk - 1;
+                if (kPartial && p.skip_dead) { dead_masks(decode_item(p, item_at(i)), row_dead, col_dead); live_range(row_dead, col_dead, jf, jl); }
+                for (int j = jf; j <= jl && ok; ++j, ++blk) {
+                    if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                     const uint32_t st = blk % kStages;
                     if (!mbar_wait_warp(bar(kKFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
                     const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
@@ -367,7 +395,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             mma_commit(bar(kSFull + qt));
                             if (qt == 1) {
                                 mma_commit(bar(kKEmpty + st));
-                                if (j == nblk - 1) mma_commit(bar(kQEmpty + buf));
+                                if (j == jl) mma_commit(bar(kQEmpty + buf));
                             }
                         }
                         __syncwarp();
@@ -383,12 +411,16 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const uint32_t d_o1 = tmem + kColO + qt * kFastOCols;         // fast form: one accumulator
             for (int i = 0; i < count && ok; ++i, ++io) {
                 if (!item_live(item_at(i))) { --io; continue; }
-                for (int j = 0; j < nblk; ++j, ++blk) {
+                uint32_t row_dead = 0u, col_dead = 0u;
+                int jf = 0, jl = nblk - 1;
+                if (kPartial && p.skip_dead) { dead_masks(decode_item(p, item_at(i)), row_dead, col_dead); live_range(row_dead, col_dead, jf, jl); }
+                for (int j = jf; j <= jl; ++j, ++blk) {
+                    if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                     const uint32_t st = blk % kStages;
                     // warp-uniform outcomes, so that the warp stays converged.  The first block of an item overwrites the
                     // accumulator: the epilogue of the item before must have read it.
                     if (!mbar_wait_warp(bar(kVFull + st), (blk / kStages) & 1, abort_flag, p.status) ||
-                        !(j > 0 || io == 0 || mbar_wait_warp(bar(kOFree + qt), (io - 1) & 1, abort_flag, p.status)) ||
+                        !(j > jf || io == 0 || mbar_wait_warp(bar(kOFree + qt), (io - 1) & 1, abort_flag, p.status)) ||
                         !mbar_wait_warp(bar(kPReady + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     if (elect_one()) {
@@ -398,12 +430,12 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             const uint64_t v = smem_desc(v_addr, kOffOnes - (kOffV + st * kContentBytes), 512, kSwizzle64B);
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk)
-                                mma_ts(d_o1, a_p + 8 * kk, v + 64 * kk, kIdescPV1, (j == 0 && kk == 0) ? 0u : 1u);
+                                mma_ts(d_o1, a_p + 8 * kk, v + 64 * kk, kIdescPV1, (j == jf && kk == 0) ? 0u : 1u);
                         } else {
                             const uint64_t v = smem_desc_at(kDesc64, v_addr);
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk)     // keys 16 kk ..: key half kk / 4 has its own accumulator
-                                mma_ts(d_o + (kk >> 2) * kD, a_p + 8 * kk, v + 64 * kk, kIdescPV, (j == 0 && (kk & 3) == 0) ? 0u : 1u);
+                                mma_ts(d_o + (kk >> 2) * kD, a_p + 8 * kk, v + 64 * kk, kIdescPV, (j == jf && (kk & 3) == 0) ? 0u : 1u);
                         }
                         mma_commit(bar(kPFree + qt));
                         mma_commit(bar(kVEmpty + st));
@@ -499,13 +531,15 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     float m_ref = 0.f;
                     float2 neg2 = make_float2(0.f, 0.f);
                     uint32_t row_dead = 0u, col_dead = 0u;
-                    if (kPartial) dead_masks(c, row_dead, col_dead);
-                    for (int j = 0; j < nblk; ++j, ++blk) {
+                    int jf = 0, jl = nblk - 1;
+                    if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                    for (int j = jf; j <= jl; ++j, ++blk) {
+                        if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
                         if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
                         tc_fence_after();
                         uint32_t sa[32], sb[32];
-                        if (j == 0) {
+                        if (j == jf) {
                             // the row's reference: the maximum over keys 0-31 of the window, the same for both key halves
                             tmem_ld32(tmem + lane_base + kColS + qt * kTile, sa);
                             tmem_wait_ld();
@@ -544,7 +578,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                             tc_fence_after();
                         }
-                        if (j == 0 && pend_ordinal >= 0) epilogue();      // that PV was the last one of the item before
+                        if (j == jf && pend_ordinal >= 0) epilogue();     // that PV was the last one of the item before
                         tmem_st16(t_p, pa);
                         tmem_st16(t_p + 16, pb);
                         tmem_wait_st();
@@ -584,8 +618,10 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     float m_used = -INFINITY, l = 0.f;
                     bool have_ref = false;            // kPartial: a block with real keys has set the reference
                     uint32_t row_dead = 0u, col_dead = 0u;
-                    if (kPartial) dead_masks(c, row_dead, col_dead);
-                    for (int j = 0; j < nblk; ++j, ++blk) {
+                    int jf = 0, jl = nblk - 1;
+                    if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                    for (int j = jf; j <= jl; ++j, ++blk) {
+                        if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
                         if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
                         tc_fence_after();
@@ -612,7 +648,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                 continue;
                             }
                         }
-                        const bool first_ref = kPartial ? !have_ref : j == 0;
+                        const bool first_ref = kPartial ? !have_ref : j == jf;
                         have_ref = true;
 #pragma unroll
                         for (int ch = 0; ch < 2; ++ch) {
@@ -641,7 +677,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                     }
                                     const float factor = need ? ex2_approx((m_used - mx) * p.scale_log2) : 1.f;
                                     if (need) { l *= factor; m_used = mx; }
-                                    if (j > 0) {
+                                    if (j > jf) {
                                         uint32_t o[32];
                                         tmem_ld32(t_o + half * kD, o);
                                         tmem_wait_ld();
@@ -802,6 +838,7 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     fp.exact_only = p.exact_softmax ? 1 : 0;
+    fp.skip_dead = kPartial && p.n / kTile >= 8 ? 1 : 0;
     fp.div_tp = make_fast_div(fp.tiles_per_item_pair); fp.div_heads = make_fast_div(p.heads);
     fp.div_nwx = make_fast_div(p.nWx); fp.div_nwy = make_fast_div(p.nWy); fp.div_per_row = make_fast_div(p.M >> 3);
     const int grid = fp.items < sm_count ? fp.items : sm_count;
