@@ -569,8 +569,8 @@ __device__ __forceinline__ bool decode_pair_token(const AuxParams& p, int pair, 
 }
 
 // One thread per (pair, token in window order): D = dO . O and lse in the layout the main kernel
-// streams, zero of this token's dQ~ accumulators; the first threads also stage bf16(Pq sqrt(d/r))
-// and clear dPq, dPk.
+// streams; the dQ~ accumulators are cleared with 16-byte stores, (d + r) / 4 per thread, as one flat array;
+// the first threads also stage bf16(Pq sqrt(d/r)) and clear dPq, dPk.
 template <int R>
 __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
 {
@@ -586,16 +586,16 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
         p.dpk[user] = 0.f;
     }
     if (t >= total) return;
+    float4* z4 = reinterpret_cast<float4*>(p.dq_acc);      // pairs * (d + r) * n floats = total * kDk / 4 vectors
+#pragma unroll
+    for (int k = 0; k < kDk / 4; ++k) z4[(size_t)k * total + t] = make_float4(0.f, 0.f, 0.f, 0.f);
     const int pair = (int)(t / p.n), w = (int)(t % p.n);
     int i; size_t tok, scalar;
-    float* z = p.dq_acc + (size_t)pair * kDk * p.n + w;
     float* ldf = reinterpret_cast<float*>(p.ld) + ((t >> 1) << 2) + (t & 1);
     if (!decode_pair_token(p, pair, w, i, tok, scalar)) {
         // a position beyond the image: as a query it gets probability 0 (exp2(-inf)) and D = 0
         ldf[0] = -INFINITY;
         ldf[2] = 0.f;
-#pragma unroll 8
-        for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
         return;
     }
     const uint4* a = reinterpret_cast<const uint4*>(p.dout + tok * kD);
@@ -614,86 +614,69 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     // per query pair (w even, w + 1): (-lse2, -lse2', -D, -D'), the operand order of the packed arithmetic
     ldf[0] = -p.lse[scalar] * 1.4426950408889634f;
     ldf[2] = -acc;
-#pragma unroll 8
-    for (int col = 0; col < kDk; ++col) z[(size_t)col * p.n] = 0.f;
 }
 
-// Finishing pass over the fp32 accumulators.  grid (n / 32, groups of pairs), 32 x 4 threads: a thread
-// owns one token position w of the window and walks a quarter of the pairs of its group; the four
-// quarters' partial sums meet in shared memory, so that one atomic per element and GROUP reaches the
-// results (these adds all land on the same n x r addresses: their number, not the traffic, set the
-// time of this kernel).  With one table for all
-// heads a group is a run of consecutive pairs; with head-wise tables it is a run of windows of one
-// head (pair = head + heads * window), so that its sums belong to one table.  Per pair it turns
-// dQ~[:, :d] / sqrt(d) into the bf16 dq row of that token, and it keeps running sums of the 16 RIB
-// columns of dQ~ (-> dPq, times 1/sqrt(r)) and of dK~ (-> dPk); the group's partial sums go to the
-// zeroed results with one vector atomic per 4 columns.
+// Finishing pass over the fp32 accumulators.  grid (n / 32, groups of pairs, R / 16), 32 x 4 threads: a thread
+// owns one token position w of the window and a quarter of the columns -- 8 of the 32 content columns of dQ~
+// (one 16-byte piece of the bf16 dq row) and 4 of the 16 RIB columns of this grid.z slice -- and walks
+// the pairs of its group.  Few registers per thread keep the SM full of warps, which is what this
+// kernel (a stream of 4-byte column reads, 128 bytes per warp) needs to reach the memory system.  With one
+// table for all heads a group is a run of consecutive pairs; with head-wise tables it is a run of windows of
+// one head (pair = head + heads * window), so that its sums belong to one table.  Per pair the thread turns its
+// piece of dQ~[:, :d] / sqrt(d) into bf16, and it keeps running sums of its RIB columns of dQ~ (-> dPq, times
+// 1/sqrt(r)) and of dK~ (-> dPk); the group's sums go to the zeroed results with one vector atomic each (these
+// adds all land on the same n x r addresses: a group is long enough that their number does not set the time).
 template <int R>
-__global__ void __launch_bounds__(128) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_thread)
+__global__ void __launch_bounds__(128, 8) rib_bwd_finish_kernel(const AuxParams p, int pairs_per_group)
 {
     constexpr int kDk = kD + R;
-    __shared__ float red[3][2][16][32];          // quarters 1-3: [dPq | dPk][column][token]
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int tx = threadIdx.x & 31, cg = threadIdx.x >> 5;
     const int w = blockIdx.x * 32 + tx;
     int pair0, pair1, step = 1;
     size_t table = 0;
     if (p.tables == 1) {
-        pair0 = (blockIdx.y * 4 + ty) * pairs_per_thread;
-        pair1 = min(p.pairs, pair0 + pairs_per_thread);
+        pair0 = blockIdx.y * pairs_per_group;
+        pair1 = min(p.pairs, pair0 + pairs_per_group);
     } else {
-        const int head = blockIdx.y % p.heads, first = ((blockIdx.y / p.heads) * 4 + ty) * pairs_per_thread;
+        const int head = blockIdx.y % p.heads, first = (blockIdx.y / p.heads) * pairs_per_group;
         step = p.heads;
         pair0 = head + first * step;
-        pair1 = min(p.pairs, pair0 + pairs_per_thread * step);
+        pair1 = min(p.pairs, pair0 + pairs_per_group * step);
         table = (size_t)head * (size_t)p.pos_head_stride;
     }
     // blockIdx.z picks 16 of the R RIB columns (grid.z = R / 16); the slice z = 0 also writes dq
-    const int col0 = 16 * blockIdx.z;
-    float sq[16], sk[16];
-#pragma unroll
-    for (int c = 0; c < 16; ++c) { sq[c] = 0.f; sk[c] = 0.f; }
+    const int col0 = 16 * blockIdx.z + 4 * cg;
+    float sq[4] = {0.f, 0.f, 0.f, 0.f}, sk[4] = {0.f, 0.f, 0.f, 0.f};
     int i = 0;
+#pragma unroll 2
     for (int pair = pair0; pair < pair1; pair += step) {
         size_t tok, scalar;
         const bool real = decode_pair_token(p, pair, w, i, tok, scalar);   // its sums are zero if not
         const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
-        if (blockIdx.z == 0 && real) {
-            uint4* dst = reinterpret_cast<uint4*>(p.dq + tok * kD);
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                float f[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * q4 + k) * p.n] * p.inv_sqrt_d;
-                dst[q4] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
-            }
-        }
         const float* srk = p.dkp + (size_t)pair * R * p.n + w;
+        float f[8], gq[4], gk[4];
+        if (blockIdx.z == 0 && real) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            sq[c] += src[(size_t)(kD + col0 + c) * p.n];
-            sk[c] += srk[(size_t)(col0 + c) * p.n];
+            for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * cg + k) * p.n];
         }
-    }
-    // (quarter 0 always has pairs: the grid is sized by the groups; later quarters may be empty and then add zeros)
-    if (ty > 0) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) { red[ty - 1][0][c][tx] = sq[c]; red[ty - 1][1][c][tx] = sk[c]; }
-    }
-    __syncthreads();
-    if (ty > 0) return;
+        for (int c = 0; c < 4; ++c) {
+            gq[c] = src[(size_t)(kD + col0 + c) * p.n];
+            gk[c] = srk[(size_t)(col0 + c) * p.n];
+        }
+        if (blockIdx.z == 0 && real) {
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        sq[c] += red[0][0][c][tx] + red[1][0][c][tx] + red[2][0][c][tx];
-        sk[c] += red[0][1][c][tx] + red[1][1][c][tx] + red[2][1][c][tx];
-    }
-    float4* out_q = reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R + col0);
-    float4* out_k = reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R + col0);
+            for (int k = 0; k < 8; ++k) f[k] *= p.inv_sqrt_d;
+            reinterpret_cast<uint4*>(p.dq + tok * kD)[cg] =
+                make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+        }
 #pragma unroll
-    for (int c4 = 0; c4 < 4; ++c4) {
-        atomicAdd(out_q + c4, make_float4(sq[4 * c4] * p.inv_sqrt_r, sq[4 * c4 + 1] * p.inv_sqrt_r, sq[4 * c4 + 2] * p.inv_sqrt_r,
-                                          sq[4 * c4 + 3] * p.inv_sqrt_r));
-        atomicAdd(out_k + c4, make_float4(sk[4 * c4], sk[4 * c4 + 1], sk[4 * c4 + 2], sk[4 * c4 + 3]));
+        for (int c = 0; c < 4; ++c) { sq[c] += gq[c]; sk[c] += gk[c]; }
     }
+    // (the first pair of a group always exists: the grid is sized by the groups; i is the token's row of the tables)
+    atomicAdd(reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R + col0),
+              make_float4(sq[0] * p.inv_sqrt_r, sq[1] * p.inv_sqrt_r, sq[2] * p.inv_sqrt_r, sq[3] * p.inv_sqrt_r));
+    atomicAdd(reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R + col0), make_float4(sk[0], sk[1], sk[2], sk[3]));
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -774,11 +757,13 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
-    const int per_group = p.pairs < 8 ? 1 : 4;
     const int windows = p.pairs / p.heads;   // pairs of one head
-    // a block takes four runs of per_group pairs (of one head, with head-wise tables)
-    const unsigned runs = (unsigned)(((tables == 1 ? p.pairs : windows) + per_group - 1) / per_group);
-    const unsigned groups = (tables == 1 ? 1u : (unsigned)p.heads) * ((runs + 3) / 4);
+    const int in_line = tables == 1 ? p.pairs : windows;      // pairs whose sums go to one table
+    // a block takes a run of per_group pairs (of one head, with head-wise tables)
+    // (measured on the training configuration: 4 or 8 pairs per block 62 us, 16: 74 us, 32: 74 us -- more blocks in flight
+    // matter more to this kernel than fewer atomics)
+    const int per_group = in_line >= 1024 ? 8 : in_line >= 16 ? 4 : 1;
+    const unsigned groups = (tables == 1 ? 1u : (unsigned)p.heads) * (unsigned)((in_line + per_group - 1) / per_group);
     dim3 grid_fin((unsigned)(p.n / 32), groups, (unsigned)(R / 16));
     { ProfileScope scope(RIB_KERNEL_BWD_FINISH, stream); rib_bwd_finish_kernel<R><<<grid_fin, 128, 0, stream>>>(ap, per_group); }
     return cudaGetLastError();

@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
             const int idx = threadIdx.x + u * kThreads;
             if (idx < 9 * D) taps[idx] = tp[u];
         }
-        if (threadIdx.x < D) { bdw[threadIdx.x] = my_bdw; bpw[threadIdx.x] = my_bpw; }
+        if (threadIdx.x < D) { bdw[threadIdx.x] = my_bdw; bpw[threadIdx.x] = 0.5f * my_bpw; }
     }
     fence_proxy_async();
     tc_fence_before();
@@ -145,44 +145,53 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
     uint32_t it = 0;
     if (warp < kFilterWarps) {
         // ===================== filter warps: halo -> depth-wise 3 x 3 -> A operand; warp 0 also requests halos and issues MMAs
-        const int c8 = threadIdx.x % kChunks, strip = threadIdx.x / kChunks;
-        const int py = strip >> 1, px0 = (strip & 1) * 8;
+        // A thread owns a chunk of 4 channels and two strips of 8 pixels of a tile row each.  Its 9 x 4 taps stay in registers
+        // as pairs (the arithmetic is the packed two-lane fp32 FMA); along a strip the 3 x 3 window slides: every halo pixel
+        // is read from shared memory and widened to fp32 once per strip (3 new pixels per output instead of 9).
+        constexpr int kChunks4 = D / 4, kStripStep = kFilterWarps * 32 / kChunks4;      // strips the filter threads cover at once (8)
+        static_assert(kStripStep * 2 == 2 * kTileH && (kFilterWarps * 32) % kChunks4 == 0, "two strips per filter thread");
+        const int c4 = threadIdx.x % kChunks4, strip0 = threadIdx.x / kChunks4;
+        float2 tap_lo[9], tap_hi[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+            const float4 w4 = *reinterpret_cast<const float4*>(taps + t * D + 4 * c4);
+            tap_lo[t] = make_float2(w4.x, w4.y); tap_hi[t] = make_float2(w4.z, w4.w);
+        }
+        const float4 b4 = *reinterpret_cast<const float4*>(bdw + 4 * c4);
+        const float2 bias_lo = make_float2(b4.x, b4.y), bias_hi = make_float2(b4.z, b4.w);
+        const uint32_t a_chunk = (uint32_t)(c4 >> 4) * L::kAAtom + (uint32_t)(c4 & 1) * 8u, a_sw = (uint32_t)((c4 & 15) >> 1);
         for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
             // the halo of this tile has landed, and the MMAs of the previous tile no longer read the A operand
             if (!__all_sync(0xffffffffu, mbar_wait(bar_halo, it & 1, abort_flag, p.status) &&
                                              (it == 0 || mbar_wait(bar, (it - 1) & 1, abort_flag, p.status)))) { ok = false; break; }
-            // A thread owns one chunk of 8 channels and a strip of 8 pixels of one tile row; its 9 x 8 taps sit in
-            // registers for the strip (the shared-memory pipe is what this phase is bound by: 9 halo reads per pixel).
-            float w[9][8];
+#pragma unroll 1
+            for (int u = 0; u < 2; ++u) {
+                const int strip = strip0 + kStripStep * u;
+                const int py = strip >> 1, px0 = (strip & 1) * 8;
+                const uint8_t* hrow = sm + L::kOffHalo + ((size_t)(py * kHaloW + px0) * D + 4 * c4) * 2;
+                float2 win_lo[3][3], win_hi[3][3];          // [column slot][row]
 #pragma unroll
-            for (int t = 0; t < 9; ++t) {
-                const float4 w0 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8);
-                const float4 w1 = *reinterpret_cast<const float4*>(taps + t * D + 8 * c8 + 4);
-                w[t][0] = w0.x; w[t][1] = w0.y; w[t][2] = w0.z; w[t][3] = w0.w;
-                w[t][4] = w1.x; w[t][5] = w1.y; w[t][6] = w1.z; w[t][7] = w1.w;
-            }
-            float bias[8];
+                for (int j = 0; j < 10; ++j) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) bias[k] = bdw[8 * c8 + k];
-#pragma unroll 2
-            for (int j = 0; j < 8; ++j) {
-                const int px = px0 + j, pix = py * kTileW + px;
-                float acc[8];
+                    for (int r = 0; r < 3; ++r) {
+                        const uint2 v = *reinterpret_cast<const uint2*>(hrow + (size_t)(r * kHaloW + j) * D * 2);
+                        win_lo[j % 3][r] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
+                        win_hi[j % 3][r] = make_float2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+                    }
+                    if (j >= 2) {
+                        float2 acc_lo = bias_lo, acc_hi = bias_hi;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) acc[k] = bias[k];
+                        for (int r = 0; r < 3; ++r)
 #pragma unroll
-                for (int t = 0; t < 9; ++t) {
-                    const int hp = (py + t / 3) * kHaloW + px + t % 3;
-                    const uint4 v = *reinterpret_cast<const uint4*>(sm + L::kOffHalo + (size_t)hp * D * 2 + c8 * 16);
-                    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        acc[2 * k] = fmaf(__uint_as_float(u[k] << 16), w[t][2 * k], acc[2 * k]);
-                        acc[2 * k + 1] = fmaf(__uint_as_float(u[k] & 0xffff0000u), w[t][2 * k + 1], acc[2 * k + 1]);
+                            for (int c = 0; c < 3; ++c) {
+                                acc_lo = __ffma2_rn(win_lo[(j - 2 + c) % 3][r], tap_lo[3 * r + c], acc_lo);
+                                acc_hi = __ffma2_rn(win_hi[(j - 2 + c) % 3][r], tap_hi[3 * r + c], acc_hi);
+                            }
+                        const int pix = py * kTileW + px0 + j - 2;
+                        *reinterpret_cast<uint2*>(sm + L::kOffA + a_chunk + pix * 128 + ((a_sw ^ (uint32_t)(pix & 7)) << 4)) =
+                            make_uint2(pack_bf16x2(acc_lo.x, acc_lo.y), pack_bf16x2(acc_hi.x, acc_hi.y));
                     }
                 }
-                *reinterpret_cast<uint4*>(sm + L::kOffA + (c8 >> 3) * L::kAAtom + pix * 128 + (((c8 & 7) ^ (pix & 7)) << 4)) =
-                    make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]), pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
             }
             fence_proxy_async();
             __syncwarp();
@@ -231,11 +240,14 @@ __global__ void __launch_bounds__(kThreads, 1) rib_cla_gate_kernel(const __grid_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_accfree);
                 }
+                // sigmoid(z) = 1/2 + 1/2 tanh(z / 2): one special-function instruction per value (bpw holds half the bias)
                 float g[16];
 #pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    const float z = __uint_as_float(a[k]) + bpw[16 * part + k];
-                    g[k] = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z));
+                for (int k = 0; k < 16; k += 2) {
+                    const float2 zh = __ffma2_rn(make_float2(__uint_as_float(a[k]), __uint_as_float(a[k + 1])), make_float2(0.5f, 0.5f),
+                                                 *reinterpret_cast<const float2*>(bpw + 16 * part + k));
+                    const float2 gg = __ffma2_rn(make_float2(tanh_approx(zh.x), tanh_approx(zh.y)), make_float2(0.5f, 0.5f), make_float2(0.5f, 0.5f));
+                    g[k] = gg.x; g[k + 1] = gg.y;
                 }
                 uint4* d16 = reinterpret_cast<uint4*>(dst + 16 * part);
                 d16[0] = make_uint4(pack_bf16x2(g[0], g[1]), pack_bf16x2(g[2], g[3]), pack_bf16x2(g[4], g[5]), pack_bf16x2(g[6], g[7]));

@@ -296,6 +296,13 @@ __device__ __forceinline__ float ex2_approx(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// tanh on the special-function unit (absolute error about 2^-11)
+__device__ __forceinline__ float tanh_approx(float x)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 // 2^x for a pair of arguments on the FMA and integer pipes (no MUFU): x = n + f with n = round(x),
 // |f| <= 1/2; 2^f by a cubic fitted to 2^f on [-1/2, 1/2] (relative error 7.5e-5, well below the bf16
 // rounding of the result), 2^n by adding n to the exponent field.  The integer n is read off the low
