@@ -149,6 +149,28 @@ size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, in
                                             int window);
 
 /*
+ * Shifted windows with a mask.  The paper's cycle of window sizes (Sec. 3.3) needs no shift; the `shift` argument of the
+ * calls above rolls the map by (-shift, -shift) before it is cut into windows, so a window of the last window row
+ * (column) holds tokens from the bottom (right) of the map and, from window position M - shift on, wrapped tokens from its
+ * top (left), and there those attend to each other.  In these two calls they do not: inside a window a query attends
+ * only to the keys of its own part (wrapped or not, in each direction separately), every other logit of Eq. 6 counts as
+ * minus infinity.  H and W must be multiples of the window (RIB_ERR_SHAPE otherwise).  pos_head_stride as in
+ * rib_window_attn_fwd_headwise (0: one table for all heads); all other arguments, layouts, error codes and the workspace
+ * (rib_window_attn_bwd_headwise_workspace) as in the unmasked calls.  With shift = 0 the results equal theirs.  The tcgen05
+ * kernels need shift % 8 == 0 (a patch of 8 x 8 tokens then lies in one part); other shifts take the any-shape kernels.
+ */
+int rib_window_attn_fwd_masked(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* out, float* lse, void* stream);
+int rib_window_attn_bwd_masked(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               const void* out, const float* lse, const void* dout,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The cyclic window strategy (Sec. 3.3: the window size cycles over the attention layers of a block, e.g.
  * {16, 32, 64, 16, 32, 64}, instead of shifting windows): one call that enqueues the forward pass of `layers`
  * attention layers over maps of one size, layer l with window windows[l] (and cyclic shift shifts[l]; shifts

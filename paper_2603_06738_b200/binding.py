@@ -27,6 +27,7 @@ EXPORTS = (
     "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
     "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
     "rib_window_attn_bwd_padded", "rib_window_attn_bwd_padded_workspace",
+    "rib_window_attn_fwd_masked", "rib_window_attn_bwd_masked",
     "rib_cla_product", "rib_cla_product_bwd", "rib_cla_gate_bwd", "rib_cla_gate_bwd_workspace",
     "rib_wait_probe", "rib_exp_probe", "rib_tensor_map_cache_counts", "rib_window_cycle_fwd",
 )
@@ -68,6 +69,10 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_fwd_padded.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd_padded.restype = ci
         lib.rib_window_attn_bwd_padded.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_attn_fwd_masked.restype = ci
+        lib.rib_window_attn_fwd_masked.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
+        lib.rib_window_attn_bwd_masked.restype = ci
+        lib.rib_window_attn_bwd_masked.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
         lib.rib_window_attn_bwd_padded_workspace.restype = ctypes.c_size_t
         lib.rib_window_attn_bwd_padded_workspace.argtypes = [ll] + [ci] * 7
         lib.rib_cla_gate.restype = ci
@@ -359,6 +364,64 @@ def rib_window_attn_bwd_padded(q, k, v, pq, pk, out, lse, dout, window, shift=0,
     dpq = torch.empty(tuple(pq.shape), dtype=torch.float32, device=q.device)
     dpk = torch.empty(tuple(pk.shape), dtype=torch.float32, device=q.device)
     rc = library().rib_window_attn_bwd_padded(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), stride, _ptr(out), _ptr(lse),
+                                              _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq), _ptr(dk), _ptr(dv),
+                                              _ptr(dpq), _ptr(dpk), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return dq, dk, dv, dpq, dpk
+
+
+def rib_window_attn_fwd_masked(q, k, v, pq, pk, window, shift=0, stream=None, want_lse=True):
+    """Forward pass with shifted windows whose wrapped parts do not attend to each other (H, W multiples of the
+    window); pq, pk are [n, r] or [heads, n, r].  Returns (out, lse)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    _check_image("k", k, q.shape)
+    _check_image("v", v, q.shape)
+    n = window * window
+    headwise = pq.dim() == 3
+    if headwise:
+        _check_pos_headwise("pq", pq, heads, n)
+        _check_pos_headwise("pk", pk, heads, n)
+    else:
+        _check_pos("pq", pq, n)
+        _check_pos("pk", pk, n)
+    r = pq.shape[-1]
+    out = torch.empty_like(q)
+    lse = torch.empty((B, heads, H, W), dtype=torch.float32, device=q.device) if want_lse else None
+    rc = library().rib_window_attn_fwd_masked(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), n * r if headwise else 0,
+                                              B, H, W, heads, d, r, window, shift, _ptr(out), _ptr(lse), _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return out, lse
+
+
+def rib_window_attn_bwd_masked(q, k, v, pq, pk, out, lse, dout, window, shift=0, workspace=None, stream=None):
+    """Backward pass of rib_window_attn_fwd_masked; pq, pk [n, r] or [heads, n, r].
+    Returns (dq, dk, dv bf16, dpq, dpk fp32 of the shape of pq)."""
+    _check_image("q", q)
+    B, H, W, heads, d = q.shape
+    for name, t in (("k", k), ("v", v), ("out", out), ("dout", dout)):
+        _check_image(name, t, q.shape)
+    n = window * window
+    headwise = pq.dim() == 3
+    if headwise:
+        _check_pos_headwise("pq", pq, heads, n)
+        _check_pos_headwise("pk", pk, heads, n)
+    else:
+        _check_pos("pq", pq, n)
+        _check_pos("pk", pk, n)
+    r = pq.shape[-1]
+    stride = n * r if headwise else 0
+    if lse.dtype != torch.float32 or tuple(lse.shape) != (B, heads, H, W) or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous fp32 tensor [B,heads,H,W]")
+    need = int(library().rib_window_attn_bwd_padded_workspace(stride, B, H, W, heads, d, r, window))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dpq = torch.empty(tuple(pq.shape), dtype=torch.float32, device=q.device)
+    dpk = torch.empty(tuple(pk.shape), dtype=torch.float32, device=q.device)
+    rc = library().rib_window_attn_bwd_masked(_ptr(q), _ptr(k), _ptr(v), _ptr(pq), _ptr(pk), stride, _ptr(out), _ptr(lse),
                                               _ptr(dout), B, H, W, heads, d, r, window, shift, _ptr(dq), _ptr(dk), _ptr(dv),
                                               _ptr(dpq), _ptr(dpk), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     if rc != RIB_OK:

@@ -62,7 +62,7 @@ void fill_shape(rib::Problem& p, int B, int H, int W, int heads, int d, int r, i
 
 int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk, long long pos_head_stride, const void* gate,
              int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream,
-             bool validate_only = false);
+             bool validate_only = false, bool masked = false);
 
 int check_pos_stride(long long stride, int window, int r)
 {
@@ -312,7 +312,8 @@ int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const 
 namespace {
 
 int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk, long long pos_head_stride, const void* gate,
-             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream, bool validate_only)
+             int B, int H, int W, int heads, int d, int r, int window, int shift, void* out, float* lse, void* stream, bool validate_only,
+             bool masked)
 {
     if (!q || !k || !v || !out || (r > 0 && (!pq || !pk))) return RIB_ERR_NULL;
     if (int rc = check_shape(B, H, W, heads, d, r, window, shift, true)) return rc;
@@ -332,6 +333,7 @@ int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const 
     p.lse_w = lse;
     p.pos_head_stride = pos_head_stride;
     p.gate = static_cast<const __nv_bfloat16*>(gate);
+    p.masked = masked;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int forced = g_forced_path.load();
@@ -406,12 +408,12 @@ size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, in
     return need;
 }
 
-int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
-                               long long pos_head_stride,
-                               const void* out, const float* lse, const void* dout,
-                               int B, int H, int W, int heads, int d, int r, int window, int shift,
-                               void* dq, void* dk, void* dv, float* dpq, float* dpk,
-                               void* workspace, size_t workspace_bytes, void* stream)
+static int bwd_impl(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                    long long pos_head_stride,
+                    const void* out, const float* lse, const void* dout,
+                    int B, int H, int W, int heads, int d, int r, int window, int shift,
+                    void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                    void* workspace, size_t workspace_bytes, void* stream, bool masked)
 {
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return RIB_ERR_NULL;
     if (r > 0 && (!pq || !pk || !dpq || !dpk)) return RIB_ERR_NULL;
@@ -442,6 +444,7 @@ int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, cons
     p.workspace = workspace;
     p.workspace_bytes = workspace_bytes;
     p.pos_head_stride = pos_head_stride;
+    p.masked = masked;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_bwd_supported(p);
@@ -450,6 +453,38 @@ int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, cons
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
     g_kernel_launches += 3;   // prepare, main, finish : rowdot, dq, dk/dv
     return RIB_OK;
+}
+
+int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               const void* out, const float* lse, const void* dout,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                               void* workspace, size_t workspace_bytes, void* stream)
+{
+    return bwd_impl(q, k, v, pq, pk, pos_head_stride, out, lse, dout, B, H, W, heads, d, r, window, shift, dq, dk, dv, dpq, dpk,
+                    workspace, workspace_bytes, stream, false);
+}
+
+int rib_window_attn_fwd_masked(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* out, float* lse, void* stream)
+{
+    if (H > 0 && W > 0 && window > 0 && (H % window || W % window)) return RIB_ERR_SHAPE;
+    return fwd_impl(q, k, v, pq, pk, pos_head_stride, nullptr, B, H, W, heads, d, r, window, shift, out, lse, stream, false, true);
+}
+
+int rib_window_attn_bwd_masked(const void* q, const void* k, const void* v, const void* pq, const void* pk,
+                               long long pos_head_stride,
+                               const void* out, const float* lse, const void* dout,
+                               int B, int H, int W, int heads, int d, int r, int window, int shift,
+                               void* dq, void* dk, void* dv, float* dpq, float* dpk,
+                               void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (H > 0 && W > 0 && window > 0 && (H % window || W % window)) return RIB_ERR_SHAPE;
+    return bwd_impl(q, k, v, pq, pk, pos_head_stride, out, lse, dout, B, H, W, heads, d, r, window, shift, dq, dk, dv, dpq, dpk,
+                    workspace, workspace_bytes, stream, true);
 }
 
 int rib_window_attn_bwd_noalloc(const void* q, const void* k, const void* v, const void* pq, const void* pk,

@@ -105,6 +105,7 @@ struct BwdParams {
     int H, W, heads, M, s, n, nWy, nWx, nblk, items;
     int Hp, Wp;                // sides of the map the windows are laid over (H, W rounded up to multiples of M)
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
+    int masked;                // kPartial: shifted windows with a mask (a query sees the keys of its own part of a border window)
     float scale_log2;          // log2(e) / sqrt(d)
     float inv_sqrt_d;
 };
@@ -342,14 +343,23 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         uint32_t g = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
-            bool key_real = true;         // kPartial: this warp's 32 key rows lie in one 8x8 patch of the key block
+            bool key_exists = true;       // kPartial: this warp's 32 key rows lie in one 8x8 patch of the key block
+            int key_part = 0, last_window = 0;   // masked shifted windows: part of the key patch; bit 1 / 0: last window row / column
             if (kPartial) {
                 const ItemCoord c = decode_item(p, item);
                 int py, px, Y0, X0;
                 patch_origin(geom, c.wy, c.wx, 2 * c.J + (quarter >> 1), py, px, Y0, X0);
-                key_real = Y0 < p.H && X0 < p.W;
+                key_exists = Y0 < p.H && X0 < p.W;
+                last_window = (c.wy == p.nWy - 1 ? 2 : 0) | (c.wx == p.nWx - 1 ? 1 : 0);
+                key_part = window_part(p.M, p.s, last_window & 2, last_window & 1, py, px);
             }
             for (int I = 0; I < p.nblk; ++I, ++g) {
+                // the 64 queries of this half-tile are one 8x8 patch as well: with a mask, one answer per warp and half-tile
+                bool key_real = key_exists;
+                if (kPartial && p.masked) {
+                    const int per_row = p.M >> 3, qp = 2 * I + h;
+                    key_real = key_exists && key_part == window_part(p.M, p.s, last_window & 2, last_window & 1, (qp / per_row) << 3, (qp % per_row) << 3);
+                }
                 const uint32_t st = g % kQStages;
                 // warp-uniform outcome: the TMEM accesses below are warp-collective
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) &&
@@ -750,6 +760,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     bp.nblk = p.n / kTile;
     bp.items = p.pairs * bp.nblk;
     bp.pos_per_head = tables > 1 ? 1 : 0;
+    bp.masked = p.masked ? 1 : 0;
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
@@ -771,7 +782,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 {
-    if (p.Hp != p.H || p.Wp != p.W) return p.r == 32 ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W || p.masked) return p.r == 32 ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
     return p.r == 32 ? launch_bwd<32, false>(p, stream) : launch_bwd<16, false>(p, stream);
 }
 

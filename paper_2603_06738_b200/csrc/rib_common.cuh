@@ -38,6 +38,7 @@ struct Problem {
     int n, nWy, nWx, pairs;           // n = M*M, windows per image, B*nWy*nWx*heads
     int* status;                      // device status word (bounded waits report here)
     bool exact_softmax;               // tcgen05 forward: every item takes the exact (running-maximum) softmax form
+    bool masked;                      // shifted windows: the wrapped parts of a border window do not attend to each other
 };
 
 // Pq/Pk tables: one shared by the heads, or one per head (Sec. 3.1, after Eq. 3: head-wise projections of the shared h).
@@ -102,6 +103,14 @@ __host__ __device__ inline void token_pixel(int H, int W, int M, int s, int wy, 
     const int y = i / M, x = i - y * M;
     Y = wy * M + y + s; if (Y >= H) Y -= H;
     X = wx * M + x + s; if (X >= W) X -= W;
+}
+
+// Shifted windows with a mask: in the last window row (column) the positions from M - s on come from the other side of
+// the map.  Part of a window position: bit 1 = wrapped rows, bit 0 = wrapped columns; two tokens of a window attend to each
+// other when their parts are equal.
+__host__ __device__ inline int window_part(int M, int s, bool last_wy, bool last_wx, int y, int x)
+{
+    return ((last_wy && y >= M - s) ? 2 : 0) | ((last_wx && x >= M - s) ? 1 : 0);
 }
 
 }  // namespace rib

@@ -115,6 +115,7 @@ struct FwdParams {
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
     int exact_only;            // 1: skip the fast form (every item takes the exact softmax)
     int skip_dead;             // kPartial: 1 = items and key blocks without tokens are skipped, 0 = walked with probability 0
+    int masked;                // kPartial: shifted windows with a mask -- a query sees the keys of its own part of a border window only
     FastDiv div_tp, div_heads, div_nwx, div_nwy, div_per_row;   // tiles_per_item_pair, heads, nWx, nWy, M / 8
 };
 
@@ -254,6 +255,20 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             int x = c.wx * p.M + 8 * lane + p.s; if (x >= p.Wp) x -= p.Wp;
             row_dead = __ballot_sync(0xffffffffu, y >= p.H);
             col_dead = __ballot_sync(0xffffffffu, x >= p.W);
+        };
+        // Masked shifted windows (p.masked, a use of the kPartial instantiation on a map the window divides): in the last window
+        // row (column) the patch rows (columns) from (M - s) / 8 on hold the wrapped part of the map.  For the query patch
+        // q_patch the patch rows and columns of the OTHER part count as dead, which hands the mask to the code that gives the
+        // keys beyond a map probability 0.  (The shift is a multiple of 8: a patch lies in one part.)
+        auto mask_masks = [&](const ItemCoord& c, int q_patch, uint32_t& row_dead, uint32_t& col_dead) {
+            const int per_row = p.M >> 3, thr = (p.M - p.s) >> 3;
+            const uint32_t in_window = per_row == 32 ? 0xffffffffu : (1u << per_row) - 1u;
+            const uint32_t wrapped = in_window & ~(thr >= 32 ? 0xffffffffu : (1u << thr) - 1u);
+            const uint32_t rows_w = c.wy == p.nWy - 1 ? wrapped : 0u, cols_w = c.wx == p.nWx - 1 ? wrapped : 0u;
+            int pr, pc;
+            p.div_per_row.divmod(q_patch, pr, pc);
+            row_dead = ((rows_w >> pr) & 1u) ? in_window & ~rows_w : rows_w;
+            col_dead = ((cols_w >> pc) & 1u) ? in_window & ~cols_w : cols_w;
         };
         auto patch_dead = [&](int sp, uint32_t row_dead, uint32_t col_dead) {
             int pr, pc;
@@ -533,6 +548,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     uint32_t row_dead = 0u, col_dead = 0u;
                     int jf = 0, jl = nblk - 1;
                     if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                    if (kPartial && p.masked) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
                     for (int j = jf; j <= jl; ++j, ++blk) {
                         if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
@@ -620,6 +636,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     uint32_t row_dead = 0u, col_dead = 0u;
                     int jf = 0, jl = nblk - 1;
                     if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                    if (kPartial && p.masked) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
                     for (int j = jf; j <= jl; ++j, ++blk) {
                         if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
@@ -811,7 +828,7 @@ bool sm100_fwd_supported(const Problem& p)
 {
     const bool partial = p.Hp != p.H || p.Wp != p.W;
     return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0 &&
-           !(partial && p.gate);
+           !((partial || p.masked) && p.gate);
 }
 
 template <int R, bool kPartial, bool kGated>
@@ -838,7 +855,8 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     fp.exact_only = p.exact_softmax ? 1 : 0;
-    fp.skip_dead = kPartial && p.n / kTile >= 8 ? 1 : 0;
+    fp.masked = p.masked ? 1 : 0;
+    fp.skip_dead = kPartial && !p.masked && p.n / kTile >= 8 ? 1 : 0;      // (a mask differs from query patch to query patch)
     fp.div_tp = make_fast_div(fp.tiles_per_item_pair); fp.div_heads = make_fast_div(p.heads);
     fp.div_nwx = make_fast_div(p.nWx); fp.div_nwy = make_fast_div(p.nWy); fp.div_per_row = make_fast_div(p.M >> 3);
     const int grid = fp.items < sm_count ? fp.items : sm_count;
@@ -848,7 +866,7 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
 {
-    if (p.Hp != p.H || p.Wp != p.W) return p.r == 32 ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W || p.masked) return p.r == 32 ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
     if (p.gate) return p.r == 32 ? launch_fwd<32, false, true>(p, stream) : launch_fwd<16, false, true>(p, stream);
     return p.r == 32 ? launch_fwd<32, false, false>(p, stream) : launch_fwd<16, false, false>(p, stream);
 }

@@ -39,6 +39,14 @@ __device__ inline bool token_exists(const Problem& p, const PairCoord& c, int i)
     return Y < p.H && X < p.W;
 }
 
+// Masked shifted windows: may query position i attend to key position j of the pair's window?
+__device__ inline bool pair_allowed(const Problem& p, const PairCoord& c, int i, int j)
+{
+    if (!p.masked) return true;
+    const bool ly = c.wy == p.nWy - 1, lx = c.wx == p.nWx - 1;
+    return window_part(p.M, p.s, ly, lx, i / p.M, i % p.M) == window_part(p.M, p.s, ly, lx, j / p.M, j % p.M);
+}
+
 // element offset of channel 0 of token i of the pair in a [B][H][W][heads][d] tensor (the token must exist)
 __device__ inline size_t token_offset(const Problem& p, const PairCoord& c, int i)
 {
@@ -127,8 +135,9 @@ __global__ void __launch_bounds__(kThreads) generic_fwd_kernel(const Problem p)
                 s0 = fmaf(a, Kt[lane * ldk + col], s0);
                 s1 = fmaf(a, Kt[(lane + 32) * ldk + col], s1);
             }
-            if (j0 + lane >= p.n || !token_exists(p, c, j0 + lane)) s0 = -INFINITY;
-            if (j0 + lane + 32 >= p.n || !token_exists(p, c, j0 + lane + 32)) s1 = -INFINITY;
+            const int qi = min(row0 + warp * kRowsPerWarp + rr, p.n - 1);
+            if (j0 + lane >= p.n || !token_exists(p, c, j0 + lane) || !pair_allowed(p, c, qi, j0 + lane)) s0 = -INFINITY;
+            if (j0 + lane + 32 >= p.n || !token_exists(p, c, j0 + lane + 32) || !pair_allowed(p, c, qi, j0 + lane + 32)) s1 = -INFINITY;
             const float m_new = fmaxf(m[rr], warp_max(fmaxf(s0, s1)));
             // -inf only while no key of the row's window has been seen yet (extended maps): nothing to add then
             const bool none = m_new == -INFINITY;
@@ -229,8 +238,9 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dq_kernel(const Problem 
                 g1 = fmaf(a, Vt[(lane + 32) * ldv + col], g1);
             }
             // keys beyond the window or, on an extended map, beyond the image have probability 0
-            const float p0 = j0 + lane < p.n && token_exists(p, c, j0 + lane) ? expf(s0 - lse[rr]) : 0.f;
-            const float p1 = j0 + lane + 32 < p.n && token_exists(p, c, j0 + lane + 32) ? expf(s1 - lse[rr]) : 0.f;
+            const int qi = min(row0 + warp * kRowsPerWarp + rr, p.n - 1);
+            const float p0 = j0 + lane < p.n && token_exists(p, c, j0 + lane) && pair_allowed(p, c, qi, j0 + lane) ? expf(s0 - lse[rr]) : 0.f;
+            const float p1 = j0 + lane + 32 < p.n && token_exists(p, c, j0 + lane + 32) && pair_allowed(p, c, qi, j0 + lane + 32) ? expf(s1 - lse[rr]) : 0.f;
             float* srow = Ss + (warp * kRowsPerWarp + rr) * kTile;
             srow[lane] = p0 * (g0 - Di[rr]);
             srow[lane + 32] = p1 * (g1 - Di[rr]);
@@ -309,8 +319,9 @@ __global__ void __launch_bounds__(kThreads) generic_bwd_dkv_kernel(const Problem
                 g0 = fmaf(a, Gt[lane * ldv + col], g0);
                 g1 = fmaf(a, Gt[(lane + 32) * ldv + col], g1);
             }
-            const float p0 = i0 + lane < p.n ? expf(s0 - Lt[lane]) : 0.f;
-            const float p1 = i0 + lane + 32 < p.n ? expf(s1 - Lt[lane + 32]) : 0.f;
+            const int kj = min(row0 + warp * kRowsPerWarp + rr, p.n - 1);
+            const float p0 = i0 + lane < p.n && pair_allowed(p, c, i0 + lane, kj) ? expf(s0 - Lt[lane]) : 0.f;
+            const float p1 = i0 + lane + 32 < p.n && pair_allowed(p, c, i0 + lane + 32, kj) ? expf(s1 - Lt[lane + 32]) : 0.f;
             float* prow = Ps + (warp * kRowsPerWarp + rr) * kTile;
             float* srow = Ss + (warp * kRowsPerWarp + rr) * kTile;
             prow[lane] = p0; prow[lane + 32] = p1;
