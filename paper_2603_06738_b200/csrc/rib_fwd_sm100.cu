@@ -39,6 +39,8 @@
 //   On maps with partial windows (kPartial) key patches in the extension of the map contribute probability 0 in
 //   both forms, the fast form takes its reference from the first block that holds real keys, and items whose query
 //   patches all lie in the extension are skipped by every role alike.
+//   Shifted windows with a mask run on the kPartial instantiation too: for a query patch the patches of the other part
+//   of its border window count as patches of the extension.
 //
 // Tiles are two 8x8-token patches (see rib_sm100_common.cuh), fetched by one TMA box each.
 //
