@@ -158,7 +158,7 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=None, help="prefix of a configuration name (default: cfg2 shape)")
+    ap.add_argument("--workload", default=None, help="prefix of a configuration name (default: the training configuration, cfg5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the timings of rank 32, head-wise tables and partial windows")
@@ -463,6 +463,14 @@ def main():
                 bf = wl.pairs * 2 * wl.n * wl.n * (5 * wl.d + 3 * r_v)
                 variants[name] = {"r": r_v, "fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_tflops": ff / (f_ms * 1e-3) / 1e12,
                                   "bwd_tflops": bf / (b_ms * 1e-3) / 1e12, "paths": [binding.rib_last_path()]}
+            # shifted windows with a region mask (the wrapped parts of a border window do not attend to each other)
+            out_m, lse_m = binding.rib_window_attn_fwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], wl.window, wl.shift)
+            f_ms = timed(lambda: binding.rib_window_attn_fwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], wl.window, wl.shift))
+            b_ms = timed(lambda: binding.rib_window_attn_bwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], out_m, lse_m, s0["dout"],
+                                                                    wl.window, wl.shift))
+            variants["masked_shift"] = {"fwd_ms": f_ms, "bwd_ms": b_ms, "paths": [binding.rib_last_path()],
+                                        "note": "same shape as the timed workload; times of the unmasked calls are `fwd.ms` and `bwd.ms`"}
+            del out_m, lse_m
             # the paper's inference frame: 360 x 640 tokens, not a multiple of the 64 x 64 window (forward only)
             fh, fw, fwin = 360, 640, 64
             fq, fk, fv = (torch.randn((1, fh, fw, wl.heads, wl.d), device=dev).to(torch.bfloat16) for _ in range(3))
