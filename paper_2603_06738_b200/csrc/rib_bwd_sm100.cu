@@ -370,6 +370,15 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const float4* ld = reinterpret_cast<const float4*>(base_ptr + kOffRing + st * kRingBytes + kRingLD) + 32 * h + 16 * cg;
                     uint8_t* ds_row = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf + row * 128;
                     uint32_t pp[2][8], dd[2][8];
+                    if (kPartial && !key_real) {
+                        // nothing of this warp's key rows meets this half-tile's queries (no tokens, or another part of a masked
+                        // window): P^T = dS^T = 0 without reading the scores; the accumulators go back to the MMA warp at once
+    #pragma unroll
+                        for (int i = 0; i < 8; ++i) { pp[0][i] = pp[1][i] = 0u; dd[0][i] = dd[1][i] = 0u; }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kSFree + h));
+                    } else
     #pragma unroll
                     for (int ch = 0; ch < 2; ++ch) {
                         uint32_t s[16], dp[16];
@@ -390,8 +399,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                             const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])),
                                                                      make_float2(t.z, t.w)));
-                            pp[ch][i] = kPartial && !key_real ? 0u : pack_bf16x2(e.x, e.y);
-                            dd[ch][i] = kPartial && !key_real ? 0u : pack_bf16x2(d.x, d.y);
+                            pp[ch][i] = pack_bf16x2(e.x, e.y);
+                            dd[ch][i] = pack_bf16x2(d.x, d.y);
                         }
                     }
                     // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
@@ -420,6 +429,13 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     for (int gq = 0; gq < 4; ++gq) t4[gq] = ld[4 * gq];       // queries 8 gq + 2 (lane % 4), + 1 of this warp's 32
                     uint8_t* ds_tile = base_ptr + kOffDS + ((g & 1) * 2 + h) * kDSHalf;
                     uint32_t pp[2][8], dd[2][8];
+                    if (kPartial && !key_real) {
+    #pragma unroll
+                        for (int i = 0; i < 8; ++i) { pp[0][i] = pp[1][i] = 0u; dd[0][i] = dd[1][i] = 0u; }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kSFree + h));
+                    } else
     #pragma unroll
                     for (int ch = 0; ch < 2; ++ch) {                          // lanes 16 ch .. 16 ch + 15 of the warp's quarter
                         uint32_t s[16], dp[16];
@@ -442,8 +458,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                 const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                                 const float2 d = __fmul2_rn(e, __fadd2_rn(make_float2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])),
                                                                          make_float2(t4[gq].z, t4[gq].w)));
-                                pp[ch][2 * gq + rr] = kPartial && !key_real ? 0u : pack_bf16x2(e.x, e.y);
-                                dd[ch][2 * gq + rr] = kPartial && !key_real ? 0u : pack_bf16x2(d.x, d.y);
+                                pp[ch][2 * gq + rr] = pack_bf16x2(e.x, e.y);
+                                dd[ch][2 * gq + rr] = pack_bf16x2(d.x, d.y);
                             }
                     }
                     // dV, dK~ of this half's previous unit still read P^T, dS^T; dQ~ of the tile before the previous one
