@@ -103,6 +103,7 @@ struct BwdParams {
     __nv_bfloat16* dv;
     int* status;
     int H, W, heads, M, s, n, nWy, nWx, nblk, items;
+    int d;                     // head width (8, 16, 24, 32): tiles are 32 wide with zeros beyond d, only d channels are stored
     int Hp, Wp;                // sides of the map the windows are laid over (H, W rounded up to multiples of M)
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
     int masked;                // kPartial: shifted windows with a mask (a query sees the keys of its own part of a border window)
@@ -521,8 +522,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             window_order_token(geom, c.wy, c.wx, c.J * kTile + row, i, Y, X);
             const bool row_real = !kPartial || (Y < p.H && X < p.W);      // no dk / dv row for a position beyond the image
             const size_t tok = row_real ? (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h : 0;
-            uint4* dst_v = reinterpret_cast<uint4*>(p.dv + tok * kD);
-            uint4* dst_k = reinterpret_cast<uint4*>(p.dk + tok * kD);
+            uint4* dst_v = reinterpret_cast<uint4*>(p.dv + tok * p.d);
+            uint4* dst_k = reinterpret_cast<uint4*>(p.dk + tok * p.d);
             float* dst_p = p.dkp + (size_t)c.pair * R * p.n + (size_t)c.J * kTile + row;
             constexpr int kParts = 4 + R / 16;
 #pragma unroll
@@ -543,6 +544,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     uint4* dst16 = (part < 2 ? dst_v : dst_k) + 2 * (part & 1);
 #pragma unroll
                     for (int q2 = 0; q2 < 2; ++q2)
+                        if (16 * (part & 1) + 8 * q2 < p.d)       // a head narrower than 32 channels: the rest is padding
                         dst16[q2] = make_uint4(pack_bf16x2(__uint_as_float(a[8 * q2 + 0]) * f, __uint_as_float(a[8 * q2 + 1]) * f),
                                                pack_bf16x2(__uint_as_float(a[8 * q2 + 2]) * f, __uint_as_float(a[8 * q2 + 3]) * f),
                                                pack_bf16x2(__uint_as_float(a[8 * q2 + 4]) * f, __uint_as_float(a[8 * q2 + 5]) * f),
@@ -574,6 +576,7 @@ struct AuxParams {
     float* dpq;
     float* dpk;
     int H, W, heads, M, s, n, nWy, nWx, pairs;
+    int d, r;                    // head width and rank of the caller's tensors (the accumulators are 32 + R columns wide)
     int Hp, Wp;                  // sides of the extended map (equal to H, W when they are multiples of the window)
     int tables;                  // Pq/Pk tables: 1 (shared by the heads) or heads
     long long pos_head_stride;   // elements between the tables in pq, dpq, dpk (pq_scaled is packed: n * 16 apart)
@@ -604,12 +607,19 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     const size_t total = (size_t)p.pairs * p.n;
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+    // staged rows are R wide (zeros from column r on), the caller's tables r wide
     const size_t per_table = (size_t)p.n * R;
     for (size_t e = t; e < per_table * p.tables; e += nthreads) {
-        const size_t user = (e / per_table) * (size_t)p.pos_head_stride + e % per_table;
-        p.pq_scaled[e] = __float2bfloat16_rn(__bfloat162float(p.pq[user]) * p.pos_scale);
-        p.dpq[user] = 0.f;
-        p.dpk[user] = 0.f;
+        const size_t tbl = e / per_table, rem = e % per_table;
+        const int row = (int)(rem / R), col = (int)(rem % R);
+        if (col < p.r) {
+            const size_t user = tbl * (size_t)p.pos_head_stride + (size_t)row * p.r + col;
+            p.pq_scaled[e] = __float2bfloat16_rn(__bfloat162float(p.pq[user]) * p.pos_scale);
+            p.dpq[user] = 0.f;
+            p.dpk[user] = 0.f;
+        } else {
+            p.pq_scaled[e] = __float2bfloat16_rn(0.f);
+        }
     }
     if (t >= total) return;
     float4* z4 = reinterpret_cast<float4*>(p.dq_acc);      // pairs * (d + r) * n floats = total * kDk / 4 vectors
@@ -624,11 +634,12 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
         ldf[2] = 0.f;
         return;
     }
-    const uint4* a = reinterpret_cast<const uint4*>(p.dout + tok * kD);
-    const uint4* b = reinterpret_cast<const uint4*>(p.out + tok * kD);
+    const uint4* a = reinterpret_cast<const uint4*>(p.dout + tok * p.d);
+    const uint4* b = reinterpret_cast<const uint4*>(p.out + tok * p.d);
     float acc = 0.f;
 #pragma unroll
     for (int q4 = 0; q4 < 4; ++q4) {
+        if (8 * q4 >= p.d) break;
         const uint4 x = __ldg(a + q4), y = __ldg(b + q4);
         const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
@@ -681,7 +692,8 @@ __global__ void __launch_bounds__(128, 8) rib_bwd_finish_kernel(const AuxParams 
         const float* src = p.dq_acc + (size_t)pair * kDk * p.n + w;
         const float* srk = p.dkp + (size_t)pair * R * p.n + w;
         float f[8], gq[4], gk[4];
-        if (blockIdx.z == 0 && real) {
+        const bool piece = blockIdx.z == 0 && real && 8 * cg < p.d;      // this thread's 8 content columns exist in the caller's dq
+        if (piece) {
 #pragma unroll
             for (int k = 0; k < 8; ++k) f[k] = src[(size_t)(8 * cg + k) * p.n];
         }
@@ -690,19 +702,20 @@ __global__ void __launch_bounds__(128, 8) rib_bwd_finish_kernel(const AuxParams 
             gq[c] = src[(size_t)(kD + col0 + c) * p.n];
             gk[c] = srk[(size_t)(col0 + c) * p.n];
         }
-        if (blockIdx.z == 0 && real) {
+        if (piece) {
 #pragma unroll
             for (int k = 0; k < 8; ++k) f[k] *= p.inv_sqrt_d;
-            reinterpret_cast<uint4*>(p.dq + tok * kD)[cg] =
+            reinterpret_cast<uint4*>(p.dq + tok * p.d)[cg] =
                 make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) { sq[c] += gq[c]; sk[c] += gk[c]; }
     }
     // (the first pair of a group always exists: the grid is sized by the groups; i is the token's row of the tables)
-    atomicAdd(reinterpret_cast<float4*>(p.dpq + table + (size_t)i * R + col0),
+    if (col0 >= p.r) return;                             // columns of the padding (ranks are multiples of 8)
+    atomicAdd(reinterpret_cast<float4*>(p.dpq + table + (size_t)i * p.r + col0),
               make_float4(sq[0] * p.inv_sqrt_r, sq[1] * p.inv_sqrt_r, sq[2] * p.inv_sqrt_r, sq[3] * p.inv_sqrt_r));
-    atomicAdd(reinterpret_cast<float4*>(p.dpk + table + (size_t)i * R + col0), make_float4(sk[0], sk[1], sk[2], sk[3]));
+    atomicAdd(reinterpret_cast<float4*>(p.dpk + table + (size_t)i * p.r + col0), make_float4(sk[0], sk[1], sk[2], sk[3]));
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -711,7 +724,7 @@ struct WorkspaceLayout { size_t ld, dq_acc, dkp, pq_scaled, total; };
 
 WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
 {
-    const int kR = r, kDk = kD + r;
+    const int kR = padded_rank(r), kDk = kD + kR;      // the accumulators carry the padded rank
     WorkspaceLayout w;
     w.ld = 0;
     w.dq_acc = w.ld + align256((size_t)pairs * n * sizeof(float2));
@@ -725,7 +738,8 @@ WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
 
 bool sm100_bwd_supported(const Problem& p)
 {
-    return p.d == sm100::kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
+    return p.d % 8 == 0 && p.d >= 8 && p.d <= sm100::kD && p.r % 8 == 0 && p.r >= 8 && p.r <= 32 && p.M % 16 == 0 && p.s % 8 == 0 &&
+           p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
 }
 
 size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r) { return workspace_layout(pairs, n, tables, r).total; }
@@ -745,8 +759,8 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
     CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
-        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * R) ||
-        !encode_pos_map_padded(&tm_pk, p.pk, p, tables, p.pos_head_stride))
+        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * R, R) ||
+        !encode_pos_map_padded(&tm_pk, p.pk, p, tables, p.pos_head_stride, p.r))
         return cudaErrorInvalidValue;
     static KernelSetup setup;       // one per instantiation of this launcher, i.e. per kernel
     int sm_count = 0;
@@ -758,6 +772,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     ap.H = p.H; ap.W = p.W; ap.heads = p.heads; ap.M = p.M; ap.s = p.s; ap.n = p.n; ap.nWy = p.nWy; ap.nWx = p.nWx;
     ap.Hp = p.Hp; ap.Wp = p.Wp;
     ap.pairs = p.pairs;
+    ap.d = p.d; ap.r = p.r;
     ap.tables = tables;
     ap.pos_head_stride = p.pos_head_stride;
     ap.pos_scale = sqrtf((float)p.d / (float)p.r);
@@ -777,6 +792,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     bp.items = p.pairs * bp.nblk;
     bp.pos_per_head = tables > 1 ? 1 : 0;
     bp.masked = p.masked ? 1 : 0;
+    bp.d = p.d;
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
@@ -798,8 +814,9 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 {
-    if (p.Hp != p.H || p.Wp != p.W || p.masked) return p.r == 32 ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
-    return p.r == 32 ? launch_bwd<32, false>(p, stream) : launch_bwd<16, false>(p, stream);
+    const bool wide = padded_rank(p.r) == 32;      // accumulators with 32 RIB columns (ranks 24 and 32), else 16 (ranks 8 and 16)
+    if (p.Hp != p.H || p.Wp != p.W || p.masked) return wide ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
+    return wide ? launch_bwd<32, false>(p, stream) : launch_bwd<16, false>(p, stream);
 }
 
 }  // namespace rib

@@ -1,7 +1,10 @@
 // Forward RIB window attention for B200 (sm_100a): tcgen05 MMAs with TMEM accumulators, TMA loads
 // whose box coordinates do the window partition and the cyclic shift, softmax in registers.
 //
-// Shapes: d = 32, r = 16 or 32 (template argument R), window side M a multiple of 16, shift a multiple of 8.
+// Shapes: head width d = 8, 16, 24 or 32 and rank r = 8, 16, 24 or 32, window side M a multiple of 16, shift a multiple
+// of 8.  Tiles are always 32 content columns and R = 16 or 32 RIB columns wide (template argument R = r rounded up):
+// a narrower head or rank is filled up with zeros by the TMA boxes (the channels beyond the tensor), which changes no
+// dot product; the scales use the true d and r and only d output channels are stored.
 // The text below describes R = 16; with R = 32 the RIB rows are 64 bytes like the content rows and take two K16 steps.
 //
 // Work item = one (batch, window, head) pair x two query tiles of 128 tokens.  A persistent CTA
@@ -107,6 +110,7 @@ struct FwdParams {
     float* lse;
     int* status;
     int H, W, heads, M, s, n, nWy, nWx;
+    int d, r;                  // head width (8, 16, 24, 32) and rank (8 .. R in steps of 8): tiles are 32 and R wide, zero beyond d and r
     int Hp, Wp;                // sides of the map the windows are laid over (H, W rounded up to multiples of M)
     int tiles_per_item_pair;   // n / 256: items per pair
     int items;
@@ -319,11 +323,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     int py, px, Y0, X0;
                     patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
                     const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
-                    const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * R);
+                    const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * p.r);
                     constexpr int kChunks = R / 8;                 // 16-byte chunks per row
                     uint4 v[kChunks];
 #pragma unroll
-                    for (int ck = 0; ck < kChunks; ++ck) v[ck] = __ldg(src + ck);
+                    for (int ck = 0; ck < kChunks; ++ck) v[ck] = 8 * ck < p.r ? __ldg(src + ck) : make_uint4(0u, 0u, 0u, 0u);
                     uint32_t* w = reinterpret_cast<uint32_t*>(v);
 #pragma unroll
                     for (int e = 0; e < 4 * kChunks; ++e) {
@@ -516,6 +520,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint4* gsrc = reinterpret_cast<const uint4*>(pend_gate);
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
+                        if (half * 16 + 8 * g >= p.d) break;          // a head narrower than 32 channels: the rest of the row is padding
                         uint32_t w[4];
                         uint4 gv = make_uint4(0u, 0u, 0u, 0u);
                         if (kGated) gv = __ldg(gsrc + g);
@@ -542,8 +547,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
                     const bool no_query = kPartial && (Y0 >= p.H || X0 >= p.W);   // a patch of the extension: no tokens, nothing to store
                     const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
-                    __nv_bfloat16* const out_row = no_query ? nullptr : p.out + tok * kD + half * 16;
-                    const __nv_bfloat16* const gate_row = kGated ? p.gate + tok * kD + half * 16 : nullptr;
+                    __nv_bfloat16* const out_row = no_query ? nullptr : p.out + tok * p.d + half * 16;
+                    const __nv_bfloat16* const gate_row = kGated ? p.gate + tok * p.d + half * 16 : nullptr;
                     float* const lse_row = (p.lse && half == 0 && !no_query) ? p.lse + (((size_t)c.b * p.heads + c.h) * p.H + Y) * p.W + X : nullptr;
                     float m_ref = 0.f;
                     float2 neg2 = make_float2(0.f, 0.f);
@@ -764,10 +769,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int Y = Y0 + ((row >> 3) & 7), X = X0 + (row & 7);   // the patch does not straddle the border
                     if (kPartial && (Y0 >= p.H || X0 >= p.W)) continue;        // a patch of the extension: no tokens, nothing to store
                     const size_t tok = (((size_t)c.b * p.H + Y) * p.W + X) * p.heads + c.h;
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kD + half * 16);
-                    const uint4* gsrc = reinterpret_cast<const uint4*>(p.gate + tok * kD + half * 16);
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * p.d + half * 16);
+                    const uint4* gsrc = reinterpret_cast<const uint4*>(p.gate + tok * p.d + half * 16);
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
+                        if (half * 16 + 8 * g >= p.d) break;          // a head narrower than 32 channels: the rest of the row is padding
                         uint32_t w[4];
                         uint4 gv = make_uint4(0u, 0u, 0u, 0u);
                         if (kGated) gv = __ldg(gsrc + g);
@@ -829,7 +835,7 @@ void tensor_map_cache_counts(long long* hits, long long* misses) { sm100::map_ca
 bool sm100_fwd_supported(const Problem& p)
 {
     const bool partial = p.Hp != p.H || p.Wp != p.W;
-    return p.d == kD && (p.r == 16 || p.r == 32) && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0 &&
+    return p.d % 8 == 0 && p.d >= 8 && p.d <= kD && p.r % 8 == 0 && p.r >= 8 && p.r <= 32 && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0 &&
            !((partial || p.masked) && p.gate);
 }
 
@@ -848,6 +854,7 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     FwdParams fp{};
     fp.pq = p.pq; fp.gate = p.gate; fp.out = p.out_w; fp.lse = p.lse_w; fp.status = p.status;
     fp.H = p.H; fp.W = p.W; fp.heads = p.heads; fp.M = p.M; fp.s = p.s; fp.n = p.n; fp.nWy = p.nWy; fp.nWx = p.nWx;
+    fp.d = p.d; fp.r = p.r;
     fp.Hp = p.Hp; fp.Wp = p.Wp;
     fp.tiles_per_item_pair = p.n / (2 * kTile);
     fp.items = p.pairs * fp.tiles_per_item_pair;
@@ -868,9 +875,10 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
 {
-    if (p.Hp != p.H || p.Wp != p.W || p.masked) return p.r == 32 ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
-    if (p.gate) return p.r == 32 ? launch_fwd<32, false, true>(p, stream) : launch_fwd<16, false, true>(p, stream);
-    return p.r == 32 ? launch_fwd<32, false, false>(p, stream) : launch_fwd<16, false, false>(p, stream);
+    const bool wide = padded_rank(p.r) == 32;      // RIB rows of 32 elements (ranks 24 and 32), else of 16 (ranks 8 and 16)
+    if (p.Hp != p.H || p.Wp != p.W || p.masked) return wide ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
+    if (p.gate) return wide ? launch_fwd<32, false, true>(p, stream) : launch_fwd<16, false, true>(p, stream);
+    return wide ? launch_fwd<32, false, false>(p, stream) : launch_fwd<16, false, false>(p, stream);
 }
 
 }  // namespace rib

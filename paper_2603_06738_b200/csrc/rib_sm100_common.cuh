@@ -141,11 +141,13 @@ inline void map_cache_counts(long long* hits, long long* misses)
     *hits = c.hits; *misses = c.misses;
 }
 
-// bf16 [B][H][W][heads][32] image tensor, box = one 8x8-token patch of one head.
+// bf16 [B][H][W][heads][d] image tensor (d = 8, 16, 24 or 32), box = one 8x8-token patch of one head, always 32 channels
+// wide: on a narrower head the channels from d on lie beyond the tensor and arrive as zeros, so a tile has one layout
+// for every head width and the zero channels change no dot product.
 inline bool encode_image_map_now(CUtensorMap* map, const void* ptr, const Problem& p)
 {
-    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)p.heads, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
-    const cuuint64_t row = (cuuint64_t)kD * 2;
+    const cuuint64_t dims[5] = {(cuuint64_t)p.d, (cuuint64_t)p.heads, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.B};
+    const cuuint64_t row = (cuuint64_t)p.d * 2;
     const cuuint64_t strides[4] = {row, row * p.heads, row * p.heads * p.W, row * p.heads * p.W * p.H};
     const cuuint32_t box[5] = {(cuuint32_t)kD, 1, 8, 8, 1};
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -159,16 +161,16 @@ inline bool encode_image_map_now(CUtensorMap* map, const void* ptr, const Proble
 // at least M * M * 16); a kernel addresses table h * (tables > 1).
 inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p)
 {
-    const MapKey key{ptr, 0, 0, 1, p.B, p.H, p.W, p.heads, 0};
+    const MapKey key{ptr, 0, 0, 1, p.B, p.H, p.W, p.heads, p.d};
     return cached_map(map, key, [&](CUtensorMap* m) { return encode_image_map_now(m, ptr, p); });
 }
 
 inline bool encode_pos_map_now(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
-                               cuuint32_t box_inner, CUtensorMapSwizzle swz)
+                               cuuint32_t box_inner, CUtensorMapSwizzle swz, int cols)
 {
-    const cuuint64_t dims[4] = {(cuuint64_t)p.r, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
-    const cuuint64_t one_table = (cuuint64_t)p.r * 2 * p.M * p.M;
-    const cuuint64_t strides[3] = {(cuuint64_t)p.r * 2, (cuuint64_t)p.r * 2 * p.M,
+    const cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
+    const cuuint64_t one_table = (cuuint64_t)cols * 2 * p.M * p.M;
+    const cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * p.M,
                                    tables > 1 ? (cuuint64_t)table_stride * 2 : one_table};
     const cuuint32_t box[4] = {box_inner, 8, 8, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -176,22 +178,26 @@ inline bool encode_pos_map_now(CUtensorMap* map, const void* ptr, const Problem&
                        CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+// `cols`: elements per row of the table in memory (the rank, or the padded rank of a table staged by the library)
 inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
-                                cuuint32_t box_inner, CUtensorMapSwizzle swz)
+                                cuuint32_t box_inner, CUtensorMapSwizzle swz, int cols)
 {
-    const MapKey key{ptr, table_stride, 0, 2, p.r, p.M, tables, (int)box_inner, (int)swz};
-    return cached_map(map, key, [&](CUtensorMap* m) { return encode_pos_map_now(m, ptr, p, tables, table_stride, box_inner, swz); });
+    const MapKey key{ptr, table_stride, 0, 2, cols, p.M, tables, (int)box_inner, (int)swz};
+    return cached_map(map, key, [&](CUtensorMap* m) { return encode_pos_map_now(m, ptr, p, tables, table_stride, box_inner, swz, cols); });
 }
+// Rows of 16 (r <= 16) or 32 (r <= 32) elements: a rank below the row width is filled up with zeros by TMA.
+inline int padded_rank(int r) { return r > 16 ? 32 : 16; }
 inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
 {
-    return encode_pos_map_impl(map, ptr, p, tables, table_stride, (cuuint32_t)p.r, p.r == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    const bool wide = padded_rank(p.r) == 32;
+    return encode_pos_map_impl(map, ptr, p, tables, table_stride, wide ? 32u : 16u, wide ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B, p.r);
 }
 // The same features fetched as 64-byte rows: the box is 32 elements wide on a 16-element dimension, so
 // TMA fills the upper half of every row with zeros.  A 64-byte-row RIB tile has the layout of a content
 // tile (SWIZZLE_64B) and can sit behind it as the second 32-column atom of one MN-major operand.
-inline bool encode_pos_map_padded(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
+inline bool encode_pos_map_padded(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride, int cols)
 {
-    return encode_pos_map_impl(map, ptr, p, tables, table_stride, kD, CU_TENSOR_MAP_SWIZZLE_64B);
+    return encode_pos_map_impl(map, ptr, p, tables, table_stride, kD, CU_TENSOR_MAP_SWIZZLE_64B, cols);
 }
 
 inline cudaError_t sm_count_of_current_device(int* count)

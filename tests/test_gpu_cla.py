@@ -55,7 +55,8 @@ def test_gate_border_pixels_see_zero_padding():
 @pytest.mark.parametrize("wl", [Workload("gated_w16_s8", 2, 32, 48, 2, 32, 16, 16, 8, seed=210),
                                 Workload("gated_w32_rank32", 1, 64, 32, 6, 32, 32, 32, 16, seed=211),
                                 Workload("gated_w8_generic", 1, 16, 24, 3, 16, 8, 8, 3, seed=212),
-                                Workload("gated_w16_headwise", 1, 32, 32, 3, 32, 16, 16, 0, seed=215, headwise=True)], ids=lambda w: w.name)
+                                Workload("gated_w16_headwise", 1, 32, 32, 3, 32, 16, 16, 0, seed=215, headwise=True),
+                                Workload("gated_w16_d16_r24", 1, 32, 32, 4, 16, 24, 16, 8, seed=216)], ids=lambda w: w.name)
 def test_gated_forward_is_attention_times_the_gate(wl, path):
     cpu, gpu = make(wl, with_dout=False)
     D = wl.heads * wl.d
@@ -68,7 +69,7 @@ def test_gated_forward_is_attention_times_the_gate(wl, path):
         binding.rib_set_path(binding.RIB_PATH_NONE)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
-    fast = path == "auto" and wl.d == 32 and wl.window % 16 == 0 and wl.shift % 8 == 0
+    fast = path == "auto" and wl.d % 8 == 0 and wl.d <= 32 and wl.window % 16 == 0 and wl.shift % 8 == 0
     assert used == (binding.RIB_PATH_SM100 if fast else binding.RIB_PATH_GENERIC)
     ref_out, ref_lse = oracle_fwd(cpu, wl)
     compare("out", to_f64(out), cla.gated_output(ref_out, to_f64(gate)))

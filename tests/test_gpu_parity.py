@@ -32,7 +32,13 @@ SMALL = [
     Workload("sst_d30_r34_w32", 1, 32, 64, 3, 30, 34, 32, 16, seed=25),
     Workload("light_d16_r24_w16", 2, 32, 32, 3, 16, 24, 16, 8, seed=26),       # d + r = 40: not a multiple of 16
     Workload("odd_d15_r7_w8", 1, 16, 16, 2, 15, 7, 8, 3, seed=27),
+    # head widths and ranks that are multiples of 8: 32-wide tiles filled up with zeros by the TMA boxes (tcgen05 kernels)
+    Workload("d16_r16_w32_s16", 1, 64, 32, 3, 16, 16, 32, 16, seed=28),
+    Workload("d24_r8_w16_s8", 2, 32, 48, 2, 24, 8, 16, 8, seed=29),
+    Workload("d8_r32_w16", 1, 32, 32, 2, 8, 32, 16, 0, seed=30),
+    Workload("d16_r24_w32_headwise", 1, 32, 64, 3, 16, 24, 32, 8, seed=31, headwise=True),
 ]
+NARROW = [wl for wl in SMALL if wl.name in ("light_d16_r24_w16", "d16_r16_w32_s16", "d24_r8_w16_s8", "d8_r32_w16", "d16_r24_w32_headwise")]
 
 
 def _inputs_for(wl):
@@ -67,6 +73,16 @@ def test_small_forward_and_backward_every_element(wl, path):
     if wl.r:
         compare("dpq", to_f64(dpq), rdpq)
         compare("dpk", to_f64(dpk), rdpk)
+
+
+@pytest.mark.parametrize("wl", NARROW, ids=lambda w: w.name)
+def test_narrow_heads_and_ranks_take_the_tcgen05_kernels(wl):
+    """d = 8, 16, 24 and r = 8, 16, 24, 32 run on the tensor-core kernels (the parity of these shapes is checked above)."""
+    _, gpu = _inputs_for(wl)
+    out, lse = run_fwd(gpu, wl)
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
+    run_bwd(gpu, wl, out, lse)
+    assert binding.rib_last_path() == binding.RIB_PATH_SM100
 
 
 def test_lse_is_optional_and_outputs_are_fully_written():
