@@ -463,6 +463,19 @@ def main():
                 bf = wl.pairs * 2 * wl.n * wl.n * (5 * wl.d + 3 * r_v)
                 variants[name] = {"r": r_v, "fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_tflops": ff / (f_ms * 1e-3) / 1e12,
                                   "bwd_tflops": bf / (b_ms * 1e-3) / 1e12, "paths": [binding.rib_last_path()]}
+            # the light-weight rows of the paper's network table: 16-channel heads with rank 24 (same map, twice the heads)
+            hq, hk, hv, hdo = (torch.randn((wl.B, wl.H, wl.W, 2 * wl.heads, 16), device=dev).to(torch.bfloat16) for _ in range(4))
+            hpq, hpk = ((0.5 * torch.randn((wl.n, 24), device=dev)).to(torch.bfloat16) for _ in range(2))
+            out_h, lse_h = binding.rib_window_attn_fwd(hq, hk, hv, hpq, hpk, wl.window, wl.shift)
+            f_ms = timed(lambda: binding.rib_window_attn_fwd(hq, hk, hv, hpq, hpk, wl.window, wl.shift))
+            b_ms = timed(lambda: binding.rib_window_attn_bwd(hq, hk, hv, hpq, hpk, out_h, lse_h, hdo, wl.window, wl.shift))
+            hp = 2 * wl.pairs
+            variants["d16_r24"] = {"heads": 2 * wl.heads, "d": 16, "r": 24, "fwd_ms": f_ms, "bwd_ms": b_ms,
+                                   "fwd_tflops": hp * 2 * wl.n * wl.n * (2 * 16 + 24) / (f_ms * 1e-3) / 1e12,
+                                   "bwd_tflops": hp * 2 * wl.n * wl.n * (5 * 16 + 3 * 24) / (b_ms * 1e-3) / 1e12,
+                                   "paths": [binding.rib_last_path()],
+                                   "note": "tiles are 32 + 32 columns wide on the tensor cores, zeros beyond d and r: the useful flops counted here are 58 % of those issued"}
+            del hq, hk, hv, hdo, out_h, lse_h
             # shifted windows with a region mask (the wrapped parts of a border window do not attend to each other)
             out_m, lse_m = binding.rib_window_attn_fwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], wl.window, wl.shift)
             f_ms = timed(lambda: binding.rib_window_attn_fwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], wl.window, wl.shift))
