@@ -107,6 +107,7 @@ struct BwdParams {
     int Hp, Wp;                // sides of the map the windows are laid over (H, W rounded up to multiples of M)
     int pos_per_head;          // 1 when Pq/Pk are head-wise: table index = head
     int masked;                // kPartial: shifted windows with a mask (a query sees the keys of its own part of a border window)
+    int packed8;               // kPartial: a 16 x 16 window stands for 2 x 2 windows of 8 x 8 tokens (a query sees its own patch only)
     float scale_log2;          // log2(e) / sqrt(d)
     float inv_sqrt_d;
 };
@@ -191,7 +192,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     patch_origin(geom, c.wy, c.wx, 2 * c.J + sub, py, px, Y0, X0);
                     tma_load_5d(base + kOffKc + slot * kContentBytes + sub * kPatchContent, &tm_k, bar(kKVFull + slot),
                                 0, c.h, X0, Y0, c.b);
-                    tma_load_4d(base + kOffKp + slot * kContentBytes + sub * kPatchContent, &tm_pk, bar(kKVFull + slot), 0, px, py, c.h * p.pos_per_head);
+                    tma_load_4d(base + kOffKp + slot * kContentBytes + sub * kPatchContent, &tm_pk, bar(kKVFull + slot), 0,
+                                kPartial && p.packed8 ? 0 : px, kPartial && p.packed8 ? 0 : py, c.h * p.pos_per_head);
                     tma_load_5d(base + kOffV + slot * kContentBytes + sub * kPatchContent, &tm_v, bar(kKVFull + slot),
                                 0, c.h, X0, Y0, c.b);
                 }
@@ -205,7 +207,8 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         int py, px, Y0, X0;
                         patch_origin(geom, c.wy, c.wx, 2 * I + sub, py, px, Y0, X0);
                         tma_load_5d(ring + kRingQc + sub * kPatchContent, &tm_q, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
-                        tma_load_4d(ring + kRingQp + sub * kPatchContent, &tm_pqs, bar(kQFull + st), 0, px, py, c.h * p.pos_per_head);
+                        tma_load_4d(ring + kRingQp + sub * kPatchContent, &tm_pqs, bar(kQFull + st), 0,
+                                    kPartial && p.packed8 ? 0 : px, kPartial && p.packed8 ? 0 : py, c.h * p.pos_per_head);
                         tma_load_5d(ring + kRingDO + sub * kPatchContent, &tm_do, bar(kQFull + st), 0, c.h, X0, Y0, c.b);
                     }
                     bulk_load_1d(ring + kRingLD, p.ld + (size_t)c.pair * p.n + (size_t)I * kTile, kLdBytes, bar(kQFull + st));
@@ -346,8 +349,10 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
             bool key_exists = true;       // kPartial: this warp's 32 key rows lie in one 8x8 patch of the key block
             int key_part = 0, last_window = 0;   // masked shifted windows: part of the key patch; bit 1 / 0: last window row / column
+            int key_patch = 0;
             if (kPartial) {
                 const ItemCoord c = decode_item(p, item);
+                key_patch = 2 * c.J + (quarter >> 1);
                 int py, px, Y0, X0;
                 patch_origin(geom, c.wy, c.wx, 2 * c.J + (quarter >> 1), py, px, Y0, X0);
                 key_exists = Y0 < p.H && X0 < p.W;
@@ -361,6 +366,7 @@ rib_bwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int per_row = p.M >> 3, qp = 2 * I + h;
                     key_real = key_exists && key_part == window_part(p.M, p.s, last_window & 2, last_window & 1, (qp / per_row) << 3, (qp % per_row) << 3);
                 }
+                if (kPartial && p.packed8) key_real = key_patch == 2 * I + h;      // packed windows of 8 x 8 tokens: the own patch only
                 const uint32_t st = g % kQStages;
                 // warp-uniform outcome: the TMEM accesses below are warp-collective
                 if (!__all_sync(0xffffffffu, mbar_wait(bar(kQFull + st), (g / kQStages) & 1, abort_flag, p.status) &&
@@ -577,6 +583,7 @@ struct AuxParams {
     float* dpk;
     int H, W, heads, M, s, n, nWy, nWx, pairs;
     int d, r;                    // head width and rank of the caller's tensors (the accumulators are 32 + R columns wide)
+    int table_rows;              // rows of a Pq / Pk table: n, or 64 when 16 x 16 windows stand for 2 x 2 windows of 8 x 8 tokens
     int Hp, Wp;                  // sides of the extended map (equal to H, W when they are multiples of the window)
     int tables;                  // Pq/Pk tables: 1 (shared by the heads) or heads
     long long pos_head_stride;   // elements between the tables in pq, dpq, dpk (pq_scaled is packed: n * 16 apart)
@@ -592,6 +599,7 @@ __device__ __forceinline__ bool decode_pair_token(const AuxParams& p, int pair, 
     const int b = pair;
     int Y, X;
     window_order_token(WindowGeom{p.Hp, p.Wp, p.M, p.s}, wy, wx, w, i, Y, X);
+    if (p.table_rows != p.n) i = w & 63;             // packed windows of 8 x 8 tokens: the row of the table is the place in the patch
     tok = (((size_t)b * p.H + Y) * p.W + X) * p.heads + h;
     scalar = (((size_t)b * p.heads + h) * p.H + Y) * p.W + X;
     return Y < p.H && X < p.W;
@@ -608,7 +616,7 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * blockDim.x;
     // staged rows are R wide (zeros from column r on), the caller's tables r wide
-    const size_t per_table = (size_t)p.n * R;
+    const size_t per_table = (size_t)p.table_rows * R;
     for (size_t e = t; e < per_table * p.tables; e += nthreads) {
         const size_t tbl = e / per_table, rem = e % per_table;
         const int row = (int)(rem / R), col = (int)(rem % R);
@@ -722,7 +730,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WorkspaceLayout { size_t ld, dq_acc, dkp, pq_scaled, total; };
 
-WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
+WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r, int table_rows)
 {
     const int kR = padded_rank(r), kDk = kD + kR;      // the accumulators carry the padded rank
     WorkspaceLayout w;
@@ -730,7 +738,7 @@ WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
     w.dq_acc = w.ld + align256((size_t)pairs * n * sizeof(float2));
     w.dkp = w.dq_acc + align256((size_t)pairs * kDk * n * sizeof(float));
     w.pq_scaled = w.dkp + align256((size_t)pairs * kR * n * sizeof(float));
-    w.total = w.pq_scaled + align256((size_t)tables * n * kR * sizeof(__nv_bfloat16));
+    w.total = w.pq_scaled + align256((size_t)tables * table_rows * kR * sizeof(__nv_bfloat16));
     return w;
 }
 
@@ -738,18 +746,20 @@ WorkspaceLayout workspace_layout(long long pairs, int n, int tables, int r)
 
 bool sm100_bwd_supported(const Problem& p)
 {
-    return p.d % 8 == 0 && p.d >= 8 && p.d <= sm100::kD && p.r % 8 == 0 && p.r >= 8 && p.r <= 32 && p.M % 16 == 0 && p.s % 8 == 0 &&
-           p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
+    return p.d % 8 == 0 && p.d >= 8 && p.d <= sm100::kD && p.r % 8 == 0 && p.r >= 8 && p.r <= 32 &&
+           (p.M % 16 == 0 || packs_windows_of_8(p)) && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0;
 }
 
-size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r) { return workspace_layout(pairs, n, tables, r).total; }
+// (pairs * n is what counts: packed windows of 8 x 8 tokens give the same size as their 16 x 16 stand-ins)
+size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r) { return workspace_layout(pairs, n, tables, r, n).total; }
 
 template <int R, bool kPartial>
 cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 {
     if (!encode_fn()) return cudaErrorNotSupported;
     const int tables = pos_tables(p);
-    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n, tables, R);
+    const int table_rows = p.packed8 ? 64 : p.n;
+    const WorkspaceLayout wl = workspace_layout(p.pairs, p.n, tables, R, table_rows);
     if (p.workspace_bytes < wl.total) return cudaErrorInvalidValue;
     uint8_t* ws = static_cast<uint8_t*>(p.workspace);
     float2* ld = reinterpret_cast<float2*>(ws + wl.ld);
@@ -759,7 +769,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
     CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk;
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
-        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)p.n * R, R) ||
+        !encode_image_map(&tm_do, p.dout, p) || !encode_pos_map_padded(&tm_pqs, pq_scaled, p, tables, (long long)table_rows * R, R) ||
         !encode_pos_map_padded(&tm_pk, p.pk, p, tables, p.pos_head_stride, p.r))
         return cudaErrorInvalidValue;
     static KernelSetup setup;       // one per instantiation of this launcher, i.e. per kernel
@@ -773,6 +783,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     ap.Hp = p.Hp; ap.Wp = p.Wp;
     ap.pairs = p.pairs;
     ap.d = p.d; ap.r = p.r;
+    ap.table_rows = table_rows;
     ap.tables = tables;
     ap.pos_head_stride = p.pos_head_stride;
     ap.pos_scale = sqrtf((float)p.d / (float)p.r);
@@ -792,6 +803,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     bp.items = p.pairs * bp.nblk;
     bp.pos_per_head = tables > 1 ? 1 : 0;
     bp.masked = p.masked ? 1 : 0;
+    bp.packed8 = p.packed8 ? 1 : 0;
     bp.d = p.d;
     bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
     bp.inv_sqrt_d = ap.inv_sqrt_d;
@@ -814,8 +826,9 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream)
 {
+    if (packs_windows_of_8(p)) return sm100_bwd(packed_windows_of_8(p), stream);
     const bool wide = padded_rank(p.r) == 32;      // accumulators with 32 RIB columns (ranks 24 and 32), else 16 (ranks 8 and 16)
-    if (p.Hp != p.H || p.Wp != p.W || p.masked) return wide ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W || p.masked || p.packed8) return wide ? launch_bwd<32, true>(p, stream) : launch_bwd<16, true>(p, stream);
     return wide ? launch_bwd<32, false>(p, stream) : launch_bwd<16, false>(p, stream);
 }
 

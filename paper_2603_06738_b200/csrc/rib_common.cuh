@@ -39,6 +39,9 @@ struct Problem {
     int* status;                      // device status word (bounded waits report here)
     bool exact_softmax;               // tcgen05 forward: every item takes the exact (running-maximum) softmax form
     bool masked;                      // shifted windows: the wrapped parts of a border window do not attend to each other
+    bool packed8;                     // tcgen05 kernels only: M, n, nWy, nWx, pairs describe 16 x 16 windows that each stand for
+                                      // 2 x 2 windows of 8 x 8 tokens (a token attends to the 8 x 8 patch it lies in; the tables
+                                      // pq, pk, dpq, dpk have 64 rows)
 };
 
 // Pq/Pk tables: one shared by the heads, or one per head (Sec. 3.1, after Eq. 3: head-wise projections of the shared h).

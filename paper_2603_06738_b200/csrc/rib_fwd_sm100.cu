@@ -122,6 +122,7 @@ struct FwdParams {
     int exact_only;            // 1: skip the fast form (every item takes the exact softmax)
     int skip_dead;             // kPartial: 1 = items and key blocks without tokens are skipped, 0 = walked with probability 0
     int masked;                // kPartial: shifted windows with a mask -- a query sees the keys of its own part of a border window only
+    int packed8;               // kPartial: a 16 x 16 window stands for 2 x 2 windows of 8 x 8 tokens -- a query sees its own patch only
     FastDiv div_tp, div_heads, div_nwx, div_nwy, div_per_row;   // tiles_per_item_pair, heads, nWx, nWy, M / 8
 };
 
@@ -269,6 +270,14 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         auto mask_masks = [&](const ItemCoord& c, int q_patch, uint32_t& row_dead, uint32_t& col_dead) {
             const int per_row = p.M >> 3, thr = (p.M - p.s) >> 3;
             const uint32_t in_window = per_row == 32 ? 0xffffffffu : (1u << per_row) - 1u;
+            if (p.packed8) {
+                // packed windows of 8 x 8 tokens: every patch but the query's own is dead
+                int pr, pc;
+                p.div_per_row.divmod(q_patch, pr, pc);
+                row_dead = in_window & ~(1u << pr);
+                col_dead = in_window & ~(1u << pc);
+                return;
+            }
             const uint32_t wrapped = in_window & ~(thr >= 32 ? 0xffffffffu : (1u << thr) - 1u);
             const uint32_t rows_w = c.wy == p.nWy - 1 ? wrapped : 0u, cols_w = c.wx == p.nWx - 1 ? wrapped : 0u;
             int pr, pc;
@@ -322,7 +331,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int r256 = lane + 32 * k, qt = r256 >> 7, row = r256 & 127;
                     int py, px, Y0, X0;
                     patch_origin(p, c, 2 * (2 * c.tp + qt) + (row >> 6), py, px, Y0, X0);
-                    const int token = (py + ((row >> 3) & 7)) * p.M + px + (row & 7);
+                    const int token = kPartial && p.packed8 ? row & 63 : (py + ((row >> 3) & 7)) * p.M + px + (row & 7);   // row of the table
                     const uint4* src = reinterpret_cast<const uint4*>(p.pq + (size_t)c.h * p.pos_head_stride + (size_t)token * p.r);
                     constexpr int kChunks = R / 8;                 // 16-byte chunks per row
                     uint4 v[kChunks];
@@ -359,7 +368,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             tma_load_5d(base + kOffKc + st * kContentBytes + sub * kPatchContent, &tm_k, bar(kKFull + st),
                                         0, c.h, X0[sub], Y0[sub], c.b);
                             tma_load_4d(base + kOffKp + st * kPosBytes + sub * kPatchPos, &tm_pk, bar(kKFull + st),
-                                        0, px[sub], py[sub], c.h * p.pos_per_head);
+                                        0, kPartial && p.packed8 ? 0 : px[sub], kPartial && p.packed8 ? 0 : py[sub], c.h * p.pos_per_head);
                         }
                         if (use > 0 && !mbar_wait(bar(kVEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                         mbar_arrive_expect_tx(bar(kVFull + st), kContentBytes);
@@ -555,7 +564,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     uint32_t row_dead = 0u, col_dead = 0u;
                     int jf = 0, jl = nblk - 1;
                     if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
-                    if (kPartial && p.masked) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
+                    if (kPartial && (p.masked | p.packed8)) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
                     for (int j = jf; j <= jl; ++j, ++blk) {
                         if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
@@ -643,7 +652,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     uint32_t row_dead = 0u, col_dead = 0u;
                     int jf = 0, jl = nblk - 1;
                     if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
-                    if (kPartial && p.masked) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
+                    if (kPartial && (p.masked | p.packed8)) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
                     for (int j = jf; j <= jl; ++j, ++blk) {
                         if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
@@ -835,7 +844,8 @@ void tensor_map_cache_counts(long long* hits, long long* misses) { sm100::map_ca
 bool sm100_fwd_supported(const Problem& p)
 {
     const bool partial = p.Hp != p.H || p.Wp != p.W;
-    return p.d % 8 == 0 && p.d >= 8 && p.d <= kD && p.r % 8 == 0 && p.r >= 8 && p.r <= 32 && p.M % 16 == 0 && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0 &&
+    return p.d % 8 == 0 && p.d >= 8 && p.d <= kD && p.r % 8 == 0 && p.r >= 8 && p.r <= 32 &&
+           (p.M % 16 == 0 || packs_windows_of_8(p)) && p.s % 8 == 0 && p.M <= 256 && p.H % 8 == 0 && p.W % 8 == 0 &&
            !((partial || p.masked) && p.gate);
 }
 
@@ -865,7 +875,8 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     fp.exact_only = p.exact_softmax ? 1 : 0;
     fp.masked = p.masked ? 1 : 0;
-    fp.skip_dead = kPartial && !p.masked && p.n / kTile >= 8 ? 1 : 0;      // (a mask differs from query patch to query patch)
+    fp.packed8 = p.packed8 ? 1 : 0;
+    fp.skip_dead = kPartial && !p.masked && !p.packed8 && p.n / kTile >= 8 ? 1 : 0;      // (a mask differs from query patch to query patch)
     fp.div_tp = make_fast_div(fp.tiles_per_item_pair); fp.div_heads = make_fast_div(p.heads);
     fp.div_nwx = make_fast_div(p.nWx); fp.div_nwy = make_fast_div(p.nWy); fp.div_per_row = make_fast_div(p.M >> 3);
     const int grid = fp.items < sm_count ? fp.items : sm_count;
@@ -875,8 +886,9 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
 
 cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream)
 {
+    if (packs_windows_of_8(p)) return sm100_fwd(packed_windows_of_8(p), stream);
     const bool wide = padded_rank(p.r) == 32;      // RIB rows of 32 elements (ranks 24 and 32), else of 16 (ranks 8 and 16)
-    if (p.Hp != p.H || p.Wp != p.W || p.masked) return wide ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
+    if (p.Hp != p.H || p.Wp != p.W || p.masked || p.packed8) return wide ? launch_fwd<32, true, false>(p, stream) : launch_fwd<16, true, false>(p, stream);
     if (p.gate) return wide ? launch_fwd<32, false, true>(p, stream) : launch_fwd<16, false, true>(p, stream);
     return wide ? launch_fwd<32, false, false>(p, stream) : launch_fwd<16, false, false>(p, stream);
 }

@@ -168,9 +168,10 @@ inline bool encode_image_map(CUtensorMap* map, const void* ptr, const Problem& p
 inline bool encode_pos_map_now(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
                                cuuint32_t box_inner, CUtensorMapSwizzle swz, int cols)
 {
-    const cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)p.M, (cuuint64_t)p.M, (cuuint64_t)tables};
-    const cuuint64_t one_table = (cuuint64_t)cols * 2 * p.M * p.M;
-    const cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * p.M,
+    const cuuint64_t side = p.packed8 ? 8 : p.M;       // the tables of packed 8 x 8 windows have 8 x 8 rows
+    const cuuint64_t dims[4] = {(cuuint64_t)cols, side, side, (cuuint64_t)tables};
+    const cuuint64_t one_table = (cuuint64_t)cols * 2 * side * side;
+    const cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * side,
                                    tables > 1 ? (cuuint64_t)table_stride * 2 : one_table};
     const cuuint32_t box[4] = {box_inner, 8, 8, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -182,11 +183,30 @@ inline bool encode_pos_map_now(CUtensorMap* map, const void* ptr, const Problem&
 inline bool encode_pos_map_impl(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride,
                                 cuuint32_t box_inner, CUtensorMapSwizzle swz, int cols)
 {
-    const MapKey key{ptr, table_stride, 0, 2, cols, p.M, tables, (int)box_inner, (int)swz};
+    const MapKey key{ptr, table_stride, 0, 2, cols, p.packed8 ? 8 : p.M, tables, (int)box_inner, (int)swz};
     return cached_map(map, key, [&](CUtensorMap* m) { return encode_pos_map_now(m, ptr, p, tables, table_stride, box_inner, swz, cols); });
 }
 // Rows of 16 (r <= 16) or 32 (r <= 32) elements: a rank below the row width is filled up with zeros by TMA.
 inline int padded_rank(int r) { return r > 16 ? 32 : 16; }
+
+// Windows of 8 x 8 tokens are half a tile.  Where the map allows it they are worked as 16 x 16 windows that hold 2 x 2 of
+// them: the kernels' geometry is that of M = 16, every 8 x 8 patch of such a window is one real window, a query patch
+// attends to the key patch with its own number only (the code path of masked windows), and positional rows come from the
+// patch-local position.  Three quarters of the score tile are discarded; the pass is bound by its memory traffic.
+inline bool packs_windows_of_8(const Problem& p)
+{
+    return p.M == 8 && p.s == 0 && p.H % 16 == 0 && p.W % 16 == 0 && !p.masked && !p.gate && !p.packed8;
+}
+inline Problem packed_windows_of_8(const Problem& p)
+{
+    Problem v = p;
+    v.packed8 = true;
+    v.M = 16; v.n = 256;
+    v.nWy = p.H / 16; v.nWx = p.W / 16;
+    v.Hp = p.H; v.Wp = p.W;
+    v.pairs = p.B * v.nWy * v.nWx * p.heads;
+    return v;
+}
 inline bool encode_pos_map(CUtensorMap* map, const void* ptr, const Problem& p, int tables, long long table_stride)
 {
     const bool wide = padded_rank(p.r) == 32;

@@ -37,8 +37,14 @@ SMALL = [
     Workload("d24_r8_w16_s8", 2, 32, 48, 2, 24, 8, 16, 8, seed=29),
     Workload("d8_r32_w16", 1, 32, 32, 2, 8, 32, 16, 0, seed=30),
     Workload("d16_r24_w32_headwise", 1, 32, 64, 3, 16, 24, 32, 8, seed=31, headwise=True),
+    # windows of 8 x 8 tokens (half a tile): worked as 16 x 16 windows that hold 2 x 2 of them on the tcgen05 kernels
+    Workload("w8_packed", 2, 32, 48, 3, 32, 16, 8, 0, seed=32),
+    Workload("w8_packed_rank32_headwise", 1, 16, 32, 2, 32, 32, 8, 0, seed=33, headwise=True),
+    Workload("w8_packed_d16_r24", 1, 32, 32, 4, 16, 24, 8, 0, seed=34),
+    Workload("w8_rows_24", 1, 24, 32, 2, 32, 16, 8, 0, seed=35),               # 24 rows: not a multiple of 16, any-shape kernels
 ]
-NARROW = [wl for wl in SMALL if wl.name in ("light_d16_r24_w16", "d16_r16_w32_s16", "d24_r8_w16_s8", "d8_r32_w16", "d16_r24_w32_headwise")]
+NARROW = [wl for wl in SMALL if wl.name in ("light_d16_r24_w16", "d16_r16_w32_s16", "d24_r8_w16_s8", "d8_r32_w16", "d16_r24_w32_headwise",
+                                             "w8_packed", "w8_packed_rank32_headwise", "w8_packed_d16_r24")]
 
 
 def _inputs_for(wl):
@@ -67,17 +73,24 @@ def test_small_forward_and_backward_every_element(wl, path):
     compare("out", to_f64(out), ref_out)
     compare("lse", to_f64(lse), ref_lse)
     rdq, rdk, rdv, rdpq, rdpk = oracle_bwd(cpu, wl)
-    compare("dq", to_f64(dq), rdq)
-    compare("dk", to_f64(dk), rdk)
+    # A window of 64 tokens averages over few keys: gradients reach 2 in size where those of the benchmark windows stay
+    # below 1.3, and a bf16 result of that size is spaced 2^-7 apart.  The absolute bound follows the size of the
+    # reference there; the relative-L2 bound is the same everywhere.
+    grad_abs = 1e-2 * max(1.0, float(np.abs(rdq).max()), float(np.abs(rdk).max())) if wl.window == 8 else 1e-2
+    compare("dq", to_f64(dq), rdq, max_abs=grad_abs)
+    compare("dk", to_f64(dk), rdk, max_abs=grad_abs)
     compare("dv", to_f64(dv), rdv)
     if wl.r:
-        compare("dpq", to_f64(dpq), rdpq)
-        compare("dpk", to_f64(dpk), rdpk)
+        # sums over every pair of the batch: bounded relative to the largest entry, as in the full-size tests
+        scale = max(1.0, float(np.abs(rdpq).max()), float(np.abs(rdpk).max()))
+        compare("dpq", to_f64(dpq), rdpq, max_abs=1e-2 * scale)
+        compare("dpk", to_f64(dpk), rdpk, max_abs=1e-2 * scale)
 
 
 @pytest.mark.parametrize("wl", NARROW, ids=lambda w: w.name)
 def test_narrow_heads_and_ranks_take_the_tcgen05_kernels(wl):
-    """d = 8, 16, 24 and r = 8, 16, 24, 32 run on the tensor-core kernels (the parity of these shapes is checked above)."""
+    """d = 8, 16, 24, r = 8, 16, 24, 32 and windows of 8 x 8 tokens run on the tensor-core kernels (the parity of these
+    shapes is checked above)."""
     _, gpu = _inputs_for(wl)
     out, lse = run_fwd(gpu, wl)
     assert binding.rib_last_path() == binding.RIB_PATH_SM100
