@@ -476,6 +476,17 @@ def main():
                                    "paths": [binding.rib_last_path()],
                                    "note": "tiles are 32 + 32 columns wide on the tensor cores, zeros beyond d and r: the useful flops counted here are 58 % of those issued"}
             del hq, hk, hv, hdo, out_h, lse_h
+            # windows of 8 x 8 tokens on the same map (memory-bound: 4 x 64 B read and 64 B written per token-head in the forward)
+            w8pq, w8pk = ((0.5 * torch.randn((64, wl.r), device=dev)).to(torch.bfloat16) for _ in range(2))
+            out_8, lse_8 = binding.rib_window_attn_fwd(s0["q"], s0["k"], s0["v"], w8pq, w8pk, 8, 0)
+            f_ms = timed(lambda: binding.rib_window_attn_fwd(s0["q"], s0["k"], s0["v"], w8pq, w8pk, 8, 0))
+            b_ms = timed(lambda: binding.rib_window_attn_bwd(s0["q"], s0["k"], s0["v"], w8pq, w8pk, out_8, lse_8, s0["dout"], 8, 0))
+            th = wl.B * wl.H * wl.W * wl.heads
+            variants["window8"] = {"fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_gbs": th * 256 / (f_ms * 1e-3) / 1e9,
+                                   "bwd_gbs": th * 516 / (b_ms * 1e-3) / 1e9, "paths": [binding.rib_last_path()],
+                                   "note": "GB/s over the algorithmic bytes: forward q, k, v read + out written (256 B per token-head), "
+                                           "backward q, k, v, out, dout, lse read + dq, dk, dv written (516 B per token-head)"}
+            del out_8, lse_8
             # shifted windows with a region mask (the wrapped parts of a border window do not attend to each other)
             out_m, lse_m = binding.rib_window_attn_fwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], wl.window, wl.shift)
             f_ms = timed(lambda: binding.rib_window_attn_fwd_masked(s0["q"], s0["k"], s0["v"], s0["pq"], s0["pk"], wl.window, wl.shift))
