@@ -647,8 +647,10 @@ __global__ void __launch_bounds__(256) rib_bwd_prepare_kernel(const AuxParams p)
     float acc = 0.f;
 #pragma unroll
     for (int q4 = 0; q4 < 4; ++q4) {
-        if (8 * q4 >= p.d) break;
-        const uint4 x = __ldg(a + q4), y = __ldg(b + q4);
+        // (predicated, not a break: the loads of all four pieces are in flight together)
+        const bool on = 8 * q4 < p.d;
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        const uint4 x = on ? __ldg(a + q4) : zero, y = on ? __ldg(b + q4) : zero;
         const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
