@@ -205,7 +205,8 @@ def test_running_maximum_rescale(direction):
     compare("lse", to_f64(lse), ref_lse, max_abs=2e-2, rel_l2=5e-3)
 
 
-@pytest.mark.parametrize("wl", [SMALL[7], SMALL[8], SMALL[12], CONFIGS[1]], ids=lambda w: w.name)
+@pytest.mark.parametrize("wl", [SMALL[7], SMALL[8], SMALL[12], CONFIGS[1]] + [w for w in SMALL if w.name in ("w8_packed", "d16_r16_w32_s16")],
+                         ids=lambda w: w.name)
 def test_exact_softmax_form_every_element(wl):
     """The tcgen05 forward kernel keeps two forms of the softmax: a fast one with a fixed per-row reference and the
     exact one with a running maximum that redoes items whose scores leave the fast form's range.  Here every item is
