@@ -228,7 +228,7 @@ int rib_window_attn_fwd_gated(const void* q, const void* k, const void* v, const
  *   dx: bf16 [B][H][W][D];  dw_dw [D][3][3], db_dw [D], dw_pw [D][D], db_pw [D]: fp32; all five overwritten.
  *   workspace: device scratch of at least rib_cla_gate_bwd_workspace(B, H, W, D) bytes (dY in fp32 and the
  *   transposed matrix), 16-byte aligned, owned by the caller, contents undefined afterwards.
- *   Any positive H and W; D = 64, 128 or 192 (RIB_ERR_UNSUPPORTED otherwise).  Four small memsets and two kernels on
+ *   Any positive H and W; D = 64, 128 or 192 (RIB_ERR_UNSUPPORTED otherwise).  Three kernels (the first one clears the four weight gradients) on
  *   `stream`: the point-wise part on the tensor cores (Y, dZ and w_pw enter the products as bf16, sums in fp32) and the
  *   depth-wise part; with rib_set_path(RIB_PATH_GENERIC) the point-wise part runs in fp32 instead (one more small
  *   kernel).  The weight gradients are fp32 sums in no fixed order (atomics): equal up to rounding from call to call.

@@ -303,7 +303,7 @@ int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const 
                                             dw_dw, db_dw, dw_pw, db_pw, workspace, fast, status, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
-    g_kernel_launches += fast ? 2 : 3;
+    g_kernel_launches += fast ? 3 : 4;     // zeroing of the weight gradients, (transpose,) point-wise part, depth-wise part
     return RIB_OK;
 }
 

@@ -729,6 +729,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) rib_cla_bwd_tc_kernel(const Cla
     }
 }
 
+// The four weight gradients start at zero (both kernels add to them): one launch instead of four memsets.
+__global__ void rib_cla_zero_grads_kernel(float* dw_dw, float* db_dw, float* dw_pw, float* db_pw, int D)
+{
+    const int n_dw = 9 * D, n_pw = D * D;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_pw; i += gridDim.x * blockDim.x) {
+        dw_pw[i] = 0.f;
+        if (i < n_dw) dw_dw[i] = 0.f;
+        if (i < D) { db_dw[i] = 0.f; db_pw[i] = 0.f; }
+    }
+}
+
 template <int D>
 cudaError_t launch_gate_bwd(const ClaBwdParams& p, bool tensor_cores, cudaStream_t stream)
 {
@@ -738,11 +749,9 @@ cudaError_t launch_gate_bwd(const ClaBwdParams& p, bool tensor_cores, cudaStream
     if (cudaError_t e = setup_pw.prepare(rib_cla_bwd_pw_kernel<D>, (uint32_t)kSmem, &sms)) return e;
     if (cudaError_t e = setup_dw.prepare(rib_cla_bwd_dw_kernel<D>, kDwSmemBytes, &sms)) return e;
     if (cudaError_t e = setup_tc.prepare(rib_cla_bwd_tc_kernel<D>, TcLayout<D>::kSmemBytes, &sms)) return e;
-    cudaError_t e = cudaMemsetAsync(p.dw_dw, 0, sizeof(float) * 9 * D, stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p.db_dw, 0, sizeof(float) * D, stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p.dw_pw, 0, sizeof(float) * D * D, stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p.db_pw, 0, sizeof(float) * D, stream);
-    if (e != cudaSuccess) return e;
+    static_assert(D * D >= 9 * D, "the zeroing kernel walks the largest of the four");
+    rib_cla_zero_grads_kernel<<<(D * D + 255) / 256, 256, 0, stream>>>(p.dw_dw, p.db_dw, p.dw_pw, p.db_pw, D);
+    if (cudaError_t e = cudaGetLastError()) return e;
     if (tensor_cores) {
         const long long tiles = (p.pixels + kTcPix - 1) / kTcPix;
         ProfileScope scope(RIB_KERNEL_CLA_BWD_TC, stream);
