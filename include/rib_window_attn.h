@@ -189,6 +189,23 @@ int rib_window_cycle_fwd(const void* const* q, const void* const* k, const void*
                          int B, int H, int W, int heads, int d, int r, void* const* out, float* const* lse, void* stream);
 
 /*
+ * The backward passes of the same layers (Sec. 3.3), in the order of the arrays: layer l computes dq[l], dk[l], dv[l] (bf16,
+ * layout of q) and dpq[l], dpk[l] (fp32 [windows[l]^2][r]) from out[l], lse[l] (results of the forward pass on q[l], k[l],
+ * v[l], pq[l], pk[l]) and dout[l], exactly as rib_window_attn_bwd_padded does for one layer.  All pointer arguments but
+ * `workspace` are HOST arrays of `layers` device pointers; no entry may be NULL.  The layers run one after the other on
+ * `stream` and share one workspace of at least rib_window_cycle_bwd_workspace(windows, layers, ...) bytes (the largest
+ * of the layers' needs; 0 = unsupported shape), 256-byte aligned, owned by the caller.  Every layer's arguments are checked
+ * before the first launch; error codes as for rib_window_attn_bwd_padded, plus RIB_ERR_SHAPE for layers outside 1..64.
+ */
+int rib_window_cycle_bwd(const void* const* q, const void* const* k, const void* const* v, const void* const* pq, const void* const* pk,
+                         const void* const* out, const float* const* lse, const void* const* dout,
+                         const int* windows, const int* shifts, int layers,
+                         int B, int H, int W, int heads, int d, int r,
+                         void* const* dq, void* const* dk, void* const* dv, float* const* dpq, float* const* dpk,
+                         void* workspace, size_t workspace_bytes, void* stream);
+size_t rib_window_cycle_bwd_workspace(const int* windows, int layers, int B, int H, int W, int heads, int d, int r);
+
+/*
  * Convolutional Local Attention (paper: Sec. 3.2, Eq. 7, Eq. 8, Eq. 9): the step right after the attention.
  *   G  = sigmoid(PWConv(DWConv3x3(X)))      X: the block's token features as an H x W map          (Eq. 8)
  *   O' = O o G                              element-wise product with the attention output           (Eq. 9)

@@ -27,7 +27,7 @@ EXPORTS = (
     "rib_window_attn_fwd_headwise", "rib_window_attn_bwd_headwise", "rib_window_attn_bwd_headwise_workspace",
     "rib_window_attn_fwd_padded", "rib_cla_gate", "rib_window_attn_fwd_gated",
     "rib_window_attn_bwd_padded", "rib_window_attn_bwd_padded_workspace",
-    "rib_window_attn_fwd_masked", "rib_window_attn_bwd_masked",
+    "rib_window_attn_fwd_masked", "rib_window_attn_bwd_masked", "rib_window_cycle_bwd", "rib_window_cycle_bwd_workspace",
     "rib_cla_product", "rib_cla_product_bwd", "rib_cla_gate_bwd", "rib_cla_gate_bwd_workspace",
     "rib_wait_probe", "rib_exp_probe", "rib_tensor_map_cache_counts", "rib_window_cycle_fwd",
 )
@@ -69,6 +69,10 @@ def library() -> ctypes.CDLL:
         lib.rib_window_attn_fwd_padded.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd_padded.restype = ci
         lib.rib_window_attn_bwd_padded.argtypes = [vp] * 5 + [ll] + [vp] * 3 + [ci] * 8 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_cycle_bwd.restype = ci
+        lib.rib_window_cycle_bwd.argtypes = [vp] * 8 + [vp, vp, ci] + [ci] * 6 + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        lib.rib_window_cycle_bwd_workspace.restype = ctypes.c_size_t
+        lib.rib_window_cycle_bwd_workspace.argtypes = [vp, ci] + [ci] * 6
         lib.rib_window_attn_fwd_masked.restype = ci
         lib.rib_window_attn_fwd_masked.argtypes = [vp] * 5 + [ll] + [ci] * 8 + [vp, fp, vp]
         lib.rib_window_attn_bwd_masked.restype = ci
@@ -336,6 +340,39 @@ def rib_window_cycle_fwd(qs, ks, vs, pqs, pks, windows, shifts=None, stream=None
     if rc != RIB_OK:
         raise RibError(rc)
     return outs, lses
+
+
+def rib_window_cycle_bwd(qs, ks, vs, pqs, pks, outs, lses, douts, windows, shifts=None, workspace=None, stream=None):
+    """Backward passes of the layers of rib_window_cycle_fwd.  Returns (dqs, dks, dvs, dpqs, dpks), one tensor per layer."""
+    layers = len(windows)
+    lists = (qs, ks, vs, pqs, pks, outs, lses, douts)
+    if any(len(x) != layers for x in lists) or (shifts is not None and len(shifts) != layers):
+        raise ValueError("one q, k, v, pq, pk, out, lse, dout (and shift) per layer")
+    _check_image("q", qs[0])
+    B, H, W, heads, d = qs[0].shape
+    r = pqs[0].shape[1]
+    for l in range(layers):
+        for name, t in (("q", qs[l]), ("k", ks[l]), ("v", vs[l]), ("out", outs[l]), ("dout", douts[l])):
+            _check_image(name, t, qs[0].shape)
+        _check_pos("pq", pqs[l], windows[l] * windows[l])
+        _check_pos("pk", pks[l], windows[l] * windows[l])
+        if lses[l].dtype != torch.float32 or tuple(lses[l].shape) != (B, heads, H, W) or not lses[l].is_contiguous():
+            raise ValueError("lse must be a contiguous fp32 tensor [B,heads,H,W]")
+    ints = lambda xs: (ctypes.c_int * layers)(*[int(x) for x in xs])
+    arr = lambda ts: (ctypes.c_void_p * layers)(*[_ptr(t) for t in ts])
+    need = int(library().rib_window_cycle_bwd_workspace(ints(windows), layers, B, H, W, heads, d, r))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=qs[0].device)
+    dqs, dks, dvs = ([torch.empty_like(qs[0]) for _ in range(layers)] for _ in range(3))
+    dpqs = [torch.empty(tuple(t.shape), dtype=torch.float32, device=t.device) for t in pqs]
+    dpks = [torch.empty(tuple(t.shape), dtype=torch.float32, device=t.device) for t in pks]
+    rc = library().rib_window_cycle_bwd(arr(qs), arr(ks), arr(vs), arr(pqs), arr(pks), arr(outs), arr(lses), arr(douts), ints(windows),
+                                        ints(shifts) if shifts is not None else None, layers, B, H, W, heads, d, r,
+                                        arr(dqs), arr(dks), arr(dvs), arr(dpqs), arr(dpks), _ptr(workspace), workspace.numel(),
+                                        _stream_ptr(stream))
+    if rc != RIB_OK:
+        raise RibError(rc)
+    return dqs, dks, dvs, dpqs, dpks
 
 
 def rib_window_attn_bwd_padded(q, k, v, pq, pk, out, lse, dout, window, shift=0, workspace=None, stream=None):

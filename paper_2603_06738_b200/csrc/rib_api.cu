@@ -413,7 +413,7 @@ static int bwd_impl(const void* q, const void* k, const void* v, const void* pq,
                     const void* out, const float* lse, const void* dout,
                     int B, int H, int W, int heads, int d, int r, int window, int shift,
                     void* dq, void* dk, void* dv, float* dpq, float* dpk,
-                    void* workspace, size_t workspace_bytes, void* stream, bool masked)
+                    void* workspace, size_t workspace_bytes, void* stream, bool masked, bool validate_only = false)
 {
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return RIB_ERR_NULL;
     if (r > 0 && (!pq || !pk || !dpq || !dpk)) return RIB_ERR_NULL;
@@ -425,6 +425,7 @@ static int bwd_impl(const void* q, const void* k, const void* v, const void* pq,
     const size_t need = rib_window_attn_bwd_padded_workspace(pos_head_stride, B, H, W, heads, d, r, window);
     if (!workspace || workspace_bytes < need) return RIB_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return RIB_ERR_ALIGN;
+    if (validate_only) return RIB_OK;
     rib::Problem p{};
     fill_shape(p, B, H, W, heads, d, r, window, shift);
     p.q = static_cast<const __nv_bfloat16*>(q);
@@ -464,6 +465,38 @@ int rib_window_attn_bwd_padded(const void* q, const void* k, const void* v, cons
 {
     return bwd_impl(q, k, v, pq, pk, pos_head_stride, out, lse, dout, B, H, W, heads, d, r, window, shift, dq, dk, dv, dpq, dpk,
                     workspace, workspace_bytes, stream, false);
+}
+
+size_t rib_window_cycle_bwd_workspace(const int* windows, int layers, int B, int H, int W, int heads, int d, int r)
+{
+    if (!windows || layers <= 0 || layers > 64) return 0;
+    size_t need = 0;
+    for (int l = 0; l < layers; ++l) {
+        const size_t one = rib_window_attn_bwd_padded_workspace(0, B, H, W, heads, d, r, windows[l]);
+        if (one == 0) return 0;
+        if (one > need) need = one;
+    }
+    return need;
+}
+
+int rib_window_cycle_bwd(const void* const* q, const void* const* k, const void* const* v, const void* const* pq, const void* const* pk,
+                         const void* const* out, const float* const* lse, const void* const* dout,
+                         const int* windows, const int* shifts, int layers,
+                         int B, int H, int W, int heads, int d, int r,
+                         void* const* dq, void* const* dk, void* const* dv, float* const* dpq, float* const* dpk,
+                         void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!q || !k || !v || !pq || !pk || !out || !lse || !dout || !windows || !dq || !dk || !dv || !dpq || !dpk) return RIB_ERR_NULL;
+    if (layers <= 0 || layers > 64) return RIB_ERR_SHAPE;
+    // every layer is checked before the first one is launched; the layers run one after the other on the stream and share the workspace
+    for (int pass = 0; pass < 2; ++pass)
+        for (int l = 0; l < layers; ++l) {
+            const int rc = bwd_impl(q[l], k[l], v[l], pq[l], pk[l], 0, out[l], lse[l], dout[l], B, H, W, heads, d, r, windows[l],
+                                    shifts ? shifts[l] : 0, dq[l], dk[l], dv[l], dpq[l], dpk[l], workspace, workspace_bytes, stream, false,
+                                    pass == 0);
+            if (rc != RIB_OK) return rc;
+        }
+    return RIB_OK;
 }
 
 int rib_window_attn_fwd_masked(const void* q, const void* k, const void* v, const void* pq, const void* pk,

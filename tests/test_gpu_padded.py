@@ -119,7 +119,8 @@ def test_plain_entry_points_still_reject_partial_windows():
 
 
 def test_window_cycle_driver_runs_the_six_layers_of_a_block():
-    """Sec. 3.3: the window size cycles over the layers of a block.  One call enqueues all six layers; every layer is
+    """Sec. 3.3: the window size cycles over the layers of a block.  One call enqueues all six layers (and one more call their
+    backward passes); every layer is
     compared with the oracle (64 does not divide the 96-row map: that layer runs on partial windows), and a repeated
     call encodes no tensor map."""
     B, H, W, heads, d, r = 1, 96, 64, 2, 32, 16
@@ -146,3 +147,17 @@ def test_window_cycle_driver_runs_the_six_layers_of_a_block():
     binding.rib_window_cycle_fwd(*args, windows)
     torch.cuda.synchronize()
     assert binding.rib_tensor_map_cache_counts()[1] == misses      # q, k, v and Pk of every layer were mapped by the first call
+    # the backward passes of the same six layers in one call, sharing one workspace
+    douts = [synthetic.bf16_tensor(320 + l, "dout", (B, H, W, heads, d), 1.0) for l in range(len(windows))]
+    launches = binding.rib_kernel_launches()
+    grads = binding.rib_window_cycle_bwd(*args, outs, lses, [t.cuda() for t in douts], windows)
+    torch.cuda.synchronize()
+    assert binding.rib_query_status() == 0 and binding.rib_kernel_launches() == launches + 18
+    for l, win in enumerate(windows):
+        f64 = {k: to_f64(v) for k, v in layers[l].items()}
+        ref = pad.bwd(f64["q"], f64["k"], f64["v"], f64["pq"], f64["pk"], to_f64(douts[l]), win, 0)
+        for name, got, want in zip(("dq", "dk", "dv"), (grads[0][l], grads[1][l], grads[2][l]), ref[:3]):
+            compare(f"layer {l} (window {win}) {name}", to_f64(got), want)
+        scale = max(1.0, float(np.abs(ref[3]).max()), float(np.abs(ref[4]).max()))
+        compare(f"layer {l} (window {win}) dpq", to_f64(grads[3][l]), ref[3], max_abs=1e-2 * scale)
+        compare(f"layer {l} (window {win}) dpk", to_f64(grads[4][l]), ref[4], max_abs=1e-2 * scale)
