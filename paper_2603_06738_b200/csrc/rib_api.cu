@@ -337,12 +337,27 @@ int fwd_impl(const void* q, const void* k, const void* v, const void* pq, const 
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int forced = g_forced_path.load();
-    const bool fast = forced != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
+    bool fast = forced != RIB_PATH_GENERIC && rib::sm100_fwd_supported(p);
     p.exact_softmax = forced == RIB_PATH_SM100_EXACT;
-    const cudaError_t e = fast ? rib::sm100_fwd(p, st) : rib::generic_fwd(p, st);
+    int launches = 1;
+    cudaError_t e;
+    if (fast) {
+        e = rib::sm100_fwd(p, st);
+    } else if (forced != RIB_PATH_GENERIC && rib::sm100_repack_supported(p)) {
+        // rows TMA cannot address (d = 30, r = 18, ...): the tensor-core kernels on zero-padded copies
+        e = rib::sm100_fwd_repacked(p, st, &launches);
+        fast = e == cudaSuccess;
+        if (e == cudaErrorMemoryAllocation) {       // no scratch to be had: the any-shape kernel needs none
+            (void)cudaGetLastError();
+            launches = 1;
+            e = rib::generic_fwd(p, st);
+        }
+    } else {
+        e = rib::generic_fwd(p, st);
+    }
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
-    g_kernel_launches += 1;
+    g_kernel_launches += launches;
     return RIB_OK;
 }
 
@@ -363,8 +378,8 @@ size_t rib_window_attn_bwd_headwise_workspace(long long pos_head_stride, int B, 
     size_t need = rowdot_bytes(B, H, W, heads);
     rib::Problem p{};
     fill_shape(p, B, H, W, heads, d, r, window, 0);
-    if (rib::sm100_bwd_supported(p)) {   // whatever the shift: one size per shape
-        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1, r);
+    if (rib::sm100_bwd_supported(p) || rib::sm100_repack_supported(p)) {   // whatever the shift: one size per shape
+        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1, rib::repacked_width(r));
         if (fast > need) need = fast;
     }
     return need;
@@ -401,8 +416,8 @@ size_t rib_window_attn_bwd_padded_workspace(long long pos_head_stride, int B, in
     size_t need = rowdot_bytes(B, H, W, heads);
     rib::Problem p{};
     fill_shape(p, B, H, W, heads, d, r, window, 0);
-    if (rib::sm100_bwd_supported(p)) {        // sized by the windows of the extended map
-        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1, r);
+    if (rib::sm100_bwd_supported(p) || rib::sm100_repack_supported(p)) {        // sized by the windows of the extended map
+        const size_t fast = rib::sm100_bwd_workspace_bytes(p.pairs, p.n, pos_head_stride ? heads : 1, rib::repacked_width(r));
         if (fast > need) need = fast;
     }
     return need;
@@ -448,11 +463,26 @@ static int bwd_impl(const void* q, const void* k, const void* v, const void* pq,
     p.masked = masked;
     if (int rc = device_status_ptr(&p.status)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool fast = g_forced_path.load() != RIB_PATH_GENERIC && rib::sm100_bwd_supported(p);
-    const cudaError_t e = fast ? rib::sm100_bwd(p, st) : rib::generic_bwd(p, st);
+    const bool allowed = g_forced_path.load() != RIB_PATH_GENERIC;
+    bool fast = allowed && rib::sm100_bwd_supported(p);
+    int launches = 3;          // prepare, main, finish : rowdot, dq, dk/dv
+    cudaError_t e;
+    if (fast) {
+        e = rib::sm100_bwd(p, st);
+    } else if (allowed && rib::sm100_repack_supported(p)) {
+        e = rib::sm100_bwd_repacked(p, st, &launches);
+        fast = e == cudaSuccess;
+        if (e == cudaErrorMemoryAllocation) {
+            (void)cudaGetLastError();
+            launches = 3;
+            e = rib::generic_bwd(p, st);
+        }
+    } else {
+        e = rib::generic_bwd(p, st);
+    }
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
-    g_kernel_launches += 3;   // prepare, main, finish : rowdot, dq, dk/dv
+    g_kernel_launches += launches;
     return RIB_OK;
 }
 

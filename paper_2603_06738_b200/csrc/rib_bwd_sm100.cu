@@ -788,9 +788,9 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     ap.table_rows = table_rows;
     ap.tables = tables;
     ap.pos_head_stride = p.pos_head_stride;
-    ap.pos_scale = sqrtf((float)p.d / (float)p.r);
-    ap.inv_sqrt_d = 1.f / sqrtf((float)p.d);
-    ap.inv_sqrt_r = 1.f / sqrtf((float)p.r);
+    ap.pos_scale = sqrtf(scale_width_d(p) / scale_width_r(p));
+    ap.inv_sqrt_d = 1.f / sqrtf(scale_width_d(p));
+    ap.inv_sqrt_r = 1.f / sqrtf(scale_width_r(p));
     const size_t tokens = (size_t)p.pairs * p.n;
     const unsigned aux_blocks = (unsigned)((tokens + 255) / 256);
     { ProfileScope scope(RIB_KERNEL_BWD_PREPARE, stream); rib_bwd_prepare_kernel<R><<<aux_blocks, 256, 0, stream>>>(ap); }
@@ -807,7 +807,7 @@ cudaError_t launch_bwd(const Problem& p, cudaStream_t stream)
     bp.masked = p.masked ? 1 : 0;
     bp.packed8 = p.packed8 ? 1 : 0;
     bp.d = p.d;
-    bp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
+    bp.scale_log2 = 1.4426950408889634f / sqrtf(scale_width_d(p));
     bp.inv_sqrt_d = ap.inv_sqrt_d;
     const int grid = bp.items < sm_count ? bp.items : sm_count;
     { ProfileScope scope(RIB_KERNEL_BWD_MAIN, stream); rib_bwd_sm100_kernel<R, kPartial><<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_pqs, tm_pk, bp); }

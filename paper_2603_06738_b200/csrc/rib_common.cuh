@@ -39,6 +39,8 @@ struct Problem {
     int* status;                      // device status word (bounded waits report here)
     bool exact_softmax;               // tcgen05 forward: every item takes the exact (running-maximum) softmax form
     bool masked;                      // shifted windows: the wrapped parts of a border window do not attend to each other
+    int d_true, r_true;               // tcgen05 kernels on zero-padded copies (rib_repack.cu): the widths the scales 1/sqrt(d),
+                                      // 1/sqrt(r) are taken from; 0 = d, r themselves
     bool packed8;                     // tcgen05 kernels only: M, n, nWy, nWx, pairs describe 16 x 16 windows that each stand for
                                       // 2 x 2 windows of 8 x 8 tokens (a token attends to the 8 x 8 patch it lies in; the tables
                                       // pq, pk, dpq, dpk have 64 rows)
@@ -52,6 +54,10 @@ inline size_t pos_extent(const Problem& p)
     return (size_t)(pos_tables(p) - 1) * (size_t)p.pos_head_stride + (size_t)p.n * p.r;
 }
 
+// The head width and the rank that the scales of Eq. 6 are taken from.
+inline float scale_width_d(const Problem& p) { return (float)(p.d_true ? p.d_true : p.d); }
+inline float scale_width_r(const Problem& p) { return (float)(p.r_true ? p.r_true : p.r); }
+
 // Launchers; each returns the cudaError_t of its launches.
 cudaError_t generic_fwd(const Problem& p, cudaStream_t stream);
 cudaError_t generic_bwd(const Problem& p, cudaStream_t stream);
@@ -62,6 +68,13 @@ cudaError_t sm100_fwd(const Problem& p, cudaStream_t stream);
 bool sm100_bwd_supported(const Problem& p);
 size_t sm100_bwd_workspace_bytes(long long pairs, int n, int tables, int r);
 cudaError_t sm100_bwd(const Problem& p, cudaStream_t stream);   // launches 3 kernels
+// Even head widths and ranks up to 32 whose rows TMA cannot address (60-byte rows of d = 30, 36-byte rows of r = 18):
+// the tensors are copied into zero-padded scratch (stream-ordered allocation), the tcgen05 kernels run on the copies,
+// and the results are copied back.  `launches` receives the number of kernels enqueued.
+bool sm100_repack_supported(const Problem& p);
+int repacked_width(int w);                    // the next multiple of 8
+cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launches);
+cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launches);
 
 bool cla_gate_supported(int H, int W, int D);
 cudaError_t cla_gate(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw, int B, int H,

@@ -868,9 +868,9 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.Hp = p.Hp; fp.Wp = p.Wp;
     fp.tiles_per_item_pair = p.n / (2 * kTile);
     fp.items = p.pairs * fp.tiles_per_item_pair;
-    fp.scale_log2 = 1.4426950408889634f / sqrtf((float)p.d);
-    fp.inv_sqrt_d = 1.f / sqrtf((float)p.d);
-    fp.pos_scale = sqrtf((float)p.d / (float)p.r);
+    fp.scale_log2 = 1.4426950408889634f / sqrtf(scale_width_d(p));
+    fp.inv_sqrt_d = 1.f / sqrtf(scale_width_d(p));
+    fp.pos_scale = sqrtf(scale_width_d(p) / scale_width_r(p));
     fp.pos_head_stride = p.pos_head_stride;
     fp.pos_per_head = p.pos_head_stride ? 1 : 0;
     fp.exact_only = p.exact_softmax ? 1 : 0;
