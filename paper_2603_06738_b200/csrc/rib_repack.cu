@@ -2,25 +2,63 @@
 // r = 18 gives 36-byte rows -- the SST rows of the paper's network table).  For even d, r <= 32 the tensors are copied
 // into scratch with every row filled up with zeros to the next multiple of 8 elements, the tcgen05 kernels run on the
 // copies (zero channels change no dot product; the scales of Eq. 6 keep the true d and r), and the results are copied
-// back.  The scratch comes from the stream-ordered allocator (cudaMallocAsync / cudaFreeAsync on the caller's stream):
-// nothing here synchronises.  The attention passes are bound by arithmetic, so the copies (a few hundred bytes per
+// back.  The scratch comes from a stream-ordered memory pool of the library's own, one per device, that keeps what is
+// freed (cudaMallocFromPoolAsync / cudaFreeAsync on the caller's stream): after the first call of a shape nothing here
+// talks to the driver's allocator and nothing synchronises.  The attention passes are bound by arithmetic, so the copies (a few hundred bytes per
 // token-head) cost little next to them; the any-shape kernels these shapes would otherwise take are about a hundred
 // times slower.
 #include "rib_common.cuh"
 
+#include <mutex>
+
 namespace rib {
 namespace {
+
+// One pool per device, created on first use with that device current; freed blocks stay in the pool (release threshold
+// at its maximum), so the steady state of a training loop reuses the same memory.
+constexpr int kMaxPoolDevices = 64;
+std::mutex g_pool_mutex;
+cudaMemPool_t g_pool[kMaxPoolDevices] = {};
+
+cudaError_t scratch_pool(cudaMemPool_t* pool)
+{
+    int dev = -1;
+    if (cudaError_t e = cudaGetDevice(&dev)) return e;
+    if (dev < 0 || dev >= kMaxPoolDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_pool_mutex);
+    if (!g_pool[dev]) {
+        cudaMemPoolProps props{};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t created = nullptr;
+        if (cudaError_t e = cudaMemPoolCreate(&created, &props)) return e;
+        unsigned long long keep = ~0ull;
+        if (cudaError_t e = cudaMemPoolSetAttribute(created, cudaMemPoolAttrReleaseThreshold, &keep)) { cudaMemPoolDestroy(created); return e; }
+        g_pool[dev] = created;
+    }
+    *pool = g_pool[dev];
+    return cudaSuccess;
+}
+
+cudaError_t scratch_alloc(uint8_t** ptr, size_t bytes, cudaStream_t stream)
+{
+    cudaMemPool_t pool = nullptr;
+    if (cudaError_t e = scratch_pool(&pool)) return e;
+    return cudaMallocFromPoolAsync(reinterpret_cast<void**>(ptr), bytes, pool, stream);
+}
 
 // dst[row][c] = src[row][c] for c < min(ws, wd), 0 for the other columns of dst; T is a pair of elements
 template <typename T>
 __global__ void __launch_bounds__(256) rib_copy_columns_kernel(const T* __restrict__ src, int ws, T* __restrict__ dst, int wd, size_t rows)
 {
-    const size_t total = rows * (size_t)wd;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-        const size_t row = e / wd;
-        const int c = (int)(e - row * wd);
+    // (32-bit index arithmetic: the launcher splits tensors of 2^32 pairs and more)
+    const unsigned total = (unsigned)rows * (unsigned)wd;
+    for (unsigned e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const unsigned row = e / (unsigned)wd, c = e - row * (unsigned)wd;
         T v{};
-        if (c < ws) v = src[row * ws + c];
+        if (c < (unsigned)ws) v = src[(size_t)row * ws + c];
         dst[e] = v;
     }
 }
@@ -28,12 +66,16 @@ __global__ void __launch_bounds__(256) rib_copy_columns_kernel(const T* __restri
 template <typename T>
 cudaError_t copy_columns(const void* src, int ws_elems, void* dst, int wd_elems, size_t rows, cudaStream_t stream, int* launches)
 {
-    const size_t total = rows * (size_t)(wd_elems / 2);
-    if (total == 0) return cudaSuccess;
-    const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
-    rib_copy_columns_kernel<T><<<blocks, 256, 0, stream>>>(static_cast<const T*>(src), ws_elems / 2, static_cast<T*>(dst), wd_elems / 2, rows);
-    ++*launches;
-    return cudaGetLastError();
+    const int ws = ws_elems / 2, wd = wd_elems / 2;
+    const size_t chunk = (size_t)0x7fffffff / (size_t)wd;          // rows per launch: their pairs fit 31 bits
+    for (size_t r0 = 0; r0 < rows; r0 += chunk) {
+        const size_t nrows = rows - r0 < chunk ? rows - r0 : chunk, total = nrows * (size_t)wd;
+        const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+        rib_copy_columns_kernel<T><<<blocks, 256, 0, stream>>>(static_cast<const T*>(src) + r0 * ws, ws, static_cast<T*>(dst) + r0 * wd, wd, nrows);
+        ++*launches;
+        if (cudaError_t e = cudaGetLastError()) return e;
+    }
+    return cudaSuccess;
 }
 
 size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -79,7 +121,7 @@ cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     const size_t rows = (size_t)p.B * p.H * p.W * p.heads;
     const size_t img = up256(rows * pp.d * sizeof(__nv_bfloat16)), tab = up256((size_t)tables * p.n * pp.r * sizeof(__nv_bfloat16));
     uint8_t* buf = nullptr;
-    if (cudaError_t e = cudaMallocAsync(reinterpret_cast<void**>(&buf), 4 * img + 2 * tab, stream)) return e;
+    if (cudaError_t e = scratch_alloc(&buf, 4 * img + 2 * tab, stream)) return e;
     __nv_bfloat16* q2 = reinterpret_cast<__nv_bfloat16*>(buf);
     __nv_bfloat16* k2 = reinterpret_cast<__nv_bfloat16*>(buf + img);
     __nv_bfloat16* v2 = reinterpret_cast<__nv_bfloat16*>(buf + 2 * img);
@@ -111,7 +153,7 @@ cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     const size_t img = up256(rows * pp.d * sizeof(__nv_bfloat16));
     const size_t tab = up256((size_t)tables * p.n * pp.r * sizeof(__nv_bfloat16)), gtab = up256((size_t)tables * p.n * pp.r * sizeof(float));
     uint8_t* buf = nullptr;
-    if (cudaError_t e = cudaMallocAsync(reinterpret_cast<void**>(&buf), 8 * img + 2 * tab + 2 * gtab, stream)) return e;
+    if (cudaError_t e = scratch_alloc(&buf, 8 * img + 2 * tab + 2 * gtab, stream)) return e;
     auto image = [&](int i) { return reinterpret_cast<__nv_bfloat16*>(buf + (size_t)i * img); };
     __nv_bfloat16* pq2 = reinterpret_cast<__nv_bfloat16*>(buf + 8 * img);
     __nv_bfloat16* pk2 = reinterpret_cast<__nv_bfloat16*>(buf + 8 * img + tab);
