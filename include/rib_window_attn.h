@@ -35,7 +35,7 @@
  * r = 18 or 34, the light-weight ones d = 16 with r = 16 or 24).  Shapes with d = 8, 16, 24 or 32, r = 8, 16, 24 or 32
  * (rows that TMA can address: multiples of 16 bytes), window a multiple of 16 and shift a multiple of 8 take the
  * tcgen05 / TMEM / TMA kernels, and so does window 8 without a shift on maps whose sides are multiples of 16.  Other
- * even d and r up to 32 (d = 30 with r = 18) take the same kernels on zero-padded copies of the tensors: those calls
+ * even d up to 32 and r up to 32 + (padding of d) (d = 30 with r = 18 or 34) take the same kernels on zero-padded copies of the tensors: those calls
  * (rib_window_attn_fwd*, rib_window_attn_bwd* except the gated forward) draw scratch from a stream-ordered memory pool
  * that the library keeps per device (no synchronisation; the pool holds on to what it has used until the process ends;
  * if it cannot grow, the call takes the any-shape kernels).  Every other supported shape takes a slower any-shape CUDA

@@ -63,6 +63,56 @@ __global__ void __launch_bounds__(256) rib_copy_columns_kernel(const T* __restri
     }
 }
 
+// Ranks above 32 (d = 30 with r = 34): the kernels hold 32 RIB columns, and the zero channels of the padded head have
+// room for the rest.  Column 32 + j of the tables goes into channel d + j of the q and k copies -- for q times sqrt(d / r),
+// so that the content scale 1 / sqrt(d) leaves 1 / sqrt(r) on the product, exactly as for the staged RIB rows -- indexed by
+// the token's place in its window; the logits are unchanged.  Geometry of the token -> window position map:
+struct PlaceGeom { int H, W, Hp, Wp, heads, M, s, d, dp, r, extra; long long table_stride; float scale; };
+
+__device__ __forceinline__ int window_place(const PlaceGeom& g, int Y, int X)
+{
+    int yr = Y - g.s, xr = X - g.s;                 // the rolled frame the windows are cut from
+    if (yr < 0) yr += g.Hp;
+    if (xr < 0) xr += g.Wp;
+    return (yr % g.M) * g.M + xr % g.M;
+}
+
+// dst[row][c]: c < d from src, d <= c < d + extra from table[place][32 + c - d] * scale, zero beyond; pairs of elements
+__global__ void __launch_bounds__(256) rib_pack_with_rank_tail_kernel(const uint32_t* __restrict__ src, uint32_t* __restrict__ dst,
+                                                                     const __nv_bfloat16* __restrict__ table, PlaceGeom g, unsigned rows)
+{
+    const unsigned wd = g.dp / 2, ws = g.d / 2, total = rows * wd;
+    for (unsigned e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const unsigned row = e / wd, c = e - row * wd;
+        uint32_t v = 0u;
+        if (c < ws) {
+            v = src[(size_t)row * ws + c];
+        } else if (2 * (int)(c - ws) < g.extra) {
+            const unsigned h = row % (unsigned)g.heads, pixel = row / (unsigned)g.heads;
+            const int X = (int)(pixel % (unsigned)g.W), Y = (int)((pixel / (unsigned)g.W) % (unsigned)g.H);
+            const __nv_bfloat16* t = table + (size_t)h * g.table_stride + (size_t)window_place(g, Y, X) * g.r + 32 + 2 * (c - ws);
+            const __nv_bfloat162 two = __floats2bfloat162_rn(__bfloat162float(t[0]) * g.scale, __bfloat162float(t[1]) * g.scale);
+            v = *reinterpret_cast<const uint32_t*>(&two);
+        }
+        dst[e] = v;
+    }
+}
+
+// the gradient of those table columns: channel d + j of dq and dk of every token, summed over the tokens of a place
+__global__ void __launch_bounds__(256) rib_rank_tail_grads_kernel(const __nv_bfloat16* __restrict__ dq, const __nv_bfloat16* __restrict__ dk,
+                                                                 float* __restrict__ dpq, float* __restrict__ dpk, PlaceGeom g, unsigned rows)
+{
+    const unsigned total = rows * (unsigned)g.extra;
+    for (unsigned e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const unsigned row = e / (unsigned)g.extra, j = e - row * (unsigned)g.extra;
+        const unsigned h = row % (unsigned)g.heads, pixel = row / (unsigned)g.heads;
+        const int X = (int)(pixel % (unsigned)g.W), Y = (int)((pixel / (unsigned)g.W) % (unsigned)g.H);
+        const size_t at = (size_t)h * g.table_stride + (size_t)window_place(g, Y, X) * g.r + 32 + j;
+        atomicAdd(dpq + at, __bfloat162float(dq[(size_t)row * g.dp + g.d + j]) * g.scale);
+        atomicAdd(dpk + at, __bfloat162float(dk[(size_t)row * g.dp + g.d + j]));
+    }
+}
+
 template <typename T>
 cudaError_t copy_columns(const void* src, int ws_elems, void* dst, int wd_elems, size_t rows, cudaStream_t stream, int* launches)
 {
@@ -90,15 +140,47 @@ cudaError_t copy_tables(const Elem* src, long long src_stride, int ws, Elem* dst
     return cudaSuccess;
 }
 
+// columns of the tables that travel in the zero channels of the padded head (ranks above 32)
+int rank_tail(const Problem& p) { return p.r > 32 ? p.r - 32 : 0; }
+
+PlaceGeom place_geom(const Problem& p)
+{
+    PlaceGeom g{};
+    g.H = p.H; g.W = p.W; g.Hp = p.Hp; g.Wp = p.Wp; g.heads = p.heads; g.M = p.M; g.s = p.s;
+    g.d = p.d; g.dp = repacked_width(p.d); g.r = p.r; g.extra = rank_tail(p);
+    g.table_stride = p.pos_head_stride;
+    g.scale = sqrtf((float)p.d / (float)p.r);
+    return g;
+}
+
 Problem padded_shape(const Problem& p)
 {
     Problem pp = p;
     pp.d = repacked_width(p.d);
-    pp.r = repacked_width(p.r);
+    pp.r = p.r > 32 ? 32 : repacked_width(p.r);
     pp.d_true = p.d;
     pp.r_true = p.r;
     if (p.pos_head_stride) pp.pos_head_stride = (long long)p.n * pp.r;
     return pp;
+}
+
+// q and k into their padded copies; with a rank above 32 the tail of the tables rides in the spare channels
+cudaError_t pack_qk(const Problem& p, const __nv_bfloat16* q, __nv_bfloat16* q2, const __nv_bfloat16* k, __nv_bfloat16* k2, size_t rows,
+                    cudaStream_t stream, int* launches)
+{
+    const int dp = repacked_width(p.d);
+    if (!rank_tail(p)) {
+        if (cudaError_t e = copy_columns<uint32_t>(q, p.d, q2, dp, rows, stream, launches)) return e;
+        return copy_columns<uint32_t>(k, p.d, k2, dp, rows, stream, launches);
+    }
+    PlaceGeom g = place_geom(p);
+    const size_t total = rows * (size_t)(dp / 2);
+    const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    rib_pack_with_rank_tail_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const uint32_t*>(q), reinterpret_cast<uint32_t*>(q2), p.pq, g, (unsigned)rows);
+    g.scale = 1.f;
+    rib_pack_with_rank_tail_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const uint32_t*>(k), reinterpret_cast<uint32_t*>(k2), p.pk, g, (unsigned)rows);
+    *launches += 2;
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -107,8 +189,10 @@ int repacked_width(int w) { return (w + 7) & ~7; }
 
 bool sm100_repack_supported(const Problem& p)
 {
-    if (p.d < 2 || p.d > 32 || p.r < 2 || p.r > 32 || (p.d & 1) || (p.r & 1) || p.gate || p.d_true || p.r_true) return false;
+    if (p.d < 2 || p.d > 32 || p.r < 2 || (p.d & 1) || (p.r & 1) || p.gate || p.d_true || p.r_true) return false;
+    if (p.r > 32 && p.r - 32 > repacked_width(p.d) - p.d) return false;      // no room for the columns above 32
     if (p.d % 8 == 0 && p.r % 8 == 0) return false;          // these run on the kernels as they are
+    if ((long long)p.B * p.H * p.W * p.heads * 16 > 0x7fffffffLL && p.r > 32) return false;   // 32-bit indices of the tail kernels
     const Problem pp = padded_shape(p);
     return sm100_fwd_supported(pp) && sm100_bwd_supported(pp);
 }
@@ -129,8 +213,7 @@ cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     __nv_bfloat16* pq2 = reinterpret_cast<__nv_bfloat16*>(buf + 4 * img);
     __nv_bfloat16* pk2 = reinterpret_cast<__nv_bfloat16*>(buf + 4 * img + tab);
     const long long tstride = (long long)p.n * pp.r;
-    cudaError_t e = copy_columns<uint32_t>(p.q, p.d, q2, pp.d, rows, stream, launches);
-    if (!e) e = copy_columns<uint32_t>(p.k, p.d, k2, pp.d, rows, stream, launches);
+    cudaError_t e = pack_qk(p, p.q, q2, p.k, k2, rows, stream, launches);
     if (!e) e = copy_columns<uint32_t>(p.v, p.d, v2, pp.d, rows, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pq, p.pos_head_stride, p.r, pq2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pk, p.pos_head_stride, p.r, pk2, tstride, pp.r, tables, p.n, stream, launches);
@@ -162,7 +245,8 @@ cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     const long long tstride = (long long)p.n * pp.r;
     const __nv_bfloat16* ins[5] = {p.q, p.k, p.v, p.out, p.dout};
     cudaError_t e = cudaSuccess;
-    for (int i = 0; i < 5 && !e; ++i) e = copy_columns<uint32_t>(ins[i], p.d, image(i), pp.d, rows, stream, launches);
+    e = pack_qk(p, p.q, image(0), p.k, image(1), rows, stream, launches);
+    for (int i = 2; i < 5 && !e; ++i) e = copy_columns<uint32_t>(ins[i], p.d, image(i), pp.d, rows, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pq, p.pos_head_stride, p.r, pq2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pk, p.pos_head_stride, p.r, pk2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) {
@@ -177,6 +261,15 @@ cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     const long long ustride = p.pos_head_stride ? p.pos_head_stride : 0;
     if (!e) e = copy_tables<float2>(dpq2, tstride, pp.r, p.dpq, ustride, p.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<float2>(dpk2, tstride, pp.r, p.dpk, ustride, p.r, tables, p.n, stream, launches);
+    if (!e && rank_tail(p)) {
+        // (the copies above have cleared the columns from 32 on: the tail's gradients are summed into them)
+        const PlaceGeom g = place_geom(p);
+        const size_t total = rows * (size_t)g.extra;
+        const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+        rib_rank_tail_grads_kernel<<<blocks, 256, 0, stream>>>(image(5), image(6), p.dpq, p.dpk, g, (unsigned)rows);
+        ++*launches;
+        e = cudaGetLastError();
+    }
     const cudaError_t f = cudaFreeAsync(buf, stream);
     return e ? e : f;
 }

@@ -60,3 +60,13 @@ def oracle_fwd(cpu, wl, pairs=None):
 
 def oracle_bwd(cpu, wl, pairs=None):
     return orc.bwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk", "dout")), wl.window, wl.shift, pairs=pairs)
+
+
+def widths_fit_tensor_cores(d: int, r: int) -> bool:
+    """Head width and rank that the tcgen05 kernels take: multiples of 8 up to 32 as they are, other even widths through
+    zero-padded copies (a rank above 32 only when its columns above 32 fit the spare channels of the padded head)."""
+    if d < 2 or d > 32 or r < 2 or d % 2 or r % 2:
+        return False
+    if d % 8 == 0 and r % 8 == 0:
+        return r <= 32
+    return r <= 32 or r - 32 <= (-d) % 8

@@ -10,7 +10,7 @@ from oracle import rib_oracle as orc
 from paper_2603_06738_b200 import binding, synthetic
 from paper_2603_06738_b200.synthetic import Workload
 
-from parity_util import compare, to_f64
+from parity_util import compare, to_f64, widths_fit_tensor_cores
 
 pytestmark = pytest.mark.gpu
 
@@ -28,12 +28,12 @@ CASES = [
     Workload("m_128x64_w64_s32", 1, 128, 64, 2, 32, 16, 64, 32, seed=90),
     Workload("m_64x64_w32_s0", 1, 64, 64, 2, 32, 16, 32, 0, seed=91),            # no shift: nothing is masked
     Workload("m_64x32_w32_s16_d16_r24", 1, 64, 32, 3, 16, 24, 32, 16, seed=93),  # narrow head, rank 24
+    Workload("m_64x32_w32_s16_d30_r18", 1, 64, 32, 3, 30, 18, 32, 16, seed=94),  # 60-byte rows: zero-padded copies
 ]
 
 
 def is_fast(wl, path):
-    return (path != "generic" and wl.d % 8 == 0 and wl.d <= 32 and wl.r % 8 == 0 and 8 <= wl.r <= 32 and wl.window % 16 == 0
-            and wl.shift % 8 == 0)
+    return path != "generic" and widths_fit_tensor_cores(wl.d, wl.r) and wl.window % 16 == 0 and wl.shift % 8 == 0
 
 
 @pytest.mark.parametrize("wl", CASES, ids=lambda w: w.name)

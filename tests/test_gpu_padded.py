@@ -9,7 +9,7 @@ from oracle import rib_padded_oracle as pad
 from paper_2603_06738_b200 import binding, synthetic
 from paper_2603_06738_b200.synthetic import Workload
 
-from parity_util import compare, to_f64
+from parity_util import compare, to_f64, widths_fit_tensor_cores
 
 pytestmark = pytest.mark.gpu
 
@@ -30,6 +30,7 @@ CASES = [
     Workload("p_8x24_w16_s8", 2, 8, 24, 2, 32, 16, 16, 8, seed=74),
     Workload("p_88x40_w32_s8", 2, 88, 40, 2, 32, 16, 32, 8, seed=75),             # whole query tiles in the extension
     Workload("p_40x56_w16_d16_r24", 1, 40, 56, 3, 16, 24, 16, 8, seed=77),         # narrow head, rank 24
+    Workload("p_40x56_w16_d30_r34", 1, 40, 56, 3, 30, 34, 16, 8, seed=78),         # 60-byte rows: zero-padded copies, rank tail in the spare channels
 ]
 
 
@@ -46,7 +47,7 @@ def test_padded_forward_every_element(wl, path):
         binding.rib_set_path(binding.RIB_PATH_NONE)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
-    fast = (path == "auto" and wl.d % 8 == 0 and wl.d <= 32 and wl.r % 8 == 0 and 8 <= wl.r <= 32 and wl.window % 16 == 0
+    fast = (path == "auto" and widths_fit_tensor_cores(wl.d, wl.r) and wl.window % 16 == 0
             and wl.shift % 8 == 0 and wl.H % 8 == 0 and wl.W % 8 == 0)
     assert used == (binding.RIB_PATH_SM100 if fast else binding.RIB_PATH_GENERIC)
     ref_out, ref_lse = pad.fwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk")), wl.window, wl.shift)
@@ -74,7 +75,7 @@ def test_padded_backward_every_element(wl, path):
         binding.rib_set_path(binding.RIB_PATH_NONE)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
-    fast = (path == "auto" and wl.d % 8 == 0 and wl.d <= 32 and wl.r % 8 == 0 and 8 <= wl.r <= 32 and wl.window % 16 == 0
+    fast = (path == "auto" and widths_fit_tensor_cores(wl.d, wl.r) and wl.window % 16 == 0
             and wl.shift % 8 == 0 and wl.H % 8 == 0 and wl.W % 8 == 0)
     assert used == (binding.RIB_PATH_SM100 if fast else binding.RIB_PATH_GENERIC)
     ref = pad.bwd(*(to_f64(cpu[k]) for k in ("q", "k", "v", "pq", "pk", "dout")), wl.window, wl.shift)

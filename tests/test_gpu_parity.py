@@ -28,11 +28,12 @@ SMALL = [
     Workload("w16_s8_rank32", 2, 32, 48, 2, 32, 32, 16, 8, seed=22),       # rank 32 (d + r = 64) on the tcgen05 kernels
     Workload("w32_s16_rank32", 1, 64, 32, 3, 32, 32, 32, 16, seed=23),
     # the head widths of the paper's other network rows (appendix table of network implementations): 60-byte rows, which the
-    # tcgen05 kernels take through zero-padded copies when d and r are even and at most 32 (r = 34 stays on the any-shape kernels)
+    # tcgen05 kernels take through zero-padded copies when d and r are even (r = 34: the two columns above 32 ride in the spare channels of d = 30)
     Workload("sst_d30_r18_w16", 1, 32, 32, 6, 30, 18, 16, 0, seed=24),
     Workload("sst_d30_r34_w32", 1, 32, 64, 3, 30, 34, 32, 16, seed=25),
     Workload("sst_d30_r18_w32_headwise", 2, 64, 32, 3, 30, 18, 32, 16, seed=36, headwise=True),   # zero-padded copies, tcgen05 kernels
     Workload("d10_r6_w16", 1, 32, 32, 2, 10, 6, 16, 8, seed=37),
+    Workload("sst_d30_r34_w16_headwise", 2, 32, 48, 3, 30, 34, 16, 8, seed=38, headwise=True),   # rank 34: two columns ride in the head's spare channels
     Workload("light_d16_r24_w16", 2, 32, 32, 3, 16, 24, 16, 8, seed=26),       # d + r = 40: not a multiple of 16
     Workload("odd_d15_r7_w8", 1, 16, 16, 2, 15, 7, 8, 3, seed=27),
     # head widths and ranks that are multiples of 8: 32-wide tiles filled up with zeros by the TMA boxes (tcgen05 kernels)
@@ -48,7 +49,7 @@ SMALL = [
 ]
 NARROW = [wl for wl in SMALL if wl.name in ("light_d16_r24_w16", "d16_r16_w32_s16", "d24_r8_w16_s8", "d8_r32_w16", "d16_r24_w32_headwise",
                                              "w8_packed", "w8_packed_rank32_headwise", "w8_packed_d16_r24",
-                                             "sst_d30_r18_w16", "sst_d30_r18_w32_headwise", "d10_r6_w16")]
+                                             "sst_d30_r18_w16", "sst_d30_r18_w32_headwise", "d10_r6_w16", "sst_d30_r34_w32", "sst_d30_r34_w16_headwise")]
 
 
 def _inputs_for(wl):
