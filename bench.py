@@ -476,6 +476,18 @@ def main():
                                    "paths": [binding.rib_last_path()],
                                    "note": "tiles are 32 + 32 columns wide on the tensor cores, zeros beyond d and r: the useful flops counted here are 58 % of those issued"}
             del hq, hk, hv, hdo, out_h, lse_h
+            # the SST rows of the paper's network table: 30-channel heads with rank 18 and 34 (60-byte rows: zero-padded copies)
+            sq, sk, sv, sdo = (torch.randn((wl.B, wl.H, wl.W, wl.heads, 30), device=dev).to(torch.bfloat16) for _ in range(4))
+            for r_s in (18, 34):
+                spq, spk = ((0.5 * torch.randn((wl.n, r_s), device=dev)).to(torch.bfloat16) for _ in range(2))
+                out_s, lse_s = binding.rib_window_attn_fwd(sq, sk, sv, spq, spk, wl.window, wl.shift)
+                f_ms = timed(lambda: binding.rib_window_attn_fwd(sq, sk, sv, spq, spk, wl.window, wl.shift))
+                b_ms = timed(lambda: binding.rib_window_attn_bwd(sq, sk, sv, spq, spk, out_s, lse_s, sdo, wl.window, wl.shift))
+                variants[f"d30_r{r_s}"] = {"d": 30, "r": r_s, "fwd_ms": f_ms, "bwd_ms": b_ms,
+                                           "fwd_tflops": wl.pairs * 2 * wl.n * wl.n * (2 * 30 + r_s) / (f_ms * 1e-3) / 1e12,
+                                           "bwd_tflops": wl.pairs * 2 * wl.n * wl.n * (5 * 30 + 3 * r_s) / (b_ms * 1e-3) / 1e12,
+                                           "paths": [binding.rib_last_path()], "note": "includes the copies into and out of the padded scratch"}
+            del sq, sk, sv, sdo, out_s, lse_s
             # windows of 8 x 8 tokens on the same map (memory-bound: 4 x 64 B read and 64 B written per token-head in the forward)
             w8pq, w8pk = ((0.5 * torch.randn((64, wl.r), device=dev)).to(torch.bfloat16) for _ in range(2))
             out_8, lse_8 = binding.rib_window_attn_fwd(s0["q"], s0["k"], s0["v"], w8pq, w8pk, 8, 0)
