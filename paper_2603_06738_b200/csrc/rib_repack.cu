@@ -113,6 +113,52 @@ __global__ void __launch_bounds__(256) rib_rank_tail_grads_kernel(const __nv_bfl
     }
 }
 
+// The image tensors (rows of bf16, widths in 4-byte words; the wide side is a multiple of 4 words): a thread moves one
+// 16-byte piece of the wide side, which is one vector access there and up to four word accesses on the narrow side.
+// kWiden: narrow src -> wide dst with zeros behind; else wide src -> narrow dst.
+template <bool kWiden>
+__global__ void __launch_bounds__(256) rib_resize_rows_kernel(const uint32_t* __restrict__ src, uint32_t* __restrict__ dst, int narrow, int wide,
+                                                             unsigned rows)
+{
+    const unsigned per_row = (unsigned)wide / 4u, total = rows * per_row;
+    for (unsigned e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const unsigned row = e / per_row, piece = e - row * per_row;
+        const int w0 = 4 * (int)piece;
+        if (kWiden) {
+            const uint32_t* in = src + (size_t)row * narrow + w0;
+            uint32_t v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[k] = w0 + k < narrow ? in[k] : 0u;
+            *reinterpret_cast<uint4*>(dst + (size_t)row * wide + w0) = make_uint4(v[0], v[1], v[2], v[3]);
+        } else {
+            const uint4 v = *reinterpret_cast<const uint4*>(src + (size_t)row * wide + w0);
+            uint32_t* out = dst + (size_t)row * narrow + w0;
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (w0 + k < narrow) out[k] = w[k];
+        }
+    }
+}
+
+// bf16 image rows of `ws` elements -> rows of `wd` elements (one of the two a multiple of 8, the other smaller or equal)
+cudaError_t resize_rows(const void* src, int ws, void* dst, int wd, size_t rows, cudaStream_t stream, int* launches)
+{
+    const int wide = (ws > wd ? ws : wd) / 2, narrow = (ws > wd ? wd : ws) / 2;      // words
+    const size_t chunk = (size_t)0x7fffffff / (size_t)wide;
+    for (size_t r0 = 0; r0 < rows; r0 += chunk) {
+        const size_t nrows = rows - r0 < chunk ? rows - r0 : chunk, total = nrows * (size_t)(wide / 4);
+        const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 32 ? (total + 255) / 256 : 148 * 32);
+        const uint32_t* s32 = static_cast<const uint32_t*>(src) + r0 * (size_t)(ws / 2);
+        uint32_t* d32 = static_cast<uint32_t*>(dst) + r0 * (size_t)(wd / 2);
+        if (wd >= ws) rib_resize_rows_kernel<true><<<blocks, 256, 0, stream>>>(s32, d32, narrow, wide, (unsigned)nrows);
+        else rib_resize_rows_kernel<false><<<blocks, 256, 0, stream>>>(s32, d32, narrow, wide, (unsigned)nrows);
+        ++*launches;
+        if (cudaError_t e = cudaGetLastError()) return e;
+    }
+    return cudaSuccess;
+}
+
 template <typename T>
 cudaError_t copy_columns(const void* src, int ws_elems, void* dst, int wd_elems, size_t rows, cudaStream_t stream, int* launches)
 {
@@ -170,8 +216,8 @@ cudaError_t pack_qk(const Problem& p, const __nv_bfloat16* q, __nv_bfloat16* q2,
 {
     const int dp = repacked_width(p.d);
     if (!rank_tail(p)) {
-        if (cudaError_t e = copy_columns<uint32_t>(q, p.d, q2, dp, rows, stream, launches)) return e;
-        return copy_columns<uint32_t>(k, p.d, k2, dp, rows, stream, launches);
+        if (cudaError_t e = resize_rows(q, p.d, q2, dp, rows, stream, launches)) return e;
+        return resize_rows(k, p.d, k2, dp, rows, stream, launches);
     }
     PlaceGeom g = place_geom(p);
     const size_t total = rows * (size_t)(dp / 2);
@@ -214,7 +260,7 @@ cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     __nv_bfloat16* pk2 = reinterpret_cast<__nv_bfloat16*>(buf + 4 * img + tab);
     const long long tstride = (long long)p.n * pp.r;
     cudaError_t e = pack_qk(p, p.q, q2, p.k, k2, rows, stream, launches);
-    if (!e) e = copy_columns<uint32_t>(p.v, p.d, v2, pp.d, rows, stream, launches);
+    if (!e) e = resize_rows(p.v, p.d, v2, pp.d, rows, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pq, p.pos_head_stride, p.r, pq2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pk, p.pos_head_stride, p.r, pk2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) {
@@ -222,7 +268,7 @@ cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launc
         e = sm100_fwd(pp, stream);
         ++*launches;
     }
-    if (!e) e = copy_columns<uint32_t>(o2, pp.d, p.out_w, p.d, rows, stream, launches);
+    if (!e) e = resize_rows(o2, pp.d, p.out_w, p.d, rows, stream, launches);
     const cudaError_t f = cudaFreeAsync(buf, stream);
     return e ? e : f;
 }
@@ -246,7 +292,7 @@ cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     const __nv_bfloat16* ins[5] = {p.q, p.k, p.v, p.out, p.dout};
     cudaError_t e = cudaSuccess;
     e = pack_qk(p, p.q, image(0), p.k, image(1), rows, stream, launches);
-    for (int i = 2; i < 5 && !e; ++i) e = copy_columns<uint32_t>(ins[i], p.d, image(i), pp.d, rows, stream, launches);
+    for (int i = 2; i < 5 && !e; ++i) e = resize_rows(ins[i], p.d, image(i), pp.d, rows, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pq, p.pos_head_stride, p.r, pq2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pk, p.pos_head_stride, p.r, pk2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) {
@@ -257,7 +303,7 @@ cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launc
         *launches += 3;
     }
     __nv_bfloat16* outs[3] = {p.dq, p.dk, p.dv};
-    for (int i = 0; i < 3 && !e; ++i) e = copy_columns<uint32_t>(image(5 + i), pp.d, outs[i], p.d, rows, stream, launches);
+    for (int i = 0; i < 3 && !e; ++i) e = resize_rows(image(5 + i), pp.d, outs[i], p.d, rows, stream, launches);
     const long long ustride = p.pos_head_stride ? p.pos_head_stride : 0;
     if (!e) e = copy_tables<float2>(dpq2, tstride, pp.r, p.dpq, ustride, p.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<float2>(dpk2, tstride, pp.r, p.dpk, ustride, p.r, tables, p.n, stream, launches);
