@@ -221,7 +221,9 @@ size_t rib_window_cycle_bwd_workspace(const int* windows, int layers, int B, int
  *   b_dw  : fp32 [D].   w_pw : fp32 [D][D], [output channel][input channel].   b_pw : fp32 [D].
  *   gate  : bf16 [B][H][W][D], overwritten (rib_cla_gate) / read (rib_window_attn_fwd_gated).
  * The paper does not state padding, stride or biases of the two convolutions; these are the readings taken.
- * rib_cla_gate supports D = 64, 128 or 192 with H a multiple of 8 and W a multiple of 16 (RIB_ERR_UNSUPPORTED
+ * rib_cla_gate supports even D up to 192 (its kernel takes 64, 128 or 192 channels; any other even D, such as 6 heads of 30
+ * or of 16 channels, runs on copies filled up with zero channels, drawn from the library's stream-ordered scratch pool)
+ * with H a multiple of 8 and W a multiple of 16 (RIB_ERR_UNSUPPORTED
  * otherwise); all pointers 16-byte aligned.  rib_window_attn_fwd_gated takes the shapes of
  * rib_window_attn_fwd_headwise (pos_head_stride = 0: one table for all heads).
  */
@@ -249,7 +251,8 @@ int rib_window_attn_fwd_gated(const void* q, const void* k, const void* v, const
  *   dx: bf16 [B][H][W][D];  dw_dw [D][3][3], db_dw [D], dw_pw [D][D], db_pw [D]: fp32; all five overwritten.
  *   workspace: device scratch of at least rib_cla_gate_bwd_workspace(B, H, W, D) bytes (dY in fp32 and the
  *   transposed matrix), 16-byte aligned, owned by the caller, contents undefined afterwards.
- *   Any positive H and W; D = 64, 128 or 192 (RIB_ERR_UNSUPPORTED otherwise).  Three kernels (the first one clears the four weight gradients) on
+ *   Any positive H and W; even D up to 192 (RIB_ERR_UNSUPPORTED otherwise; 64, 128 and 192 as they are, other counts on copies
+ *   filled up with zero channels from the library's scratch pool).  Three kernels (the first one clears the four weight gradients) on
  *   `stream`: the point-wise part on the tensor cores (Y, dZ and w_pw enter the products as bf16, sums in fp32) and the
  *   depth-wise part; with rib_set_path(RIB_PATH_GENERIC) the point-wise part runs in fp32 instead (one more small
  *   kernel).  The weight gradients are fp32 sums in no fixed order (atomics): equal up to rounding from call to call.

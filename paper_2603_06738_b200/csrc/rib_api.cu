@@ -234,16 +234,21 @@ int rib_cla_gate(const void* x, const float* w_dw, const float* b_dw, const floa
 {
     if (!x || !w_dw || !b_dw || !w_pw || !b_pw || !gate) return RIB_ERR_NULL;
     if (B <= 0 || H <= 0 || W <= 0 || D <= 0) return RIB_ERR_SHAPE;
-    if (!rib::cla_gate_supported(H, W, D)) return RIB_ERR_UNSUPPORTED;
+    // other even channel counts up to 192 (6 heads of 30 or 16 channels) run on zero-padded copies
+    const bool native = rib::cla_gate_supported(H, W, D);
+    if (!native && !(rib::cla_padded_channels(D) && rib::cla_gate_supported(H, W, rib::cla_padded_channels(D)))) return RIB_ERR_UNSUPPORTED;
     const void* ptrs[] = {x, w_dw, b_dw, w_pw, b_pw, gate};
     for (const void* ptr : ptrs)
         if (!aligned16(ptr)) return RIB_ERR_ALIGN;
     int* status = nullptr;
     if (int rc = device_status_ptr(&status)) return rc;
-    const cudaError_t e = rib::cla_gate(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw, B, H, W, D,
-                                        static_cast<__nv_bfloat16*>(gate), status, static_cast<cudaStream_t>(stream));
+    int launches = 1;
+    const cudaError_t e = native ? rib::cla_gate(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw, B, H, W, D,
+                                                 static_cast<__nv_bfloat16*>(gate), status, static_cast<cudaStream_t>(stream))
+                                 : rib::cla_gate_padded(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw, B, H, W, D,
+                                                        static_cast<__nv_bfloat16*>(gate), status, static_cast<cudaStream_t>(stream), &launches);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
-    g_kernel_launches += 1;
+    g_kernel_launches += launches;
     return RIB_OK;
 }
 
@@ -280,6 +285,7 @@ int rib_cla_product_bwd(const void* out, const void* gate, const void* dout_gate
 size_t rib_cla_gate_bwd_workspace(int B, int H, int W, int D)
 {
     if (B <= 0 || H <= 0 || W <= 0 || D <= 0) return 0;
+    if (!rib::cla_gate_bwd_supported(D) && rib::cla_padded_channels(D)) D = rib::cla_padded_channels(D);     // runs on padded copies
     return rib::cla_gate_bwd_workspace_bytes((long long)B * H * W, D);
 }
 
@@ -290,7 +296,8 @@ int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const 
 {
     if (!x || !w_dw || !b_dw || !w_pw || !b_pw || !dgate || !dx || !dw_dw || !db_dw || !dw_pw || !db_pw) return RIB_ERR_NULL;
     if (B <= 0 || H <= 0 || W <= 0 || D <= 0) return RIB_ERR_SHAPE;
-    if (!rib::cla_gate_bwd_supported(D)) return RIB_ERR_UNSUPPORTED;
+    const bool native = rib::cla_gate_bwd_supported(D);
+    if (!native && !rib::cla_padded_channels(D)) return RIB_ERR_UNSUPPORTED;
     const void* ptrs[] = {x, w_dw, b_dw, w_pw, b_pw, dgate, dx, dw_dw, db_dw, dw_pw, db_pw, workspace};
     for (const void* ptr : ptrs)
         if (!aligned16(ptr)) return RIB_ERR_ALIGN;
@@ -298,12 +305,17 @@ int rib_cla_gate_bwd(const void* x, const float* w_dw, const float* b_dw, const 
     int* status = nullptr;
     if (int rc = device_status_ptr(&status)) return rc;
     const bool fast = g_forced_path.load() != RIB_PATH_GENERIC;
-    const cudaError_t e = rib::cla_gate_bwd(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw,
-                                            static_cast<const __nv_bfloat16*>(dgate), B, H, W, D, static_cast<__nv_bfloat16*>(dx),
-                                            dw_dw, db_dw, dw_pw, db_pw, workspace, fast, status, static_cast<cudaStream_t>(stream));
+    int launches = fast ? 3 : 4;           // zeroing of the weight gradients, (transpose,) point-wise part, depth-wise part
+    const cudaError_t e =
+        native ? rib::cla_gate_bwd(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw, static_cast<const __nv_bfloat16*>(dgate), B, H,
+                                   W, D, static_cast<__nv_bfloat16*>(dx), dw_dw, db_dw, dw_pw, db_pw, workspace, fast, status,
+                                   static_cast<cudaStream_t>(stream))
+               : rib::cla_gate_bwd_padded(static_cast<const __nv_bfloat16*>(x), w_dw, b_dw, w_pw, b_pw, static_cast<const __nv_bfloat16*>(dgate),
+                                          B, H, W, D, static_cast<__nv_bfloat16*>(dx), dw_dw, db_dw, dw_pw, db_pw, workspace, fast, status,
+                                          static_cast<cudaStream_t>(stream), &launches);
     if (e != cudaSuccess) return RIB_ERR_CUDA;
     t_last_path = fast ? RIB_PATH_SM100 : RIB_PATH_GENERIC;
-    g_kernel_launches += fast ? 3 : 4;     // zeroing of the weight gradients, (transpose,) point-wise part, depth-wise part
+    g_kernel_launches += launches;
     return RIB_OK;
 }
 

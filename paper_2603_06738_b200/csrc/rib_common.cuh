@@ -76,6 +76,13 @@ int repacked_width(int w);                    // the next multiple of 8
 cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launches);
 cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launches);
 
+// Channel counts the gate kernels do not take (even D up to 192): zero-padded copies in the library's scratch pool.
+int cla_padded_channels(int D);               // 64, 128 or 192; 0 = not paddable
+cudaError_t cla_gate_padded(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw, int B, int H,
+                            int W, int D, __nv_bfloat16* gate, int* status, cudaStream_t stream, int* launches);
+cudaError_t cla_gate_bwd_padded(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
+                                const __nv_bfloat16* dgate, int B, int H, int W, int D, __nv_bfloat16* dx, float* dw_dw, float* db_dw,
+                                float* dw_pw, float* db_pw, void* workspace, bool tensor_cores, int* status, cudaStream_t stream, int* launches);
 bool cla_gate_supported(int H, int W, int D);
 cudaError_t cla_gate(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw, int B, int H,
                      int W, int D, __nv_bfloat16* gate, int* status, cudaStream_t stream);

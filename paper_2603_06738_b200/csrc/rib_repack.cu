@@ -235,7 +235,7 @@ int repacked_width(int w) { return (w + 7) & ~7; }
 
 bool sm100_repack_supported(const Problem& p)
 {
-    if (p.d < 2 || p.d > 32 || p.r < 2 || (p.d & 1) || (p.r & 1) || p.gate || p.d_true || p.r_true) return false;
+    if (p.d < 2 || p.d > 32 || p.r < 2 || (p.d & 1) || (p.r & 1) || p.d_true || p.r_true) return false;
     if (p.r > 32 && p.r - 32 > repacked_width(p.d) - p.d) return false;      // no room for the columns above 32
     if (p.d % 8 == 0 && p.r % 8 == 0) return false;          // these run on the kernels as they are
     if ((long long)p.B * p.H * p.W * p.heads * 16 > 0x7fffffffLL && p.r > 32) return false;   // 32-bit indices of the tail kernels
@@ -251,16 +251,18 @@ cudaError_t sm100_fwd_repacked(const Problem& p, cudaStream_t stream, int* launc
     const size_t rows = (size_t)p.B * p.H * p.W * p.heads;
     const size_t img = up256(rows * pp.d * sizeof(__nv_bfloat16)), tab = up256((size_t)tables * p.n * pp.r * sizeof(__nv_bfloat16));
     uint8_t* buf = nullptr;
-    if (cudaError_t e = scratch_alloc(&buf, 4 * img + 2 * tab, stream)) return e;
+    if (cudaError_t e = scratch_alloc(&buf, 5 * img + 2 * tab, stream)) return e;
     __nv_bfloat16* q2 = reinterpret_cast<__nv_bfloat16*>(buf);
     __nv_bfloat16* k2 = reinterpret_cast<__nv_bfloat16*>(buf + img);
     __nv_bfloat16* v2 = reinterpret_cast<__nv_bfloat16*>(buf + 2 * img);
     __nv_bfloat16* o2 = reinterpret_cast<__nv_bfloat16*>(buf + 3 * img);
-    __nv_bfloat16* pq2 = reinterpret_cast<__nv_bfloat16*>(buf + 4 * img);
-    __nv_bfloat16* pk2 = reinterpret_cast<__nv_bfloat16*>(buf + 4 * img + tab);
+    __nv_bfloat16* g2 = reinterpret_cast<__nv_bfloat16*>(buf + 4 * img);          // the CLA gate, if any (layout of out)
+    __nv_bfloat16* pq2 = reinterpret_cast<__nv_bfloat16*>(buf + 5 * img);
+    __nv_bfloat16* pk2 = reinterpret_cast<__nv_bfloat16*>(buf + 5 * img + tab);
     const long long tstride = (long long)p.n * pp.r;
     cudaError_t e = pack_qk(p, p.q, q2, p.k, k2, rows, stream, launches);
     if (!e) e = resize_rows(p.v, p.d, v2, pp.d, rows, stream, launches);
+    if (!e && p.gate) { e = resize_rows(p.gate, p.d, g2, pp.d, rows, stream, launches); pp.gate = g2; }
     if (!e) e = copy_tables<uint32_t>(p.pq, p.pos_head_stride, p.r, pq2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) e = copy_tables<uint32_t>(p.pk, p.pos_head_stride, p.r, pk2, tstride, pp.r, tables, p.n, stream, launches);
     if (!e) {
@@ -316,6 +318,110 @@ cudaError_t sm100_bwd_repacked(const Problem& p, cudaStream_t stream, int* launc
         ++*launches;
         e = cudaGetLastError();
     }
+    const cudaError_t f = cudaFreeAsync(buf, stream);
+    return e ? e : f;
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// The CLA gate kernels take D = 64, 128 or 192 channels.  Other even D up to 192 (6 heads of 30 or of 16 channels: 180,
+// 96) run on them through copies with the channel dimension filled up with zeros: zero weights keep the added channels
+// out of every real one (their own gate is sigmoid(0), which is dropped), and their gradients are zero.
+// ------------------------------------------------------------------------------------------------------------------
+namespace {
+
+// dst[r][c] = src[r][c] where both have the entry, 0 elsewhere (fp32 matrices: weights in, gradients out)
+__global__ void __launch_bounds__(256) rib_fit_matrix_kernel(const float* __restrict__ src, int rs, int cs, float* __restrict__ dst, int rd, int cd)
+{
+    const int total = rd * cd;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const int r = e / cd, c = e - r * cd;
+        dst[e] = r < rs && c < cs ? src[r * cs + c] : 0.f;
+    }
+}
+
+cudaError_t fit_matrix(const float* src, int rs, int cs, float* dst, int rd, int cd, cudaStream_t stream, int* launches)
+{
+    rib_fit_matrix_kernel<<<(rd * cd + 255) / 256, 256, 0, stream>>>(src, rs, cs, dst, rd, cd);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+struct PaddedWeights { float *w_dw, *b_dw, *w_pw, *b_pw; size_t bytes; };
+
+size_t weight_bytes(int Dp) { return up256((size_t)Dp * 9 * 4) + 2 * up256((size_t)Dp * 4) + up256((size_t)Dp * Dp * 4); }
+
+PaddedWeights weight_layout(uint8_t* base, int Dp)
+{
+    PaddedWeights w;
+    size_t off = 0;
+    w.w_dw = reinterpret_cast<float*>(base + off); off += up256((size_t)Dp * 9 * 4);
+    w.b_dw = reinterpret_cast<float*>(base + off); off += up256((size_t)Dp * 4);
+    w.w_pw = reinterpret_cast<float*>(base + off); off += up256((size_t)Dp * Dp * 4);
+    w.b_pw = reinterpret_cast<float*>(base + off); off += up256((size_t)Dp * 4);
+    w.bytes = off;
+    return w;
+}
+
+}  // namespace
+
+int cla_padded_channels(int D)
+{
+    if (D <= 0 || D > 192 || (D & 1)) return 0;
+    return D <= 64 ? 64 : D <= 128 ? 128 : 192;
+}
+
+cudaError_t cla_gate_padded(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw, int B, int H,
+                            int W, int D, __nv_bfloat16* gate, int* status, cudaStream_t stream, int* launches)
+{
+    *launches = 0;
+    const int Dp = cla_padded_channels(D);
+    const size_t pixels = (size_t)B * H * W, img = up256(pixels * Dp * 2);
+    const size_t wbytes = weight_bytes(Dp);
+    uint8_t* buf = nullptr;
+    if (cudaError_t e = scratch_alloc(&buf, 2 * img + wbytes, stream)) return e;
+    __nv_bfloat16* x2 = reinterpret_cast<__nv_bfloat16*>(buf);
+    __nv_bfloat16* g2 = reinterpret_cast<__nv_bfloat16*>(buf + img);
+    const PaddedWeights w = weight_layout(buf + 2 * img, Dp);
+    cudaError_t e = resize_rows(x, D, x2, Dp, pixels, stream, launches);
+    if (!e) e = fit_matrix(w_dw, D, 9, w.w_dw, Dp, 9, stream, launches);
+    if (!e) e = fit_matrix(b_dw, 1, D, w.b_dw, 1, Dp, stream, launches);
+    if (!e) e = fit_matrix(w_pw, D, D, w.w_pw, Dp, Dp, stream, launches);
+    if (!e) e = fit_matrix(b_pw, 1, D, w.b_pw, 1, Dp, stream, launches);
+    if (!e) { e = cla_gate(x2, w.w_dw, w.b_dw, w.w_pw, w.b_pw, B, H, W, Dp, g2, status, stream); ++*launches; }
+    if (!e) e = resize_rows(g2, Dp, gate, D, pixels, stream, launches);
+    const cudaError_t f = cudaFreeAsync(buf, stream);
+    return e ? e : f;
+}
+
+cudaError_t cla_gate_bwd_padded(const __nv_bfloat16* x, const float* w_dw, const float* b_dw, const float* w_pw, const float* b_pw,
+                                const __nv_bfloat16* dgate, int B, int H, int W, int D, __nv_bfloat16* dx, float* dw_dw, float* db_dw,
+                                float* dw_pw, float* db_pw, void* workspace, bool tensor_cores, int* status, cudaStream_t stream, int* launches)
+{
+    *launches = 0;
+    const int Dp = cla_padded_channels(D);
+    const size_t pixels = (size_t)B * H * W, img = up256(pixels * Dp * 2);
+    const size_t wbytes = weight_bytes(Dp);
+    uint8_t* buf = nullptr;
+    if (cudaError_t e = scratch_alloc(&buf, 3 * img + 2 * wbytes, stream)) return e;
+    __nv_bfloat16* x2 = reinterpret_cast<__nv_bfloat16*>(buf);
+    __nv_bfloat16* dg2 = reinterpret_cast<__nv_bfloat16*>(buf + img);
+    __nv_bfloat16* dx2 = reinterpret_cast<__nv_bfloat16*>(buf + 2 * img);
+    const PaddedWeights w = weight_layout(buf + 3 * img, Dp), g = weight_layout(buf + 3 * img + wbytes, Dp);
+    cudaError_t e = resize_rows(x, D, x2, Dp, pixels, stream, launches);
+    if (!e) e = resize_rows(dgate, D, dg2, Dp, pixels, stream, launches);
+    if (!e) e = fit_matrix(w_dw, D, 9, w.w_dw, Dp, 9, stream, launches);
+    if (!e) e = fit_matrix(b_dw, 1, D, w.b_dw, 1, Dp, stream, launches);
+    if (!e) e = fit_matrix(w_pw, D, D, w.w_pw, Dp, Dp, stream, launches);
+    if (!e) e = fit_matrix(b_pw, 1, D, w.b_pw, 1, Dp, stream, launches);
+    if (!e) {
+        e = cla_gate_bwd(x2, w.w_dw, w.b_dw, w.w_pw, w.b_pw, dg2, B, H, W, Dp, dx2, g.w_dw, g.b_dw, g.w_pw, g.b_pw, workspace, tensor_cores, status, stream);
+        *launches += tensor_cores ? 3 : 4;
+    }
+    if (!e) e = resize_rows(dx2, Dp, dx, D, pixels, stream, launches);
+    if (!e) e = fit_matrix(g.w_dw, Dp, 9, dw_dw, D, 9, stream, launches);
+    if (!e) e = fit_matrix(g.b_dw, 1, Dp, db_dw, 1, D, stream, launches);
+    if (!e) e = fit_matrix(g.w_pw, Dp, Dp, dw_pw, D, D, stream, launches);
+    if (!e) e = fit_matrix(g.b_pw, 1, Dp, db_pw, 1, D, stream, launches);
     const cudaError_t f = cudaFreeAsync(buf, stream);
     return e ? e : f;
 }

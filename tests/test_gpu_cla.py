@@ -8,7 +8,7 @@ from oracle import cla_oracle as cla
 from paper_2603_06738_b200 import binding, synthetic
 from paper_2603_06738_b200.synthetic import Workload
 
-from parity_util import compare, make, oracle_fwd, to_f64
+from parity_util import compare, make, oracle_fwd, to_f64, widths_fit_tensor_cores
 
 pytestmark = pytest.mark.gpu
 
@@ -25,7 +25,8 @@ def gate_inputs(seed, B, H, W, D):
 
 # the last three shapes give every persistent CTA several tiles (the benchmark shape: 576 tiles on 148 CTAs)
 @pytest.mark.parametrize("B,H,W,D", [(1, 8, 16, 64), (2, 16, 32, 192), (1, 24, 48, 128), (3, 40, 16, 192), (1, 96, 96, 192),
-                                     (8, 96, 96, 192), (2, 160, 160, 64), (4, 88, 96, 128)])
+                                     (8, 96, 96, 192), (2, 160, 160, 64), (4, 88, 96, 128),
+                                     (2, 16, 32, 180), (1, 24, 48, 96), (1, 8, 16, 30)])      # 6 x 30, 6 x 16 channels: zero-padded copies
 def test_gate_matches_the_oracle(B, H, W, D):
     x, ws = gate_inputs(200 + D + H, B, H, W, D)
     g = binding.rib_cla_gate(x.cuda(), *[torch.from_numpy(w).cuda() for w in ws])
@@ -56,7 +57,8 @@ def test_gate_border_pixels_see_zero_padding():
                                 Workload("gated_w32_rank32", 1, 64, 32, 6, 32, 32, 32, 16, seed=211),
                                 Workload("gated_w8_generic", 1, 16, 24, 3, 16, 8, 8, 3, seed=212),
                                 Workload("gated_w16_headwise", 1, 32, 32, 3, 32, 16, 16, 0, seed=215, headwise=True),
-                                Workload("gated_w16_d16_r24", 1, 32, 32, 4, 16, 24, 16, 8, seed=216)], ids=lambda w: w.name)
+                                Workload("gated_w16_d16_r24", 1, 32, 32, 4, 16, 24, 16, 8, seed=216),
+                                Workload("gated_w16_d30_r18", 1, 32, 32, 6, 30, 18, 16, 8, seed=217)], ids=lambda w: w.name)
 def test_gated_forward_is_attention_times_the_gate(wl, path):
     cpu, gpu = make(wl, with_dout=False)
     D = wl.heads * wl.d
@@ -69,7 +71,7 @@ def test_gated_forward_is_attention_times_the_gate(wl, path):
         binding.rib_set_path(binding.RIB_PATH_NONE)
     torch.cuda.synchronize()
     assert binding.rib_query_status() == 0
-    fast = path == "auto" and wl.d % 8 == 0 and wl.d <= 32 and wl.window % 16 == 0 and wl.shift % 8 == 0
+    fast = path == "auto" and widths_fit_tensor_cores(wl.d, wl.r) and wl.window % 16 == 0 and wl.shift % 8 == 0
     assert used == (binding.RIB_PATH_SM100 if fast else binding.RIB_PATH_GENERIC)
     ref_out, ref_lse = oracle_fwd(cpu, wl)
     compare("out", to_f64(out), cla.gated_output(ref_out, to_f64(gate)))
@@ -95,7 +97,8 @@ def test_gate_rejects_unsupported_sizes():
     w = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
     ptrs = [x.data_ptr()] + [w.data_ptr()] * 4
     launches = binding.rib_kernel_launches()
-    assert lib.rib_cla_gate(*ptrs, 1, 8, 16, 96, x.data_ptr(), None) == -3     # channels not 64, 128 or 192
+    assert lib.rib_cla_gate(*ptrs, 1, 8, 16, 95, x.data_ptr(), None) == -3     # an odd number of channels
+    assert lib.rib_cla_gate(*ptrs, 1, 8, 16, 200, x.data_ptr(), None) == -3    # more than 192 channels
     assert lib.rib_cla_gate(*ptrs, 1, 8, 24, 64, x.data_ptr(), None) == -3     # W not a multiple of 16
     assert lib.rib_cla_gate(*ptrs, 1, 12, 16, 64, x.data_ptr(), None) == -3    # H not a multiple of 8
     assert lib.rib_cla_gate(*ptrs, 0, 8, 16, 64, x.data_ptr(), None) == -2
@@ -113,7 +116,8 @@ def dgate_input(seed, shape):
 @pytest.mark.parametrize("B,H,W,D", [(1, 5, 7, 64), (2, 16, 32, 192), (1, 24, 47, 128), (3, 9, 16, 192), (1, 1, 1, 64),
                                      (1, 96, 96, 192), (2, 40, 56, 64),
                                      # several tiles per persistent CTA / block, the last one with ragged H and W
-                                     (8, 96, 96, 192), (2, 160, 160, 64), (4, 90, 100, 128)])
+                                     (8, 96, 96, 192), (2, 160, 160, 64), (4, 90, 100, 128),
+                                     (2, 19, 32, 180), (1, 24, 48, 96)])         # 6 x 30, 6 x 16 channels: zero-padded copies
 def test_gate_backward_matches_the_oracle(B, H, W, D, path):
     x, ws = gate_inputs(300 + D + H, B, H, W, D)
     dgate = dgate_input(301 + D + H, (B, H, W, D))
@@ -171,7 +175,7 @@ def test_gate_backward_rejects_unsupported_channels_without_launching():
     x = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
     w = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
     launches = binding.rib_kernel_launches()
-    assert lib.rib_cla_gate_bwd(x.data_ptr(), *[w.data_ptr()] * 4, x.data_ptr(), 1, 4, 4, 96, x.data_ptr(), *[w.data_ptr()] * 4,
+    assert lib.rib_cla_gate_bwd(x.data_ptr(), *[w.data_ptr()] * 4, x.data_ptr(), 1, 4, 4, 95, x.data_ptr(), *[w.data_ptr()] * 4,
                                 w.data_ptr(), 1 << 18, None) == -3
     assert binding.rib_kernel_launches() == launches
 
