@@ -129,7 +129,9 @@ def test_cla_backward_entry_points_validate_before_any_cuda_call(lib):
     assert call(ins=[None] + a[1:]) == -1
     assert call(outs=outs[:4] + [None]) == -1
     assert call(B=0) == -2
-    assert call(D=96) == -3
+    assert call(D=95) == -3                                                        # an odd channel count
+    assert call(D=200) == -3                                                       # more than 192 channels
+    assert lib.rib_cla_gate_bwd_workspace(1, 5, 7, 96) == (5 * 7 * 128 + 128 * 128) * 4   # 96 channels run as 128
     assert call(outs=[2050] + outs[1:]) == -4
     assert call(ws=None) == -5
     assert call(ws_bytes=need - 1) == -5
