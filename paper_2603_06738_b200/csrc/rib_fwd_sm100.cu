@@ -68,6 +68,10 @@ using namespace sm100;
 constexpr int kStages = 4;            // K/V ring depth
 constexpr int kThreads = 640;
 constexpr int kMaxRedo = 64;          // items a CTA can note for the exact pass (more: all of its items are redone)
+constexpr int kMaxListed = 1023;      // kPartial: items of a CTA whose masks are worked out once and kept in shared memory
+
+// kPartial with skipping: an item of the CTA that holds tokens, with what every role needs to walk it
+struct ItemRec { int item; uint32_t row_dead, col_dead, range; };       // range = first | last << 16 key block with tokens
 constexpr uint32_t kPolyMask = RIB_FWD_POLY_MASK;
 
 // kSFull .. kOFree: one per query tile; kDrain: one per issuing warp; kMerge: 4 * tile + quarter of the rows
@@ -90,7 +94,9 @@ struct Layout {
     static constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;                 // tmem base, abort flags, redo count
     static constexpr uint32_t kOffRedo = kOffMisc + 16;                          // [kMaxRedo] item ordinals of the exact pass
     static constexpr uint32_t kOffMerge = kOffRedo + kMaxRedo * 4;               // [2 tiles][2 halves][128 rows] (max, sum)
-    static constexpr uint32_t kSmemBytes = kOffMerge + 4 * kTile * 8 + 1024;     // + slack for manual alignment
+    static constexpr uint32_t kOffItems = kOffMerge + 4 * kTile * 8;             // [1 + kMaxListed] ItemRec; entry 0 holds the count
+    static constexpr uint32_t kSmemBytes = kOffItems + (1 + kMaxListed) * 16 + 1024;   // + slack for manual alignment
+    static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
     static_assert(kOffV % 1024 == 0 && kOffOnes % 1024 == 0, "swizzle atoms need aligned tiles");
 };
 
@@ -227,6 +233,55 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // kPartial: one warp works out, once, which of this CTA's items hold tokens and their dead-patch masks; every role then
+    // walks that list instead of testing every item itself (the tests were the cost of skipping: a few hundred cycles per
+    // role and item).
+    ItemRec* const item_list = reinterpret_cast<ItemRec*>(base_ptr + L::kOffItems) + 1;
+    int* const list_count = reinterpret_cast<int*>(base_ptr + L::kOffItems);
+    const bool listed = kPartial && !p.masked && !p.packed8 && my_items <= kMaxListed;     // the same for every thread of the CTA
+    if (listed) {
+        if (warp == 4) {
+            const int per_row = p.M >> 3;
+            const uint32_t in_window = per_row == 32 ? 0xffffffffu : (1u << per_row) - 1u;
+            int kept = 0;
+            for (int i0 = 0; i0 < my_items; i0 += 32) {
+                const int i = i0 + lane;
+                bool live = false;
+                ItemRec rec{};
+                if (i < my_items) {
+                    rec.item = (int)blockIdx.x + i * (int)gridDim.x;
+                    const ItemCoord c = decode_item(p, rec.item);
+                    for (int l = 0; l < per_row; ++l) {
+                        int y = c.wy * p.M + 8 * l + p.s; if (y >= p.Hp) y -= p.Hp;
+                        int x = c.wx * p.M + 8 * l + p.s; if (x >= p.Wp) x -= p.Wp;
+                        rec.row_dead |= (uint32_t)(y >= p.H) << l;
+                        rec.col_dead |= (uint32_t)(x >= p.W) << l;
+                    }
+                    for (int sp = 0; sp < 4; ++sp) {
+                        int pr, pc;
+                        p.div_per_row.divmod(4 * c.tp + sp, pr, pc);
+                        live = live || (((rec.row_dead >> pr) | (rec.col_dead >> pc)) & 1u) == 0u;
+                    }
+                    const uint32_t rows = ~rec.row_dead & in_window;
+                    const uint32_t pairs = ~(rec.col_dead & (rec.col_dead >> 1)) & 0x55555555u & in_window;
+                    const int jf = (__ffs(rows) - 1) * (per_row >> 1) + ((__ffs(pairs) - 1) >> 1);
+                    const int jl = (31 - __clz(rows)) * (per_row >> 1) + ((31 - __clz(pairs)) >> 1);
+                    rec.range = (uint32_t)jf | ((uint32_t)jl << 16);
+                    if (!p.skip_dead) {                  // small windows: everything is walked, the list only saves the roles the masks
+                        live = true;
+                        rec.range = (uint32_t)(nblk - 1) << 16;
+                    }
+                }
+                const uint32_t votes = __ballot_sync(0xffffffffu, live);
+                if (live) item_list[kept + __popc(votes & ((1u << lane) - 1u))] = rec;
+                kept += __popc(votes);
+            }
+            if (lane == 0) *list_count = kept;
+        }
+        __syncthreads();
+    }
+    const int live_items = listed ? *list_count : my_items;
+
     // Role state that carries over from the first pass to the exact pass: block and item counters give the barrier phases.
     uint32_t blk = 0, io = 0, nmerge = 0;
     uint32_t q_armed = 0, k_armed = 0, v_armed = 0;
@@ -237,14 +292,15 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         // pass 0: every item of this CTA; pass 1: the items noted by the fast form (all of them when the notes overflowed)
         const int noted = pass == 0 ? 0 : *redo_count;
         const bool all_items = pass == 0 || noted > kMaxRedo;
-        const int count = all_items ? my_items : noted;
-        auto item_at = [&](int i) { return (int)blockIdx.x + (all_items ? i : redo_list[i]) * (int)gridDim.x; };
+        const int count = all_items ? live_items : noted;
+        auto ordinal = [&](int i) { return all_items ? i : (int)redo_list[i]; };      // place in the CTA's sequence of items
+        auto item_at = [&](int i) { return listed ? item_list[ordinal(i)].item : (int)blockIdx.x + ordinal(i) * (int)gridDim.x; };
         // kPartial: an item whose four query patches all lie in the extension of the map has nothing to compute; every role
         // skips it by the same test, so the item and block counters that give the barrier phases stay in step.  The tests cost
         // every role some hundred cycles per item, which pays from windows of 32 x 32 tokens on (skip_dead); in smaller
         // windows an item is a block or two long and everything is walked.
         auto item_live = [&](int item) {
-            if (!kPartial || !p.skip_dead) return true;
+            if (!kPartial || !p.skip_dead || listed) return true;         // (a listed item is walked)
             const ItemCoord c = decode_item(p, item);
             bool live = false;
 #pragma unroll
@@ -307,6 +363,17 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             jf = (__ffs(rows) - 1) * (per_row >> 1) + ((__ffs(pairs) - 1) >> 1);
             jl = (31 - __clz(rows)) * (per_row >> 1) + ((31 - __clz(pairs)) >> 1);
         };
+        // the masks and the block range of item i of this pass: from the list, or worked out here (warp-collective)
+        auto item_masks = [&](int i, const ItemCoord& c, uint32_t& row_dead, uint32_t& col_dead, int& jf, int& jl) {
+            if (listed) {
+                const ItemRec rec = item_list[ordinal(i)];
+                row_dead = rec.row_dead; col_dead = rec.col_dead;
+                jf = (int)(rec.range & 0xffffu); jl = (int)(rec.range >> 16);
+            } else {
+                dead_masks(c, row_dead, col_dead);
+                if (p.skip_dead) live_range(row_dead, col_dead, jf, jl);
+            }
+        };
 
         if (warp == 0) {
             // ===================== TMA producer (lane 0) and query RIB rows bf16(Pq * sqrt(d/r)) of the same item (whole warp)
@@ -353,11 +420,11 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 __syncwarp();
                 uint32_t row_dead = 0u, col_dead = 0u;
                 int jf = 0, jl = nblk - 1;
-                if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                if (kPartial) item_masks(i, c, row_dead, col_dead, jf, jl);
                 if (lane == 0) {
                     mbar_arrive(bar(kQPos + buf));
                     for (int j = jf; j <= jl; ++j, ++blk) {
-                        if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
+                        if (kPartial && p.skip_dead && (row_dead | col_dead) != 0u && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         const uint32_t st = blk % kStages, use = blk / kStages;
                         if (use > 0 && !mbar_wait(bar(kKEmpty + st), (use - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                         mbar_arrive_expect_tx(bar(kKFull + st), kContentBytes + kPosBytes);
@@ -402,9 +469,9 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     !mbar_wait_warp(bar(kQPos + buf), (io >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
                 uint32_t row_dead = 0u, col_dead = 0u;
                 int jf = 0, jl = nblk - 1;
-                if (kPartial && p.skip_dead) { dead_masks(decode_item(p, item_at(i)), row_dead, col_dead); live_range(row_dead, col_dead, jf, jl); }
+                if (kPartial && (p.skip_dead || listed)) item_masks(i, listed ? ItemCoord{} : decode_item(p, item_at(i)), row_dead, col_dead, jf, jl);
                 for (int j = jf; j <= jl && ok; ++j, ++blk) {
-                    if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
+                    if (kPartial && p.skip_dead && (row_dead | col_dead) != 0u && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                     const uint32_t st = blk % kStages;
                     if (!mbar_wait_warp(bar(kKFull + st), (blk / kStages) & 1, abort_flag, p.status)) { ok = false; break; }
                     const uint64_t kc = smem_desc_at(kDesc64, base + kOffKc + st * kContentBytes);
@@ -443,9 +510,9 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!item_live(item_at(i))) { --io; continue; }
                 uint32_t row_dead = 0u, col_dead = 0u;
                 int jf = 0, jl = nblk - 1;
-                if (kPartial && p.skip_dead) { dead_masks(decode_item(p, item_at(i)), row_dead, col_dead); live_range(row_dead, col_dead, jf, jl); }
+                if (kPartial && (p.skip_dead || listed)) item_masks(i, listed ? ItemCoord{} : decode_item(p, item_at(i)), row_dead, col_dead, jf, jl);
                 for (int j = jf; j <= jl; ++j, ++blk) {
-                    if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
+                    if (kPartial && p.skip_dead && (row_dead | col_dead) != 0u && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                     const uint32_t st = blk % kStages;
                     // warp-uniform outcomes, so that the warp stays converged.  The first block of an item overwrites the
                     // accumulator: the epilogue of the item before must have read it.
@@ -563,10 +630,10 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     float2 neg2 = make_float2(0.f, 0.f);
                     uint32_t row_dead = 0u, col_dead = 0u;
                     int jf = 0, jl = nblk - 1;
-                    if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                    if (kPartial) item_masks(i, c, row_dead, col_dead, jf, jl);
                     if (kPartial && (p.masked | p.packed8)) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
                     for (int j = jf; j <= jl; ++j, ++blk) {
-                        if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
+                        if (kPartial && p.skip_dead && (row_dead | col_dead) != 0u && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
                         if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
                         tc_fence_after();
@@ -594,7 +661,7 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         if (lane == 0) mbar_arrive(bar(kSFree + qt));   // the next block's scores may overwrite the accumulator
                         uint32_t pa[16], pb[16];
                         float2 sc2 = scale2, ng2 = neg2;
-                        if (kPartial && patch_dead(2 * j + half, row_dead, col_dead)) {
+                        if (kPartial && (row_dead | col_dead) != 0u && patch_dead(2 * j + half, row_dead, col_dead)) {
                             // This thread's 64 keys are one 8x8 patch; in the extension of the map it holds no tokens.  The block
                             // runs through the same instructions with scale 0 and offset -119: each such key gets the weight
                             // 2^-119 (the smallest both exponential paths deliver), its zero-filled value row adds nothing to
@@ -651,10 +718,10 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     bool have_ref = false;            // kPartial: a block with real keys has set the reference
                     uint32_t row_dead = 0u, col_dead = 0u;
                     int jf = 0, jl = nblk - 1;
-                    if (kPartial) { dead_masks(c, row_dead, col_dead); if (p.skip_dead) live_range(row_dead, col_dead, jf, jl); }
+                    if (kPartial) item_masks(i, c, row_dead, col_dead, jf, jl);
                     if (kPartial && (p.masked | p.packed8)) mask_masks(c, 2 * (2 * c.tp + qt) + (row >> 6), row_dead, col_dead);
                     for (int j = jf; j <= jl; ++j, ++blk) {
-                        if (kPartial && p.skip_dead && block_dead(j, row_dead, col_dead)) { --blk; continue; }
+                        if (kPartial && p.skip_dead && (row_dead | col_dead) != 0u && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
                         if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
                         tc_fence_after();
@@ -876,7 +943,9 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     fp.exact_only = p.exact_softmax ? 1 : 0;
     fp.masked = p.masked ? 1 : 0;
     fp.packed8 = p.packed8 ? 1 : 0;
-    fp.skip_dead = kPartial && !p.masked && !p.packed8 && p.n / kTile >= 8 ? 1 : 0;      // (a mask differs from query patch to query patch)
+    // (a mask differs from query patch to query patch; in windows below 32 x 32 an item is a block or two long and the tests of
+    // the blocks cost more than the skipped ones save: measured +6 % at 16 x 16 even with the per-CTA list of live items)
+    fp.skip_dead = kPartial && !p.masked && !p.packed8 && p.n / kTile >= 8 ? 1 : 0;
     fp.div_tp = make_fast_div(fp.tiles_per_item_pair); fp.div_heads = make_fast_div(p.heads);
     fp.div_nwx = make_fast_div(p.nWx); fp.div_nwy = make_fast_div(p.nWy); fp.div_per_row = make_fast_div(p.M >> 3);
     const int grid = fp.items < sm_count ? fp.items : sm_count;
