@@ -95,8 +95,9 @@ struct Layout {
     static constexpr uint32_t kOffRedo = kOffMisc + 16;                          // [kMaxRedo] item ordinals of the exact pass
     static constexpr uint32_t kOffMerge = kOffRedo + kMaxRedo * 4;               // [2 tiles][2 halves][128 rows] (max, sum)
     static constexpr uint32_t kOffItems = kOffMerge + 4 * kTile * 8;             // [1 + kMaxListed] ItemRec; entry 0 holds the count
-    static constexpr uint32_t kSmemBytes = kOffItems + (1 + kMaxListed) * 16 + 1024;   // + slack for manual alignment
-    static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+    static constexpr uint32_t kSmemBytes = kOffItems + 1024;                           // + slack for manual alignment
+    static constexpr uint32_t kSmemBytesPartial = kOffItems + (1 + kMaxListed) * 16 + 1024;   // kPartial instantiations: with the item list
+    static_assert(kSmemBytesPartial <= 232448, "shared memory of one CTA");
     static_assert(kOffV % 1024 == 0 && kOffOnes % 1024 == 0, "swizzle atoms need aligned tiles");
 };
 
@@ -292,9 +293,12 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         // pass 0: every item of this CTA; pass 1: the items noted by the fast form (all of them when the notes overflowed)
         const int noted = pass == 0 ? 0 : *redo_count;
         const bool all_items = pass == 0 || noted > kMaxRedo;
-        const int count = all_items ? live_items : noted;
+        const int count = all_items ? (kPartial ? live_items : my_items) : noted;
         auto ordinal = [&](int i) { return all_items ? i : (int)redo_list[i]; };      // place in the CTA's sequence of items
-        auto item_at = [&](int i) { return listed ? item_list[ordinal(i)].item : (int)blockIdx.x + ordinal(i) * (int)gridDim.x; };
+        auto item_at = [&](int i) {
+            if (kPartial && listed) return item_list[ordinal(i)].item;
+            return (int)blockIdx.x + (all_items ? i : redo_list[i]) * (int)gridDim.x;
+        };
         // kPartial: an item whose four query patches all lie in the extension of the map has nothing to compute; every role
         // skips it by the same test, so the item and block counters that give the barrier phases stay in step.  The tests cost
         // every role some hundred cycles per item, which pays from windows of 32 x 32 tokens on (skip_dead); in smaller
@@ -924,7 +928,7 @@ cudaError_t launch_fwd(const Problem& p, cudaStream_t stream)
     if (!encode_image_map(&tm_q, p.q, p) || !encode_image_map(&tm_k, p.k, p) || !encode_image_map(&tm_v, p.v, p) ||
         !encode_pos_map(&tm_pk, p.pk, p, pos_tables(p), p.pos_head_stride))
         return cudaErrorInvalidValue;
-    constexpr uint32_t kSmemBytes = Layout<R>::kSmemBytes;
+    constexpr uint32_t kSmemBytes = kPartial ? Layout<R>::kSmemBytesPartial : Layout<R>::kSmemBytes;
     static KernelSetup setup;       // one per instantiation of this launcher, i.e. per kernel
     int sm_count = 0;
     if (cudaError_t e = setup.prepare(rib_fwd_sm100_kernel<R, kPartial, kGated>, kSmemBytes, &sm_count)) return e;
