@@ -576,6 +576,12 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 float* pend_lse = nullptr;
                 float pend_ref = 0.f;
                 int pend_ordinal = -1;                      // -1: nothing pending
+                // Full windows: the wait for the next block's scores is asked between the stores of P and their completion,
+                // in straight-line code (with a branch around the question the gain is gone: 3 % of the kernel).  After the
+                // last block of the pass no scores follow; there the question names the phase just used, which is complete,
+                // so that no warp sits out the time limit of a wait that nothing answers.
+                bool s_polled = false, s_ready = false;
+                const uint32_t last_blk = blk + (uint32_t)count * (uint32_t)nblk - 1u;
                 // O and l of the pending item are complete (the caller has waited for its last PV): normalise, store, note overflow
                 auto epilogue = [&]() {
                     uint32_t o[16], lsum[1];
@@ -639,7 +645,8 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     for (int j = jf; j <= jl; ++j, ++blk) {
                         if (kPartial && p.skip_dead && (row_dead | col_dead) != 0u && block_dead(j, row_dead, col_dead)) { --blk; continue; }
                         // warp-uniform outcome: the TMEM loads below are warp-collective
-                        if (!mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
+                        if (!(s_polled && __all_sync(0xffffffffu, s_ready)) && !mbar_wait_warp(bar(kSFull + qt), blk & 1, abort_flag, p.status)) { ok = false; break; }
+                        s_polled = false;
                         tc_fence_after();
                         uint32_t sa[32], sb[32];
                         if (j == jf) {
@@ -674,16 +681,22 @@ rib_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             sc2 = make_float2(0.f, 0.f);
                             ng2 = make_float2(-119.f, -119.f);
                         }
+                        // P of the tile is free once the previous block's PV has completed (long ago, as a rule).  Full windows ask
+                        // before the exponentials, so that the answer is there when they are done.
+                        const bool p_free = blk == 0 || (!kPartial && mbar_try_wait(b_free, (blk - 1) & 1));
                         exp_chunk1(sa, sc2, ng2, pa);
                         exp_chunk1(sb, sc2, ng2, pb);
-                        // P of the tile is free once the previous block's PV has completed (long ago, as a rule)
                         if (blk > 0) {
-                            if (!mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+                            if (!__all_sync(0xffffffffu, p_free) && !mbar_wait_warp(b_free, (blk - 1) & 1, abort_flag, p.status)) { ok = false; break; }
                             tc_fence_after();
                         }
                         if (j == jf && pend_ordinal >= 0) epilogue();     // that PV was the last one of the item before
                         tmem_st16(t_p, pa);
                         tmem_st16(t_p + 16, pb);
+                        if (!kPartial) {
+                            s_ready = mbar_try_wait(bar(kSFull + qt), (blk + (blk != last_blk ? 1u : 0u)) & 1);
+                            s_polled = true;
+                        }
                         tmem_wait_st();
                         tc_fence_before();
                         __syncwarp();
